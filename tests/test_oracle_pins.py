@@ -1,0 +1,347 @@
+"""Pins for the float64 oracle: each check compares an oracle function with
+something the paper or the mathematics fixes independently of it."""
+import os
+
+import numpy as np
+import pytest
+
+from oracle import gptaq_oracle as orc
+import workloads as wl
+
+GOLDEN = os.path.join(os.path.dirname(__file__), "golden")
+
+
+def tiny(n=24, m=5, k=200, seed=0, noise=0.1):
+    r = np.random.default_rng(seed)
+    Xfp = r.standard_normal((k, n))
+    Xfp[:, :2] *= 8.0
+    X = Xfp + noise * np.abs(Xfp) * r.standard_normal((k, n))
+    W = 0.05 * r.standard_normal((m, n))
+    return W, X, Xfp
+
+
+def stats_of(X, Xfp, split=3):
+    st = orc.new_stats(X.shape[1], True)
+    for a in np.array_split(np.arange(X.shape[0]), split):
+        orc.accumulate(st, X[a], Xfp[a])
+    return st
+
+
+# ---------------------------------------------------------------- statistics
+def test_statistics_brute_force():
+    _, X, Xfp = tiny(n=6, k=11)
+    st = stats_of(X, Xfp, split=2)
+    n, k = 6, 11
+    for i in range(n):
+        for j in range(n):
+            h = sum(X[t, i] * X[t, j] for t in range(k))
+            d = sum((Xfp[t, i] - X[t, i]) * X[t, j] for t in range(k))
+            assert abs(st.H[i, j] - h) < 1e-12 * (1 + abs(h))
+            assert abs(st.D[i, j] - d) < 1e-12 * (1 + abs(d))
+    assert st.tokens == k
+
+
+def test_statistics_invariants():
+    _, X, Xfp = tiny()
+    st = stats_of(X, Xfp)
+    assert np.allclose(st.H, st.H.T, rtol=0, atol=1e-12)
+    assert np.linalg.eigvalsh(st.H).min() > -1e-9
+    st0 = stats_of(X, X)
+    assert np.all(st0.D == 0.0)
+    c = 0.37
+    stc = stats_of(X, (1 + c) * X)
+    assert np.allclose(stc.D, c * stc.H, rtol=1e-12, atol=1e-10)
+    # float32 inputs are widened before any product
+    st32 = stats_of(X.astype(np.float32), Xfp.astype(np.float32))
+    ref = stats_of(X.astype(np.float32).astype(np.float64), Xfp.astype(np.float32).astype(np.float64))
+    assert np.array_equal(st32.H, ref.H) and np.array_equal(st32.D, ref.D)
+
+
+# ---------------------------------------------------------------- factor
+def test_factor_is_inverse_cholesky_and_spd():
+    _, X, Xfp = tiny()
+    st = stats_of(X, Xfp)
+    U, dead = orc.factor(st.H, st.tokens, 0.01)
+    Hd, _ = orc.damped_hessian(st.H, st.tokens, 0.01)
+    n = U.shape[0]
+    assert not dead.any()
+    assert np.allclose(np.tril(U, -1), 0.0) and np.all(np.diag(U) > 0)
+    assert np.allclose(U.T @ U @ Hd, np.eye(n), atol=1e-10)
+    assert np.linalg.eigvalsh(Hd).min() > 0
+    lam = 0.01 * np.mean(np.diag(st.H / st.tokens))
+    assert np.allclose(Hd, st.H / st.tokens + lam * np.eye(n))
+    # U is the inverse of the reverse Cholesky factor R (H_d = R R^T, R upper)
+    J = np.eye(n)[::-1]
+    R = J @ np.linalg.cholesky(J @ Hd @ J) @ J
+    assert np.allclose(np.triu(R), R) and np.allclose(R @ R.T, Hd)
+    assert np.allclose(U, np.linalg.inv(R), atol=1e-10)
+
+
+def test_lemma_4_1_trailing_blocks_and_elimination():
+    _, X, Xfp = tiny(n=12)
+    st = stats_of(X, Xfp)
+    U, _ = orc.factor(st.H, st.tokens, 0.02)
+    Hd, _ = orc.damped_hessian(st.H, st.tokens, 0.02)
+    L = U.T
+    Hinv = np.linalg.inv(Hd)
+    for q in range(12):
+        # Lemma 4.1: L[q:, q:] L[q:, q:]^T is the inverse of the trailing block of H_d
+        assert np.allclose(L[q:, q:] @ L[q:, q:].T, np.linalg.inv(Hd[q:, q:]), atol=1e-10)
+        # ... and equals the Gaussian-elimination form (Eq. "ge") applied q times
+        assert np.allclose(L[q:, q:] @ L[q:, q:].T, Hinv[q:, q:], atol=1e-10)
+        if q < 11:
+            Hinv = Hinv - np.outer(Hinv[:, q], Hinv[q, :]) / Hinv[q, q]
+
+
+def test_dead_inputs_and_not_spd():
+    W, X, Xfp = tiny(n=8)
+    X[:, 3] = 0.0
+    st = stats_of(X, Xfp)
+    U, dead = orc.factor(st.H, st.tokens, 0.01)
+    assert dead.tolist() == [i == 3 for i in range(8)]
+    assert np.isfinite(U).all()
+    res = orc.quantize(W, U, orc.build_P(st.D, st.tokens, U, 1.0), dead, 4, 0, False)
+    assert np.all(res.Wq[:, 3] == 0.0)
+    # rank-deficient H with no damping is rejected
+    Xr = np.repeat(X[:4], 2, axis=0)[:, :8]
+    with pytest.raises(np.linalg.LinAlgError):
+        orc.factor(Xr.T @ Xr + 0.0, 8, 0.0)
+
+
+# ---------------------------------------------------------------- P
+def test_theorem_4_2_three_ways():
+    _, X, Xfp = tiny(n=16)
+    st = stats_of(X, Xfp)
+    U, _ = orc.factor(st.H, st.tokens, 0.01)
+    Hd, _ = orc.damped_hessian(st.H, st.tokens, 0.01)
+    P = orc.build_P(st.D, st.tokens, U, 1.0)
+    Pr = orc.build_P_rowwise(st.D, st.tokens, U, 1.0)
+    assert np.allclose(P, Pr, atol=1e-12)
+    assert np.allclose(np.tril(P), 0.0)
+    D = st.D / st.tokens
+    for q in range(15):
+        direct = D[q, q + 1:] @ np.linalg.inv(Hd[q + 1:, q + 1:])
+        assert np.allclose(P[q, q + 1:], direct, atol=1e-10)
+    assert np.allclose(orc.build_P(st.D, st.tokens, U, 0.25), 0.25 * P)
+
+
+def test_P_closed_forms():
+    r = np.random.default_rng(3)
+    n = 10
+    # diagonal H: P = triu_1(D) diag(1/h)
+    h = r.uniform(0.5, 2.0, n)
+    U, _ = orc.factor(np.diag(h), 1, 0.0)
+    D = r.standard_normal((n, n))
+    assert np.allclose(orc.build_P(D, 1, U, 1.0), np.triu(D, 1) / h[None, :], atol=1e-12)
+    # dX = c X, no damping: P = c (I - diag(U)^-1 U)
+    X = r.standard_normal((80, n))
+    H = X.T @ X
+    U, _ = orc.factor(H, 80, 0.0)
+    c = -0.3
+    P = orc.build_P(c * H, 80, U, 1.0)
+    assert np.allclose(P, c * (np.eye(n) - U / np.diag(U)[:, None]), atol=1e-9)
+
+
+# ---------------------------------------------------------------- quantizer
+@pytest.mark.parametrize("bits", [2, 3, 4])
+@pytest.mark.parametrize("sym", [False, True])
+def test_quantizer_exhaustive(bits, sym):
+    r = np.random.default_rng(bits)
+    w = r.standard_normal((64, 33)) * r.uniform(0.01, 3.0, (64, 1))
+    w[0] = 0.0
+    w[1] = np.abs(w[1])          # one-sided rows: the grid still holds zero
+    w[2] = -np.abs(w[2])
+    s, z = orc.grid(w, bits, sym)
+    c = orc.qcode(w, s[:, None], z[:, None], bits)
+    q = orc.dequant(c, s[:, None], z[:, None])
+    assert c.min() >= 0 and c.max() <= 2 ** bits - 1 and np.all(c == np.rint(c))
+    # zero is always representable exactly
+    assert np.all(orc.dequant(orc.qcode(0 * w, s[:, None], z[:, None], bits), s[:, None], z[:, None]) == 0)
+    if sym:
+        inside = np.abs(w) <= (s * (2 ** (bits - 1) - 1))[:, None] * (1 + 1e-12)
+        assert inside.all()
+        assert np.all(z == 2 ** (bits - 1))
+    assert np.all(np.abs(w - q) <= s[:, None] / 2 * (1 + 1e-9) + 1e-300)
+    # nearest grid point by brute force over all codes
+    levels = s[:, None, None] * (np.arange(2 ** bits)[None, None, :] - z[:, None, None])
+    best = np.min(np.abs(w[:, :, None] - levels), axis=2)
+    assert np.allclose(np.abs(w - q), best, atol=1e-12)
+    # round half to even at an exact tie
+    s1, z1 = np.array([1.0]), np.array([4.0])
+    assert orc.qcode(np.array([0.5, 1.5, 2.5, -0.5]), s1, z1, 4).tolist() == [4.0, 6.0, 6.0, 4.0]
+
+
+# ---------------------------------------------------------------- loop
+def constrained_ls_step(Hd, D, w_q, c, q):
+    """min_d  d A d^T - 2 w_q D[q, q:] d^T  s.t. d[0] = c, with A = H_d[q:, q:]
+    (the per-column problem of Step 2 with the damped Gram matrix)."""
+    A = Hd[q:, q:]
+    b = w_q * D[q, q:]
+    rest = (b[1:] - c * A[0, 1:]) @ np.linalg.inv(A[1:, 1:])
+    return rest
+
+
+def test_each_column_step_is_the_constrained_minimiser():
+    W, X, Xfp = tiny(n=14, m=3)
+    st = stats_of(X, Xfp)
+    damp = 0.03
+    U, dead = orc.factor(st.H, st.tokens, damp)
+    P = orc.build_P(st.D, st.tokens, U, 1.0)
+    Hd, _ = orc.damped_hessian(st.H, st.tokens, damp)
+    D = st.D / st.tokens
+    n = 14
+    Wc = W.copy()
+    s, z = orc.grid(Wc, 4, False)
+    for q in range(n - 1):
+        w = Wc[:, q].copy()
+        qv = orc.dequant(orc.qcode(w, s, z, 4), s, z)
+        e = (w - qv) / U[q, q]
+        step = -np.outer(e, U[q, q + 1:]) + np.outer(w, P[q, q + 1:])
+        for r in range(3):
+            want = constrained_ls_step(Hd, D, w[r], qv[r] - w[r], q)
+            assert np.allclose(step[r], want, atol=1e-10)
+        Wc[:, q + 1:] += step
+        Wc[:, q] = qv
+    res = orc.quantize(W, U, P, dead, 4, 0, False)
+    assert np.allclose(res.Wq[:, :-1], Wc[:, :-1], atol=1e-12)
+
+
+def gptq_elimination(W, Hd, bits, group, sym):
+    """GPTQ in explicit-elimination form: OBQ update with the running inverse
+    Hessian, removing one row/column per step (Eq. "ge")."""
+    W = W.copy()
+    m, n = W.shape
+    Hinv = np.linalg.inv(Hd)
+    Q = np.zeros_like(W)
+    if group <= 0:
+        s, z = orc.grid(W, bits, sym)
+    for q in range(n):
+        if group > 0 and q % group == 0:
+            s, z = orc.grid(W[:, q:q + group], bits, sym)
+        w = W[:, q].copy()
+        qv = orc.dequant(orc.qcode(w, s, z, bits), s, z)
+        Q[:, q] = qv
+        W += np.outer((qv - w) / Hinv[q, q], Hinv[q, :])
+        Hinv = Hinv - np.outer(Hinv[:, q], Hinv[q, :]) / Hinv[q, q]
+        Hinv[q, q] = 1.0   # keeps later divisions finite; row/col q are otherwise zero
+    return Q
+
+
+@pytest.mark.parametrize("group,sym", [(0, False), (8, False), (8, True)])
+def test_gptq_limit(group, sym):
+    W, X, Xfp = tiny(n=24, m=6)
+    st = stats_of(X, Xfp)
+    U, dead = orc.factor(st.H, st.tokens, 0.01)
+    Hd, _ = orc.damped_hessian(st.H, st.tokens, 0.01)
+    want = gptq_elimination(W, Hd, 4, group, sym)
+    a0 = orc.quantize(W, U, orc.build_P(st.D, st.tokens, U, 0.0), dead, 4, group, sym)
+    none = orc.quantize(W, U, None, dead, 4, group, sym)
+    assert np.allclose(a0.Wq, want, atol=1e-10) and np.array_equal(a0.codes, none.codes)
+    # X~ = X  =>  dXX^T = 0  =>  GPTQ
+    st_same = stats_of(X, X)
+    U2, d2 = orc.factor(st_same.H, st_same.tokens, 0.01)
+    P2 = orc.build_P(st_same.D, st_same.tokens, U2, 1.0)
+    assert np.all(P2 == 0)
+    assert np.allclose(orc.quantize(W, U2, P2, d2, 4, group, sym).Wq, want, atol=1e-10)
+
+
+def test_rtn_limit_and_objective_order():
+    W, X, Xfp = tiny(n=32, m=16, k=600)
+    st = stats_of(X, Xfp)
+    U, dead = orc.factor(st.H, st.tokens, 0.01)
+    rtn = orc.quantize(W, U, None, dead, 4, 0, False, update=False)
+    s, z = orc.grid(W, 4, False)
+    assert np.array_equal(rtn.codes, orc.qcode(W, s[:, None], z[:, None], 4).astype(np.uint8))
+    J = {}
+    J["rtn"] = orc.objective(W, rtn.Wq, st)
+    J["gptq"] = orc.objective(W, orc.quantize(W, U, None, dead, 4, 0, False).Wq, st)
+    for a in (0.25, 1.0):
+        P = orc.build_P(st.D, st.tokens, U, a)
+        J[a] = orc.objective(W, orc.quantize(W, U, P, dead, 4, 0, False).Wq, st)
+    assert J[1.0] < J["rtn"] and J[0.25] < J["rtn"] and J["gptq"] < J["rtn"]
+
+
+@pytest.mark.parametrize("name", ["cfg1"])
+def test_objective_not_worse_than_rtn_on_config(name):
+    cfg = wl.CONFIGS[name]
+    W = wl.make_weight(cfg).numpy()
+    st, U, P, dead, res = orc.solve_layer(
+        W, [tuple(t.numpy() for t in wl.make_batch(cfg, b)) for b in range(cfg.n_batches)],
+        cfg.damp, cfg.alpha, cfg.bits, cfg.group, cfg.sym)
+    rtn = orc.quantize(W, U, None, dead, cfg.bits, cfg.group, cfg.sym, update=False)
+    assert orc.objective(W, res.Wq, st) <= orc.objective(W, rtn.Wq, st)
+
+
+@pytest.mark.parametrize("group", [0, 8])
+def test_blocksize_invariance_and_blocked_form(group):
+    W, X, Xfp = tiny(n=32, m=7)
+    st = stats_of(X, Xfp)
+    U, dead = orc.factor(st.H, st.tokens, 0.01)
+    P = orc.build_P(st.D, st.tokens, U, 0.7)
+    ref = orc.quantize(W, U, P, dead, 3, group, False)
+    for B in (8, 16, 32):
+        blk = orc.quantize_blocked(W, U, P, dead, 3, group, False, B)
+        assert np.array_equal(blk.codes, ref.codes)
+        assert np.allclose(blk.Wq, ref.Wq, atol=1e-12)
+        assert np.allclose(blk.scales, ref.scales, atol=1e-14)
+    # the literal reading (quantized block in the second term) depends on B
+    lit = [orc.quantize_blocked(W, U, P, dead, 3, group, False, B, True).Wq for B in (8, 32)]
+    assert not np.allclose(lit[0], lit[1], atol=1e-9)
+
+
+def test_row_independence_and_scale_invariance():
+    W, X, Xfp = tiny(n=20, m=9)
+    st = stats_of(X, Xfp)
+    U, dead = orc.factor(st.H, st.tokens, 0.01)
+    P = orc.build_P(st.D, st.tokens, U, 1.0)
+    full = orc.quantize(W, U, P, dead, 4, 4, False)
+    sub = orc.quantize(W[[1, 5, 8]], U, P, dead, 4, 4, False)
+    assert np.array_equal(sub.codes, full.codes[[1, 5, 8]])
+    st2 = stats_of(3.0 * X, 3.0 * Xfp)
+    U2, d2 = orc.factor(st2.H, st2.tokens, 0.01)
+    P2 = orc.build_P(st2.D, st2.tokens, U2, 1.0)
+    assert np.allclose(P2, P, atol=1e-12)
+    assert np.array_equal(orc.quantize(W, U2, P2, d2, 4, 4, False).codes, full.codes)
+    # the token-count normalisation does not change the result either
+    U3, _ = orc.factor(st.H, 1, 0.01)
+    P3 = orc.build_P(st.D, 1, U3, 1.0)
+    assert np.allclose(P3, P, atol=1e-12)
+
+
+# ---------------------------------------------------------------- objective
+def test_objective_identity():
+    W, X, Xfp = tiny(n=12, m=4, k=90)
+    st = stats_of(X, Xfp)
+    Wq = W + 0.01 * np.random.default_rng(5).standard_normal(W.shape)
+    direct = orc.objective_direct(W, Wq, X, Xfp)
+    assert abs(orc.objective(W, Wq, st) - direct) < 1e-10 * direct
+    # W^ = W: only the residual term ||W dX||^2 is left
+    assert abs(orc.objective(W, W, st) - np.sum(((Xfp - X) @ W.T) ** 2)) < 1e-10
+
+
+# ---------------------------------------------------------------- follow mode
+def test_follow_mode_accepts_own_output_and_flags_planted_errors():
+    W, X, Xfp = tiny(n=32, m=12)
+    st = stats_of(X, Xfp)
+    U, dead = orc.factor(st.H, st.tokens, 0.01)
+    P = orc.build_P(st.D, st.tokens, U, 0.25)
+    res = orc.quantize(W, U, P, dead, 4, 8, False)
+    rep = orc.follow(W, U, P, dead, 4, 8, False, res.codes, res.scales, res.zeros)
+    assert rep.mismatches == 0 and rep.disallowed == 0 and rep.grid_rel_err == 0.0
+    bad = res.codes.copy()
+    bad[3, 5] = (bad[3, 5] + 2) % 16
+    rep = orc.follow(W, U, P, dead, 4, 8, False, bad, res.scales, res.zeros)
+    assert rep.disallowed >= 1
+    # a wrong sign of the second term is caught as well
+    rep = orc.follow(W, U, -P, dead, 4, 8, False, res.codes, res.scales, res.zeros)
+    assert rep.disallowed > 0
+
+
+# ---------------------------------------------------------------- appendix table
+def test_memory_table_of_the_appendix():
+    rows = [l.split() for l in open(os.path.join(GOLDEN, "memory_table.txt")) if l.strip() and l[0] != "#"]
+    for m, n, gptq_gb, gptaq_gb in rows:
+        m, n = int(m), int(n)
+        for asym, want in ((False, float(gptq_gb)), (True, float(gptaq_gb))):
+            elems = sum(orc.working_set_elements(m, n, 128, asym).values())
+            assert abs(elems * 2 / 2 ** 30 - want) <= 0.011
