@@ -1,0 +1,327 @@
+#!/usr/bin/env python
+"""Benchmark of the GPTAQ per-layer solve on B200.
+
+One step = one pass of the whole hot path over one synthetic layer:
+reset -> accumulate (all token batches) -> factor -> build_P -> quantize.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload cfg2]
+    python bench.py --impl reference ...     # the float64 CPU oracle, bounded sample
+
+Prints ONE JSON line (rank 0).  With N > 1 (launched by torchrun) every rank
+solves its own independent layer of the same shape (layers are independent
+problems; no data-path collective), and the value is the time per layer of
+the whole job.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+import torch
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+import workloads as wl  # noqa: E402
+
+METRIC = "ms per layer (GPTAQ solve: accumulate + factor + P + quantize)"
+
+
+def peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        d = json.load(open(p))
+        return {"hbm_gbs": d["hbm_gbs"], "bf16_burst": d["bf16_tflops"],
+                "bf16_sustained": d.get("bf16_tflops_sustained", d["bf16_tflops"]), "source": "measured"}
+    return {"hbm_gbs": 6650.0, "bf16_burst": 1590.0, "bf16_sustained": 1400.0, "source": "fallback"}
+
+
+class ClockSampler:
+    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+    Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+         "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+         "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index, self.rows, self.stop, self.th = index, [], threading.Event(), None
+
+    def _run(self):
+        while not self.stop.is_set():
+            try:
+                out = subprocess.run(["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits",
+                                      "-i", str(self.index)], capture_output=True, text=True, timeout=5).stdout
+                self.rows.append([c.strip() for c in out.strip().split(",")])
+            except Exception:
+                pass
+            self.stop.wait(0.2)
+
+    def __enter__(self):
+        self.th = threading.Thread(target=self._run, daemon=True)
+        self.th.start()
+        return self
+
+    def __exit__(self, *a):
+        self.stop.set()
+        self.th.join(timeout=6)
+
+    def summary(self):
+        sm, mx, reasons = [], [], set()
+        for r in self.rows:
+            if len(r) < 8:
+                continue
+            try:
+                sm.append(float(r[0])); mx.append(float(r[1]))
+            except ValueError:
+                continue
+            for name, v in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), r[4:8]):
+                if v.lower().startswith("active"):
+                    reasons.add(name)
+        if not sm:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        sm.sort()
+        return {"sm_mhz": sm[len(sm) // 2], "sm_max_mhz": max(mx), "reasons": sorted(reasons), "samples": len(sm)}
+
+
+# --------------------------------------------------------------------------- CPU oracle leg
+def oracle_sample(cfg: wl.LayerConfig, sample_tokens: int, sample_rows: int):
+    """Times the float64 oracle, as it stands, on a bounded sample of the
+    workload and scales linearly to the whole layer (statistics are linear in
+    tokens, rows of W are independent).  Returns (ms per layer, description)."""
+    from oracle import gptaq_oracle as orc
+    threads = torch.get_num_threads()
+    sample_tokens = min(sample_tokens, cfg.batch_tokens)
+    sample_rows = min(sample_rows, cfg.m)
+    X, Xfp = (t.numpy() for t in wl.make_batch(cfg, 0, "cpu", sample_tokens))
+    W = wl.make_weight(cfg, "cpu", rows=sample_rows).numpy()
+    st = orc.new_stats(cfg.n)
+    t0 = time.perf_counter()
+    orc.accumulate(st, X, Xfp)
+    t_acc = time.perf_counter() - t0
+    t0 = time.perf_counter()
+    U, dead = orc.factor(st.H, st.tokens, max(cfg.damp, 0.05))   # few tokens: keep the sample SPD
+    t_fac = time.perf_counter() - t0
+    t0 = time.perf_counter()
+    P = orc.build_P(st.D, st.tokens, U, cfg.alpha)
+    t_p = time.perf_counter() - t0
+    t0 = time.perf_counter()
+    orc.quantize(W, U, P, dead, cfg.bits, cfg.group, cfg.sym)
+    t_q = time.perf_counter() - t0
+    total = t_acc * (cfg.tokens / sample_tokens) + t_fac + t_p + t_q * (cfg.m / sample_rows)
+    desc = (f"accumulate on {sample_tokens} of {cfg.tokens} tokens ({t_acc:.2f} s, scaled by tokens); "
+            f"factor ({t_fac:.2f} s) and P ({t_p:.2f} s) in full; column loop on {sample_rows} of {cfg.m} rows "
+            f"({t_q:.2f} s, scaled by rows)")
+    return total * 1e3, desc, threads
+
+
+def run_reference(args, cfg):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    times = []
+    desc, threads = "", 0
+    for i in range(args.warmup + args.steps):
+        ms, desc, threads = oracle_sample(cfg, args.ref_tokens, args.ref_rows)
+        if i >= args.warmup:
+            times.append(ms)
+    v = sum(times) / len(times)
+    line = {
+        "impl": "reference", "metric": METRIC, "value": v, "unit": "ms", "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": v, "higher_is_better": False,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": dict(wl.describe(cfg), parallelism="cpu oracle, rank 0 only"),
+        "cpu_baseline": {"value": v, "unit": "ms", "cores": threads, "kind": "oracle", "sample": desc},
+        "e2e": {"value": v, "unit": "ms", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line), flush=True)
+
+
+# --------------------------------------------------------------------------- CUDA leg
+def run_ours(args, cfg):
+    import paper_2504_02692_b200 as g
+    from paper_2504_02692_b200 import build as gbuild
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=dev)
+    if rank == 0:
+        gbuild.build()
+    if world > 1:
+        dist.barrier()
+    g.load_library()
+    pk = peaks()
+
+    # inputs resident in HBM before the timed region (each rank its own layer: seed = rank)
+    cfg_r = wl.scaled(cfg, seed=cfg.seed + rank)
+    batches = [wl.make_batch(cfg_r, b, dev) for b in range(cfg.n_batches)]
+    W0 = wl.make_weight(cfg_r, dev)
+    if cfg.w_bf16:
+        W0 = W0.to(torch.bfloat16)
+    G = 1 if cfg.group <= 0 else (cfg.n + cfg.group - 1) // cfg.group
+    codes = torch.empty((cfg.m, cfg.n), dtype=torch.uint8, device=dev)
+    scales = torch.empty((cfg.m, G), dtype=torch.float32, device=dev)
+    zeros = torch.empty((cfg.m, G), dtype=torch.float32, device=dev)
+    Wq = torch.empty((cfg.m, cfg.n), dtype=torch.float32, device=dev)
+    st = g.LayerState(cfg.n, cfg.m, cfg.batch_tokens, cfg.blocksize, dev)
+    h = st.handle
+    stream = torch.cuda.current_stream()
+
+    def ev():
+        return torch.cuda.Event(enable_timing=True)
+
+    def step(marks=None):
+        g.gptaq_reset(h)
+        acc_ev = []
+        for X, Xfp in batches:
+            if marks is not None:
+                a, b = ev(), ev()
+                a.record(stream)
+            g.gptaq_accumulate(h, X, Xfp)
+            if marks is not None:
+                b.record(stream)
+                acc_ev.append((a, b))
+        e1 = ev(); e1.record(stream)
+        g.gptaq_factor(h, cfg.damp)
+        e2 = ev(); e2.record(stream)
+        g.gptaq_build_P(h, cfg.alpha)
+        e3 = ev(); e3.record(stream)
+        g.gptaq_quantize(h, W0, cfg.bits, cfg.group, cfg.sym, cfg.blocksize, codes, scales, zeros, Wq)
+        e4 = ev(); e4.record(stream)
+        if marks is not None:
+            marks.append((acc_ev, e1, e2, e3, e4))
+
+    def sync_all():
+        torch.cuda.synchronize()
+        if world > 1:
+            dist.barrier()
+            torch.cuda.synchronize()
+
+    for _ in range(args.warmup):
+        step()
+    status = g.gptaq_sync_status(h)
+    if status[0] != g.GPTAQ_OK:
+        raise RuntimeError(f"device status {status}")
+
+    marks = []
+    sync_all()
+    l0 = g.gptaq_launch_count(h)
+    t_beg, t_end = ev(), ev()
+    with ClockSampler(local) as clk:
+        t_beg.record(stream)
+        for _ in range(args.steps):
+            step(marks)
+        t_end.record(stream)
+        sync_all()
+    launches = g.gptaq_launch_count(h) - l0
+    ms_total = t_beg.elapsed_time(t_end)
+    if world > 1:
+        t = torch.tensor([ms_total], device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms_total = float(t.item())
+    ms_step = ms_total / args.steps
+    ms_layer = ms_step / world           # `world` independent layers per step
+
+    acc_ms = [a.elapsed_time(b) for m in marks for (a, b) in m[0]]
+    acc_call_ms = sum(acc_ms) / len(acc_ms)
+    acc_step_ms = sum(acc_ms) / args.steps
+    fac_ms = sum(m[1].elapsed_time(m[2]) for m in marks) / args.steps
+    p_ms = sum(m[2].elapsed_time(m[3]) for m in marks) / args.steps
+    q_ms = sum(m[3].elapsed_time(m[4]) for m in marks) / args.steps
+    flops_call = 3.0 * cfg.n * cfg.n * cfg.batch_tokens
+    achieved = flops_call / (acc_call_ms * 1e-3) / 1e12
+    peak = pk["bf16_sustained"]
+
+    # end to end through the host entry points: pinned host buffers in, host results out
+    e2e = None
+    if not args.no_e2e:
+        hb = [(X.cpu().pin_memory(), Xfp.cpu().pin_memory()) for X, Xfp in batches]
+        hW = (W0.float() if cfg.w_bf16 else W0).cpu().pin_memory()
+        hcodes = torch.empty((cfg.m, cfg.n), dtype=torch.uint8).pin_memory()
+        hs = torch.empty((cfg.m, G), dtype=torch.float32).pin_memory()
+        hz = torch.empty((cfg.m, G), dtype=torch.float32).pin_memory()
+        stage = torch.empty(max(2 * cfg.batch_tokens * cfg.n * 4, g.gptaq_quantize_stage_bytes(cfg.m, cfg.n, cfg.group)),
+                            dtype=torch.uint8, device=dev)
+
+        def step_host():
+            g.gptaq_reset(h)
+            for X, Xfp in hb:
+                g.gptaq_accumulate_host(h, X, Xfp, stage)
+            g.gptaq_factor(h, cfg.damp)
+            g.gptaq_build_P(h, cfg.alpha)
+            g.gptaq_quantize_host(h, hW, cfg.bits, cfg.group, cfg.sym, cfg.blocksize, hcodes, hs, hz, stage)
+
+        step_host()
+        sync_all()
+        a, b = ev(), ev()
+        a.record(stream)
+        ke = max(1, min(args.steps, 3))
+        for _ in range(ke):
+            step_host()
+        b.record(stream)
+        sync_all()
+        ems = a.elapsed_time(b) / ke
+        if world > 1:
+            t = torch.tensor([ems], device=dev)
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            ems = float(t.item())
+        h2d = sum(x.numel() * 4 * 2 for x, _ in hb) + hW.numel() * 4
+        d2h = hcodes.numel() + (hs.numel() + hz.numel()) * 4
+        e2e = {"value": ems / world, "unit": "ms", "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h}
+
+    if rank != 0:
+        return
+    cpu = None
+    if world == 1 and not args.no_cpu_baseline:
+        v, desc, threads = oracle_sample(cfg, args.ref_tokens, args.ref_rows)
+        cpu = {"value": v, "unit": "ms", "cores": threads, "kind": "oracle", "sample": desc}
+    line = {
+        "metric": METRIC, "value": ms_layer, "unit": "ms", "n_gpus": world, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": False, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+        "config": dict(wl.describe(cfg), parallelism=f"{world} independent layer(s), one per GPU",
+                       l2="inputs (%.1f GB per step) exceed L2" % (2 * cfg.tokens * cfg.n * 4 / 1e9)),
+        "stages_ms": {"accumulate": acc_step_ms, "factor": fac_ms, "build_P": p_ms, "quantize": q_ms,
+                      "layer_quantize": fac_ms + p_ms + q_ms},
+        "accumulate_tflops": achieved,
+        "roofline": {"kernel": "gptaq_accumulate (one token batch)", "bound": "tensor", "achieved": achieved,
+                     "peak": peak, "unit": "TFLOP/s", "frac": achieved / peak, "traffic": None,
+                     "peak_source": pk["source"] + " bf16 cuBLAS, sustained",
+                     "algorithmic_flops_per_launch": flops_call},
+        "cpu_baseline": cpu, "e2e": e2e, "gpu_launches": launches, "clocks": clk.summary(),
+    }
+    print(json.dumps(line), flush=True)
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=5)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="cfg2", choices=sorted(wl.CONFIGS))
+    ap.add_argument("--ref-tokens", type=int, default=1024)
+    ap.add_argument("--ref-rows", type=int, default=32)
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    cfg = wl.CONFIGS[args.workload]
+    if args.impl == "reference":
+        run_reference(args, cfg)
+    else:
+        if not torch.cuda.is_available():
+            raise SystemExit("bench.py needs a CUDA device (there is no CPU fallback); "
+                             "use --impl reference for the CPU oracle")
+        run_ours(args, cfg)
+
+
+if __name__ == "__main__":
+    main()

@@ -1,0 +1,166 @@
+/*
+ * gptaq.h -- C ABI of the B200 (sm_100a) GPTAQ per-layer solve.
+ *
+ * GPTAQ quantizes one linear layer W (m x n, rows = output channels) so that
+ * the quantized layer fed with the quantized model's input X reproduces the
+ * full-precision layer fed with the full-precision input X~ (the paper's
+ * asymmetric calibration objective, Eq. "asym obj", Section 4).  The calls
+ * follow Algorithm 1 of the paper line by line:
+ *
+ *   gptaq_accumulate   line 2   H += X X^T,  dXX^T += (X~ - X) X^T
+ *   gptaq_factor       line 3   L = Inverse_Cholesky(H + lambda_1 I), kept as U = L^T
+ *   gptaq_build_P      line 4   P = ((dXX^T L) .* M_U) L^T          (Theorem 4.2)
+ *   gptaq_quantize     l. 5-13  blocked column loop + lazy-batch trailing update
+ *
+ * Conventions
+ *  - Every pointer named d_* is DEVICE memory, every pointer named h_* is
+ *    HOST memory.  All device memory is allocated and owned by the caller;
+ *    the library allocates no device memory.  The handle itself is a small
+ *    host object owned by the library between gptaq_create / gptaq_destroy.
+ *  - Matrices are row-major float32 unless stated.  Activations are
+ *    token-major: X is passed as X^T, [tokens x n] with leading dimension ld.
+ *  - `stream` is a cudaStream_t passed as void* (NULL = the default stream).
+ *    Calls only enqueue work and return; host-side argument and call-order
+ *    errors are returned at once, conditions found on the device (a
+ *    non-positive pivot, a non-finite value, a bounded wait that ran out) are
+ *    recorded in a device status word that gptaq_sync_status() reads.  Nothing
+ *    traps or asserts on the device.
+ *  - Call order: create -> accumulate* -> factor -> build_P -> quantize*.
+ *    Anything else returns GPTAQ_ERR_BAD_STATE.  gptaq_reset() returns a
+ *    handle to the state right after create.  quantize may be called many
+ *    times on one state (layers that share an input share H, U and P).
+ *  - A handle is not thread-safe; distinct handles are independent.
+ */
+#ifndef GPTAQ_H_
+#define GPTAQ_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct gptaq_ctx *gptaq_handle_t;
+typedef void *gptaq_stream_t; /* a cudaStream_t */
+
+typedef enum {
+    GPTAQ_OK = 0,
+    GPTAQ_ERR_INVALID_ARG = 1,  /* null pointer, negative size, misaligned buffer */
+    GPTAQ_ERR_BAD_STATE = 2,    /* call out of order */
+    GPTAQ_ERR_WORKSPACE = 3,    /* state / workspace / staging buffer too small */
+    GPTAQ_ERR_NOT_SPD = 4,      /* device: a pivot of the damped H was <= 0; info = its index */
+    GPTAQ_ERR_NONFINITE = 5,    /* device: NaN/Inf met in H or W; info = row or column index */
+    GPTAQ_ERR_TIMEOUT = 6,      /* device: a bounded wait ran out; info = where */
+    GPTAQ_ERR_UNSUPPORTED = 7,  /* argument combination outside the supported set */
+    GPTAQ_ERR_CUDA = 8          /* a CUDA runtime call failed; see gptaq_last_cuda_error */
+} gptaq_status_t;
+
+enum { GPTAQ_W_FP32 = 0, GPTAQ_W_BF16 = 1 };
+
+/* Bytes of the caller-owned device state for layer width n: a header (status
+ * word, pivot index), H (n x n), dXX^T (n x n) and the dead-input flags.
+ * After gptaq_factor, U overwrites H; after gptaq_build_P, P overwrites dXX^T. */
+size_t gptaq_state_bytes(int64_t n);
+
+/* Bytes of caller-owned device scratch that factor / build_P / quantize need
+ * for width n, at most m_max weight rows and the given lazy-batch block size
+ * (Algorithm 1, input B).  max_batch_tokens is the largest `tokens` that
+ * gptaq_accumulate will be given. */
+size_t gptaq_workspace_bytes(int64_t n, int64_t m_max, int64_t max_batch_tokens, int blocksize);
+
+/* Creates a handle over caller-owned device buffers (both 256-byte aligned)
+ * on the current CUDA device and enqueues the zeroing of H and dXX^T
+ * (Algorithm 1, line 2 starts from empty sums). */
+gptaq_status_t gptaq_create(gptaq_handle_t *out, int64_t n, void *d_state, size_t state_bytes,
+                            void *d_workspace, size_t workspace_bytes, gptaq_stream_t stream);
+
+/* Back to the state right after gptaq_create (sums zeroed, token count 0). */
+gptaq_status_t gptaq_reset(gptaq_handle_t h, gptaq_stream_t stream);
+
+gptaq_status_t gptaq_destroy(gptaq_handle_t h);
+
+/* Algorithm 1, line 2, one token batch:  H += X X^T,  dXX^T += (X~ - X) X^T.
+ * d_X, d_Xfp: [tokens x n] float32, leading dimension ld >= n, read only.
+ * The difference X~ - X is formed in float32 before any product.
+ * tokens == 0 is a no-op.  Only the upper triangle of H is maintained. */
+gptaq_status_t gptaq_accumulate(gptaq_handle_t h, const float *d_X, const float *d_Xfp,
+                                int64_t tokens, int64_t ld, gptaq_stream_t stream);
+
+/* Same with HOST inputs (pinned memory for asynchronous copies): copies the
+ * batch into d_stage (device, >= 2 * tokens * n * 4 bytes) on `stream`, then
+ * accumulates from there. */
+gptaq_status_t gptaq_accumulate_host(gptaq_handle_t h, const float *h_X, const float *h_Xfp,
+                                     int64_t tokens, int64_t ld, void *d_stage, size_t stage_bytes,
+                                     gptaq_stream_t stream);
+
+/* Algorithm 1, line 3 with the "standard GPTQ procedure" of Section 4:
+ * H <- H / tokens; inputs with H_qq == 0 get H_qq = 1 (their weight columns
+ * are zeroed by gptaq_quantize); H_d = H + damp * mean(diag H) * I; then the
+ * upper factor U of H_d^-1 = U^T U (U = L^T of the paper) overwrites H
+ * (strict lower triangle zeroed).  Needs at least one accumulated token. */
+gptaq_status_t gptaq_factor(gptaq_handle_t h, float damp, gptaq_stream_t stream);
+
+/* Algorithm 1, line 4 / Theorem 4.2:  P = alpha * ((dXX^T U^T) .* M_U) U with
+ * dXX^T normalised by the token count like H, M_U the strictly-upper mask.
+ * alpha = 1 is the paper's P; alpha = 0 reduces the solve to GPTQ.
+ * P overwrites dXX^T (lower triangle and diagonal zero). */
+gptaq_status_t gptaq_build_P(gptaq_handle_t h, float alpha, gptaq_stream_t stream);
+
+/* Algorithm 1, lines 5-13, for one weight matrix sharing this state.
+ *   d_W      [m x ldw], float32 or bf16 (w_dtype); consumed: float32 weights are
+ *            updated in place and hold the dequantized result on return
+ *            (column j becomes Q[:, j] at step j); bf16 weights are read only
+ *            and the float32 working copy lives in d_Wq, which is then required.
+ *   bits     2..8;  group: 0 = one grid per output channel taken from the
+ *            original row, else a grid per `group` consecutive columns taken
+ *            from the current (already updated) weights at the group's first
+ *            column; requires blocksize % group == 0.
+ *   sym      0: asymmetric min/max grid containing zero, zero point = rint(-lo/scale);
+ *            1: symmetric grid, scale = max|w| / (2^(bits-1) - 1), stored code
+ *            = s + 2^(bits-1).  Rounding is round-half-to-even.
+ *   blocksize  lazy-batch block B in {32, 64, 128}.
+ *   d_codes  [m x n] uint8 out;  d_scales, d_zeros [m x G] float32 out,
+ *            G = 1 (group == 0) or ceil(n / group).
+ *   d_Wq     [m x n] float32 out, dequantized weights (ld n); may be NULL for
+ *            float32 weights.
+ * m == 0 is a no-op. */
+gptaq_status_t gptaq_quantize(gptaq_handle_t h, void *d_W, int w_dtype, int64_t m, int64_t ldw,
+                              int bits, int group, int sym, int blocksize,
+                              uint8_t *d_codes, float *d_scales, float *d_zeros, float *d_Wq,
+                              gptaq_stream_t stream);
+
+/* Same with HOST weights in and HOST codes / scales / zeros out: copies W into
+ * d_stage (device, >= gptaq_quantize_stage_bytes(m, n, group)), quantizes there and copies
+ * the three results back; all on `stream`, asynchronous if the host memory is
+ * pinned.  h_Wq (dequantized float32, [m x n]) may be NULL. */
+size_t gptaq_quantize_stage_bytes(int64_t m, int64_t n, int group);
+gptaq_status_t gptaq_quantize_host(gptaq_handle_t h, const float *h_W, int64_t m, int64_t ldw,
+                                   int bits, int group, int sym, int blocksize,
+                                   uint8_t *h_codes, float *h_scales, float *h_zeros, float *h_Wq,
+                                   void *d_stage, size_t stage_bytes, gptaq_stream_t stream);
+
+/* Synchronises `stream`, then returns the device status word (GPTAQ_OK, or the
+ * first device-side condition recorded since create/reset) and, in *info, the
+ * index that goes with it (may be NULL). */
+gptaq_status_t gptaq_sync_status(gptaq_handle_t h, int64_t *info, gptaq_stream_t stream);
+
+/* Device views into the state (n x n, leading dimension n), for tests and for
+ * callers that checkpoint the sums: H / U and dXX^T / P share storage. */
+float *gptaq_H(gptaq_handle_t h);
+float *gptaq_D(gptaq_handle_t h);
+int64_t gptaq_tokens(gptaq_handle_t h);
+/* Sets the token count (for callers that restore checkpointed sums). */
+gptaq_status_t gptaq_set_tokens(gptaq_handle_t h, int64_t tokens);
+
+/* Number of kernels this handle has launched since create (bookkeeping for benchmarks). */
+int64_t gptaq_launch_count(gptaq_handle_t h);
+
+const char *gptaq_status_string(gptaq_status_t s);
+/* Text of the last CUDA runtime error seen by this handle ("" if none). */
+const char *gptaq_last_cuda_error(gptaq_handle_t h);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* GPTAQ_H_ */

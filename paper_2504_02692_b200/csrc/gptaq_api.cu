@@ -1,0 +1,448 @@
+// C ABI of the GPTAQ layer solve: handle, argument checks, launch sequences.
+// Every arithmetic step runs in the kernels of this library; the host code
+// below only validates, carves the caller's workspace and enqueues launches.
+#include "../../include/gptaq.h"
+
+#include <cuda_runtime.h>
+
+#include <cmath>
+#include <cstring>
+#include <new>
+#include <string>
+
+#include "kernels.cuh"
+#include "simt_gemm.cuh"
+
+using namespace gptaq;
+
+namespace {
+
+constexpr size_t ALIGN = 256;
+inline size_t round_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+
+enum Stage { STAGE_ACCUM = 0, STAGE_FACTORED = 1, STAGE_P = 2 };
+
+}  // namespace
+
+struct gptaq_ctx {
+    int64_t n;
+    int device;
+    int num_sms;
+    char *state;
+    size_t state_bytes;
+    char *ws;
+    size_t ws_bytes;
+    StateHeader *hd;
+    float *H, *D;
+    uint8_t *dead;
+    int stage;
+    int64_t tokens;
+    int64_t launches;
+    std::string cuda_error;
+};
+
+namespace {
+
+struct Layout {
+    size_t h_off, d_off, dead_off, total;
+};
+
+Layout state_layout(int64_t n) {
+    Layout l;
+    size_t mat = round_up((size_t)n * (size_t)n * sizeof(float), ALIGN);
+    l.h_off = ALIGN;
+    l.d_off = l.h_off + mat;
+    l.dead_off = l.d_off + mat;
+    l.total = l.dead_off + round_up((size_t)n, ALIGN);
+    return l;
+}
+
+struct WsLayout {
+    size_t t_off, rinv_off, ew_off, total;
+};
+
+WsLayout ws_layout(int64_t n, int64_t m_max, int blocksize) {
+    WsLayout w;
+    size_t nb = (size_t)((n + NB - 1) / NB);
+    w.t_off = 0;
+    w.rinv_off = w.t_off + round_up((size_t)n * (size_t)n * sizeof(float), ALIGN);
+    w.ew_off = w.rinv_off + round_up(nb * NB * NB * sizeof(float), ALIGN);
+    w.total = w.ew_off + round_up((size_t)m_max * 2 * (size_t)blocksize * sizeof(float), ALIGN);
+    return w;
+}
+
+gptaq_status_t cuda_fail(gptaq_ctx *h, cudaError_t e) {
+    if (h) h->cuda_error = cudaGetErrorString(e);
+    return GPTAQ_ERR_CUDA;
+}
+
+#define CU(call)                                             \
+    do {                                                     \
+        cudaError_t e__ = (call);                            \
+        if (e__ != cudaSuccess) return cuda_fail(h, e__);    \
+    } while (0)
+
+#define LAUNCHED()                                           \
+    do {                                                     \
+        cudaError_t e__ = cudaGetLastError();                \
+        if (e__ != cudaSuccess) return cuda_fail(h, e__);    \
+        h->launches++;                                       \
+    } while (0)
+
+gptaq_status_t gemm(gptaq_ctx *h, const GemmProblem &p, bool a_rc, bool b_rc, cudaStream_t s) {
+    if (p.M <= 0 || p.N <= 0 || p.nbatch <= 0) return GPTAQ_OK;
+    cudaError_t e = launch_simt_gemm(p, a_rc, b_rc, s);
+    if (e != cudaSuccess) return cuda_fail(h, e);
+    h->launches++;
+    return GPTAQ_OK;
+}
+
+#define OK(call)                                  \
+    do {                                          \
+        gptaq_status_t s__ = (call);              \
+        if (s__ != GPTAQ_OK) return s__;          \
+    } while (0)
+
+bool valid_block(int b) { return b == 32 || b == 64 || b == 128; }
+
+}  // namespace
+
+extern "C" {
+
+size_t gptaq_state_bytes(int64_t n) {
+    if (n <= 0) return 0;
+    return state_layout(n).total;
+}
+
+size_t gptaq_workspace_bytes(int64_t n, int64_t m_max, int64_t max_batch_tokens, int blocksize) {
+    (void)max_batch_tokens;
+    if (n <= 0 || m_max < 0 || !valid_block(blocksize)) return 0;
+    return ws_layout(n, m_max, blocksize).total;
+}
+
+gptaq_status_t gptaq_create(gptaq_handle_t *out, int64_t n, void *d_state, size_t state_bytes,
+                            void *d_workspace, size_t workspace_bytes, gptaq_stream_t stream) {
+    if (!out) return GPTAQ_ERR_INVALID_ARG;
+    *out = nullptr;
+    if (n <= 0 || n > (int64_t)1 << 20 || !d_state || !d_workspace) return GPTAQ_ERR_INVALID_ARG;
+    if ((reinterpret_cast<uintptr_t>(d_state) % ALIGN) || (reinterpret_cast<uintptr_t>(d_workspace) % ALIGN))
+        return GPTAQ_ERR_INVALID_ARG;
+    Layout l = state_layout(n);
+    if (state_bytes < l.total) return GPTAQ_ERR_WORKSPACE;
+    if (workspace_bytes < ws_layout(n, 0, 32).total) return GPTAQ_ERR_WORKSPACE;
+    gptaq_ctx *h = new (std::nothrow) gptaq_ctx();
+    if (!h) return GPTAQ_ERR_INVALID_ARG;
+    h->n = n;
+    h->state = static_cast<char *>(d_state);
+    h->state_bytes = state_bytes;
+    h->ws = static_cast<char *>(d_workspace);
+    h->ws_bytes = workspace_bytes;
+    h->hd = reinterpret_cast<StateHeader *>(h->state);
+    h->H = reinterpret_cast<float *>(h->state + l.h_off);
+    h->D = reinterpret_cast<float *>(h->state + l.d_off);
+    h->dead = reinterpret_cast<uint8_t *>(h->state + l.dead_off);
+    h->launches = 0;
+    cudaError_t e = cudaGetDevice(&h->device);
+    if (e == cudaSuccess) e = cudaDeviceGetAttribute(&h->num_sms, cudaDevAttrMultiProcessorCount, h->device);
+    if (e == cudaSuccess)
+        e = cudaFuncSetAttribute(chol_diag_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)DIAG_SMEM);
+    if (e == cudaSuccess)
+        e = cudaFuncSetAttribute(column_loop_kernel<4>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 2 * 128 * 128 * (int)sizeof(float));
+    if (e == cudaSuccess)
+        e = cudaFuncSetAttribute(column_loop_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 2 * 64 * 64 * (int)sizeof(float));
+    if (e != cudaSuccess) {
+        delete h;
+        return GPTAQ_ERR_CUDA;
+    }
+    gptaq_status_t st = gptaq_reset(h, stream);
+    if (st != GPTAQ_OK) {
+        delete h;
+        return st;
+    }
+    *out = h;
+    return GPTAQ_OK;
+}
+
+gptaq_status_t gptaq_reset(gptaq_handle_t h, gptaq_stream_t stream) {
+    if (!h) return GPTAQ_ERR_INVALID_ARG;
+    Layout l = state_layout(h->n);
+    CU(cudaMemsetAsync(h->state, 0, l.total, static_cast<cudaStream_t>(stream)));
+    h->stage = STAGE_ACCUM;
+    h->tokens = 0;
+    return GPTAQ_OK;
+}
+
+gptaq_status_t gptaq_destroy(gptaq_handle_t h) {
+    if (!h) return GPTAQ_ERR_INVALID_ARG;
+    delete h;
+    return GPTAQ_OK;
+}
+
+gptaq_status_t gptaq_accumulate(gptaq_handle_t h, const float *d_X, const float *d_Xfp,
+                                int64_t tokens, int64_t ld, gptaq_stream_t stream) {
+    if (!h || tokens < 0 || tokens > INT32_MAX) return GPTAQ_ERR_INVALID_ARG;
+    if (h->stage != STAGE_ACCUM) return GPTAQ_ERR_BAD_STATE;
+    if (tokens == 0) return GPTAQ_OK;
+    if (!d_X || !d_Xfp || ld < h->n) return GPTAQ_ERR_INVALID_ARG;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    const int n = (int)h->n;
+    // H (upper tiles) += X X^T
+    Operand xa = make_operand(d_X, 1, ld);
+    GemmProblem ph = make_problem(xa, xa, h->H, n, n, n, (int)tokens, 1.f, 1.f, GEMM_UPPER_TILES);
+    OK(gemm(h, ph, true, true, s));
+    // dXX^T += (X~ - X) X^T, the difference taken in float32 at load time
+    Operand da = xa;
+    da.sub = d_Xfp;
+    GemmProblem pd = make_problem(da, xa, h->D, n, n, n, (int)tokens, 1.f, 1.f, GEMM_FULL);
+    OK(gemm(h, pd, true, true, s));
+    h->tokens += tokens;
+    return GPTAQ_OK;
+}
+
+gptaq_status_t gptaq_accumulate_host(gptaq_handle_t h, const float *h_X, const float *h_Xfp,
+                                     int64_t tokens, int64_t ld, void *d_stage, size_t stage_bytes,
+                                     gptaq_stream_t stream) {
+    if (!h || tokens < 0) return GPTAQ_ERR_INVALID_ARG;
+    if (h->stage != STAGE_ACCUM) return GPTAQ_ERR_BAD_STATE;
+    if (tokens == 0) return GPTAQ_OK;
+    if (!h_X || !h_Xfp || !d_stage || ld < h->n) return GPTAQ_ERR_INVALID_ARG;
+    size_t one = (size_t)tokens * (size_t)h->n * sizeof(float);
+    if (stage_bytes < 2 * one) return GPTAQ_ERR_WORKSPACE;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    float *dx = static_cast<float *>(d_stage);
+    float *dxfp = dx + (size_t)tokens * (size_t)h->n;
+    size_t rowb = (size_t)h->n * sizeof(float);
+    CU(cudaMemcpy2DAsync(dx, rowb, h_X, (size_t)ld * sizeof(float), rowb, (size_t)tokens,
+                         cudaMemcpyHostToDevice, s));
+    CU(cudaMemcpy2DAsync(dxfp, rowb, h_Xfp, (size_t)ld * sizeof(float), rowb, (size_t)tokens,
+                         cudaMemcpyHostToDevice, s));
+    return gptaq_accumulate(h, dx, dxfp, tokens, h->n, stream);
+}
+
+gptaq_status_t gptaq_factor(gptaq_handle_t h, float damp, gptaq_stream_t stream) {
+    if (!h || !(damp >= 0.f) || !std::isfinite(damp)) return GPTAQ_ERR_INVALID_ARG;
+    if (h->stage != STAGE_ACCUM || h->tokens <= 0) return GPTAQ_ERR_BAD_STATE;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    const int n = (int)h->n;
+    const int nb = (n + NB - 1) / NB;
+    WsLayout wl = ws_layout(h->n, 0, 32);
+    float *T = reinterpret_cast<float *>(h->ws + wl.t_off);
+    float *Rinv = reinterpret_cast<float *>(h->ws + wl.rinv_off);
+    float *H = h->H;
+
+    diag_stats_kernel<<<1, 1024, 0, s>>>(H, n, (float)(1.0 / (double)h->tokens), damp, h->hd, h->dead);
+    LAUNCHED();
+    scale_damp_kernel<<<dim3((n + 63) / 64, (n + 63) / 64), 256, 0, s>>>(H, n, h->hd, h->dead);
+    LAUNCHED();
+
+    // reverse Cholesky H_d = R R^T, R upper, from the last block column upwards
+    for (int p = nb - 1; p >= 0; --p) {
+        const int b0 = p * NB, bw = std::min(NB, n - b0);
+        float *Rp = Rinv + (size_t)p * NB * NB;
+        chol_diag_kernel<<<1, DIAG_THREADS, DIAG_SMEM, s>>>(H, n, b0, Rp, h->hd);
+        LAUNCHED();
+        if (p == 0) break;
+        // R[0:b0, blk] = A[0:b0, blk] * inv(R_pp)^T
+        GemmProblem pp = make_problem(make_operand(H + b0, n, 1), make_operand(Rp, NB, 1), H + b0, n,
+                                      b0, bw, bw, 1.f, 0.f, GEMM_FULL);
+        OK(gemm(h, pp, false, false, s));
+        // A[0:b0, 0:b0] -= R[0:b0, blk] R[0:b0, blk]^T  (upper tiles)
+        Operand rp = make_operand(H + b0, n, 1);
+        GemmProblem ps = make_problem(rp, rp, H, n, b0, b0, bw, -1.f, 1.f, GEMM_UPPER_TILES);
+        OK(gemm(h, ps, false, false, s));
+    }
+
+    // U = R^-1: inverted diagonal blocks, then off-diagonal blocks by doubling:
+    // inv([[A, B], [0, C]]) = [[A^-1, -A^-1 B C^-1], [0, C^-1]]
+    place_diag_inverse_kernel<<<nb, 256, 0, s>>>(H, n, Rinv);
+    LAUNCHED();
+    for (int64_t sz = NB; sz < n; sz *= 2) {
+        const int np = (int)((n - sz + 2 * sz - 1) / (2 * sz));
+        const int tail = (int)(n - (2 * sz * (np - 1) + sz));
+        const int64_t bstride = 2 * sz * ((int64_t)n + 1);
+        // T = B * C^-1
+        GemmProblem p1 = make_problem(make_operand(H + sz, n, 1),
+                                      make_operand(H + sz * n + sz, 1, n), T + sz, n,
+                                      (int)sz, (int)sz, (int)sz, 1.f, 0.f, GEMM_TRI_RIGHT);
+        p1.nbatch = np; p1.batchA = p1.batchB = p1.batchC = bstride;
+        p1.batchN_last = tail; p1.batchK_last = tail;
+        OK(gemm(h, p1, false, true, s));
+        // B <- -A^-1 * T
+        GemmProblem p2 = make_problem(make_operand(H, n, 1), make_operand(T + sz, 1, n), H + sz, n,
+                                      (int)sz, (int)sz, (int)sz, -1.f, 0.f, GEMM_TRI_LEFT);
+        p2.nbatch = np; p2.batchA = p2.batchB = p2.batchC = bstride;
+        p2.batchN_last = tail;
+        OK(gemm(h, p2, false, true, s));
+    }
+    h->stage = STAGE_FACTORED;
+    return GPTAQ_OK;
+}
+
+gptaq_status_t gptaq_build_P(gptaq_handle_t h, float alpha, gptaq_stream_t stream) {
+    if (!h || !std::isfinite(alpha)) return GPTAQ_ERR_INVALID_ARG;
+    if (h->stage != STAGE_FACTORED) return GPTAQ_ERR_BAD_STATE;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    const int n = (int)h->n;
+    WsLayout wl = ws_layout(h->n, 0, 32);
+    float *O = reinterpret_cast<float *>(h->ws + wl.t_off);
+    // O = (dXX^T U^T) .* M_U
+    GemmProblem po = make_problem(make_operand(h->D, n, 1), make_operand(h->H, n, 1), O, n, n, n, n,
+                                  1.f, 0.f, GEMM_O);
+    OK(gemm(h, po, false, false, s));
+    // P = (alpha / tokens) * O U
+    GemmProblem pp = make_problem(make_operand(O, n, 1), make_operand(h->H, 1, n), h->D, n, n, n, n,
+                                  (float)((double)alpha / (double)h->tokens), 0.f, GEMM_P);
+    OK(gemm(h, pp, false, true, s));
+    h->stage = STAGE_P;
+    return GPTAQ_OK;
+}
+
+gptaq_status_t gptaq_quantize(gptaq_handle_t h, void *d_W, int w_dtype, int64_t m, int64_t ldw,
+                              int bits, int group, int sym, int blocksize,
+                              uint8_t *d_codes, float *d_scales, float *d_zeros, float *d_Wq,
+                              gptaq_stream_t stream) {
+    if (!h || m < 0 || m > INT32_MAX) return GPTAQ_ERR_INVALID_ARG;
+    if (h->stage != STAGE_P) return GPTAQ_ERR_BAD_STATE;
+    if (bits < 2 || bits > 8 || !valid_block(blocksize) || group < 0 ||
+        (w_dtype != GPTAQ_W_FP32 && w_dtype != GPTAQ_W_BF16))
+        return GPTAQ_ERR_UNSUPPORTED;
+    if (group > 0 && (blocksize % group) != 0) return GPTAQ_ERR_UNSUPPORTED;
+    if (m == 0) return GPTAQ_OK;
+    if (!d_W || !d_codes || !d_scales || !d_zeros || ldw < h->n) return GPTAQ_ERR_INVALID_ARG;
+    if (w_dtype == GPTAQ_W_BF16 && !d_Wq) return GPTAQ_ERR_INVALID_ARG;
+    const int n = (int)h->n;
+    WsLayout wl = ws_layout(h->n, m, blocksize);
+    if (h->ws_bytes < wl.total) return GPTAQ_ERR_WORKSPACE;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    float *EW = reinterpret_cast<float *>(h->ws + wl.ew_off);
+
+    float *Wk = static_cast<float *>(d_W);
+    int64_t ldk = ldw;
+    if (w_dtype == GPTAQ_W_BF16) {
+        bf16_to_f32_kernel<<<h->num_sms * 8, 256, 0, s>>>(static_cast<const __nv_bfloat16 *>(d_W), ldw,
+                                                         d_Wq, n, (int)m, n);
+        LAUNCHED();
+        Wk = d_Wq; ldk = n;
+    } else if (d_Wq && d_Wq != d_W) {
+        copy2d_kernel<<<h->num_sms * 8, 256, 0, s>>>(static_cast<const float *>(d_W), ldw, d_Wq, n,
+                                                    (int)m, n);
+        LAUNCHED();
+        Wk = d_Wq; ldk = n;
+    }
+
+    const int G = group > 0 ? (n + group - 1) / group : 1;
+    if (group <= 0) {
+        row_grid_kernel<<<(unsigned)((m + 7) / 8), 256, 0, s>>>(Wk, ldk, (int)m, n, h->dead, bits, sym,
+                                                               d_scales, d_zeros);
+        LAUNCHED();
+    }
+
+    int nw = (int)((m + h->num_sms - 1) / h->num_sms);
+    nw = std::max(1, std::min(32, nw));
+    const unsigned cl_grid = (unsigned)((m + nw - 1) / nw);
+    const int T = blocksize / 32;
+    const size_t cl_smem = 2 * (size_t)blocksize * blocksize * sizeof(float);
+
+    for (int i0 = 0; i0 < n; i0 += blocksize) {
+        ColumnLoopArgs a;
+        a.W = Wk; a.ldw = ldk; a.m = (int)m; a.n = n; a.U = h->H; a.P = h->D; a.dead = h->dead;
+        a.i0 = i0; a.bw = std::min(blocksize, n - i0);
+        a.bits = bits; a.group = group; a.sym = sym;
+        a.codes = d_codes; a.scales = d_scales; a.zeros = d_zeros; a.G = G; a.EW = EW; a.hd = h->hd;
+        if (T == 4) column_loop_kernel<4><<<cl_grid, nw * 32, cl_smem, s>>>(a);
+        else if (T == 2) column_loop_kernel<2><<<cl_grid, nw * 32, cl_smem, s>>>(a);
+        else column_loop_kernel<1><<<cl_grid, nw * 32, cl_smem, s>>>(a);
+        LAUNCHED();
+        const int i2 = i0 + blocksize;
+        if (i2 < n) {
+            // W[:, i2:] += [-Err | Wpre] * [U[blk, i2:] ; P[blk, i2:]]   (lazy-batch update)
+            Operand bop = make_operand(h->H + (int64_t)i0 * n + i2, 1, n);
+            bop.p2 = h->D + (int64_t)i0 * n + i2;
+            bop.k_split = blocksize;
+            GemmProblem pt = make_problem(make_operand(EW, 2 * blocksize, 1), bop, Wk + i2, ldk,
+                                          (int)m, n - i2, 2 * blocksize, 1.f, 1.f, GEMM_FULL);
+            OK(gemm(h, pt, false, true, s));
+        }
+    }
+    return GPTAQ_OK;
+}
+
+size_t gptaq_quantize_stage_bytes(int64_t m, int64_t n, int group) {
+    if (m < 0 || n <= 0 || group < 0) return 0;
+    size_t G = group > 0 ? (size_t)((n + group - 1) / group) : 1;
+    return round_up((size_t)m * n * sizeof(float), ALIGN) + round_up((size_t)m * n, ALIGN) +
+           2 * round_up((size_t)m * G * sizeof(float), ALIGN);
+}
+
+gptaq_status_t gptaq_quantize_host(gptaq_handle_t h, const float *h_W, int64_t m, int64_t ldw,
+                                   int bits, int group, int sym, int blocksize,
+                                   uint8_t *h_codes, float *h_scales, float *h_zeros, float *h_Wq,
+                                   void *d_stage, size_t stage_bytes, gptaq_stream_t stream) {
+    if (!h || m < 0) return GPTAQ_ERR_INVALID_ARG;
+    if (h->stage != STAGE_P) return GPTAQ_ERR_BAD_STATE;
+    if (m == 0) return GPTAQ_OK;
+    if (!h_W || !h_codes || !h_scales || !h_zeros || !d_stage || ldw < h->n || group < 0)
+        return GPTAQ_ERR_INVALID_ARG;
+    if (stage_bytes < gptaq_quantize_stage_bytes(m, h->n, group)) return GPTAQ_ERR_WORKSPACE;
+    const size_t n = (size_t)h->n;
+    const size_t G = group > 0 ? (n + group - 1) / group : 1;
+    char *base = static_cast<char *>(d_stage);
+    float *dW = reinterpret_cast<float *>(base);
+    uint8_t *dC = reinterpret_cast<uint8_t *>(base + round_up((size_t)m * n * sizeof(float), ALIGN));
+    float *dS = reinterpret_cast<float *>(reinterpret_cast<char *>(dC) + round_up((size_t)m * n, ALIGN));
+    float *dZ = reinterpret_cast<float *>(reinterpret_cast<char *>(dS) + round_up((size_t)m * G * sizeof(float), ALIGN));
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    CU(cudaMemcpy2DAsync(dW, n * sizeof(float), h_W, (size_t)ldw * sizeof(float), n * sizeof(float),
+                         (size_t)m, cudaMemcpyHostToDevice, s));
+    OK(gptaq_quantize(h, dW, GPTAQ_W_FP32, m, (int64_t)n, bits, group, sym, blocksize, dC, dS, dZ, nullptr,
+                      stream));
+    CU(cudaMemcpyAsync(h_codes, dC, (size_t)m * n, cudaMemcpyDeviceToHost, s));
+    CU(cudaMemcpyAsync(h_scales, dS, (size_t)m * G * sizeof(float), cudaMemcpyDeviceToHost, s));
+    CU(cudaMemcpyAsync(h_zeros, dZ, (size_t)m * G * sizeof(float), cudaMemcpyDeviceToHost, s));
+    if (h_Wq) CU(cudaMemcpyAsync(h_Wq, dW, (size_t)m * n * sizeof(float), cudaMemcpyDeviceToHost, s));
+    return GPTAQ_OK;
+}
+
+gptaq_status_t gptaq_sync_status(gptaq_handle_t h, int64_t *info, gptaq_stream_t stream) {
+    if (!h) return GPTAQ_ERR_INVALID_ARG;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    StateHeader hd;
+    CU(cudaMemcpyAsync(&hd, h->hd, sizeof(hd), cudaMemcpyDeviceToHost, s));
+    CU(cudaStreamSynchronize(s));
+    if (info) *info = hd.info;
+    return static_cast<gptaq_status_t>(hd.status);
+}
+
+float *gptaq_H(gptaq_handle_t h) { return h ? h->H : nullptr; }
+float *gptaq_D(gptaq_handle_t h) { return h ? h->D : nullptr; }
+int64_t gptaq_tokens(gptaq_handle_t h) { return h ? h->tokens : -1; }
+
+gptaq_status_t gptaq_set_tokens(gptaq_handle_t h, int64_t tokens) {
+    if (!h || tokens < 0) return GPTAQ_ERR_INVALID_ARG;
+    if (h->stage != STAGE_ACCUM) return GPTAQ_ERR_BAD_STATE;
+    h->tokens = tokens;
+    return GPTAQ_OK;
+}
+
+int64_t gptaq_launch_count(gptaq_handle_t h) { return h ? h->launches : -1; }
+
+const char *gptaq_status_string(gptaq_status_t s) {
+    switch (s) {
+        case GPTAQ_OK: return "ok";
+        case GPTAQ_ERR_INVALID_ARG: return "invalid argument";
+        case GPTAQ_ERR_BAD_STATE: return "call out of order";
+        case GPTAQ_ERR_WORKSPACE: return "buffer too small";
+        case GPTAQ_ERR_NOT_SPD: return "damped H is not positive definite";
+        case GPTAQ_ERR_NONFINITE: return "non-finite value";
+        case GPTAQ_ERR_TIMEOUT: return "bounded device wait ran out";
+        case GPTAQ_ERR_UNSUPPORTED: return "unsupported argument combination";
+        case GPTAQ_ERR_CUDA: return "CUDA runtime error";
+    }
+    return "unknown status";
+}
+
+const char *gptaq_last_cuda_error(gptaq_handle_t h) { return h ? h->cuda_error.c_str() : ""; }
+
+}  // extern "C"

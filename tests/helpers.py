@@ -1,0 +1,128 @@
+"""Shared helpers of the GPU parity tests: run a layer through the C-ABI
+binding and through the float64 oracle on the same seeded inputs."""
+from __future__ import annotations
+
+import dataclasses
+
+import numpy as np
+import torch
+
+import paper_2504_02692_b200 as g
+import workloads as wl
+from oracle import gptaq_oracle as orc
+
+# Parity bounds of the benchmark spec.
+TOL_OBJECTIVE = 1e-3      # relative difference of the layer objective
+TOL_FACTOR = 1e-4         # relative Frobenius error of U
+TOL_FLIP_BAND = 1e-4      # distance to a rounding boundary that excuses a flip
+TOL_FLIP_RATE = 1e-3      # at most 0.1 % excused flips
+
+
+@dataclasses.dataclass
+class GpuRun:
+    H: np.ndarray | None
+    D: np.ndarray | None
+    U: np.ndarray
+    P: np.ndarray
+    codes: np.ndarray
+    scales: np.ndarray
+    zeros: np.ndarray
+    Wq: np.ndarray
+    status: tuple
+
+
+def n_groups(n, group):
+    return 1 if group <= 0 else (n + group - 1) // group
+
+
+def gpu_layer(cfg: wl.LayerConfig, W: torch.Tensor, batches, keep_stats=True, rows=None) -> GpuRun:
+    """Runs create -> accumulate* -> factor -> build_P -> quantize through the binding."""
+    dev = "cuda"
+    m = W.shape[0]
+    st = g.LayerState(cfg.n, m, cfg.batch_tokens, cfg.blocksize, dev)
+    try:
+        for X, Xfp in batches:
+            g.gptaq_accumulate(st.handle, X.to(dev), Xfp.to(dev))
+        H = D = None
+        if keep_stats:
+            H = st.H().cpu().numpy().astype(np.float64)
+            D = st.D().cpu().numpy().astype(np.float64)
+        g.gptaq_factor(st.handle, cfg.damp)
+        g.gptaq_build_P(st.handle, cfg.alpha)
+        U = st.H().cpu().numpy().astype(np.float64)
+        P = st.D().cpu().numpy().astype(np.float64)
+        G = n_groups(cfg.n, cfg.group)
+        codes = torch.empty((m, cfg.n), dtype=torch.uint8, device=dev)
+        scales = torch.empty((m, G), dtype=torch.float32, device=dev)
+        zeros = torch.empty((m, G), dtype=torch.float32, device=dev)
+        Wd = W.to(dev)
+        if cfg.w_bf16:
+            Wd = Wd.to(torch.bfloat16)
+        Wq = torch.empty((m, cfg.n), dtype=torch.float32, device=dev)
+        g.gptaq_quantize(st.handle, Wd, cfg.bits, cfg.group, cfg.sym, cfg.blocksize, codes, scales, zeros, Wq)
+        status = g.gptaq_sync_status(st.handle)
+        return GpuRun(H, D, U, P, codes.cpu().numpy(), scales.cpu().numpy().astype(np.float64),
+                      zeros.cpu().numpy().astype(np.float64), Wq.cpu().numpy().astype(np.float64), status)
+    finally:
+        st.close()
+
+
+def oracle_stats(cfg, batches):
+    st = orc.new_stats(cfg.n, True)
+    for X, Xfp in batches:
+        orc.accumulate(st, X.cpu().numpy(), Xfp.cpu().numpy())
+    return st
+
+
+def rel_fro(a, b):
+    return float(np.linalg.norm(a - b) / np.linalg.norm(b))
+
+
+def check_layer(cfg, W, batches, rows=None, report=None):
+    """Full parity of one layer against the oracle; returns a dict of numbers."""
+    Wn = W.cpu().numpy().astype(np.float64)
+    run = gpu_layer(cfg, W, batches)
+    assert run.status[0] == g.GPTAQ_OK, run.status
+    st = oracle_stats(cfg, batches)
+    U, dead = orc.factor(st.H, st.tokens, cfg.damp)
+    P = orc.build_P(st.D, st.tokens, U, cfg.alpha)
+    out = {}
+    iu = np.triu_indices(cfg.n)
+    out["H_rel"] = float(np.linalg.norm((run.H - st.H)[iu]) / np.linalg.norm(st.H[iu]))
+    out["D_rel"] = rel_fro(run.D, st.D)
+    out["U_rel"] = rel_fro(np.triu(run.U), U)
+    out["U_lower_max"] = float(np.abs(np.tril(run.U, -1)).max()) if cfg.n > 1 else 0.0
+    out["P_rel"] = rel_fro(np.triu(run.P, 1), P) if np.linalg.norm(P) > 0 else float(np.abs(run.P).max())
+    out["P_lower_max"] = float(np.abs(np.tril(run.P)).max())
+    sel = slice(None) if rows is None else rows
+    res = orc.quantize(Wn[sel], U, P, dead, cfg.bits, cfg.group, cfg.sym)
+    rep = orc.follow(Wn[sel], U, P, dead, cfg.bits, cfg.group, cfg.sym,
+                     run.codes[sel], run.scales[sel], run.zeros[sel], band=TOL_FLIP_BAND)
+    out["follow"] = rep
+    out["free_mismatch_rate"] = float(np.mean(run.codes[sel] != res.codes))
+    J_gpu = orc.objective(Wn[sel], run.Wq[sel], st)
+    J_orc = orc.objective(Wn[sel], res.Wq, st)
+    rtn = orc.quantize(Wn[sel], U, None, dead, cfg.bits, cfg.group, cfg.sym, update=False)
+    out["J_gpu"], out["J_oracle"], out["J_rtn"] = J_gpu, J_orc, orc.objective(Wn[sel], rtn.Wq, st)
+    out["J_rel"] = abs(J_gpu - J_orc) / J_orc
+    # the dequantized output must be exactly what the codes and grids say
+    gsz = cfg.group if cfg.group > 0 else cfg.n
+    sc = np.repeat(run.scales[sel].astype(np.float32), gsz, axis=1)[:, :cfg.n]
+    zp = np.repeat(run.zeros[sel].astype(np.float32), gsz, axis=1)[:, :cfg.n]
+    deq = sc * (run.codes[sel].astype(np.float32) - zp)
+    out["dequant_consistent"] = bool(np.array_equal(deq.astype(np.float32), run.Wq[sel].astype(np.float32)))
+    if report is not None:
+        report.update(out)
+    return out
+
+
+def assert_parity(out):
+    rep = out["follow"]
+    assert out["U_rel"] <= TOL_FACTOR, out
+    assert out["U_lower_max"] == 0.0 and out["P_lower_max"] == 0.0, out
+    assert out["J_rel"] <= TOL_OBJECTIVE, out
+    assert rep.disallowed == 0, rep
+    assert rep.allowed <= TOL_FLIP_RATE * rep.total, rep
+    assert rep.grid_rel_err <= 1e-5 and rep.zero_mismatch == 0, rep
+    assert out["dequant_consistent"], out
+    assert out["J_gpu"] <= out["J_rtn"], out

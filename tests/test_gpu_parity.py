@@ -1,0 +1,202 @@
+"""CUDA path vs float64 oracle, through the C-ABI binding (needs a B200)."""
+import numpy as np
+import pytest
+import torch
+
+import paper_2504_02692_b200 as g
+import workloads as wl
+from oracle import gptaq_oracle as orc
+from tests import helpers as hp
+
+pytestmark = pytest.mark.gpu
+
+
+def batches_of(cfg, device="cpu", n_batches=None, tokens=None):
+    nb = cfg.n_batches if n_batches is None else n_batches
+    return [wl.make_batch(cfg, b, device, tokens) for b in range(nb)]
+
+
+def test_library_is_the_cuda_one():
+    lib = g.load_library()
+    assert lib._name.endswith("libgptaq.so")
+
+
+def test_cfg1_full_parity():
+    cfg = wl.CONFIGS["cfg1"]
+    out = hp.check_layer(cfg, wl.make_weight(cfg), batches_of(cfg))
+    hp.assert_parity(out)
+    assert out["H_rel"] < 1e-5 and out["D_rel"] < 1e-5 and out["P_rel"] < 1e-4
+
+
+@pytest.mark.parametrize("alpha", [0.0, 1.0])
+def test_cfg1_alpha_limits(alpha):
+    cfg = wl.scaled(wl.CONFIGS["cfg1"], alpha=alpha)
+    out = hp.check_layer(cfg, wl.make_weight(cfg), batches_of(cfg))
+    hp.assert_parity(out)
+    if alpha == 0.0:
+        assert out["P_rel"] == 0.0   # P == 0 exactly: the solve is GPTQ
+
+
+@pytest.mark.parametrize("n,m,tokens,nb,bits,group,sym,B", [
+    (200, 37, 333, 2, 4, 0, False, 32),      # ragged everything, per-channel
+    (200, 37, 333, 2, 3, 8, False, 32),      # small groups, ragged last group/block
+    (328, 70, 1000, 1, 4, 32, True, 64),     # symmetric groups, B = 64
+    (520, 150, 2048, 2, 2, 128, False, 128), # 2-bit, several 128-blocks plus a ragged tail
+    (1, 5, 16, 1, 4, 0, False, 32),          # a single input neuron
+    (129, 3, 700, 1, 8, 0, True, 128),       # one column beyond a tile
+])
+def test_ragged_shapes(n, m, tokens, nb, bits, group, sym, B):
+    cfg = wl.scaled(wl.CONFIGS["cfg1"], name="ragged", n=n, m=m, batch_tokens=tokens, n_batches=nb,
+                    bits=bits, group=group, sym=sym, blocksize=B, outlier_channels=min(2, n),
+                    act="student")
+    out = hp.check_layer(cfg, wl.make_weight(cfg), batches_of(cfg))
+    hp.assert_parity(out)
+
+
+def test_cfg4_shape_row_subset():
+    """ViT-shaped layer at full n and tokens; the oracle loop replays a seeded row subset
+    (rows are independent)."""
+    cfg = wl.CONFIGS["cfg4"]
+    W = wl.make_weight(cfg)
+    rows = np.sort(np.random.default_rng(0).choice(cfg.m, 192, replace=False))
+    out = hp.check_layer(cfg, W, batches_of(cfg), rows=rows)
+    hp.assert_parity(out)
+
+
+def test_mid_llama_like_groups():
+    """LLaMA-like recipe (Student-t, outlier channels, W4 g128) at n = 1024."""
+    cfg = wl.scaled(wl.CONFIGS["cfg2"], name="cfg2_small", n=1024, m=512, batch_tokens=4096, n_batches=4,
+                    outlier_channels=10)
+    out = hp.check_layer(cfg, wl.make_weight(cfg), batches_of(cfg), rows=np.arange(0, 512, 4))
+    hp.assert_parity(out)
+
+
+def test_gated_3bit_bf16_weights():
+    cfg = wl.scaled(wl.CONFIGS["cfg5"], name="cfg5_small", n=768, m=256, batch_tokens=2048, n_batches=3)
+    out = hp.check_layer(cfg, wl.make_weight(cfg), batches_of(cfg), rows=np.arange(0, 256, 2))
+    hp.assert_parity(out)
+
+
+def test_deterministic_and_host_entry_points_agree():
+    cfg = wl.scaled(wl.CONFIGS["cfg1"], n=256, m=96, batch_tokens=700, n_batches=2, group=32, blocksize=64)
+    W = wl.make_weight(cfg)
+    bt = batches_of(cfg)
+    a = hp.gpu_layer(cfg, W, bt)
+    b = hp.gpu_layer(cfg, W, bt)
+    assert np.array_equal(a.codes, b.codes) and np.array_equal(a.U, b.U) and np.array_equal(a.P, b.P)
+    # host entry points: pinned host buffers in, host results out
+    st = g.LayerState(cfg.n, cfg.m, cfg.batch_tokens, cfg.blocksize)
+    stage = torch.empty(max(2 * cfg.batch_tokens * cfg.n * 4, g.gptaq_quantize_stage_bytes(cfg.m, cfg.n, cfg.group)),
+                        dtype=torch.uint8, device="cuda")
+    for X, Xfp in bt:
+        g.gptaq_accumulate_host(st.handle, X.pin_memory(), Xfp.pin_memory(), stage)
+        torch.cuda.synchronize()
+    g.gptaq_factor(st.handle, cfg.damp)
+    g.gptaq_build_P(st.handle, cfg.alpha)
+    G = hp.n_groups(cfg.n, cfg.group)
+    codes = torch.empty((cfg.m, cfg.n), dtype=torch.uint8).pin_memory()
+    scales = torch.empty((cfg.m, G), dtype=torch.float32).pin_memory()
+    zeros = torch.empty((cfg.m, G), dtype=torch.float32).pin_memory()
+    Wq = torch.empty((cfg.m, cfg.n), dtype=torch.float32).pin_memory()
+    g.gptaq_quantize_host(st.handle, W.pin_memory(), cfg.bits, cfg.group, cfg.sym, cfg.blocksize,
+                          codes, scales, zeros, stage, Wq)
+    assert g.gptaq_sync_status(st.handle)[0] == g.GPTAQ_OK
+    assert np.array_equal(codes.numpy(), a.codes)
+    assert np.array_equal(Wq.numpy().astype(np.float64), a.Wq)
+    assert g.gptaq_launch_count(st.handle) > 0
+    st.close()
+
+
+def test_shared_state_quantizes_several_matrices_and_in_place():
+    cfg = wl.scaled(wl.CONFIGS["cfg1"], n=192, m=64, batch_tokens=600, group=0, blocksize=64)
+    bt = batches_of(cfg)
+    W = wl.make_weight(cfg)
+    ref = hp.gpu_layer(cfg, W, bt)
+    st = g.LayerState(cfg.n, cfg.m, cfg.batch_tokens, cfg.blocksize)
+    for X, Xfp in bt:
+        g.gptaq_accumulate(st.handle, X.cuda(), Xfp.cuda())
+    g.gptaq_factor(st.handle, cfg.damp)
+    g.gptaq_build_P(st.handle, cfg.alpha)
+    for rep in range(2):      # q/k/v-style: same statistics, several weights
+        Wd = W.cuda().clone()
+        codes = torch.empty((cfg.m, cfg.n), dtype=torch.uint8, device="cuda")
+        sc = torch.empty((cfg.m, 1), dtype=torch.float32, device="cuda")
+        zp = torch.empty((cfg.m, 1), dtype=torch.float32, device="cuda")
+        g.gptaq_quantize(st.handle, Wd, cfg.bits, cfg.group, cfg.sym, cfg.blocksize, codes, sc, zp, None)
+        assert g.gptaq_sync_status(st.handle)[0] == g.GPTAQ_OK
+        assert np.array_equal(codes.cpu().numpy(), ref.codes)
+        assert np.array_equal(Wd.cpu().numpy().astype(np.float64), ref.Wq)   # in place when d_Wq is NULL
+    st.close()
+
+
+def test_call_order_empty_inputs_and_bad_arguments():
+    n, m = 96, 8
+    st = g.LayerState(n, m, 64, 32)
+    h = st.handle
+    X = torch.randn(64, n, device="cuda")
+    with pytest.raises(g.GptaqError) as e:
+        g.gptaq_factor(h, 0.01)                      # nothing accumulated yet
+    assert e.value.status == g.GPTAQ_ERR_BAD_STATE
+    with pytest.raises(g.GptaqError) as e:
+        g.gptaq_build_P(h, 1.0)
+    assert e.value.status == g.GPTAQ_ERR_BAD_STATE
+    g.gptaq_accumulate(h, X[:0], X[:0])              # empty batch: no-op
+    assert g.gptaq_tokens(h) == 0
+    g.gptaq_accumulate(h, X, X)
+    assert g.gptaq_tokens(h) == 64
+    g.gptaq_factor(h, 0.01)
+    with pytest.raises(g.GptaqError) as e:
+        g.gptaq_accumulate(h, X, X)                  # sums are gone after factor
+    assert e.value.status == g.GPTAQ_ERR_BAD_STATE
+    g.gptaq_build_P(h, 0.5)
+    W = torch.randn(m, n, device="cuda")
+    codes = torch.empty((m, n), dtype=torch.uint8, device="cuda")
+    s = torch.empty((m, 1), device="cuda"); z = torch.empty((m, 1), device="cuda")
+    for kw in (dict(bits=1), dict(bits=9), dict(blocksize=48), dict(group=24)):
+        a = dict(bits=4, group=0, blocksize=32); a.update(kw)
+        with pytest.raises(g.GptaqError) as e:
+            g.gptaq_quantize(h, W, a["bits"], a["group"], False, a["blocksize"], codes, s, z)
+        assert e.value.status == g.GPTAQ_ERR_UNSUPPORTED
+    g.gptaq_quantize(h, W[:0], 4, 0, False, 32, codes[:0], s[:0], z[:0])   # m == 0: no-op
+    assert g.gptaq_sync_status(h)[0] == g.GPTAQ_OK
+    # X~ == X gave dXX^T == 0 exactly, hence P == 0
+    assert float(st.D().abs().max()) == 0.0
+    g.gptaq_reset(h)
+    assert g.gptaq_tokens(h) == 0
+    g.gptaq_accumulate(h, X, X)
+    st.close()
+
+
+def test_device_side_conditions_are_reported_not_trapped():
+    n = 64
+    st = g.LayerState(n, 4, 16, 32)
+    h = st.handle
+    X = torch.randn(16, n, device="cuda")            # rank 16 < n and no damping
+    g.gptaq_accumulate(h, X, X)
+    g.gptaq_factor(h, 0.0)
+    status, info = g.gptaq_sync_status(h)
+    assert status == g.GPTAQ_ERR_NOT_SPD and 0 <= info < n
+    # the context is still usable: damped, the same statistics factor fine
+    g.gptaq_reset(h)
+    g.gptaq_accumulate(h, X, X)
+    g.gptaq_factor(h, 0.01)
+    assert g.gptaq_sync_status(h)[0] == g.GPTAQ_OK
+    # a NaN in the input is reported by factor
+    g.gptaq_reset(h)
+    Xn = X.clone(); Xn[3, 5] = float("nan")
+    g.gptaq_accumulate(h, Xn, Xn)
+    g.gptaq_factor(h, 0.01)
+    status, info = g.gptaq_sync_status(h)
+    assert status == g.GPTAQ_ERR_NONFINITE
+    st.close()
+
+
+def test_dead_inputs():
+    cfg = wl.scaled(wl.CONFIGS["cfg1"], n=160, m=24, batch_tokens=500, group=32, blocksize=32)
+    W = wl.make_weight(cfg)
+    bt = [(X.clone(), Xfp.clone()) for X, Xfp in batches_of(cfg)]
+    for X, Xfp in bt:
+        X[:, 7] = 0.0
+        X[:, 100] = 0.0
+    out = hp.check_layer(cfg, W, bt)
+    hp.assert_parity(out)
