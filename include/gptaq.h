@@ -58,6 +58,14 @@ typedef enum {
 
 enum { GPTAQ_W_FP32 = 0, GPTAQ_W_BF16 = 1 };
 
+/* Arithmetic of the statistics (Algorithm 1, line 2).
+ * GPTAQ_STATS_FP16_TENSOR (default): X and X~ - X (the difference taken in float32 first) are
+ *   rounded to fp16, scaled by a power of two if the batch would leave the fp16 range, and
+ *   multiplied on the tensor cores with float32 accumulation.  Used for n >= 256; smaller
+ *   layers always take the float32 path.
+ * GPTAQ_STATS_FP32: float32 products and sums on the plain FMA pipes (exact inputs). */
+enum { GPTAQ_STATS_FP16_TENSOR = 0, GPTAQ_STATS_FP32 = 1 };
+
 /* Bytes of the caller-owned device state for layer width n: a header (status
  * word, pivot index), H (n x n), dXX^T (n x n) and the dead-input flags.
  * After gptaq_factor, U overwrites H; after gptaq_build_P, P overwrites dXX^T. */
@@ -66,7 +74,8 @@ size_t gptaq_state_bytes(int64_t n);
 /* Bytes of caller-owned device scratch that factor / build_P / quantize need
  * for width n, at most m_max weight rows and the given lazy-batch block size
  * (Algorithm 1, input B).  max_batch_tokens is the largest `tokens` that
- * gptaq_accumulate will be given. */
+ * gptaq_accumulate will be given in one call (larger batches still work: they
+ * are processed in chunks that fit). */
 size_t gptaq_workspace_bytes(int64_t n, int64_t m_max, int64_t max_batch_tokens, int blocksize);
 
 /* Creates a handle over caller-owned device buffers (both 256-byte aligned)
@@ -108,10 +117,11 @@ gptaq_status_t gptaq_factor(gptaq_handle_t h, float damp, gptaq_stream_t stream)
 gptaq_status_t gptaq_build_P(gptaq_handle_t h, float alpha, gptaq_stream_t stream);
 
 /* Algorithm 1, lines 5-13, for one weight matrix sharing this state.
- *   d_W      [m x ldw], float32 or bf16 (w_dtype); consumed: float32 weights are
+ *   d_W      [m x ldw], float32 or bf16 (w_dtype).  If d_Wq is given, d_W is read
+ *            only and the float32 working copy lives in d_Wq (required for bf16
+ *            weights).  If d_Wq is NULL (or equal to d_W), float32 weights are
  *            updated in place and hold the dequantized result on return
- *            (column j becomes Q[:, j] at step j); bf16 weights are read only
- *            and the float32 working copy lives in d_Wq, which is then required.
+ *            (column j becomes Q[:, j] at step j).
  *   bits     2..8;  group: 0 = one grid per output channel taken from the
  *            original row, else a grid per `group` consecutive columns taken
  *            from the current (already updated) weights at the group's first
@@ -152,6 +162,9 @@ float *gptaq_D(gptaq_handle_t h);
 int64_t gptaq_tokens(gptaq_handle_t h);
 /* Sets the token count (for callers that restore checkpointed sums). */
 gptaq_status_t gptaq_set_tokens(gptaq_handle_t h, int64_t tokens);
+
+/* Chooses the arithmetic of gptaq_accumulate (see GPTAQ_STATS_*). */
+gptaq_status_t gptaq_set_stats_precision(gptaq_handle_t h, int precision);
 
 /* Number of kernels this handle has launched since create (bookkeeping for benchmarks). */
 int64_t gptaq_launch_count(gptaq_handle_t h);

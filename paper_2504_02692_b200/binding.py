@@ -26,6 +26,8 @@ GPTAQ_ERR_UNSUPPORTED = 7
 GPTAQ_ERR_CUDA = 8
 GPTAQ_W_FP32 = 0
 GPTAQ_W_BF16 = 1
+GPTAQ_STATS_FP16_TENSOR = 0
+GPTAQ_STATS_FP32 = 1
 
 _vp, _i64, _int, _sz, _f = C.c_void_p, C.c_int64, C.c_int, C.c_size_t, C.c_float
 
@@ -48,6 +50,7 @@ SIGNATURES = {
     "gptaq_D": (_vp, [_vp]),
     "gptaq_tokens": (_i64, [_vp]),
     "gptaq_set_tokens": (_int, [_vp, _i64]),
+    "gptaq_set_stats_precision": (_int, [_vp, _int]),
     "gptaq_launch_count": (_i64, [_vp]),
     "gptaq_status_string": (C.c_char_p, [_int]),
     "gptaq_last_cuda_error": (C.c_char_p, [_vp]),
@@ -219,6 +222,10 @@ def gptaq_tokens(h) -> int:
 
 def gptaq_set_tokens(h, tokens: int):
     _check(load_library().gptaq_set_tokens(h, tokens), "gptaq_set_tokens", h)
+
+
+def gptaq_set_stats_precision(h, precision: int):
+    _check(load_library().gptaq_set_stats_precision(h, precision), "gptaq_set_stats_precision", h)
 
 
 def gptaq_launch_count(h) -> int:

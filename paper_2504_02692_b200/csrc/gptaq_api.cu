@@ -12,6 +12,7 @@
 
 #include "kernels.cuh"
 #include "simt_gemm.cuh"
+#include "umma_gemm.cuh"
 
 using namespace gptaq;
 
@@ -38,6 +39,7 @@ struct gptaq_ctx {
     int stage;
     int64_t tokens;
     int64_t launches;
+    int stats_precision;   // GPTAQ_STATS_*
     std::string cuda_error;
 };
 
@@ -103,6 +105,87 @@ gptaq_status_t gemm(gptaq_ctx *h, const GemmProblem &p, bool a_rc, bool b_rc, cu
         if (s__ != GPTAQ_OK) return s__;          \
     } while (0)
 
+// cuTensorMapEncodeTiled through the runtime's driver entry point (no link-time libcuda).
+typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
+                                  const cuuint64_t *, const cuuint32_t *, const cuuint32_t *,
+                                  CUtensorMapInterleave, CUtensorMapSwizzle, CUtensorMapL2promotion,
+                                  CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_tiled_fn() {
+    static EncodeTiledFn fn = nullptr;
+    if (!fn) {
+        void *p = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
+            q == cudaDriverEntryPointSuccess)
+            fn = reinterpret_cast<EncodeTiledFn>(p);
+    }
+    return fn;
+}
+
+// fp16 matrix [rows][kp] (K contiguous), box = 64 x box_rows, 128-byte swizzle.
+bool make_kmajor_map(CUtensorMap *map, const void *ptr, int64_t rows, int64_t kp, int box_rows) {
+    EncodeTiledFn fn = encode_tiled_fn();
+    if (!fn) return false;
+    cuuint64_t dims[2] = {(cuuint64_t)kp, (cuuint64_t)rows};
+    cuuint64_t strides[1] = {(cuuint64_t)kp * 2};
+    cuuint32_t box[2] = {(cuuint32_t)UBK, (cuuint32_t)box_rows};
+    cuuint32_t estr[2] = {1, 1};
+    return fn(map, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 2, const_cast<void *>(ptr), dims, strides, box, estr,
+              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+// Largest token chunk (multiple of 64) whose two fp16 operand copies fit the workspace.
+int64_t tc_chunk_tokens(const gptaq_ctx *h) {
+    int64_t per_token = 2 * h->n * 2;   // X^T and dX^T, fp16
+    int64_t cap = (int64_t)(h->ws_bytes / (size_t)per_token);
+    cap = cap / UBK * UBK;
+    return std::min<int64_t>(cap, 1 << 20);
+}
+
+bool tc_eligible(const gptaq_ctx *h) {
+    return h->stats_precision == GPTAQ_STATS_FP16_TENSOR && h->n >= UBN && tc_chunk_tokens(h) >= UBK &&
+           encode_tiled_fn() != nullptr;
+}
+
+gptaq_status_t accumulate_tc(gptaq_ctx *h, const float *X, const float *Xfp, int64_t tokens, int64_t ld,
+                             cudaStream_t s) {
+    const int n = (int)h->n;
+    const int64_t chunk = tc_chunk_tokens(h);
+    const int TM = (n + UBM - 1) / UBM, TN = (n + UBN - 1) / UBN;
+    int64_t ntiles = (int64_t)TM * TN;
+    for (int tm = 0; tm < TM; ++tm) ntiles += TN - (tm * UBM) / UBN;
+    for (int64_t t0 = 0; t0 < tokens; t0 += chunk) {
+        const int tk = (int)std::min<int64_t>(chunk, tokens - t0);
+        const int kp = (tk + UBK - 1) / UBK * UBK;
+        __half *Xt = reinterpret_cast<__half *>(h->ws);
+        __half *dXt = Xt + (size_t)n * kp;
+        CU(cudaMemsetAsync(h->hd->amax, 0, 2 * sizeof(unsigned), s));
+        ConvertArgs ca;
+        ca.X = X + t0 * ld; ca.Xfp = Xfp + t0 * ld; ca.ld = ld; ca.tokens = tk; ca.n = n; ca.kp = kp;
+        ca.Xt = Xt; ca.dXt = dXt; ca.amax = h->hd->amax;
+        dim3 cgrid(kp / 64, (n + 63) / 64);
+        convert_transpose_kernel<0><<<cgrid, 256, 0, s>>>(ca);
+        LAUNCHED();
+        convert_transpose_kernel<1><<<cgrid, 256, 0, s>>>(ca);
+        LAUNCHED();
+        CUtensorMap mXa, mDa, mXb;
+        if (!make_kmajor_map(&mXa, Xt, n, kp, UBM) || !make_kmajor_map(&mDa, dXt, n, kp, UBM) ||
+            !make_kmajor_map(&mXb, Xt, n, kp, UBN)) {
+            h->cuda_error = "cuTensorMapEncodeTiled failed";
+            return GPTAQ_ERR_CUDA;
+        }
+        StatsGemmArgs ga;
+        ga.H = h->H; ga.D = h->D; ga.n = n; ga.kblocks = kp / UBK; ga.amax = h->hd->amax; ga.hd = h->hd;
+        const int grid = (int)std::min<int64_t>(ntiles, h->num_sms);
+        stats_umma_kernel<<<grid, UMMA_THREADS, UMMA_SMEM, s>>>(mXa, mDa, mXb, ga);
+        LAUNCHED();
+    }
+    h->tokens += tokens;
+    return GPTAQ_OK;
+}
+
 bool valid_block(int b) { return b == 32 || b == 64 || b == 128; }
 
 }  // namespace
@@ -115,9 +198,11 @@ size_t gptaq_state_bytes(int64_t n) {
 }
 
 size_t gptaq_workspace_bytes(int64_t n, int64_t m_max, int64_t max_batch_tokens, int blocksize) {
-    (void)max_batch_tokens;
-    if (n <= 0 || m_max < 0 || !valid_block(blocksize)) return 0;
-    return ws_layout(n, m_max, blocksize).total;
+    if (n <= 0 || m_max < 0 || max_batch_tokens < 0 || !valid_block(blocksize)) return 0;
+    // the fp16 operand copies of one token batch share the space of the later steps' scratch
+    size_t kp = round_up((size_t)max_batch_tokens, (size_t)UBK);
+    size_t xt = round_up(2 * (size_t)n * kp * 2, ALIGN);
+    return std::max(ws_layout(n, m_max, blocksize).total, xt);
 }
 
 gptaq_status_t gptaq_create(gptaq_handle_t *out, int64_t n, void *d_state, size_t state_bytes,
@@ -142,6 +227,7 @@ gptaq_status_t gptaq_create(gptaq_handle_t *out, int64_t n, void *d_state, size_
     h->D = reinterpret_cast<float *>(h->state + l.d_off);
     h->dead = reinterpret_cast<uint8_t *>(h->state + l.dead_off);
     h->launches = 0;
+    h->stats_precision = GPTAQ_STATS_FP16_TENSOR;
     cudaError_t e = cudaGetDevice(&h->device);
     if (e == cudaSuccess) e = cudaDeviceGetAttribute(&h->num_sms, cudaDevAttrMultiProcessorCount, h->device);
     if (e == cudaSuccess)
@@ -149,6 +235,8 @@ gptaq_status_t gptaq_create(gptaq_handle_t *out, int64_t n, void *d_state, size_
     if (e == cudaSuccess)
         e = cudaFuncSetAttribute(column_loop_kernel<4>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                  2 * 128 * 128 * (int)sizeof(float));
+    if (e == cudaSuccess)
+        e = cudaFuncSetAttribute(stats_umma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)UMMA_SMEM);
     if (e == cudaSuccess)
         e = cudaFuncSetAttribute(column_loop_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                  2 * 64 * 64 * (int)sizeof(float));
@@ -188,6 +276,7 @@ gptaq_status_t gptaq_accumulate(gptaq_handle_t h, const float *d_X, const float 
     if (!d_X || !d_Xfp || ld < h->n) return GPTAQ_ERR_INVALID_ARG;
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     const int n = (int)h->n;
+    if (tc_eligible(h)) return accumulate_tc(h, d_X, d_Xfp, tokens, ld, s);
     // H (upper tiles) += X X^T
     Operand xa = make_operand(d_X, 1, ld);
     GemmProblem ph = make_problem(xa, xa, h->H, n, n, n, (int)tokens, 1.f, 1.f, GEMM_UPPER_TILES);
@@ -423,6 +512,13 @@ gptaq_status_t gptaq_set_tokens(gptaq_handle_t h, int64_t tokens) {
     if (!h || tokens < 0) return GPTAQ_ERR_INVALID_ARG;
     if (h->stage != STAGE_ACCUM) return GPTAQ_ERR_BAD_STATE;
     h->tokens = tokens;
+    return GPTAQ_OK;
+}
+
+gptaq_status_t gptaq_set_stats_precision(gptaq_handle_t h, int precision) {
+    if (!h) return GPTAQ_ERR_INVALID_ARG;
+    if (precision != GPTAQ_STATS_FP16_TENSOR && precision != GPTAQ_STATS_FP32) return GPTAQ_ERR_UNSUPPORTED;
+    h->stats_precision = precision;
     return GPTAQ_OK;
 }
 

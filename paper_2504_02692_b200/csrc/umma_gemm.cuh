@@ -1,0 +1,385 @@
+// Tensor-core statistics kernel for sm_100a: C += A * B^T with fp16 operands in
+// K-major shared-memory tiles (TMA, 128-byte swizzle), tcgen05.mma with fp32
+// accumulators in tensor memory, and a read-modify-write epilogue into the fp32
+// sums.  Persistent, warp-specialised: warp 0 issues TMA loads, warp 1 issues
+// the MMAs and owns the TMEM allocation, warps 2-5 drain the accumulators.
+// Two 128 x 256 accumulators are kept in TMEM so that the epilogue of one tile
+// overlaps the main loop of the next.
+//
+// Every wait on an mbarrier is bounded by a clock limit; when it runs out the
+// kernel records GPTAQ_ERR_TIMEOUT in the state header, lets outstanding copies
+// land (bounded as well), frees its tensor memory and returns.
+#pragma once
+#include <cuda.h>
+#include <cuda_fp16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "kernels.cuh"
+
+namespace gptaq {
+
+constexpr int UBM = 128, UBN = 256, UBK = 64, USTAGES = 4;
+constexpr int UA_BYTES = UBM * UBK * 2;
+constexpr int UB_BYTES = UBN * UBK * 2;
+constexpr int USTAGE_BYTES = UA_BYTES + UB_BYTES;
+constexpr int UMMA_THREADS = 192;
+constexpr size_t UMMA_SMEM = (size_t)USTAGES * USTAGE_BYTES + 1024 /*alignment slack*/ + 256 /*barriers*/;
+constexpr long long WAIT_LIMIT_CYCLES = 4000000000LL;   // about two seconds
+
+// fp16 range management: operands are scaled by a power of two when the
+// batch's absolute maximum is outside [2^-8, 2^15]; the epilogue undoes it.
+__host__ __device__ __forceinline__ float pick_scale(float amax) {
+    if (!(amax > 0.f) || !isfinite(amax)) return 1.f;
+    if (amax <= 32768.f && amax >= 0.00390625f) return 1.f;
+    int e;
+    frexpf(amax, &e);                 // amax = f * 2^e, f in [0.5, 1)
+    return ldexpf(1.f, 14 - e);       // scaled maximum in [2^13, 2^14)
+}
+
+// ---------------------------------------------------------------------------
+// Prologue: token-major fp32 X, X~  ->  channel-major (K-major) fp16 X^T and
+// (X~ - X)^T with the token dimension zero-padded to kp; the difference is
+// taken in fp32 before the down-conversion.  PASS 0 converts with scale 1 and
+// records the absolute maxima; PASS 1 redoes the conversion only if a maximum
+// fell outside the fp16 comfort range.
+// ---------------------------------------------------------------------------
+struct ConvertArgs {
+    const float *X, *Xfp;
+    int64_t ld;
+    int tokens, n, kp;
+    __half *Xt, *dXt;       // [n][kp]
+    unsigned *amax;          // [2]: bit patterns of max|X|, max|X~ - X|
+};
+
+template <int PASS>
+__global__ void __launch_bounds__(256) convert_transpose_kernel(ConvertArgs a) {
+    __shared__ __half sx[64][72];
+    __shared__ __half sd[64][72];
+    float scx = 1.f, scd = 1.f;
+    if (PASS == 1) {
+        scx = pick_scale(__uint_as_float(a.amax[0]));
+        scd = pick_scale(__uint_as_float(a.amax[1]));
+        if (scx == 1.f && scd == 1.f) return;
+    }
+    const int t0 = blockIdx.x * 64, c0 = blockIdx.y * 64;
+    const int tid = threadIdx.x;
+    float mx = 0.f, md = 0.f;
+#pragma unroll
+    for (int it = 0; it < 4; ++it) {
+        int idx = tid + it * 256;          // 0..1023: 64 tokens x 16 float4
+        int tl = idx >> 4, cl = (idx & 15) * 4;
+        int t = t0 + tl, c = c0 + cl;
+        float x[4] = {0.f, 0.f, 0.f, 0.f}, f[4] = {0.f, 0.f, 0.f, 0.f};
+        if (t < a.tokens) {
+            const float *px = a.X + (int64_t)t * a.ld + c;
+            const float *pf = a.Xfp + (int64_t)t * a.ld + c;
+            if (c + 3 < a.n && ((reinterpret_cast<uintptr_t>(px) | reinterpret_cast<uintptr_t>(pf)) & 15) == 0) {
+                float4 vx = *reinterpret_cast<const float4 *>(px);
+                float4 vf = *reinterpret_cast<const float4 *>(pf);
+                x[0] = vx.x; x[1] = vx.y; x[2] = vx.z; x[3] = vx.w;
+                f[0] = vf.x; f[1] = vf.y; f[2] = vf.z; f[3] = vf.w;
+            } else {
+#pragma unroll
+                for (int e = 0; e < 4; ++e)
+                    if (c + e < a.n) { x[e] = px[e]; f[e] = pf[e]; }
+            }
+        }
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+            float d = f[e] - x[e];
+            if (PASS == 0) {
+                // NaN compares false everywhere, so fold it in through the bit pattern below
+                mx = fmaxf(mx, fabsf(x[e])); md = fmaxf(md, fabsf(d));
+                if (x[e] != x[e] || d != d) { mx = __int_as_float(0x7fc00000); }
+            }
+            sx[cl + e][tl] = __float2half_rn(x[e] * scx);
+            sd[cl + e][tl] = __float2half_rn(d * scd);
+        }
+    }
+    if (PASS == 0) {
+        unsigned ux = __float_as_uint(mx), ud = __float_as_uint(md);
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) {
+            ux = max(ux, __shfl_xor_sync(0xffffffffu, ux, o));
+            ud = max(ud, __shfl_xor_sync(0xffffffffu, ud, o));
+        }
+        if ((tid & 31) == 0) { atomicMax(&a.amax[0], ux); atomicMax(&a.amax[1], ud); }
+    }
+    __syncthreads();
+    // 64 channels x 8 chunks of 8 halves (16 bytes) per matrix
+#pragma unroll
+    for (int it = 0; it < 2; ++it) {
+        int idx = tid + it * 256;          // 0..511
+        int cl = idx >> 3, ch = (idx & 7) * 8;
+        int c = c0 + cl, t = t0 + ch;
+        if (c < a.n && t < a.kp) {
+            *reinterpret_cast<uint4 *>(a.Xt + (int64_t)c * a.kp + t) = *reinterpret_cast<const uint4 *>(&sx[cl][ch]);
+            *reinterpret_cast<uint4 *>(a.dXt + (int64_t)c * a.kp + t) = *reinterpret_cast<const uint4 *>(&sd[cl][ch]);
+        }
+    }
+}
+
+// ---------------------------------------------------------------------------
+// PTX wrappers
+// ---------------------------------------------------------------------------
+__device__ __forceinline__ uint32_t smem_u32(const void *p) {
+    return static_cast<uint32_t>(__cvta_generic_to_shared(p));
+}
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_try(uint32_t bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+    return ok != 0;
+}
+// Bounded wait: false if the clock limit ran out or another role gave up.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag) {
+    if (mbar_try(bar, parity)) return true;
+    const long long t0 = clock64();
+    for (uint32_t it = 1;; ++it) {
+        if (mbar_try(bar, parity)) return true;
+        if ((it & 63) == 0) {
+            if (*abort_flag) return false;
+            if (clock64() - t0 > WAIT_LIMIT_CYCLES) { *abort_flag = 1; return false; }
+        }
+    }
+}
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap *map, int c0, int c1, uint32_t bar) {
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
+        ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(bar), "r"(c0), "r"(c1) : "memory");
+}
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void umma_f16(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t acc) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(acc) : "memory");
+}
+__device__ __forceinline__ void umma_commit(uint32_t bar) {
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+          "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
+          "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
+          "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+        : "r"(taddr) : "memory");
+}
+__device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+
+// K-major, 128-byte-swizzled operand tile: rows of 128 bytes, 8-row groups 1024 bytes apart.
+__device__ __forceinline__ uint64_t make_kmajor_desc(uint32_t smem_addr) {
+    uint64_t d = 0;
+    d |= (uint64_t)((smem_addr >> 4) & 0x3FFF);
+    d |= (uint64_t)1 << 16;                 // leading byte offset (unused for swizzled K-major)
+    d |= (uint64_t)(1024 >> 4) << 32;       // stride byte offset between 8-row groups
+    d |= (uint64_t)1 << 46;                 // descriptor version of sm_100
+    d |= (uint64_t)2 << 61;                 // 128-byte swizzle
+    return d;
+}
+
+// kind::f16 instruction descriptor: fp16 A and B (both K-major), fp32 D, M = 128, N = 256.
+constexpr uint32_t UMMA_IDESC_F16 = (1u << 4) | (0u << 7) | (0u << 10) | ((UBN >> 3) << 17) | ((UBM >> 4) << 24);
+
+struct StatsGemmArgs {
+    float *H, *D;            // n x n, ld n
+    int n;
+    int kblocks;             // kp / 64
+    const unsigned *amax;    // scales are recomputed from the recorded maxima
+    StateHeader *hd;
+};
+
+// Tile enumeration shared by all roles: row-major over (row tile, column tile);
+// rows [0, TM) belong to H (tiles entirely below the diagonal are not
+// enumerated), rows [TM, 2 TM) to dXX^T.
+struct TileIter {
+    int TM, TN, r, tn, left;      // left: tiles still to skip before the next one of this CTA
+    __device__ TileIter(int n, int first) : TM((n + UBM - 1) / UBM), TN((n + UBN - 1) / UBN), r(0), tn(0), left(first) {
+        tn = first_tn(0);
+    }
+    __device__ int first_tn(int row) const { return row < TM ? (row * UBM) / UBN : 0; }
+    // Advances to the tile `left` positions ahead; false when the list is exhausted.
+    __device__ bool seek() {
+        while (r < 2 * TM) {
+            int avail = TN - tn;
+            if (left < avail) { tn += left; left = 0; return true; }
+            left -= avail;
+            ++r;
+            tn = first_tn(r);
+        }
+        return false;
+    }
+};
+
+__global__ void __launch_bounds__(UMMA_THREADS, 1)
+stats_umma_kernel(const __grid_constant__ CUtensorMap mapXa, const __grid_constant__ CUtensorMap mapDa,
+                  const __grid_constant__ CUtensorMap mapXb, StatsGemmArgs a) {
+    extern __shared__ uint8_t smem_raw[];
+    // 1024-byte alignment for the swizzled tiles
+    const uint32_t raw = smem_u32(smem_raw);
+    const uint32_t base = (raw + 1023u) & ~1023u;
+    uint8_t *aligned = smem_raw + (base - raw);
+    const uint32_t bar0 = base + USTAGES * USTAGE_BYTES;
+    // barrier slots (8 bytes each): full[4], empty[4], tfull[2], tempty[2]; then tmem slot, abort flag
+    auto full_bar = [&](int s) { return bar0 + 8u * s; };
+    auto empty_bar = [&](int s) { return bar0 + 8u * (USTAGES + s); };
+    auto tfull_bar = [&](int b) { return bar0 + 8u * (2 * USTAGES + b); };
+    auto tempty_bar = [&](int b) { return bar0 + 8u * (2 * USTAGES + 2 + b); };
+    volatile uint32_t *tmem_slot = reinterpret_cast<volatile uint32_t *>(aligned + USTAGES * USTAGE_BYTES + 8 * (2 * USTAGES + 4));
+    volatile int *abort_flag = reinterpret_cast<volatile int *>(tmem_slot + 1);
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < USTAGES; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
+        for (int b = 0; b < 2; ++b) { mbar_init(tfull_bar(b), 1); mbar_init(tempty_bar(b), 4); }
+        *abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 1) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
+                     ::"r"(smem_u32(const_cast<uint32_t *>(tmem_slot))), "r"(512u) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = *tmem_slot;
+    const int KB = a.kblocks;
+
+    if (warp == 0) {
+        // ------------------------------------------------------------ TMA producer
+        if (lane == 0) {
+            TileIter it(a.n, blockIdx.x);
+            uint32_t stage = 0, phase = 0;
+            int issued = 0;
+            bool ok = true;
+            while (ok && it.seek()) {
+                const bool isD = it.r >= it.TM;
+                const CUtensorMap *mapA = isD ? &mapDa : &mapXa;
+                const int row0 = (isD ? it.r - it.TM : it.r) * UBM, col0 = it.tn * UBN;
+                for (int kb = 0; kb < KB; ++kb) {
+                    if (!mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag)) { ok = false; break; }
+                    const uint32_t sa = base + stage * USTAGE_BYTES, sb = sa + UA_BYTES;
+                    mbar_expect_tx(full_bar(stage), USTAGE_BYTES);
+                    tma_load_2d(sa, mapA, kb * UBK, row0, full_bar(stage));
+                    tma_load_2d(sb, &mapXb, kb * UBK, col0, full_bar(stage));
+                    ++issued;
+                    if (++stage == USTAGES) { stage = 0; phase ^= 1u; }
+                }
+                it.left = gridDim.x;
+            }
+            if (!ok) {
+                // give copies that are still in flight time to land before the CTA exits
+                const long long t0 = clock64();
+                while (issued > 0 && clock64() - t0 < 4000000LL) {}
+            }
+        }
+    } else if (warp == 1) {
+        // ------------------------------------------------------------ MMA issuer
+        if (lane == 0) {
+            TileIter it(a.n, blockIdx.x);
+            uint32_t stage = 0, phase = 0, tcount = 0;
+            bool ok = true;
+            while (ok && it.seek()) {
+                const uint32_t buf = tcount & 1u, tphase = (tcount >> 1) & 1u;
+                if (!mbar_wait(tempty_bar(buf), tphase ^ 1u, abort_flag)) { ok = false; break; }
+                tc_fence_after();
+                const uint32_t d_tmem = tmem_base + buf * UBN;
+                for (int kb = 0; kb < KB; ++kb) {
+                    if (!mbar_wait(full_bar(stage), phase, abort_flag)) { ok = false; break; }
+                    tc_fence_after();
+                    const uint32_t sa = base + stage * USTAGE_BYTES, sb = sa + UA_BYTES;
+                    const uint64_t ad = make_kmajor_desc(sa), bd = make_kmajor_desc(sb);
+#pragma unroll
+                    for (int k = 0; k < UBK / 16; ++k)
+                        umma_f16(d_tmem, ad + (uint64_t)(k * 2), bd + (uint64_t)(k * 2), UMMA_IDESC_F16,
+                                 (kb | k) != 0 ? 1u : 0u);
+                    umma_commit(empty_bar(stage));
+                    if (++stage == USTAGES) { stage = 0; phase ^= 1u; }
+                }
+                if (!ok) break;
+                umma_commit(tfull_bar(buf));
+                ++tcount;
+                it.left = gridDim.x;
+            }
+        }
+    } else {
+        // ------------------------------------------------------------ epilogue (warps 2..5)
+        const int quarter = warp & 3;           // TMEM lanes 32 * quarter .. + 31
+        TileIter it(a.n, blockIdx.x);
+        uint32_t tcount = 0;
+        bool ok = true;
+        const float sx = pick_scale(__uint_as_float(a.amax[0]));
+        const float sd = pick_scale(__uint_as_float(a.amax[1]));
+        while (ok && it.seek()) {
+            const uint32_t buf = tcount & 1u, tphase = (tcount >> 1) & 1u;
+            const bool isD = it.r >= it.TM;
+            const int row = (isD ? it.r - it.TM : it.r) * UBM + quarter * 32 + lane;
+            const int col0 = it.tn * UBN;
+            float *C = isD ? a.D : a.H;
+            const float inv = 1.f / (sx * (isD ? sd : sx));
+            if (!mbar_wait(tfull_bar(buf), tphase, abort_flag)) { ok = false; break; }
+            tc_fence_after();
+            const uint32_t taddr = tmem_base + buf * UBN + ((uint32_t)(quarter * 32) << 16);
+#pragma unroll 1
+            for (int cc = 0; cc < UBN; cc += 32) {
+                uint32_t v[32];
+                tmem_ld32(taddr + cc, v);
+                tmem_ld_wait();
+                const int col = col0 + cc;
+                if (row < a.n && col < a.n) {
+                    float *cp = C + (int64_t)row * a.n + col;
+                    if (col + 31 < a.n && (reinterpret_cast<uintptr_t>(cp) & 15) == 0) {
+#pragma unroll
+                        for (int q = 0; q < 8; ++q) {
+                            float4 c4 = *reinterpret_cast<float4 *>(cp + 4 * q);
+                            c4.x = fmaf(__uint_as_float(v[4 * q + 0]), inv, c4.x);
+                            c4.y = fmaf(__uint_as_float(v[4 * q + 1]), inv, c4.y);
+                            c4.z = fmaf(__uint_as_float(v[4 * q + 2]), inv, c4.z);
+                            c4.w = fmaf(__uint_as_float(v[4 * q + 3]), inv, c4.w);
+                            *reinterpret_cast<float4 *>(cp + 4 * q) = c4;
+                        }
+                    } else {
+#pragma unroll
+                        for (int q = 0; q < 32; ++q)
+                            if (col + q < a.n) cp[q] = fmaf(__uint_as_float(v[q]), inv, cp[q]);
+                    }
+                }
+            }
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(tempty_bar(buf));
+            ++tcount;
+            it.left = gridDim.x;
+        }
+    }
+
+    tc_fence_before();
+    __syncthreads();
+    if (*abort_flag && threadIdx.x == 0) record_status(a.hd, ST_TIMEOUT, blockIdx.x);
+    if (warp == 1) {
+        tc_fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(512u) : "memory");
+    }
+}
+
+}  // namespace gptaq

@@ -200,3 +200,48 @@ def test_dead_inputs():
         X[:, 100] = 0.0
     out = hp.check_layer(cfg, W, bt)
     hp.assert_parity(out)
+
+
+def _stats_only(cfg, bt, precision, scale=1.0):
+    st = g.LayerState(cfg.n, 8, cfg.batch_tokens, cfg.blocksize)
+    g.gptaq_set_stats_precision(st.handle, precision)
+    for X, Xfp in bt:
+        g.gptaq_accumulate(st.handle, (X * scale).cuda(), (Xfp * scale).cuda())
+    assert g.gptaq_sync_status(st.handle)[0] == g.GPTAQ_OK
+    H = st.H().cpu().numpy().astype(np.float64)
+    D = st.D().cpu().numpy().astype(np.float64)
+    st.close()
+    return H, D
+
+
+@pytest.mark.parametrize("n,tokens,nb", [(256, 64, 1), (384, 1000, 2), (1024, 4112, 2), (2052, 777, 1)])
+def test_tensor_core_statistics_against_oracle(n, tokens, nb):
+    """fp16 tensor-core sums vs float64: elementwise error bounded by the fp16 rounding
+    of the operands (2^-11 relative per factor) times sqrt(H_ii H_jj)."""
+    cfg = wl.scaled(wl.CONFIGS["cfg2"], name="stats", n=n, m=8, batch_tokens=tokens, n_batches=nb,
+                    outlier_channels=max(1, n // 100))
+    bt = batches_of(cfg)
+    so = hp.oracle_stats(cfg, bt)
+    iu = np.triu_indices(n)
+    d = np.sqrt(np.diag(so.H))
+    for prec, tol in ((g.GPTAQ_STATS_FP16_TENSOR, 2.0 ** -10), (g.GPTAQ_STATS_FP32, 1e-5)):
+        H, D = _stats_only(cfg, bt, prec)
+        errH = np.abs(H - so.H)[iu] / np.outer(d, d)[iu]
+        assert errH.max() < tol, (prec, errH.max())
+        # dXX^T: bound with the norms of the delta rows
+        dd = np.sqrt(np.diag(so.G))
+        errD = np.abs(D - so.D) / np.outer(dd, d)
+        assert errD.max() < tol, (prec, errD.max())
+        assert hp.rel_fro(D, so.D) < tol and np.linalg.norm((H - so.H)[iu]) / np.linalg.norm(so.H[iu]) < tol
+
+
+@pytest.mark.parametrize("scale", [3e5, 1e-7])
+def test_tensor_core_statistics_rescale_out_of_range_batches(scale):
+    cfg = wl.scaled(wl.CONFIGS["cfg2"], name="stats", n=512, m=8, batch_tokens=640, n_batches=1, outlier_channels=5)
+    bt = batches_of(cfg)
+    H, D = _stats_only(cfg, bt, g.GPTAQ_STATS_FP16_TENSOR, scale)
+    so = hp.oracle_stats(cfg, [(X * scale, Xfp * scale) for X, Xfp in bt])
+    iu = np.triu_indices(cfg.n)
+    assert np.isfinite(H).all() and np.isfinite(D).all()
+    assert np.linalg.norm((H - so.H)[iu]) / np.linalg.norm(so.H[iu]) < 2.0 ** -10
+    assert hp.rel_fro(D, so.D) < 2.0 ** -10
