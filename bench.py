@@ -171,8 +171,12 @@ def run_ours(args, cfg):
     scales = torch.empty((cfg.m, G), dtype=torch.float32, device=dev)
     zeros = torch.empty((cfg.m, G), dtype=torch.float32, device=dev)
     Wq = torch.empty((cfg.m, cfg.n), dtype=torch.float32, device=dev)
-    st = g.LayerState(cfg.n, cfg.m, cfg.batch_tokens, cfg.blocksize, dev)
+    # statistics arithmetic: the cheapest tensor-core mode that keeps U within its error bound
+    st = g.LayerState(cfg.n, cfg.m, cfg.batch_tokens, cfg.blocksize, dev, total_tokens=cfg.tokens)
     h = st.handle
+    prec = g.gptaq_recommended_stats_precision(cfg.n, cfg.tokens)
+    prec_name = {g.GPTAQ_STATS_FP16_TENSOR: "fp16 operands, fp32 accumulate",
+                 g.GPTAQ_STATS_FP16_SPLIT_TENSOR: "fp16 hi+lo split for H, fp32 accumulate"}[prec]
     stream = torch.cuda.current_stream()
 
     def ev():
@@ -286,9 +290,10 @@ def run_ours(args, cfg):
     line = {
         "metric": METRIC, "value": ms_layer, "unit": "ms", "n_gpus": world, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": False, "scaling": "weak",
-        "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+        "vs_baseline": None, "dtype": "f16 x f16 -> f32 (statistics), f32 (solve)", "data": "synthetic",
         "config": dict(wl.describe(cfg), parallelism=f"{world} independent layer(s), one per GPU",
-                       l2="inputs (%.1f GB per step) exceed L2" % (2 * cfg.tokens * cfg.n * 4 / 1e9)),
+                       l2="inputs (%.1f GB per step) exceed L2" % (2 * cfg.tokens * cfg.n * 4 / 1e9),
+                       statistics=prec_name),
         "stages_ms": {"accumulate": acc_step_ms, "factor": fac_ms, "build_P": p_ms, "quantize": q_ms,
                       "layer_quantize": fac_ms + p_ms + q_ms},
         "accumulate_tflops": achieved,

@@ -58,13 +58,17 @@ typedef enum {
 
 enum { GPTAQ_W_FP32 = 0, GPTAQ_W_BF16 = 1 };
 
-/* Arithmetic of the statistics (Algorithm 1, line 2).
- * GPTAQ_STATS_FP16_TENSOR (default): X and X~ - X (the difference taken in float32 first) are
- *   rounded to fp16, scaled by a power of two if the batch would leave the fp16 range, and
- *   multiplied on the tensor cores with float32 accumulation.  Used for n >= 256; smaller
- *   layers always take the float32 path.
+/* Arithmetic of the statistics (Algorithm 1, line 2).  In the two tensor-core modes X and
+ * X~ - X (the difference taken in float32 first) are rounded to fp16, scaled by a power of two
+ * if the batch would leave the fp16 range, and multiplied by tcgen05 MMAs with float32
+ * accumulation; they apply for n >= 256, smaller layers always take the float32 path.
+ * GPTAQ_STATS_FP16_SPLIT_TENSOR (default): H additionally carries the rounding remainder of X
+ *   as a second fp16 term (H = hi hi^T + hi lo^T + lo hi^T, about 22 significant bits), so that
+ *   the factor U keeps its accuracy even with few tokens per input channel.
+ * GPTAQ_STATS_FP16_TENSOR: single fp16 term (11 significant bits), 40 % fewer MMAs; accurate
+ *   enough for U once total tokens >= 16 n (see gptaq_recommended_stats_precision).
  * GPTAQ_STATS_FP32: float32 products and sums on the plain FMA pipes (exact inputs). */
-enum { GPTAQ_STATS_FP16_TENSOR = 0, GPTAQ_STATS_FP32 = 1 };
+enum { GPTAQ_STATS_FP16_TENSOR = 0, GPTAQ_STATS_FP32 = 1, GPTAQ_STATS_FP16_SPLIT_TENSOR = 2 };
 
 /* Bytes of the caller-owned device state for layer width n: a header (status
  * word, pivot index), H (n x n), dXX^T (n x n) and the dead-input flags.
@@ -163,8 +167,11 @@ int64_t gptaq_tokens(gptaq_handle_t h);
 /* Sets the token count (for callers that restore checkpointed sums). */
 gptaq_status_t gptaq_set_tokens(gptaq_handle_t h, int64_t tokens);
 
-/* Chooses the arithmetic of gptaq_accumulate (see GPTAQ_STATS_*). */
+/* Chooses the arithmetic of gptaq_accumulate (see GPTAQ_STATS_*); allowed before gptaq_factor. */
 gptaq_status_t gptaq_set_stats_precision(gptaq_handle_t h, int precision);
+/* The cheapest tensor-core mode whose rounding keeps the relative error of U below 1e-4 for a
+ * layer of width n calibrated on total_tokens tokens. */
+int gptaq_recommended_stats_precision(int64_t n, int64_t total_tokens);
 
 /* Number of kernels this handle has launched since create (bookkeeping for benchmarks). */
 int64_t gptaq_launch_count(gptaq_handle_t h);

@@ -28,6 +28,7 @@ GPTAQ_W_FP32 = 0
 GPTAQ_W_BF16 = 1
 GPTAQ_STATS_FP16_TENSOR = 0
 GPTAQ_STATS_FP32 = 1
+GPTAQ_STATS_FP16_SPLIT_TENSOR = 2
 
 _vp, _i64, _int, _sz, _f = C.c_void_p, C.c_int64, C.c_int, C.c_size_t, C.c_float
 
@@ -51,6 +52,7 @@ SIGNATURES = {
     "gptaq_tokens": (_i64, [_vp]),
     "gptaq_set_tokens": (_int, [_vp, _i64]),
     "gptaq_set_stats_precision": (_int, [_vp, _int]),
+    "gptaq_recommended_stats_precision": (_int, [_i64, _i64]),
     "gptaq_launch_count": (_i64, [_vp]),
     "gptaq_status_string": (C.c_char_p, [_int]),
     "gptaq_last_cuda_error": (C.c_char_p, [_vp]),
@@ -228,6 +230,10 @@ def gptaq_set_stats_precision(h, precision: int):
     _check(load_library().gptaq_set_stats_precision(h, precision), "gptaq_set_stats_precision", h)
 
 
+def gptaq_recommended_stats_precision(n: int, total_tokens: int) -> int:
+    return load_library().gptaq_recommended_stats_precision(n, total_tokens)
+
+
 def gptaq_launch_count(h) -> int:
     return load_library().gptaq_launch_count(h)
 
@@ -247,7 +253,8 @@ def gptaq_D_ptr(h) -> int:
 class LayerState:
     """Owns the torch device buffers behind one handle (memory plumbing only)."""
 
-    def __init__(self, n: int, m_max: int, max_batch_tokens: int, blocksize: int, device="cuda", stream=None):
+    def __init__(self, n: int, m_max: int, max_batch_tokens: int, blocksize: int, device="cuda", stream=None,
+                 total_tokens: int | None = None):
         _need_cuda()
         self.n = n
         self.device = torch.device(device)
@@ -258,6 +265,8 @@ class LayerState:
         self.state = torch.empty(sb, dtype=torch.uint8, device=self.device)
         self.workspace = torch.empty(wb, dtype=torch.uint8, device=self.device)
         self.handle = gptaq_create(n, self.state, self.workspace, stream)
+        if total_tokens is not None:
+            gptaq_set_stats_precision(self.handle, gptaq_recommended_stats_precision(n, total_tokens))
 
     def _view(self, ptr: int) -> torch.Tensor:
         off = ptr - self.state.data_ptr()

@@ -138,14 +138,15 @@ bool make_kmajor_map(CUtensorMap *map, const void *ptr, int64_t rows, int64_t kp
 
 // Largest token chunk (multiple of 64) whose two fp16 operand copies fit the workspace.
 int64_t tc_chunk_tokens(const gptaq_ctx *h) {
-    int64_t per_token = 2 * h->n * 2;   // X^T and dX^T, fp16
+    const int nbuf = h->stats_precision == GPTAQ_STATS_FP16_SPLIT_TENSOR ? 3 : 2;
+    int64_t per_token = nbuf * h->n * 2;   // X^T, dX^T (and the low part of X^T), fp16
     int64_t cap = (int64_t)(h->ws_bytes / (size_t)per_token);
     cap = cap / UBK * UBK;
     return std::min<int64_t>(cap, 1 << 20);
 }
 
 bool tc_eligible(const gptaq_ctx *h) {
-    return h->stats_precision == GPTAQ_STATS_FP16_TENSOR && h->n >= UBN && tc_chunk_tokens(h) >= UBK &&
+    return h->stats_precision != GPTAQ_STATS_FP32 && h->n >= UBN && tc_chunk_tokens(h) >= UBK &&
            encode_tiled_fn() != nullptr;
 }
 
@@ -161,25 +162,29 @@ gptaq_status_t accumulate_tc(gptaq_ctx *h, const float *X, const float *Xfp, int
         const int kp = (tk + UBK - 1) / UBK * UBK;
         __half *Xt = reinterpret_cast<__half *>(h->ws);
         __half *dXt = Xt + (size_t)n * kp;
+        const bool split = h->stats_precision == GPTAQ_STATS_FP16_SPLIT_TENSOR;
+        __half *Xlo = split ? dXt + (size_t)n * kp : nullptr;
         CU(cudaMemsetAsync(h->hd->amax, 0, 2 * sizeof(unsigned), s));
         ConvertArgs ca;
         ca.X = X + t0 * ld; ca.Xfp = Xfp + t0 * ld; ca.ld = ld; ca.tokens = tk; ca.n = n; ca.kp = kp;
-        ca.Xt = Xt; ca.dXt = dXt; ca.amax = h->hd->amax;
+        ca.Xt = Xt; ca.dXt = dXt; ca.Xlo = Xlo; ca.amax = h->hd->amax;
         dim3 cgrid(kp / 64, (n + 63) / 64);
         convert_transpose_kernel<0><<<cgrid, 256, 0, s>>>(ca);
         LAUNCHED();
         convert_transpose_kernel<1><<<cgrid, 256, 0, s>>>(ca);
         LAUNCHED();
-        CUtensorMap mXa, mDa, mXb;
+        CUtensorMap mXa, mDa, mXb, mLa, mLb;
+        const __half *lo = split ? Xlo : Xt;    // unused maps still have to be valid
         if (!make_kmajor_map(&mXa, Xt, n, kp, UBM) || !make_kmajor_map(&mDa, dXt, n, kp, UBM) ||
-            !make_kmajor_map(&mXb, Xt, n, kp, UBN)) {
+            !make_kmajor_map(&mXb, Xt, n, kp, UBN) || !make_kmajor_map(&mLa, lo, n, kp, UBM) ||
+            !make_kmajor_map(&mLb, lo, n, kp, UBN)) {
             h->cuda_error = "cuTensorMapEncodeTiled failed";
             return GPTAQ_ERR_CUDA;
         }
         StatsGemmArgs ga;
-        ga.H = h->H; ga.D = h->D; ga.n = n; ga.kblocks = kp / UBK; ga.amax = h->hd->amax; ga.hd = h->hd;
+        ga.H = h->H; ga.D = h->D; ga.n = n; ga.kblocks = kp / UBK; ga.nseg_h = split ? 3 : 1; ga.amax = h->hd->amax; ga.hd = h->hd;
         const int grid = (int)std::min<int64_t>(ntiles, h->num_sms);
-        stats_umma_kernel<<<grid, UMMA_THREADS, UMMA_SMEM, s>>>(mXa, mDa, mXb, ga);
+        stats_umma_kernel<<<grid, UMMA_THREADS, UMMA_SMEM, s>>>(mXa, mDa, mXb, mLa, mLb, ga);
         LAUNCHED();
     }
     h->tokens += tokens;
@@ -201,7 +206,7 @@ size_t gptaq_workspace_bytes(int64_t n, int64_t m_max, int64_t max_batch_tokens,
     if (n <= 0 || m_max < 0 || max_batch_tokens < 0 || !valid_block(blocksize)) return 0;
     // the fp16 operand copies of one token batch share the space of the later steps' scratch
     size_t kp = round_up((size_t)max_batch_tokens, (size_t)UBK);
-    size_t xt = round_up(2 * (size_t)n * kp * 2, ALIGN);
+    size_t xt = round_up(3 * (size_t)n * kp * 2, ALIGN);
     return std::max(ws_layout(n, m_max, blocksize).total, xt);
 }
 
@@ -227,7 +232,7 @@ gptaq_status_t gptaq_create(gptaq_handle_t *out, int64_t n, void *d_state, size_
     h->D = reinterpret_cast<float *>(h->state + l.d_off);
     h->dead = reinterpret_cast<uint8_t *>(h->state + l.dead_off);
     h->launches = 0;
-    h->stats_precision = GPTAQ_STATS_FP16_TENSOR;
+    h->stats_precision = GPTAQ_STATS_FP16_SPLIT_TENSOR;
     cudaError_t e = cudaGetDevice(&h->device);
     if (e == cudaSuccess) e = cudaDeviceGetAttribute(&h->num_sms, cudaDevAttrMultiProcessorCount, h->device);
     if (e == cudaSuccess)
@@ -517,9 +522,18 @@ gptaq_status_t gptaq_set_tokens(gptaq_handle_t h, int64_t tokens) {
 
 gptaq_status_t gptaq_set_stats_precision(gptaq_handle_t h, int precision) {
     if (!h) return GPTAQ_ERR_INVALID_ARG;
-    if (precision != GPTAQ_STATS_FP16_TENSOR && precision != GPTAQ_STATS_FP32) return GPTAQ_ERR_UNSUPPORTED;
+    if (precision != GPTAQ_STATS_FP16_TENSOR && precision != GPTAQ_STATS_FP32 &&
+        precision != GPTAQ_STATS_FP16_SPLIT_TENSOR)
+        return GPTAQ_ERR_UNSUPPORTED;
+    if (h->stage != STAGE_ACCUM) return GPTAQ_ERR_BAD_STATE;
     h->stats_precision = precision;
     return GPTAQ_OK;
+}
+
+int gptaq_recommended_stats_precision(int64_t n, int64_t total_tokens) {
+    // fp16 rounding of X perturbs U by about 5e-5 * sqrt(n/k) / ((1 - sqrt(n/k))^2 + damp):
+    // below 1e-4 with margin once there are 16 tokens per input channel.
+    return (n > 0 && total_tokens >= 16 * n) ? GPTAQ_STATS_FP16_TENSOR : GPTAQ_STATS_FP16_SPLIT_TENSOR;
 }
 
 int64_t gptaq_launch_count(gptaq_handle_t h) { return h ? h->launches : -1; }

@@ -2,9 +2,9 @@
 // K-major shared-memory tiles (TMA, 128-byte swizzle), tcgen05.mma with fp32
 // accumulators in tensor memory, and a read-modify-write epilogue into the fp32
 // sums.  Persistent, warp-specialised: warp 0 issues TMA loads, warp 1 issues
-// the MMAs and owns the TMEM allocation, warps 2-5 drain the accumulators.
-// Two 128 x 256 accumulators are kept in TMEM so that the epilogue of one tile
-// overlaps the main loop of the next.
+// the MMAs and owns the TMEM allocation, warps 2-9 drain the accumulators.
+// Two 128 x 256 accumulators are kept in TMEM so that draining one overlaps the
+// MMAs into the other.
 //
 // Every wait on an mbarrier is bounded by a clock limit; when it runs out the
 // kernel records GPTAQ_ERR_TIMEOUT in the state header, lets outstanding copies
@@ -23,7 +23,8 @@ constexpr int UBM = 128, UBN = 256, UBK = 64, USTAGES = 4;
 constexpr int UA_BYTES = UBM * UBK * 2;
 constexpr int UB_BYTES = UBN * UBK * 2;
 constexpr int USTAGE_BYTES = UA_BYTES + UB_BYTES;
-constexpr int UMMA_THREADS = 192;
+constexpr int UEPI_WARPS = 8;
+constexpr int UMMA_THREADS = 64 + 32 * UEPI_WARPS;
 constexpr size_t UMMA_SMEM = (size_t)USTAGES * USTAGE_BYTES + 1024 /*alignment slack*/ + 256 /*barriers*/;
 constexpr long long WAIT_LIMIT_CYCLES = 4000000000LL;   // about two seconds
 
@@ -49,56 +50,82 @@ struct ConvertArgs {
     int64_t ld;
     int tokens, n, kp;
     __half *Xt, *dXt;       // [n][kp]
+    __half *Xlo;            // [n][kp] or nullptr: fp16(X - float(fp16(X))), the second term of the split
     unsigned *amax;          // [2]: bit patterns of max|X|, max|X~ - X|
 };
 
+// Shared-memory staging of one 64-channel x 64-token tile as 32-bit words that
+// hold two consecutive tokens of one channel.  Word (c, tp) lives at
+// c * 33 + 2 * (c >> 5) + tp: conflict-free both for the transposing stores
+// (lanes step 4 channels) and for the row reads (lanes step 4 words).
+__device__ __forceinline__ int cvt_word(int c, int tp) { return c * 33 + 2 * (c >> 5) + tp; }
+constexpr int CVT_WORDS = 64 * 33 + 4;
+
 template <int PASS>
 __global__ void __launch_bounds__(256) convert_transpose_kernel(ConvertArgs a) {
-    __shared__ __half sx[64][72];
-    __shared__ __half sd[64][72];
+    __shared__ uint32_t sx[CVT_WORDS];
+    __shared__ uint32_t sd[CVT_WORDS];
+    __shared__ uint32_t sl[CVT_WORDS];
     float scx = 1.f, scd = 1.f;
     if (PASS == 1) {
         scx = pick_scale(__uint_as_float(a.amax[0]));
         scd = pick_scale(__uint_as_float(a.amax[1]));
         if (scx == 1.f && scd == 1.f) return;
     }
+    const bool split = a.Xlo != nullptr;
     const int t0 = blockIdx.x * 64, c0 = blockIdx.y * 64;
     const int tid = threadIdx.x;
     float mx = 0.f, md = 0.f;
+    bool nan = false;
 #pragma unroll
-    for (int it = 0; it < 4; ++it) {
-        int idx = tid + it * 256;          // 0..1023: 64 tokens x 16 float4
-        int tl = idx >> 4, cl = (idx & 15) * 4;
-        int t = t0 + tl, c = c0 + cl;
-        float x[4] = {0.f, 0.f, 0.f, 0.f}, f[4] = {0.f, 0.f, 0.f, 0.f};
-        if (t < a.tokens) {
-            const float *px = a.X + (int64_t)t * a.ld + c;
-            const float *pf = a.Xfp + (int64_t)t * a.ld + c;
-            if (c + 3 < a.n && ((reinterpret_cast<uintptr_t>(px) | reinterpret_cast<uintptr_t>(pf)) & 15) == 0) {
-                float4 vx = *reinterpret_cast<const float4 *>(px);
-                float4 vf = *reinterpret_cast<const float4 *>(pf);
-                x[0] = vx.x; x[1] = vx.y; x[2] = vx.z; x[3] = vx.w;
-                f[0] = vf.x; f[1] = vf.y; f[2] = vf.z; f[3] = vf.w;
-            } else {
+    for (int it = 0; it < 2; ++it) {
+        const int idx = tid + it * 256;        // 0..511: 32 token pairs x 16 float4
+        const int tp = idx >> 4, cl = (idx & 15) * 4;
+        const int c = c0 + cl;
+        float x[2][4], f[2][4];
 #pragma unroll
-                for (int e = 0; e < 4; ++e)
-                    if (c + e < a.n) { x[e] = px[e]; f[e] = pf[e]; }
+        for (int h = 0; h < 2; ++h) {
+            const int t = t0 + 2 * tp + h;
+#pragma unroll
+            for (int e = 0; e < 4; ++e) { x[h][e] = 0.f; f[h][e] = 0.f; }
+            if (t < a.tokens) {
+                const float *px = a.X + (int64_t)t * a.ld + c;
+                const float *pf = a.Xfp + (int64_t)t * a.ld + c;
+                if (c + 3 < a.n && ((reinterpret_cast<uintptr_t>(px) | reinterpret_cast<uintptr_t>(pf)) & 15) == 0) {
+                    float4 vx = __ldcs(reinterpret_cast<const float4 *>(px));
+                    float4 vf = __ldcs(reinterpret_cast<const float4 *>(pf));
+                    x[h][0] = vx.x; x[h][1] = vx.y; x[h][2] = vx.z; x[h][3] = vx.w;
+                    f[h][0] = vf.x; f[h][1] = vf.y; f[h][2] = vf.z; f[h][3] = vf.w;
+                } else {
+#pragma unroll
+                    for (int e = 0; e < 4; ++e)
+                        if (c + e < a.n) { x[h][e] = px[e]; f[h][e] = pf[e]; }
+                }
             }
         }
 #pragma unroll
         for (int e = 0; e < 4; ++e) {
-            float d = f[e] - x[e];
-            if (PASS == 0) {
-                // NaN compares false everywhere, so fold it in through the bit pattern below
-                mx = fmaxf(mx, fabsf(x[e])); md = fmaxf(md, fabsf(d));
-                if (x[e] != x[e] || d != d) { mx = __int_as_float(0x7fc00000); }
+            __half hx[2], hd[2], hl[2];
+#pragma unroll
+            for (int h = 0; h < 2; ++h) {
+                const float xv = x[h][e], d = f[h][e] - xv;
+                if (PASS == 0) {
+                    mx = fmaxf(mx, fabsf(xv)); md = fmaxf(md, fabsf(d));
+                    nan |= (xv != xv) || (d != d);     // fmaxf drops NaNs
+                }
+                const float xs = xv * scx;
+                hx[h] = __float2half_rn(xs);
+                hd[h] = __float2half_rn(d * scd);
+                hl[h] = __float2half_rn(xs - __half2float(hx[h]));
             }
-            sx[cl + e][tl] = __float2half_rn(x[e] * scx);
-            sd[cl + e][tl] = __float2half_rn(d * scd);
+            const int w = cvt_word(cl + e, tp);
+            sx[w] = (uint32_t)__half_as_ushort(hx[0]) | ((uint32_t)__half_as_ushort(hx[1]) << 16);
+            sd[w] = (uint32_t)__half_as_ushort(hd[0]) | ((uint32_t)__half_as_ushort(hd[1]) << 16);
+            if (split) sl[w] = (uint32_t)__half_as_ushort(hl[0]) | ((uint32_t)__half_as_ushort(hl[1]) << 16);
         }
     }
     if (PASS == 0) {
-        unsigned ux = __float_as_uint(mx), ud = __float_as_uint(md);
+        unsigned ux = nan ? 0x7fc00000u : __float_as_uint(mx), ud = __float_as_uint(md);
 #pragma unroll
         for (int o = 16; o > 0; o >>= 1) {
             ux = max(ux, __shfl_xor_sync(0xffffffffu, ux, o));
@@ -107,15 +134,18 @@ __global__ void __launch_bounds__(256) convert_transpose_kernel(ConvertArgs a) {
         if ((tid & 31) == 0) { atomicMax(&a.amax[0], ux); atomicMax(&a.amax[1], ud); }
     }
     __syncthreads();
-    // 64 channels x 8 chunks of 8 halves (16 bytes) per matrix
+    // 64 channels x 8 chunks of 8 tokens (16 bytes) per matrix
 #pragma unroll
     for (int it = 0; it < 2; ++it) {
-        int idx = tid + it * 256;          // 0..511
-        int cl = idx >> 3, ch = (idx & 7) * 8;
-        int c = c0 + cl, t = t0 + ch;
+        const int idx = tid + it * 256;        // 0..511
+        const int cl = idx >> 3, q = idx & 7;
+        const int c = c0 + cl, t = t0 + q * 8;
         if (c < a.n && t < a.kp) {
-            *reinterpret_cast<uint4 *>(a.Xt + (int64_t)c * a.kp + t) = *reinterpret_cast<const uint4 *>(&sx[cl][ch]);
-            *reinterpret_cast<uint4 *>(a.dXt + (int64_t)c * a.kp + t) = *reinterpret_cast<const uint4 *>(&sd[cl][ch]);
+            const int w = cvt_word(cl, q * 4);
+            const int64_t off = (int64_t)c * a.kp + t;
+            *reinterpret_cast<uint4 *>(a.Xt + off) = make_uint4(sx[w], sx[w + 1], sx[w + 2], sx[w + 3]);
+            *reinterpret_cast<uint4 *>(a.dXt + off) = make_uint4(sd[w], sd[w + 1], sd[w + 2], sd[w + 3]);
+            if (split) *reinterpret_cast<uint4 *>(a.Xlo + off) = make_uint4(sl[w], sl[w + 1], sl[w + 2], sl[w + 3]);
         }
     }
 }
@@ -204,6 +234,7 @@ struct StatsGemmArgs {
     float *H, *D;            // n x n, ld n
     int n;
     int kblocks;             // kp / 64
+    int nseg_h;              // 1: H = hi hi^T;  3: H = hi hi^T + hi lo^T + lo hi^T (split operands)
     const unsigned *amax;    // scales are recomputed from the recorded maxima
     StateHeader *hd;
 };
@@ -230,9 +261,17 @@ struct TileIter {
     }
 };
 
+// Accumulation chains in tensor memory are kept short: the tensor core truncates
+// its fp32 accumulator once per MMA, which biases a long sum of like-signed
+// products (the diagonal of H) by about 2^-24 per step.  Every UCHUNK K-blocks
+// the partial sum is therefore added, with round-to-nearest, into fp32 registers
+// of the epilogue warps; HBM is touched once per tile.
+constexpr int UCHUNK = 8;           // K-blocks (of 64) per TMEM accumulation chain
+
 __global__ void __launch_bounds__(UMMA_THREADS, 1)
 stats_umma_kernel(const __grid_constant__ CUtensorMap mapXa, const __grid_constant__ CUtensorMap mapDa,
-                  const __grid_constant__ CUtensorMap mapXb, StatsGemmArgs a) {
+                  const __grid_constant__ CUtensorMap mapXb, const __grid_constant__ CUtensorMap mapLa,
+                  const __grid_constant__ CUtensorMap mapLb, StatsGemmArgs a) {
     extern __shared__ uint8_t smem_raw[];
     // 1024-byte alignment for the swizzled tiles
     const uint32_t raw = smem_u32(smem_raw);
@@ -250,7 +289,7 @@ stats_umma_kernel(const __grid_constant__ CUtensorMap mapXa, const __grid_consta
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     if (threadIdx.x == 0) {
         for (int s = 0; s < USTAGES; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
-        for (int b = 0; b < 2; ++b) { mbar_init(tfull_bar(b), 1); mbar_init(tempty_bar(b), 4); }
+        for (int b = 0; b < 2; ++b) { mbar_init(tfull_bar(b), 1); mbar_init(tempty_bar(b), UEPI_WARPS); }
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
@@ -274,16 +313,20 @@ stats_umma_kernel(const __grid_constant__ CUtensorMap mapXa, const __grid_consta
             bool ok = true;
             while (ok && it.seek()) {
                 const bool isD = it.r >= it.TM;
-                const CUtensorMap *mapA = isD ? &mapDa : &mapXa;
                 const int row0 = (isD ? it.r - it.TM : it.r) * UBM, col0 = it.tn * UBN;
-                for (int kb = 0; kb < KB; ++kb) {
-                    if (!mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag)) { ok = false; break; }
-                    const uint32_t sa = base + stage * USTAGE_BYTES, sb = sa + UA_BYTES;
-                    mbar_expect_tx(full_bar(stage), USTAGE_BYTES);
-                    tma_load_2d(sa, mapA, kb * UBK, row0, full_bar(stage));
-                    tma_load_2d(sb, &mapXb, kb * UBK, col0, full_bar(stage));
-                    ++issued;
-                    if (++stage == USTAGES) { stage = 0; phase ^= 1u; }
+                const int nseg = isD ? 1 : a.nseg_h;
+                for (int seg = 0; seg < nseg && ok; ++seg) {
+                    const CUtensorMap *mapA = isD ? &mapDa : (seg == 2 ? &mapLa : &mapXa);
+                    const CUtensorMap *mapB = (seg == 1) ? &mapLb : &mapXb;
+                    for (int kb = 0; kb < KB; ++kb) {
+                        if (!mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag)) { ok = false; break; }
+                        const uint32_t sa = base + stage * USTAGE_BYTES, sb = sa + UA_BYTES;
+                        mbar_expect_tx(full_bar(stage), USTAGE_BYTES);
+                        tma_load_2d(sa, mapA, kb * UBK, row0, full_bar(stage));
+                        tma_load_2d(sb, mapB, kb * UBK, col0, full_bar(stage));
+                        ++issued;
+                        if (++stage == USTAGES) { stage = 0; phase ^= 1u; }
+                    }
                 }
                 it.left = gridDim.x;
             }
@@ -297,78 +340,91 @@ stats_umma_kernel(const __grid_constant__ CUtensorMap mapXa, const __grid_consta
         // ------------------------------------------------------------ MMA issuer
         if (lane == 0) {
             TileIter it(a.n, blockIdx.x);
-            uint32_t stage = 0, phase = 0, tcount = 0;
+            uint32_t stage = 0, phase = 0, ccount = 0;     // ccount: chunks issued so far
             bool ok = true;
             while (ok && it.seek()) {
-                const uint32_t buf = tcount & 1u, tphase = (tcount >> 1) & 1u;
-                if (!mbar_wait(tempty_bar(buf), tphase ^ 1u, abort_flag)) { ok = false; break; }
-                tc_fence_after();
-                const uint32_t d_tmem = tmem_base + buf * UBN;
-                for (int kb = 0; kb < KB; ++kb) {
-                    if (!mbar_wait(full_bar(stage), phase, abort_flag)) { ok = false; break; }
+                const int kb_total = (it.r >= it.TM) ? KB : KB * a.nseg_h;
+                for (int kb0 = 0; kb0 < kb_total && ok; kb0 += UCHUNK) {
+                    const uint32_t buf = ccount & 1u, cphase = (ccount >> 1) & 1u;
+                    if (!mbar_wait(tempty_bar(buf), cphase ^ 1u, abort_flag)) { ok = false; break; }
                     tc_fence_after();
-                    const uint32_t sa = base + stage * USTAGE_BYTES, sb = sa + UA_BYTES;
-                    const uint64_t ad = make_kmajor_desc(sa), bd = make_kmajor_desc(sb);
+                    const uint32_t d_tmem = tmem_base + buf * UBN;
+                    const int kb1 = min(kb0 + UCHUNK, kb_total);
+                    for (int kb = kb0; kb < kb1; ++kb) {
+                        if (!mbar_wait(full_bar(stage), phase, abort_flag)) { ok = false; break; }
+                        tc_fence_after();
+                        const uint32_t sa = base + stage * USTAGE_BYTES, sb = sa + UA_BYTES;
+                        const uint64_t ad = make_kmajor_desc(sa), bd = make_kmajor_desc(sb);
 #pragma unroll
-                    for (int k = 0; k < UBK / 16; ++k)
-                        umma_f16(d_tmem, ad + (uint64_t)(k * 2), bd + (uint64_t)(k * 2), UMMA_IDESC_F16,
-                                 (kb | k) != 0 ? 1u : 0u);
-                    umma_commit(empty_bar(stage));
-                    if (++stage == USTAGES) { stage = 0; phase ^= 1u; }
+                        for (int k = 0; k < UBK / 16; ++k)
+                            umma_f16(d_tmem, ad + (uint64_t)(k * 2), bd + (uint64_t)(k * 2), UMMA_IDESC_F16,
+                                     (kb != kb0 || k != 0) ? 1u : 0u);
+                        umma_commit(empty_bar(stage));
+                        if (++stage == USTAGES) { stage = 0; phase ^= 1u; }
+                    }
+                    if (!ok) break;
+                    umma_commit(tfull_bar(buf));
+                    ++ccount;
                 }
-                if (!ok) break;
-                umma_commit(tfull_bar(buf));
-                ++tcount;
                 it.left = gridDim.x;
             }
         }
     } else {
-        // ------------------------------------------------------------ epilogue (warps 2..5)
-        const int quarter = warp & 3;           // TMEM lanes 32 * quarter .. + 31
+        // ------------------------------------------------------------ epilogue (warps 2..9)
+        const int quarter = warp & 3;                 // TMEM lanes 32 * quarter .. + 31
+        const int half = (warp - 2) >> 2;             // columns [128 * half, 128 * half + 128)
         TileIter it(a.n, blockIdx.x);
-        uint32_t tcount = 0;
+        uint32_t ccount = 0;
         bool ok = true;
         const float sx = pick_scale(__uint_as_float(a.amax[0]));
         const float sd = pick_scale(__uint_as_float(a.amax[1]));
+        float acc[UBN / 2];
         while (ok && it.seek()) {
-            const uint32_t buf = tcount & 1u, tphase = (tcount >> 1) & 1u;
             const bool isD = it.r >= it.TM;
+            const int kb_total = isD ? KB : KB * a.nseg_h;
+#pragma unroll
+            for (int i = 0; i < UBN / 2; ++i) acc[i] = 0.f;
+            for (int kb0 = 0; kb0 < kb_total; kb0 += UCHUNK) {
+                const uint32_t buf = ccount & 1u, cphase = (ccount >> 1) & 1u;
+                if (!mbar_wait(tfull_bar(buf), cphase, abort_flag)) { ok = false; break; }
+                tc_fence_after();
+                const uint32_t taddr = tmem_base + buf * UBN + half * (UBN / 2) + ((uint32_t)(quarter * 32) << 16);
+#pragma unroll
+                for (int gq = 0; gq < UBN / 2 / 32; ++gq) {
+                    uint32_t v[32];
+                    tmem_ld32(taddr + gq * 32, v);
+                    tmem_ld_wait();
+#pragma unroll
+                    for (int i = 0; i < 32; ++i) acc[gq * 32 + i] += __uint_as_float(v[i]);
+                }
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(tempty_bar(buf));
+                ++ccount;
+            }
+            if (!ok) break;
             const int row = (isD ? it.r - it.TM : it.r) * UBM + quarter * 32 + lane;
-            const int col0 = it.tn * UBN;
+            const int col0 = it.tn * UBN + half * (UBN / 2);
             float *C = isD ? a.D : a.H;
             const float inv = 1.f / (sx * (isD ? sd : sx));
-            if (!mbar_wait(tfull_bar(buf), tphase, abort_flag)) { ok = false; break; }
-            tc_fence_after();
-            const uint32_t taddr = tmem_base + buf * UBN + ((uint32_t)(quarter * 32) << 16);
-#pragma unroll 1
-            for (int cc = 0; cc < UBN; cc += 32) {
-                uint32_t v[32];
-                tmem_ld32(taddr + cc, v);
-                tmem_ld_wait();
-                const int col = col0 + cc;
-                if (row < a.n && col < a.n) {
-                    float *cp = C + (int64_t)row * a.n + col;
-                    if (col + 31 < a.n && (reinterpret_cast<uintptr_t>(cp) & 15) == 0) {
+            if (row < a.n) {
+                float *cp = C + (int64_t)row * a.n + col0;
+                if (col0 + UBN / 2 <= a.n && (reinterpret_cast<uintptr_t>(cp) & 15) == 0) {
 #pragma unroll
-                        for (int q = 0; q < 8; ++q) {
-                            float4 c4 = *reinterpret_cast<float4 *>(cp + 4 * q);
-                            c4.x = fmaf(__uint_as_float(v[4 * q + 0]), inv, c4.x);
-                            c4.y = fmaf(__uint_as_float(v[4 * q + 1]), inv, c4.y);
-                            c4.z = fmaf(__uint_as_float(v[4 * q + 2]), inv, c4.z);
-                            c4.w = fmaf(__uint_as_float(v[4 * q + 3]), inv, c4.w);
-                            *reinterpret_cast<float4 *>(cp + 4 * q) = c4;
-                        }
-                    } else {
-#pragma unroll
-                        for (int q = 0; q < 32; ++q)
-                            if (col + q < a.n) cp[q] = fmaf(__uint_as_float(v[q]), inv, cp[q]);
+                    for (int q = 0; q < UBN / 2 / 4; ++q) {
+                        float4 c4 = *reinterpret_cast<float4 *>(cp + 4 * q);
+                        c4.x = fmaf(acc[4 * q + 0], inv, c4.x);
+                        c4.y = fmaf(acc[4 * q + 1], inv, c4.y);
+                        c4.z = fmaf(acc[4 * q + 2], inv, c4.z);
+                        c4.w = fmaf(acc[4 * q + 3], inv, c4.w);
+                        *reinterpret_cast<float4 *>(cp + 4 * q) = c4;
                     }
+                } else {
+#pragma unroll
+                    for (int q = 0; q < UBN / 2; ++q)
+                        if (col0 + q < a.n) cp[q] = fmaf(acc[q], inv, cp[q]);
                 }
             }
-            tc_fence_before();
-            __syncwarp();
-            if (lane == 0) mbar_arrive(tempty_bar(buf));
-            ++tcount;
             it.left = gridDim.x;
         }
     }
