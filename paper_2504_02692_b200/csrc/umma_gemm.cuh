@@ -125,13 +125,22 @@ __global__ void __launch_bounds__(256) convert_transpose_kernel(ConvertArgs a) {
         }
     }
     if (PASS == 0) {
+        // block maximum first; the shared word is only touched when it would grow
+        __shared__ unsigned bmax[2];
+        if (tid == 0) { bmax[0] = 0u; bmax[1] = 0u; }
+        __syncthreads();
         unsigned ux = nan ? 0x7fc00000u : __float_as_uint(mx), ud = __float_as_uint(md);
 #pragma unroll
         for (int o = 16; o > 0; o >>= 1) {
             ux = max(ux, __shfl_xor_sync(0xffffffffu, ux, o));
             ud = max(ud, __shfl_xor_sync(0xffffffffu, ud, o));
         }
-        if ((tid & 31) == 0) { atomicMax(&a.amax[0], ux); atomicMax(&a.amax[1], ud); }
+        if ((tid & 31) == 0) { atomicMax(&bmax[0], ux); atomicMax(&bmax[1], ud); }
+        __syncthreads();
+        if (tid == 0) {
+            if (bmax[0] > *reinterpret_cast<volatile unsigned *>(&a.amax[0])) atomicMax(&a.amax[0], bmax[0]);
+            if (bmax[1] > *reinterpret_cast<volatile unsigned *>(&a.amax[1])) atomicMax(&a.amax[1], bmax[1]);
+        }
     }
     __syncthreads();
     // 64 channels x 8 chunks of 8 tokens (16 bytes) per matrix
@@ -410,15 +419,13 @@ stats_umma_kernel(const __grid_constant__ CUtensorMap mapXa, const __grid_consta
             if (row < a.n) {
                 float *cp = C + (int64_t)row * a.n + col0;
                 if (col0 + UBN / 2 <= a.n && (reinterpret_cast<uintptr_t>(cp) & 15) == 0) {
+                    // each element belongs to exactly one CTA per launch: a reduction without
+                    // return value is a plain, order-independent "+=" that needs no round trip
 #pragma unroll
-                    for (int q = 0; q < UBN / 2 / 4; ++q) {
-                        float4 c4 = *reinterpret_cast<float4 *>(cp + 4 * q);
-                        c4.x = fmaf(acc[4 * q + 0], inv, c4.x);
-                        c4.y = fmaf(acc[4 * q + 1], inv, c4.y);
-                        c4.z = fmaf(acc[4 * q + 2], inv, c4.z);
-                        c4.w = fmaf(acc[4 * q + 3], inv, c4.w);
-                        *reinterpret_cast<float4 *>(cp + 4 * q) = c4;
-                    }
+                    for (int q = 0; q < UBN / 2 / 4; ++q)
+                        asm volatile("red.global.add.v4.f32 [%0], {%1, %2, %3, %4};" ::"l"(cp + 4 * q),
+                                     "f"(acc[4 * q + 0] * inv), "f"(acc[4 * q + 1] * inv),
+                                     "f"(acc[4 * q + 2] * inv), "f"(acc[4 * q + 3] * inv) : "memory");
                 } else {
 #pragma unroll
                     for (int q = 0; q < UBN / 2; ++q)
