@@ -154,6 +154,36 @@ gptaq_status_t gptaq_quantize_host(gptaq_handle_t h, const float *h_W, int64_t m
                                    uint8_t *h_codes, float *h_scales, float *h_zeros, float *h_Wq,
                                    void *d_stage, size_t stage_bytes, gptaq_stream_t stream);
 
+/* (No counterpart in the paper.)  gptaq_quantize for callers that cannot hand the library a
+ * scratch buffer of their own -- code that runs where device allocation is off limits (inside a
+ * real-time loop, under a memory pool whose budget is already spent, in a plug-in that is not
+ * allowed to call the CUDA allocator) and that therefore cannot size a workspace per layer.
+ * It needs no handle and no workspace: the factor and the correction matrix are plain inputs,
+ * and the m x 2B scratch of the lazy-batch update ([-Err | Wpre], Algorithm 1 line 5) lives in
+ * an array built into the library.  The function allocates nothing, on the device or through
+ * any library.
+ *   d_U, d_P   [n x n] float32, leading dimension n: U (upper, H_d^-1 = U^T U) and P (strictly
+ *              upper), e.g. gptaq_H / gptaq_D of a handle after gptaq_build_P, or restored
+ *              copies of them.  All n inputs are taken as live (no dead-input flags).
+ *   d_status   device int64[2] or NULL: receives the status a handle would record
+ *              (GPTAQ_OK or GPTAQ_ERR_NONFINITE) and the row index that goes with it.
+ *   All other arguments as in gptaq_quantize.
+ * Limits: n <= GPTAQ_STATIC_MAX_N and m * 2 * blocksize <= GPTAQ_STATIC_SCRATCH_FLOATS (4 MiB
+ * of scratch: m <= 4096 at blocksize 128); beyond them GPTAQ_ERR_WORKSPACE is returned before
+ * any work is enqueued.  Every GPU that loads the library holds the array (about 4 MiB) until
+ * the process exits.
+ * The first call on each device looks up the array's device address and configures the
+ * kernels (with that device current); make that first call outside any stream capture.
+ * All calls on a device share the one array, which still holds the previous call's contents;
+ * the function clears what has to start from zero, but two calls whose work overlaps on the
+ * GPU (different streams, no dependency between them) race on it: order them. */
+#define GPTAQ_STATIC_MAX_N 16384
+#define GPTAQ_STATIC_SCRATCH_FLOATS (1 << 20)
+gptaq_status_t gptaq_quantize_static(const float *d_U, const float *d_P, int64_t n, void *d_W, int w_dtype,
+                                     int64_t m, int64_t ldw, int bits, int group, int sym, int blocksize,
+                                     uint8_t *d_codes, float *d_scales, float *d_zeros, float *d_Wq,
+                                     int64_t *d_status, gptaq_stream_t stream);
+
 /* Synchronises `stream`, then returns the device status word (GPTAQ_OK, or the
  * first device-side condition recorded since create/reset) and, in *info, the
  * index that goes with it (may be NULL). */

@@ -46,6 +46,8 @@ SIGNATURES = {
     "gptaq_quantize": (_int, [_vp, _vp, _int, _i64, _i64, _int, _int, _int, _int, _vp, _vp, _vp, _vp, _vp]),
     "gptaq_quantize_stage_bytes": (_sz, [_i64, _i64, _int]),
     "gptaq_quantize_host": (_int, [_vp, _vp, _i64, _i64, _int, _int, _int, _int, _vp, _vp, _vp, _vp, _vp, _sz, _vp]),
+    "gptaq_quantize_static": (_int, [_vp, _vp, _i64, _vp, _int, _i64, _i64, _int, _int, _int, _int, _vp, _vp, _vp, _vp,
+                                     _vp, _vp]),
     "gptaq_sync_status": (_int, [_vp, C.POINTER(_i64), _vp]),
     "gptaq_H": (_vp, [_vp]),
     "gptaq_D": (_vp, [_vp]),
@@ -208,6 +210,43 @@ def gptaq_quantize_host(h, h_W: torch.Tensor, bits: int, group: int, sym: bool, 
                                             _ptr(d_stage), d_stage.numel() * d_stage.element_size(),
                                             _stream(stream))
     _check(st, "gptaq_quantize_host", h)
+
+
+GPTAQ_STATIC_MAX_N = 16384
+GPTAQ_STATIC_SCRATCH_FLOATS = 1 << 20
+
+
+def gptaq_quantize_static(d_U: torch.Tensor, d_P: torch.Tensor, d_W: torch.Tensor, bits: int, group: int,
+                          sym: bool, blocksize: int, d_codes: torch.Tensor, d_scales: torch.Tensor,
+                          d_zeros: torch.Tensor, d_Wq: torch.Tensor | None = None,
+                          d_status: torch.Tensor | None = None, stream=None):
+    """``gptaq_quantize`` without handle or workspace, for callers that may not allocate device
+    memory: ``d_U`` / ``d_P`` are ``[n, n]`` float32 inputs and the scratch is an array built
+    into the library (limits: ``n <= GPTAQ_STATIC_MAX_N``,
+    ``m * 2 * blocksize <= GPTAQ_STATIC_SCRATCH_FLOATS``).  ``d_status``: optional int64[2]
+    CUDA tensor that receives the device status and its index."""
+    _need_cuda(d_U, d_P, d_W, d_codes, d_scales, d_zeros, d_Wq, d_status)
+    n = d_U.shape[0]
+    assert d_U.dtype == torch.float32 and d_P.dtype == torch.float32
+    assert d_U.shape == (n, n) and d_P.shape == (n, n) and d_U.is_contiguous() and d_P.is_contiguous()
+    assert d_W.dim() == 2 and d_W.stride(1) == 1 and d_W.shape[1] == n
+    dt = {torch.float32: GPTAQ_W_FP32, torch.bfloat16: GPTAQ_W_BF16}[d_W.dtype]
+    m = d_W.shape[0]
+    ldw = d_W.stride(0) if m > 1 else d_W.shape[1]
+    assert d_codes.dtype == torch.uint8 and d_codes.is_contiguous()
+    assert d_scales.dtype == torch.float32 and d_zeros.dtype == torch.float32
+    if d_Wq is not None:
+        assert d_Wq.dtype == torch.float32 and d_Wq.is_contiguous() and d_Wq.shape == d_W.shape
+    if d_status is not None:
+        assert d_status.dtype == torch.int64 and d_status.numel() >= 2 and d_status.is_contiguous()
+    st = load_library().gptaq_quantize_static(_ptr(d_U), _ptr(d_P), n, _ptr(d_W), dt, m, ldw, bits, group,
+                                              int(bool(sym)), blocksize, _ptr(d_codes), _ptr(d_scales),
+                                              _ptr(d_zeros), _ptr(d_Wq), _ptr(d_status), _stream(stream))
+    if st == GPTAQ_ERR_WORKSPACE:
+        raise GptaqError(st, "gptaq_quantize_static",
+                         f"n = {n} (limit {GPTAQ_STATIC_MAX_N}) or m * 2 * blocksize = {m * 2 * blocksize} "
+                         f"(limit {GPTAQ_STATIC_SCRATCH_FLOATS}) exceeds the built-in scratch")
+    _check(st, "gptaq_quantize_static")
 
 
 # ---------------------------------------------------------------- status and views

@@ -7,6 +7,7 @@
 
 #include <cmath>
 #include <cstring>
+#include <mutex>
 #include <new>
 #include <string>
 
@@ -192,6 +193,153 @@ gptaq_status_t accumulate_tc(gptaq_ctx *h, const float *X, const float *Xfp, int
 }
 
 bool valid_block(int b) { return b == 32 || b == 64 || b == 128; }
+
+// What the column loop and the trailing update work on: the factor U, the matrix P, the
+// dead-input flags, the device status header and the m x 2B scratch for [-Err | Wpre].
+struct QuantizeTarget {
+    int n;
+    const float *U, *P;
+    const uint8_t *dead;
+    StateHeader *hd;
+    float *EW;
+    int num_sms;
+};
+
+gptaq_status_t check_quantize_args(int64_t n, const void *d_W, int w_dtype, int64_t m, int64_t ldw, int bits,
+                                   int group, int blocksize, const uint8_t *d_codes, const float *d_scales,
+                                   const float *d_zeros, const float *d_Wq) {
+    if (bits < 2 || bits > 8 || !valid_block(blocksize) || group < 0 ||
+        (w_dtype != GPTAQ_W_FP32 && w_dtype != GPTAQ_W_BF16))
+        return GPTAQ_ERR_UNSUPPORTED;
+    if (group > 0 && (blocksize % group) != 0) return GPTAQ_ERR_UNSUPPORTED;
+    if (m == 0) return GPTAQ_OK;
+    if (!d_W || !d_codes || !d_scales || !d_zeros || ldw < n) return GPTAQ_ERR_INVALID_ARG;
+    if (w_dtype == GPTAQ_W_BF16 && !d_Wq) return GPTAQ_ERR_INVALID_ARG;
+    return GPTAQ_OK;
+}
+
+#define QLAUNCHED()                                          \
+    do {                                                     \
+        cudaError_t e__ = cudaGetLastError();                \
+        if (e__ != cudaSuccess) { *err = e__; return GPTAQ_ERR_CUDA; } \
+        ++*launches;                                         \
+    } while (0)
+
+// Algorithm 1, lines 5-13: launch sequence shared by the entry points that quantize.
+gptaq_status_t quantize_core(const QuantizeTarget &t, void *d_W, int w_dtype, int64_t m, int64_t ldw,
+                             int bits, int group, int sym, int blocksize, uint8_t *d_codes, float *d_scales,
+                             float *d_zeros, float *d_Wq, cudaStream_t s, int64_t *launches, cudaError_t *err) {
+    const int n = t.n;
+    float *EW = t.EW;
+    float *Wk = static_cast<float *>(d_W);
+    int64_t ldk = ldw;
+    if (w_dtype == GPTAQ_W_BF16) {
+        bf16_to_f32_kernel<<<t.num_sms * 8, 256, 0, s>>>(static_cast<const __nv_bfloat16 *>(d_W), ldw,
+                                                        d_Wq, n, (int)m, n);
+        QLAUNCHED();
+        Wk = d_Wq; ldk = n;
+    } else if (d_Wq && d_Wq != d_W) {
+        copy2d_kernel<<<t.num_sms * 8, 256, 0, s>>>(static_cast<const float *>(d_W), ldw, d_Wq, n,
+                                                   (int)m, n);
+        QLAUNCHED();
+        Wk = d_Wq; ldk = n;
+    }
+
+    const int G = group > 0 ? (n + group - 1) / group : 1;
+    if (group <= 0) {
+        row_grid_kernel<<<(unsigned)((m + 7) / 8), 256, 0, s>>>(Wk, ldk, (int)m, n, t.dead, bits, sym,
+                                                               d_scales, d_zeros);
+        QLAUNCHED();
+    }
+
+    int nw = (int)((m + t.num_sms - 1) / t.num_sms);
+    nw = std::max(1, std::min(32, nw));
+    const unsigned cl_grid = (unsigned)((m + nw - 1) / nw);
+    const int T = blocksize / 32;
+    const size_t cl_smem = 2 * (size_t)blocksize * blocksize * sizeof(float);
+
+    for (int i0 = 0; i0 < n; i0 += blocksize) {
+        ColumnLoopArgs a;
+        a.W = Wk; a.ldw = ldk; a.m = (int)m; a.n = n; a.U = t.U; a.P = t.P; a.dead = t.dead;
+        a.i0 = i0; a.bw = std::min(blocksize, n - i0);
+        a.bits = bits; a.group = group; a.sym = sym;
+        a.codes = d_codes; a.scales = d_scales; a.zeros = d_zeros; a.G = G; a.EW = EW; a.hd = t.hd;
+        if (T == 4) column_loop_kernel<4><<<cl_grid, nw * 32, cl_smem, s>>>(a);
+        else if (T == 2) column_loop_kernel<2><<<cl_grid, nw * 32, cl_smem, s>>>(a);
+        else column_loop_kernel<1><<<cl_grid, nw * 32, cl_smem, s>>>(a);
+        QLAUNCHED();
+        const int i2 = i0 + blocksize;
+        if (i2 < n) {
+            // W[:, i2:] += [-Err | Wpre] * [U[blk, i2:] ; P[blk, i2:]]   (lazy-batch update)
+            Operand bop = make_operand(t.U + (int64_t)i0 * n + i2, 1, n);
+            bop.p2 = t.P + (int64_t)i0 * n + i2;
+            bop.k_split = blocksize;
+            GemmProblem pt = make_problem(make_operand(EW, 2 * blocksize, 1), bop, Wk + i2, ldk,
+                                          (int)m, n - i2, 2 * blocksize, 1.f, 1.f, GEMM_FULL);
+            *err = launch_simt_gemm(pt, false, true, s);
+            if (*err != cudaSuccess) return GPTAQ_ERR_CUDA;
+            ++*launches;
+        }
+    }
+    return GPTAQ_OK;
+}
+
+
+// ---------------------------------------------------------------------------
+// Built-in scratch of gptaq_quantize_static: one array per GPU that loads the library, held
+// until the process exits.  Layout: status header | dead-input flags (all zero) | [-Err | Wpre].
+// In host code the array's name is only a stand-in for the symbol, not a device address; the
+// address that kernels may use is looked up once per device with cudaGetSymbolAddress.
+// ---------------------------------------------------------------------------
+constexpr size_t STATIC_FLAGS_OFFSET = 256;
+constexpr size_t STATIC_EW_OFFSET = STATIC_FLAGS_OFFSET + GPTAQ_STATIC_MAX_N;
+constexpr size_t STATIC_SCRATCH_BYTES = STATIC_EW_OFFSET + (size_t)GPTAQ_STATIC_SCRATCH_FLOATS * sizeof(float);
+static_assert(STATIC_EW_OFFSET % 256 == 0, "scratch alignment");
+static_assert(sizeof(StateHeader) <= STATIC_FLAGS_OFFSET, "header fits");
+
+static __device__ __align__(256) unsigned char g_static_scratch[STATIC_SCRATCH_BYTES];
+
+struct StaticScratch {
+    bool ready;
+    uint8_t *base;
+    int num_sms;
+};
+constexpr int MAX_DEVICES = 64;
+StaticScratch g_static_table[MAX_DEVICES];
+std::mutex g_static_mutex;
+
+__global__ void export_status_kernel(const StateHeader *hd, int64_t *out) {
+    out[0] = hd->status;
+    out[1] = hd->info;
+}
+
+// Set-up on first use, once per device, with that device current: resolves the device address
+// of the scratch array and raises the shared-memory limit of the column-loop kernels.
+cudaError_t static_scratch_for_current_device(StaticScratch **out) {
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    if (dev < 0 || dev >= MAX_DEVICES) return cudaErrorInvalidDevice;
+    std::lock_guard<std::mutex> lock(g_static_mutex);
+    StaticScratch &sc = g_static_table[dev];
+    if (!sc.ready) {
+        void *ptr = nullptr;
+        e = cudaGetSymbolAddress(&ptr, g_static_scratch);
+        if (e != cudaSuccess) return e;
+        e = cudaDeviceGetAttribute(&sc.num_sms, cudaDevAttrMultiProcessorCount, dev);
+        if (e != cudaSuccess) return e;
+        e = cudaFuncSetAttribute(column_loop_kernel<4>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 2 * 128 * 128 * (int)sizeof(float));
+        if (e != cudaSuccess) return e;
+        e = cudaFuncSetAttribute(column_loop_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 2 * 64 * 64 * (int)sizeof(float));
+        if (e != cudaSuccess) return e;
+        sc.base = static_cast<uint8_t *>(ptr);
+        sc.ready = true;
+    }
+    *out = &sc;
+    return cudaSuccess;
+}
 
 }  // namespace
 
@@ -399,68 +547,20 @@ gptaq_status_t gptaq_quantize(gptaq_handle_t h, void *d_W, int w_dtype, int64_t 
                               gptaq_stream_t stream) {
     if (!h || m < 0 || m > INT32_MAX) return GPTAQ_ERR_INVALID_ARG;
     if (h->stage != STAGE_P) return GPTAQ_ERR_BAD_STATE;
-    if (bits < 2 || bits > 8 || !valid_block(blocksize) || group < 0 ||
-        (w_dtype != GPTAQ_W_FP32 && w_dtype != GPTAQ_W_BF16))
-        return GPTAQ_ERR_UNSUPPORTED;
-    if (group > 0 && (blocksize % group) != 0) return GPTAQ_ERR_UNSUPPORTED;
-    if (m == 0) return GPTAQ_OK;
-    if (!d_W || !d_codes || !d_scales || !d_zeros || ldw < h->n) return GPTAQ_ERR_INVALID_ARG;
-    if (w_dtype == GPTAQ_W_BF16 && !d_Wq) return GPTAQ_ERR_INVALID_ARG;
-    const int n = (int)h->n;
+    gptaq_status_t st = check_quantize_args(h->n, d_W, w_dtype, m, ldw, bits, group, blocksize, d_codes,
+                                            d_scales, d_zeros, d_Wq);
+    if (st != GPTAQ_OK || m == 0) return st;
     WsLayout wl = ws_layout(h->n, m, blocksize);
     if (h->ws_bytes < wl.total) return GPTAQ_ERR_WORKSPACE;
-    cudaStream_t s = static_cast<cudaStream_t>(stream);
-    float *EW = reinterpret_cast<float *>(h->ws + wl.ew_off);
-
-    float *Wk = static_cast<float *>(d_W);
-    int64_t ldk = ldw;
-    if (w_dtype == GPTAQ_W_BF16) {
-        bf16_to_f32_kernel<<<h->num_sms * 8, 256, 0, s>>>(static_cast<const __nv_bfloat16 *>(d_W), ldw,
-                                                         d_Wq, n, (int)m, n);
-        LAUNCHED();
-        Wk = d_Wq; ldk = n;
-    } else if (d_Wq && d_Wq != d_W) {
-        copy2d_kernel<<<h->num_sms * 8, 256, 0, s>>>(static_cast<const float *>(d_W), ldw, d_Wq, n,
-                                                    (int)m, n);
-        LAUNCHED();
-        Wk = d_Wq; ldk = n;
-    }
-
-    const int G = group > 0 ? (n + group - 1) / group : 1;
-    if (group <= 0) {
-        row_grid_kernel<<<(unsigned)((m + 7) / 8), 256, 0, s>>>(Wk, ldk, (int)m, n, h->dead, bits, sym,
-                                                               d_scales, d_zeros);
-        LAUNCHED();
-    }
-
-    int nw = (int)((m + h->num_sms - 1) / h->num_sms);
-    nw = std::max(1, std::min(32, nw));
-    const unsigned cl_grid = (unsigned)((m + nw - 1) / nw);
-    const int T = blocksize / 32;
-    const size_t cl_smem = 2 * (size_t)blocksize * blocksize * sizeof(float);
-
-    for (int i0 = 0; i0 < n; i0 += blocksize) {
-        ColumnLoopArgs a;
-        a.W = Wk; a.ldw = ldk; a.m = (int)m; a.n = n; a.U = h->H; a.P = h->D; a.dead = h->dead;
-        a.i0 = i0; a.bw = std::min(blocksize, n - i0);
-        a.bits = bits; a.group = group; a.sym = sym;
-        a.codes = d_codes; a.scales = d_scales; a.zeros = d_zeros; a.G = G; a.EW = EW; a.hd = h->hd;
-        if (T == 4) column_loop_kernel<4><<<cl_grid, nw * 32, cl_smem, s>>>(a);
-        else if (T == 2) column_loop_kernel<2><<<cl_grid, nw * 32, cl_smem, s>>>(a);
-        else column_loop_kernel<1><<<cl_grid, nw * 32, cl_smem, s>>>(a);
-        LAUNCHED();
-        const int i2 = i0 + blocksize;
-        if (i2 < n) {
-            // W[:, i2:] += [-Err | Wpre] * [U[blk, i2:] ; P[blk, i2:]]   (lazy-batch update)
-            Operand bop = make_operand(h->H + (int64_t)i0 * n + i2, 1, n);
-            bop.p2 = h->D + (int64_t)i0 * n + i2;
-            bop.k_split = blocksize;
-            GemmProblem pt = make_problem(make_operand(EW, 2 * blocksize, 1), bop, Wk + i2, ldk,
-                                          (int)m, n - i2, 2 * blocksize, 1.f, 1.f, GEMM_FULL);
-            OK(gemm(h, pt, false, true, s));
-        }
-    }
-    return GPTAQ_OK;
+    QuantizeTarget t;
+    t.n = (int)h->n; t.U = h->H; t.P = h->D; t.dead = h->dead; t.hd = h->hd;
+    t.EW = reinterpret_cast<float *>(h->ws + wl.ew_off);
+    t.num_sms = h->num_sms;
+    cudaError_t e = cudaSuccess;
+    st = quantize_core(t, d_W, w_dtype, m, ldw, bits, group, sym, blocksize, d_codes, d_scales, d_zeros, d_Wq,
+                       static_cast<cudaStream_t>(stream), &h->launches, &e);
+    if (st == GPTAQ_ERR_CUDA) h->cuda_error = cudaGetErrorString(e);
+    return st;
 }
 
 size_t gptaq_quantize_stage_bytes(int64_t m, int64_t n, int group) {
@@ -496,6 +596,43 @@ gptaq_status_t gptaq_quantize_host(gptaq_handle_t h, const float *h_W, int64_t m
     CU(cudaMemcpyAsync(h_scales, dS, (size_t)m * G * sizeof(float), cudaMemcpyDeviceToHost, s));
     CU(cudaMemcpyAsync(h_zeros, dZ, (size_t)m * G * sizeof(float), cudaMemcpyDeviceToHost, s));
     if (h_Wq) CU(cudaMemcpyAsync(h_Wq, dW, (size_t)m * n * sizeof(float), cudaMemcpyDeviceToHost, s));
+    return GPTAQ_OK;
+}
+
+gptaq_status_t gptaq_quantize_static(const float *d_U, const float *d_P, int64_t n, void *d_W, int w_dtype,
+                                     int64_t m, int64_t ldw, int bits, int group, int sym, int blocksize,
+                                     uint8_t *d_codes, float *d_scales, float *d_zeros, float *d_Wq,
+                                     int64_t *d_status, gptaq_stream_t stream) {
+    if (!d_U || !d_P || n <= 0 || m < 0 || m > INT32_MAX) return GPTAQ_ERR_INVALID_ARG;
+    gptaq_status_t st = check_quantize_args(n, d_W, w_dtype, m, ldw, bits, group, blocksize, d_codes, d_scales,
+                                            d_zeros, d_Wq);
+    if (st != GPTAQ_OK) return st;
+    // the limits of the built-in scratch come before anything touches the device
+    if (n > GPTAQ_STATIC_MAX_N || (int64_t)m * 2 * blocksize > GPTAQ_STATIC_SCRATCH_FLOATS)
+        return GPTAQ_ERR_WORKSPACE;
+    if (m == 0) return GPTAQ_OK;
+    StaticScratch *sc = nullptr;
+    cudaError_t e = static_scratch_for_current_device(&sc);
+    if (e != cudaSuccess) return GPTAQ_ERR_CUDA;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    // every call shares the array and finds the last call's contents: the status header and
+    // the all-zero dead-input flags have to start from zero
+    e = cudaMemsetAsync(sc->base, 0, STATIC_EW_OFFSET, s);
+    if (e != cudaSuccess) return GPTAQ_ERR_CUDA;
+    QuantizeTarget t;
+    t.n = (int)n; t.U = d_U; t.P = d_P;
+    t.hd = reinterpret_cast<StateHeader *>(sc->base);
+    t.dead = sc->base + STATIC_FLAGS_OFFSET;
+    t.EW = reinterpret_cast<float *>(sc->base + STATIC_EW_OFFSET);
+    t.num_sms = sc->num_sms;
+    int64_t launches = 0;
+    st = quantize_core(t, d_W, w_dtype, m, ldw, bits, group, sym, blocksize, d_codes, d_scales, d_zeros, d_Wq, s,
+                       &launches, &e);
+    if (st != GPTAQ_OK) return st;
+    if (d_status) {
+        export_status_kernel<<<1, 1, 0, s>>>(t.hd, d_status);
+        if (cudaGetLastError() != cudaSuccess) return GPTAQ_ERR_CUDA;
+    }
     return GPTAQ_OK;
 }
 
