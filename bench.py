@@ -172,9 +172,9 @@ def run_ours(args, cfg):
     zeros = torch.empty((cfg.m, G), dtype=torch.float32, device=dev)
     Wq = torch.empty((cfg.m, cfg.n), dtype=torch.float32, device=dev)
     # statistics arithmetic: the cheapest tensor-core mode that keeps U within its error bound
-    st = g.LayerState(cfg.n, cfg.m, cfg.batch_tokens, cfg.blocksize, dev, total_tokens=cfg.tokens)
+    st = g.LayerState(cfg.n, cfg.m, cfg.batch_tokens, cfg.blocksize, dev, total_tokens=args.full_tokens)
     h = st.handle
-    prec = g.gptaq_recommended_stats_precision(cfg.n, cfg.tokens)
+    prec = g.gptaq_recommended_stats_precision(cfg.n, args.full_tokens)
     prec_name = {g.GPTAQ_STATS_FP16_TENSOR: "fp16 operands, fp32 accumulate",
                  g.GPTAQ_STATS_FP16_SPLIT_TENSOR: "fp16 hi+lo split for H, fp32 accumulate"}[prec]
     stream = torch.cuda.current_stream()
@@ -303,6 +303,8 @@ def run_ours(args, cfg):
                      "algorithmic_flops_per_launch": flops_call},
         "cpu_baseline": cpu, "e2e": e2e, "gpu_launches": launches, "clocks": clk.summary(),
     }
+    if args.batches > 0:
+        line["truncated"] = f"{cfg.n_batches} token batches only: not a benchmark value"
     print(json.dumps(line), flush=True)
 
 
@@ -315,10 +317,16 @@ def main():
     ap.add_argument("--workload", default="cfg2", choices=sorted(wl.CONFIGS))
     ap.add_argument("--ref-tokens", type=int, default=1024)
     ap.add_argument("--ref-rows", type=int, default=32)
+    ap.add_argument("--batches", type=int, default=0,
+                    help="profiler captures only: keep this many token batches (the line is marked truncated)")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()
     cfg = wl.CONFIGS[args.workload]
+    full_tokens = cfg.tokens
+    if args.batches > 0:
+        cfg = wl.scaled(cfg, n_batches=min(args.batches, cfg.n_batches))
+    args.full_tokens = full_tokens
     if args.impl == "reference":
         run_reference(args, cfg)
     else:
