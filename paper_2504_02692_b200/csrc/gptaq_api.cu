@@ -14,6 +14,7 @@
 #include "kernels.cuh"
 #include "simt_gemm.cuh"
 #include "umma_gemm.cuh"
+#include "tc_gemm.cuh"
 
 using namespace gptaq;
 
@@ -41,6 +42,7 @@ struct gptaq_ctx {
     int64_t tokens;
     int64_t launches;
     int stats_precision;   // GPTAQ_STATS_*
+    bool tensor;           // float32-grade tensor-core GEMMs for factor / P / trailing update
     std::string cuda_error;
 };
 
@@ -60,17 +62,33 @@ Layout state_layout(int64_t n) {
     return l;
 }
 
+// float32-grade tensor-core path (tc_gemm.cuh): widths whose rows are 16-byte multiples (a TMA
+// stride rule) and that are large enough for 128 x 256 tiles to pay.
+constexpr int64_t TC_MIN_N = 512;
+inline bool tc_shape_ok(int64_t n) { return n >= TC_MIN_N && (n % 4) == 0; }
+
 struct WsLayout {
-    size_t t_off, rinv_off, ew_off, total;
+    size_t t_off, rinv_off;
+    size_t s_off[6];        // split operand matrices (n x n each): S1 hi/lo, S2 hi/lo, S3 hi/lo
+    size_t pan_off[2];      // split copy of one factor panel (n x 128), hi/lo
+    size_t ew_off, ew_lo_off, total;
+    bool tensor;
 };
 
 WsLayout ws_layout(int64_t n, int64_t m_max, int blocksize) {
     WsLayout w;
     size_t nb = (size_t)((n + NB - 1) / NB);
+    const size_t mat = round_up((size_t)n * (size_t)n * sizeof(float), ALIGN);
+    w.tensor = tc_shape_ok(n);
     w.t_off = 0;
-    w.rinv_off = w.t_off + round_up((size_t)n * (size_t)n * sizeof(float), ALIGN);
-    w.ew_off = w.rinv_off + round_up(nb * NB * NB * sizeof(float), ALIGN);
-    w.total = w.ew_off + round_up((size_t)m_max * 2 * (size_t)blocksize * sizeof(float), ALIGN);
+    w.rinv_off = w.t_off + mat;
+    size_t off = w.rinv_off + round_up(nb * NB * NB * sizeof(float), ALIGN);
+    for (int i = 0; i < 6; ++i) { w.s_off[i] = off; if (w.tensor) off += mat; }
+    for (int i = 0; i < 2; ++i) { w.pan_off[i] = off; if (w.tensor) off += round_up((size_t)n * NB * sizeof(float), ALIGN); }
+    const size_t ew = round_up((size_t)m_max * 2 * (size_t)blocksize * sizeof(float), ALIGN);
+    w.ew_off = off;
+    w.ew_lo_off = off + ew;
+    w.total = off + (w.tensor ? 2 * ew : ew);
     return w;
 }
 
@@ -135,6 +153,67 @@ bool make_kmajor_map(CUtensorMap *map, const void *ptr, int64_t rows, int64_t kp
     return fn(map, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 2, const_cast<void *>(ptr), dims, strides, box, estr,
               CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+// float32 matrix [rows][ld] with `cols` valid K-contiguous elements per row; box = 32 x box_rows,
+// 128-byte swizzle, out-of-range elements read as zero.
+bool make_f32_map(CUtensorMap *map, const void *ptr, int64_t rows, int64_t cols, int64_t ld, int box_rows) {
+    EncodeTiledFn fn = encode_tiled_fn();
+    if (!fn) return false;
+    cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
+    cuuint64_t strides[1] = {(cuuint64_t)ld * 4};
+    cuuint32_t box[2] = {(cuuint32_t)TBK, (cuuint32_t)box_rows};
+    cuuint32_t estr[2] = {1, 1};
+    return fn(map, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, const_cast<void *>(ptr), dims, strides, box, estr,
+              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+// A split operand (hi / lo arrays of the same shape) as seen by the tensor-core GEMM.
+struct SplitOperand {
+    const float *hi, *lo;
+    int64_t rows, cols, ld;
+};
+
+struct TcMaps {
+    CUtensorMap a_hi, a_lo, b_hi, b_lo, b2_hi, b2_lo;
+};
+
+bool make_tc_maps(TcMaps *m, const SplitOperand &A, const SplitOperand &B, const SplitOperand *B2) {
+    const SplitOperand &b2 = B2 ? *B2 : B;
+    return make_f32_map(&m->a_hi, A.hi, A.rows, A.cols, A.ld, TBM) && make_f32_map(&m->a_lo, A.lo, A.rows, A.cols, A.ld, TBM) &&
+           make_f32_map(&m->b_hi, B.hi, B.rows, B.cols, B.ld, TBN) && make_f32_map(&m->b_lo, B.lo, B.rows, B.cols, B.ld, TBN) &&
+           make_f32_map(&m->b2_hi, b2.hi, b2.rows, b2.cols, b2.ld, TBN) &&
+           make_f32_map(&m->b2_lo, b2.lo, b2.rows, b2.cols, b2.ld, TBN);
+}
+
+TcGemmArgs tc_args(float *C, int64_t ldc, int M, int N, int K, float alpha, float beta, int mode, int mask,
+                   StateHeader *hd) {
+    TcGemmArgs a;
+    std::memset(&a, 0, sizeof(a));
+    a.C = C; a.ldc = ldc; a.M = M; a.N = N; a.K = K; a.nbatch = 1;
+    a.alpha = alpha; a.beta = beta; a.mode = mode; a.mask = mask; a.hd = hd;
+    return a;
+}
+
+cudaError_t launch_tc_gemm(const TcMaps &m, const TcGemmArgs &a, int num_sms, cudaStream_t s) {
+    if (a.M <= 0 || a.N <= 0 || a.nbatch <= 0) return cudaSuccess;
+    const int64_t tiles = (int64_t)a.nbatch * ((a.M + TBM - 1) / TBM) * ((a.N + TBN - 1) / TBN);
+    const int grid = (int)std::min<int64_t>(tiles, num_sms);
+    tc_gemm_kernel<<<grid, TC_THREADS, TC_SMEM, s>>>(m.a_hi, m.a_lo, m.b_hi, m.b_lo, m.b2_hi, m.b2_lo, a);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_split(const float *src, int64_t lds, float *hi, float *lo, int64_t ldd, int rows, int cols,
+                         bool transpose, int mask, float scale, cudaStream_t s) {
+    if (rows <= 0 || cols <= 0) return cudaSuccess;
+    SplitArgs a;
+    a.src = src; a.lds = lds; a.src_bstride = 0; a.hi = hi; a.lo = lo; a.ldd = ldd; a.dst_bstride = 0;
+    a.rows = rows; a.cols = cols; a.rows_last = a.cols_last = 0; a.nbatch = 1;
+    a.transpose = transpose ? 1 : 0; a.mask = mask; a.scale = scale;
+    dim3 grid((cols + 63) / 64, (rows + 63) / 64, 1);
+    split_kernel<<<grid, 256, 0, s>>>(a);
+    return cudaGetLastError();
 }
 
 // Largest token chunk (multiple of 64) whose two fp16 operand copies fit the workspace.
@@ -203,6 +282,10 @@ struct QuantizeTarget {
     StateHeader *hd;
     float *EW;
     int num_sms;
+    // float32-grade tensor-core trailing update: split copies of U^T and P^T (n x n, ld n) and
+    // the low part of [-Err | Wpre]; all null on the plain-FMA path
+    const float *UT_hi, *UT_lo, *PT_hi, *PT_lo;
+    float *EW_lo;
 };
 
 gptaq_status_t check_quantize_args(int64_t n, const void *d_W, int w_dtype, int64_t m, int64_t ldw, int bits,
@@ -258,18 +341,33 @@ gptaq_status_t quantize_core(const QuantizeTarget &t, void *d_W, int w_dtype, in
     const int T = blocksize / 32;
     const size_t cl_smem = 2 * (size_t)blocksize * blocksize * sizeof(float);
 
+    const bool tensor = t.EW_lo != nullptr;
+    TcMaps maps;
+    if (tensor) {
+        const SplitOperand A{EW, t.EW_lo, m, 2 * blocksize, 2 * blocksize};
+        const SplitOperand B{t.UT_hi, t.UT_lo, n, n, n}, B2{t.PT_hi, t.PT_lo, n, n, n};
+        if (!make_tc_maps(&maps, A, B, &B2)) { *err = cudaErrorUnknown; return GPTAQ_ERR_CUDA; }
+    }
     for (int i0 = 0; i0 < n; i0 += blocksize) {
         ColumnLoopArgs a;
         a.W = Wk; a.ldw = ldk; a.m = (int)m; a.n = n; a.U = t.U; a.P = t.P; a.dead = t.dead;
         a.i0 = i0; a.bw = std::min(blocksize, n - i0);
         a.bits = bits; a.group = group; a.sym = sym;
-        a.codes = d_codes; a.scales = d_scales; a.zeros = d_zeros; a.G = G; a.EW = EW; a.hd = t.hd;
+        a.codes = d_codes; a.scales = d_scales; a.zeros = d_zeros; a.G = G; a.EW = EW; a.EW_lo = t.EW_lo; a.hd = t.hd;
         if (T == 4) column_loop_kernel<4><<<cl_grid, nw * 32, cl_smem, s>>>(a);
         else if (T == 2) column_loop_kernel<2><<<cl_grid, nw * 32, cl_smem, s>>>(a);
         else column_loop_kernel<1><<<cl_grid, nw * 32, cl_smem, s>>>(a);
         QLAUNCHED();
         const int i2 = i0 + blocksize;
-        if (i2 < n) {
+        if (i2 < n && tensor) {
+            // W[:, i2:] += [-Err | Wpre] * [U[blk, i2:] ; P[blk, i2:]] on the tensor cores: B operand rows
+            // are rows i2.. of U^T (first B contraction steps) and of P^T (the next B)
+            TcGemmArgs g = tc_args(Wk + i2, ldk, (int)m, n - i2, 2 * blocksize, 1.f, 1.f, TC_FULL, TC_MASK_NONE, t.hd);
+            g.b_row0 = i2; g.b_k0 = i0; g.k_split = blocksize; g.b2_k0 = i0;
+            *err = launch_tc_gemm(maps, g, t.num_sms, s);
+            if (*err != cudaSuccess) return GPTAQ_ERR_CUDA;
+            ++*launches;
+        } else if (i2 < n) {
             // W[:, i2:] += [-Err | Wpre] * [U[blk, i2:] ; P[blk, i2:]]   (lazy-batch update)
             Operand bop = make_operand(t.U + (int64_t)i0 * n + i2, 1, n);
             bop.p2 = t.P + (int64_t)i0 * n + i2;
@@ -381,6 +479,7 @@ gptaq_status_t gptaq_create(gptaq_handle_t *out, int64_t n, void *d_state, size_
     h->dead = reinterpret_cast<uint8_t *>(h->state + l.dead_off);
     h->launches = 0;
     h->stats_precision = GPTAQ_STATS_FP16_SPLIT_TENSOR;
+    h->tensor = tc_shape_ok(n) && encode_tiled_fn() != nullptr;
     cudaError_t e = cudaGetDevice(&h->device);
     if (e == cudaSuccess) e = cudaDeviceGetAttribute(&h->num_sms, cudaDevAttrMultiProcessorCount, h->device);
     if (e == cudaSuccess)
@@ -390,6 +489,8 @@ gptaq_status_t gptaq_create(gptaq_handle_t *out, int64_t n, void *d_state, size_
                                  2 * 128 * 128 * (int)sizeof(float));
     if (e == cudaSuccess)
         e = cudaFuncSetAttribute(stats_umma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)UMMA_SMEM);
+    if (e == cudaSuccess)
+        e = cudaFuncSetAttribute(tc_gemm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)TC_SMEM);
     if (e == cudaSuccess)
         e = cudaFuncSetAttribute(column_loop_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                  2 * 64 * 64 * (int)sizeof(float));
@@ -518,6 +619,16 @@ gptaq_status_t gptaq_factor(gptaq_handle_t h, float damp, gptaq_stream_t stream)
         p2.batchN_last = tail;
         OK(gemm(h, p2, false, true, s));
     }
+    if (h->tensor) {
+        // operand copies of U for the products that follow: S1 = split(U), S2 = split(U^T)
+        WsLayout w = ws_layout(h->n, 0, 32);
+        float *S1h = reinterpret_cast<float *>(h->ws + w.s_off[0]), *S1l = reinterpret_cast<float *>(h->ws + w.s_off[1]);
+        float *S2h = reinterpret_cast<float *>(h->ws + w.s_off[2]), *S2l = reinterpret_cast<float *>(h->ws + w.s_off[3]);
+        CU(launch_split(H, n, S1h, S1l, n, n, n, false, SPLIT_UPPER, 1.f, s));
+        h->launches++;
+        CU(launch_split(H, n, S2h, S2l, n, n, n, true, SPLIT_UPPER, 1.f, s));
+        h->launches++;
+    }
     h->stage = STAGE_FACTORED;
     return GPTAQ_OK;
 }
@@ -529,6 +640,29 @@ gptaq_status_t gptaq_build_P(gptaq_handle_t h, float alpha, gptaq_stream_t strea
     const int n = (int)h->n;
     WsLayout wl = ws_layout(h->n, 0, 32);
     float *O = reinterpret_cast<float *>(h->ws + wl.t_off);
+    if (h->tensor) {
+        float *S[6];
+        for (int i = 0; i < 6; ++i) S[i] = reinterpret_cast<float *>(h->ws + wl.s_off[i]);
+        const SplitOperand Us{S[0], S[1], n, n, n}, UTs{S[2], S[3], n, n, n}, S3{S[4], S[5], n, n, n};
+        TcMaps maps;
+        // S3 = split(dXX^T / tokens);  O = (S3 U^T) .* M_U  (contraction over k >= column, U[a][k] = 0 below)
+        CU(launch_split(h->D, n, S[4], S[5], n, n, n, false, SPLIT_ALL, (float)(1.0 / (double)h->tokens), s));
+        h->launches++;
+        if (!make_tc_maps(&maps, S3, Us, nullptr)) { h->cuda_error = "cuTensorMapEncodeTiled failed"; return GPTAQ_ERR_CUDA; }
+        CU(launch_tc_gemm(maps, tc_args(O, n, n, n, n, 1.f, 0.f, TC_O, TC_MASK_STRICT_ZERO, h->hd), h->num_sms, s));
+        h->launches++;
+        // S3 = split(O);  P = alpha * O U  (B operand rows are rows of U^T)
+        CU(launch_split(O, n, S[4], S[5], n, n, n, false, SPLIT_STRICT_UPPER, 1.f, s));
+        h->launches++;
+        if (!make_tc_maps(&maps, S3, UTs, nullptr)) { h->cuda_error = "cuTensorMapEncodeTiled failed"; return GPTAQ_ERR_CUDA; }
+        CU(launch_tc_gemm(maps, tc_args(h->D, n, n, n, n, alpha, 0.f, TC_P, TC_MASK_STRICT_ZERO, h->hd), h->num_sms, s));
+        h->launches++;
+        // S3 = split(P^T) for the lazy-batch updates of gptaq_quantize
+        CU(launch_split(h->D, n, S[4], S[5], n, n, n, true, SPLIT_STRICT_UPPER, 1.f, s));
+        h->launches++;
+        h->stage = STAGE_P;
+        return GPTAQ_OK;
+    }
     // O = (dXX^T U^T) .* M_U
     GemmProblem po = make_problem(make_operand(h->D, n, 1), make_operand(h->H, n, 1), O, n, n, n, n,
                                   1.f, 0.f, GEMM_O);
@@ -556,6 +690,12 @@ gptaq_status_t gptaq_quantize(gptaq_handle_t h, void *d_W, int w_dtype, int64_t 
     t.n = (int)h->n; t.U = h->H; t.P = h->D; t.dead = h->dead; t.hd = h->hd;
     t.EW = reinterpret_cast<float *>(h->ws + wl.ew_off);
     t.num_sms = h->num_sms;
+    t.UT_hi = t.UT_lo = t.PT_hi = t.PT_lo = nullptr; t.EW_lo = nullptr;
+    if (h->tensor) {
+        t.UT_hi = reinterpret_cast<float *>(h->ws + wl.s_off[2]); t.UT_lo = reinterpret_cast<float *>(h->ws + wl.s_off[3]);
+        t.PT_hi = reinterpret_cast<float *>(h->ws + wl.s_off[4]); t.PT_lo = reinterpret_cast<float *>(h->ws + wl.s_off[5]);
+        t.EW_lo = reinterpret_cast<float *>(h->ws + wl.ew_lo_off);
+    }
     cudaError_t e = cudaSuccess;
     st = quantize_core(t, d_W, w_dtype, m, ldw, bits, group, sym, blocksize, d_codes, d_scales, d_zeros, d_Wq,
                        static_cast<cudaStream_t>(stream), &h->launches, &e);
@@ -625,6 +765,7 @@ gptaq_status_t gptaq_quantize_static(const float *d_U, const float *d_P, int64_t
     t.dead = sc->base + STATIC_FLAGS_OFFSET;
     t.EW = reinterpret_cast<float *>(sc->base + STATIC_EW_OFFSET);
     t.num_sms = sc->num_sms;
+    t.UT_hi = t.UT_lo = t.PT_hi = t.PT_lo = nullptr; t.EW_lo = nullptr;
     int64_t launches = 0;
     st = quantize_core(t, d_W, w_dtype, m, ldw, bits, group, sym, blocksize, d_codes, d_scales, d_zeros, d_Wq, s,
                        &launches, &e);

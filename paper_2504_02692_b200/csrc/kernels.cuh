@@ -21,6 +21,13 @@ static_assert(sizeof(StateHeader) == 128, "header size");
 
 constexpr int ST_NOT_SPD = 4, ST_NONFINITE = 5, ST_TIMEOUT = 6;
 
+// Round to the nearest TF32 value (10 explicit mantissa bits), kept in a float.
+__device__ __forceinline__ float tf32_rn(float x) {
+    uint32_t r;
+    asm("cvt.rna.tf32.f32 %0, %1;" : "=r"(r) : "f"(x));
+    return __uint_as_float(r);
+}
+
 __device__ __forceinline__ void record_status(StateHeader *hd, int code, long long info) {
     if (atomicCAS(&hd->status, 0, code) == 0) hd->info = info;
 }
@@ -221,6 +228,7 @@ struct ColumnLoopArgs {
     float *scales, *zeros;     // m x G
     int G;
     float *EW;                 // m x (2 * 32 * T): [-Err | Wpre]
+    float *EW_lo;              // nullptr, or: EW receives the TF32 value of each entry and EW_lo the remainder
     StateHeader *hd;
 };
 
@@ -309,12 +317,19 @@ __global__ void __launch_bounds__(1024) column_loop_kernel(ColumnLoopArgs a) {
 
     bool bad = false;
     float *ew = a.EW + (int64_t)row * (2 * BW);
+    float *ewl = a.EW_lo ? a.EW_lo + (int64_t)row * (2 * BW) : nullptr;
     uint8_t *crow = a.codes + (int64_t)row * n + i0;
 #pragma unroll
     for (int t = 0; t < T; ++t) {
         int c = lane + 32 * t;
-        ew[c] = nerr[t];
-        ew[BW + c] = pre[t];
+        if (ewl) {
+            const float eh = tf32_rn(nerr[t]), ph = tf32_rn(pre[t]);
+            ew[c] = eh; ewl[c] = tf32_rn(nerr[t] - eh);
+            ew[BW + c] = ph; ewl[BW + c] = tf32_rn(pre[t] - ph);
+        } else {
+            ew[c] = nerr[t];
+            ew[BW + c] = pre[t];
+        }
         if (c < bw) {
             wrow[c] = w[t];
             crow[c] = (uint8_t)code[t];
