@@ -483,7 +483,7 @@ gptaq_status_t gptaq_create(gptaq_handle_t *out, int64_t n, void *d_state, size_
     cudaError_t e = cudaGetDevice(&h->device);
     if (e == cudaSuccess) e = cudaDeviceGetAttribute(&h->num_sms, cudaDevAttrMultiProcessorCount, h->device);
     if (e == cudaSuccess)
-        e = cudaFuncSetAttribute(chol_diag_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)DIAG_SMEM);
+        e = cudaFuncSetAttribute(factor_panel_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)FP_SMEM);
     if (e == cudaSuccess)
         e = cudaFuncSetAttribute(column_loop_kernel<4>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                  2 * 128 * 128 * (int)sizeof(float));
@@ -581,20 +581,33 @@ gptaq_status_t gptaq_factor(gptaq_handle_t h, float damp, gptaq_stream_t stream)
     LAUNCHED();
 
     // reverse Cholesky H_d = R R^T, R upper, from the last block column upwards
+    float *pan_hi = h->tensor ? reinterpret_cast<float *>(h->ws + wl.pan_off[0]) : nullptr;
+    float *pan_lo = h->tensor ? reinterpret_cast<float *>(h->ws + wl.pan_off[1]) : nullptr;
+    TcMaps pan_maps;
+    if (h->tensor) {
+        const SplitOperand pan{pan_hi, pan_lo, n, NB, NB};
+        if (!make_tc_maps(&pan_maps, pan, pan, nullptr)) { h->cuda_error = "cuTensorMapEncodeTiled failed"; return GPTAQ_ERR_CUDA; }
+    }
     for (int p = nb - 1; p >= 0; --p) {
-        const int b0 = p * NB, bw = std::min(NB, n - b0);
-        float *Rp = Rinv + (size_t)p * NB * NB;
-        chol_diag_kernel<<<1, DIAG_THREADS, DIAG_SMEM, s>>>(H, n, b0, Rp, h->hd);
+        const int b0 = p * NB;
+        // diagonal block (factor + inverse) and the panel above it: R[0:b0, blk] = A[0:b0, blk] inv(R_pp)^T
+        FactorPanelArgs fa;
+        fa.H = H; fa.n = n; fa.b0 = b0; fa.Rinv = Rinv + (size_t)p * NB * NB;
+        fa.pan_hi = pan_hi; fa.pan_lo = pan_lo; fa.hd = h->hd;
+        const int fgrid = std::max(1, std::min(b0 / NB, h->num_sms));
+        factor_panel_kernel<<<fgrid, FP_THREADS, FP_SMEM, s>>>(fa);
         LAUNCHED();
         if (p == 0) break;
-        // R[0:b0, blk] = A[0:b0, blk] * inv(R_pp)^T
-        GemmProblem pp = make_problem(make_operand(H + b0, n, 1), make_operand(Rp, NB, 1), H + b0, n,
-                                      b0, bw, bw, 1.f, 0.f, GEMM_FULL);
-        OK(gemm(h, pp, false, false, s));
-        // A[0:b0, 0:b0] -= R[0:b0, blk] R[0:b0, blk]^T  (upper tiles)
-        Operand rp = make_operand(H + b0, n, 1);
-        GemmProblem ps = make_problem(rp, rp, H, n, b0, b0, bw, -1.f, 1.f, GEMM_UPPER_TILES);
-        OK(gemm(h, ps, false, false, s));
+        // A[0:b0, 0:b0] -= R[0:b0, blk] R[0:b0, blk]^T  (upper part)
+        if (h->tensor && b0 >= TC_MIN_N) {
+            TcGemmArgs g = tc_args(H, n, b0, b0, NB, -1.f, 1.f, TC_UPPER_TILES, TC_MASK_UPPER_KEEP, h->hd);
+            CU(launch_tc_gemm(pan_maps, g, h->num_sms, s));
+            h->launches++;
+        } else {
+            Operand rp = make_operand(H + b0, n, 1);
+            GemmProblem ps = make_problem(rp, rp, H, n, b0, b0, std::min(NB, n - b0), -1.f, 1.f, GEMM_UPPER_TILES);
+            OK(gemm(h, ps, false, false, s));
+        }
     }
 
     // U = R^-1: inverted diagonal blocks, then off-diagonal blocks by doubling:

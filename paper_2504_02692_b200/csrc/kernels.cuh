@@ -79,30 +79,45 @@ __global__ void __launch_bounds__(256) scale_damp_kernel(float *H, int n, const 
 }
 
 // ---------------------------------------------------------------------------
-// Diagonal block of the reverse Cholesky  H_d = R R^T (R upper):  factor the
-// NB x NB block in shared memory from its last row/column upwards, write R_pp
-// back in place (lower part zero) and its inverse to Rinv (NB x NB, ld NB).
+// One panel step of the reverse Cholesky  H_d = R R^T  (R upper), block column
+// [b0, b0 + NB):
+//   1. factor the NB x NB diagonal block from its last row/column upwards and invert the
+//      factor, both in shared memory (32-wide sub-blocks: one warp factors and inverts a
+//      32 x 32 block in registers, all warps apply it);
+//   2. rows above the block:  R[0:b0, blk] = A[0:b0, blk] * inv(R_pp)^T, written back in
+//      place and, if asked for, as TF32 hi/lo parts for the tensor-core rank-NB update.
+// Every CTA repeats step 1 (it is short and the other SMs would idle) and then takes row
+// tiles of step 2; CTA 0 stores inv(R_pp).  R_pp itself is not stored: nothing reads it.
 // Rows/columns beyond n are padded with the identity.
 // ---------------------------------------------------------------------------
 constexpr int NB = 128;
-constexpr int DIAG_THREADS = 1024;
-constexpr size_t DIAG_SMEM = 2 * NB * (NB + 1) * sizeof(float);
+constexpr int FP_THREADS = 1024;
+constexpr int FP_LD = NB + 4;
+constexpr size_t FP_SMEM = (2 * NB * FP_LD + 32 + 2 * 32 * 33) * sizeof(float);
 
-__global__ void __launch_bounds__(DIAG_THREADS) chol_diag_kernel(float *H, int n, int b0,
-                                                                 float *Rinv, StateHeader *hd) {
+struct FactorPanelArgs {
+    float *H; int n; int b0;
+    float *Rinv;               // NB x NB (ld NB): inverse of the diagonal factor
+    float *pan_hi, *pan_lo;    // nullptr, or [n][NB]: TF32 parts of the panel rows
+    StateHeader *hd;
+};
+
+__global__ void __launch_bounds__(FP_THREADS, 1) factor_panel_kernel(FactorPanelArgs a) {
     extern __shared__ float smem_f[];
-    float (*S)[NB + 1] = reinterpret_cast<float (*)[NB + 1]>(smem_f);
-    float (*X)[NB + 1] = reinterpret_cast<float (*)[NB + 1]>(smem_f + NB * (NB + 1));
-    const int tid = threadIdx.x;
-    const int tx = tid & 31, ty = tid >> 5;
+    float (*S)[FP_LD] = reinterpret_cast<float (*)[FP_LD]>(smem_f);
+    float (*X)[FP_LD] = reinterpret_cast<float (*)[FP_LD]>(smem_f + NB * FP_LD);
+    float *colbuf = smem_f + 2 * NB * FP_LD;
+    float (*T32)[32][33] = reinterpret_cast<float (*)[32][33]>(colbuf + 32);
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int n = a.n, b0 = a.b0;
     const int nv = min(NB, n - b0);
 
-    for (int i = ty; i < NB; i += 32)
-        for (int j = tx; j < NB; j += 32) {
+    for (int i = warp; i < NB; i += 32)
+        for (int j = lane; j < NB; j += 32) {
             float v;
             if (i < nv && j < nv) {
-                int a = min(i, j), b = max(i, j);
-                v = H[(int64_t)(b0 + a) * n + (b0 + b)];
+                const int lo = min(i, j), hi = max(i, j);
+                v = a.H[(int64_t)(b0 + lo) * n + (b0 + hi)];
             } else {
                 v = (i == j) ? 1.f : 0.f;
             }
@@ -111,48 +126,159 @@ __global__ void __launch_bounds__(DIAG_THREADS) chol_diag_kernel(float *H, int n
         }
     __syncthreads();
 
-    for (int k = NB - 1; k >= 0; --k) {
-        float piv = S[k][k];
-        bool bad = !(piv > 0.f) || !isfinite(piv);
-        if (bad) {
-            if (tid == 0) record_status(hd, ST_NOT_SPD, b0 + k);
-            piv = 1.f;
+    for (int sb = NB / 32 - 1; sb >= 0; --sb) {
+        const int o = 32 * sb;
+        if (warp == 0) {
+            // ---- 32 x 32 reverse Cholesky, lane = row, then its inverse, lane = column
+            float d[32];
+#pragma unroll
+            for (int j = 0; j < 32; ++j) d[j] = S[o + lane][o + j];
+#pragma unroll
+            for (int k = 31; k >= 0; --k) {
+                float piv = __shfl_sync(0xffffffffu, d[k], k);
+                if (!(piv > 0.f) || !isfinite(piv)) {
+                    if (lane == 0 && blockIdx.x == 0) record_status(a.hd, ST_NOT_SPD, b0 + o + k);
+                    piv = 1.f;
+                }
+                const float r = sqrtf(piv);
+                const float c = lane < k ? d[k] / r : 0.f;
+                d[k] = lane < k ? c : (lane == k ? r : 0.f);
+                colbuf[lane] = c;
+                __syncwarp();
+#pragma unroll
+                for (int j = 0; j < k; ++j) d[j] = fmaf(-c, colbuf[j], d[j]);
+                __syncwarp();
+            }
+#pragma unroll
+            for (int j = 0; j < 32; ++j) S[o + lane][o + j] = j >= lane ? d[j] : 0.f;
+            __syncwarp();
+            float x[32];
+#pragma unroll
+            for (int i = 31; i >= 0; --i) {
+                float sum = (i == lane) ? 1.f : 0.f;
+#pragma unroll
+                for (int k = i + 1; k < 32; ++k) sum = fmaf(-S[o + i][o + k], x[k], sum);
+                x[i] = i <= lane ? sum / S[o + i][o + i] : 0.f;
+            }
+#pragma unroll
+            for (int i = 0; i < 32; ++i) X[o + i][o + lane] = x[i];
         }
-        float r = sqrtf(piv);
         __syncthreads();
-        if (tid < k) S[tid][k] = S[tid][k] / r;
-        else if (tid == k) S[k][k] = r;
-        __syncthreads();
-        for (int i = ty; i < k; i += 32) {
-            float rik = S[i][k];
-            for (int j = tx; j < k; j += 32)
-                if (j >= i) S[i][j] = fmaf(-rik, S[j][k], S[i][j]);
+        // ---- rows above: R[i, sub] = S[i, sub] * inv(R_ss)^T   (one warp per row, in place)
+        for (int i = warp; i < o; i += 32) {
+            float acc = 0.f;
+#pragma unroll 8
+            for (int k = 0; k < 32; ++k) acc = fmaf(S[i][o + k], X[o + lane][o + k], acc);
+            __syncwarp();
+            S[i][o + lane] = acc;
         }
-        // the next iteration's pivot read is ordered by the sync below
+        __syncthreads();
+        // ---- leading part: S[i][j] -= R[i, sub] . R[j, sub]  (kept symmetric)
+        for (int idx = tid; idx < o * o; idx += FP_THREADS) {
+            const int i = idx / o, j = idx - i * o;
+            if (j < i) continue;
+            float acc = 0.f;
+#pragma unroll 8
+            for (int k = 0; k < 32; ++k) acc = fmaf(S[i][o + k], S[j][o + k], acc);
+            const float v = S[i][j] - acc;
+            S[i][j] = v;
+            S[j][i] = v;
+        }
         __syncthreads();
     }
 
-    // X = R^-1 (upper): column j by back substitution, 8 lanes per column.
-    {
-        const int j = tid >> 3, l = tid & 7;
-        for (int i = NB - 1; i >= 0; --i) {
-            float part = 0.f;
-            if (i < j)
-                for (int s = i + 1 + l; s <= j; s += 8) part = fmaf(S[i][s], X[s][j], part);
-            part += __shfl_xor_sync(0xffffffffu, part, 1);
-            part += __shfl_xor_sync(0xffffffffu, part, 2);
-            part += __shfl_xor_sync(0xffffffffu, part, 4);
-            if (l == 0 && i <= j) X[i][j] = ((i == j ? 1.f : 0.f) - part) / S[i][i];
-            __syncwarp();
-        }
+    // ---- off-diagonal blocks of X = R^-1:  X12 = -X11 (R12 X22), 32 -> 64 -> 128
+    for (int idx = tid; idx < 2 * 1024; idx += FP_THREADS) {
+        const int pr = idx >> 10, i = (idx >> 5) & 31, j = idx & 31;
+        const int oa = 64 * pr, oc = oa + 32;
+        float acc = 0.f;
+        for (int k = 0; k <= j; ++k) acc = fmaf(S[oa + i][oc + k], X[oc + k][oc + j], acc);
+        T32[pr][i][j] = acc;
     }
     __syncthreads();
+    for (int idx = tid; idx < 2 * 1024; idx += FP_THREADS) {
+        const int pr = idx >> 10, i = (idx >> 5) & 31, j = idx & 31;
+        const int oa = 64 * pr, oc = oa + 32;
+        float acc = 0.f;
+        for (int k = i; k < 32; ++k) acc = fmaf(X[oa + i][oa + k], T32[pr][k][j], acc);
+        X[oa + i][oc + j] = -acc;
+    }
+    __syncthreads();
+    // T64 = R[0:64, 64:128] X[64:128, 64:128], parked in the (still unused) lower-left of X
+    for (int idx = tid; idx < 64 * 64; idx += FP_THREADS) {
+        const int i = idx >> 6, j = idx & 63;
+        float acc = 0.f;
+        for (int k = 0; k <= j; ++k) acc = fmaf(S[i][64 + k], X[64 + k][64 + j], acc);
+        X[64 + i][j] = acc;
+    }
+    __syncthreads();
+    for (int idx = tid; idx < 64 * 64; idx += FP_THREADS) {
+        const int i = idx >> 6, j = idx & 63;
+        float acc = 0.f;
+        for (int k = i; k < 64; ++k) acc = fmaf(X[i][k], X[64 + k][j], acc);
+        X[i][64 + j] = -acc;
+    }
+    __syncthreads();
+    for (int idx = tid; idx < 64 * 64; idx += FP_THREADS) X[64 + (idx >> 6)][idx & 63] = 0.f;
+    __syncthreads();
+    if (blockIdx.x == 0)
+        for (int idx = tid; idx < NB * NB; idx += FP_THREADS) a.Rinv[idx] = X[idx >> 7][idx & 127];
+    if (b0 == 0) return;
 
-    for (int i = ty; i < NB; i += 32)
-        for (int j = tx; j < NB; j += 32) {
-            if (i < nv && j < nv) H[(int64_t)(b0 + i) * n + (b0 + j)] = (j >= i) ? S[i][j] : 0.f;
-            Rinv[i * NB + j] = (j >= i) ? X[i][j] : 0.f;
+    // ---- X <- X^T in place, so that a thread reads four consecutive columns of inv(R_pp)^T at once
+    for (int idx = tid; idx < NB * NB; idx += FP_THREADS) {
+        const int i = idx >> 7, j = idx & 127;
+        if (j > i) { const float u = X[i][j]; X[i][j] = X[j][i]; X[j][i] = u; }
+    }
+    // (the first tile's load below ends with a barrier)
+
+    const int ntiles = b0 / NB;              // b0 is a multiple of NB
+    const int ty = tid >> 5, tx = tid & 31;  // rows 4 ty .. 4 ty + 3, columns 4 tx .. 4 tx + 3
+    const bool vec = (n & 3) == 0 && (reinterpret_cast<uintptr_t>(a.H) & 15) == 0 && nv == NB;
+    for (int rt = blockIdx.x; rt < ntiles; rt += gridDim.x) {
+        const int r0 = rt * NB;
+        __syncthreads();                     // previous tile's reads of S are done
+        for (int i = warp; i < NB; i += 32) {
+            const float *src = a.H + (int64_t)(r0 + i) * n + b0;
+            for (int k = lane; k < NB; k += 32) S[i][k] = k < nv ? src[k] : 0.f;
         }
+        __syncthreads();
+        float acc[4][4];
+#pragma unroll
+        for (int e = 0; e < 4; ++e)
+#pragma unroll
+            for (int f = 0; f < 4; ++f) acc[e][f] = 0.f;
+#pragma unroll 4
+        for (int k = 0; k < NB; ++k) {
+            const float4 b = *reinterpret_cast<const float4 *>(&X[k][4 * tx]);
+            float av[4];
+#pragma unroll
+            for (int e = 0; e < 4; ++e) av[e] = S[4 * ty + e][k];
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+                acc[e][0] = fmaf(av[e], b.x, acc[e][0]); acc[e][1] = fmaf(av[e], b.y, acc[e][1]);
+                acc[e][2] = fmaf(av[e], b.z, acc[e][2]); acc[e][3] = fmaf(av[e], b.w, acc[e][3]);
+            }
+        }
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+            const int row = r0 + 4 * ty + e;
+            float *dst = a.H + (int64_t)row * n + b0 + 4 * tx;
+            if (vec) {
+                *reinterpret_cast<float4 *>(dst) = make_float4(acc[e][0], acc[e][1], acc[e][2], acc[e][3]);
+            } else {
+#pragma unroll
+                for (int f = 0; f < 4; ++f) if (4 * tx + f < nv) dst[f] = acc[e][f];
+            }
+            if (a.pan_hi) {
+                float hv[4], lv[4];
+#pragma unroll
+                for (int f = 0; f < 4; ++f) { hv[f] = tf32_rn(acc[e][f]); lv[f] = tf32_rn(acc[e][f] - hv[f]); }
+                *reinterpret_cast<float4 *>(a.pan_hi + (int64_t)row * NB + 4 * tx) = make_float4(hv[0], hv[1], hv[2], hv[3]);
+                *reinterpret_cast<float4 *>(a.pan_lo + (int64_t)row * NB + 4 * tx) = make_float4(lv[0], lv[1], lv[2], lv[3]);
+            }
+        }
+    }
 }
 
 // Copies the inverted diagonal blocks (NB x NB each) onto the diagonal of H.
