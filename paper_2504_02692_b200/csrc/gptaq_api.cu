@@ -204,14 +204,21 @@ cudaError_t launch_tc_gemm(const TcMaps &m, const TcGemmArgs &a, int num_sms, cu
     return cudaGetLastError();
 }
 
+struct SplitBatch {
+    int nbatch = 1;
+    int64_t src_bstride = 0, dst_bstride = 0;
+    int rows_last = 0, cols_last = 0;
+};
+
 cudaError_t launch_split(const float *src, int64_t lds, float *hi, float *lo, int64_t ldd, int rows, int cols,
-                         bool transpose, int mask, float scale, cudaStream_t s) {
-    if (rows <= 0 || cols <= 0) return cudaSuccess;
+                         bool transpose, int mask, float scale, cudaStream_t s, const SplitBatch &b = SplitBatch()) {
+    if (rows <= 0 || cols <= 0 || b.nbatch <= 0) return cudaSuccess;
     SplitArgs a;
-    a.src = src; a.lds = lds; a.src_bstride = 0; a.hi = hi; a.lo = lo; a.ldd = ldd; a.dst_bstride = 0;
-    a.rows = rows; a.cols = cols; a.rows_last = a.cols_last = 0; a.nbatch = 1;
+    a.src = src; a.lds = lds; a.src_bstride = b.src_bstride; a.hi = hi; a.lo = lo; a.ldd = ldd;
+    a.dst_bstride = b.dst_bstride;
+    a.rows = rows; a.cols = cols; a.rows_last = b.rows_last; a.cols_last = b.cols_last; a.nbatch = b.nbatch;
     a.transpose = transpose ? 1 : 0; a.mask = mask; a.scale = scale;
-    dim3 grid((cols + 63) / 64, (rows + 63) / 64, 1);
+    dim3 grid((cols + 63) / 64, (rows + 63) / 64, b.nbatch);
     split_kernel<<<grid, 256, 0, s>>>(a);
     return cudaGetLastError();
 }
@@ -488,6 +495,8 @@ gptaq_status_t gptaq_create(gptaq_handle_t *out, int64_t n, void *d_state, size_
         e = cudaFuncSetAttribute(column_loop_kernel<4>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                  2 * 128 * 128 * (int)sizeof(float));
     if (e == cudaSuccess)
+        e = cudaFuncSetAttribute(invert_diag_blocks_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)ID_SMEM);
+    if (e == cudaSuccess)
         e = cudaFuncSetAttribute(stats_umma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)UMMA_SMEM);
     if (e == cudaSuccess)
         e = cudaFuncSetAttribute(tc_gemm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)TC_SMEM);
@@ -592,9 +601,10 @@ gptaq_status_t gptaq_factor(gptaq_handle_t h, float damp, gptaq_stream_t stream)
         const int b0 = p * NB;
         // diagonal block (factor + inverse) and the panel above it: R[0:b0, blk] = A[0:b0, blk] inv(R_pp)^T
         FactorPanelArgs fa;
-        fa.H = H; fa.n = n; fa.b0 = b0; fa.Rinv = Rinv + (size_t)p * NB * NB;
+        fa.H = H; fa.n = n; fa.b0 = b0; fa.Rdiag = Rinv + (size_t)p * NB * NB;
         fa.pan_hi = pan_hi; fa.pan_lo = pan_lo; fa.hd = h->hd;
         const int fgrid = std::max(1, std::min(b0 / NB, h->num_sms));
+        fa.rows_per_cta = ((b0 + fgrid - 1) / fgrid + NB - 1) / NB * NB;
         factor_panel_kernel<<<fgrid, FP_THREADS, FP_SMEM, s>>>(fa);
         LAUNCHED();
         if (p == 0) break;
@@ -612,12 +622,49 @@ gptaq_status_t gptaq_factor(gptaq_handle_t h, float damp, gptaq_stream_t stream)
 
     // U = R^-1: inverted diagonal blocks, then off-diagonal blocks by doubling:
     // inv([[A, B], [0, C]]) = [[A^-1, -A^-1 B C^-1], [0, C^-1]]
-    place_diag_inverse_kernel<<<nb, 256, 0, s>>>(H, n, Rinv);
+    invert_diag_blocks_kernel<<<nb, ID_THREADS, ID_SMEM, s>>>(H, n, Rinv);
     LAUNCHED();
+    float *S1h = nullptr, *S1l = nullptr, *S2h = nullptr, *S2l = nullptr;
+    TcMaps inv_maps;
+    if (h->tensor) {
+        S1h = reinterpret_cast<float *>(h->ws + wl.s_off[0]); S1l = reinterpret_cast<float *>(h->ws + wl.s_off[1]);
+        S2h = reinterpret_cast<float *>(h->ws + wl.s_off[2]); S2l = reinterpret_cast<float *>(h->ws + wl.s_off[3]);
+        const SplitOperand A{S1h, S1l, n, n, n}, B{S2h, S2l, n, n, n};
+        if (!make_tc_maps(&inv_maps, A, B, nullptr)) { h->cuda_error = "cuTensorMapEncodeTiled failed"; return GPTAQ_ERR_CUDA; }
+    }
     for (int64_t sz = NB; sz < n; sz *= 2) {
         const int np = (int)((n - sz + 2 * sz - 1) / (2 * sz));
         const int tail = (int)(n - (2 * sz * (np - 1) + sz));
         const int64_t bstride = 2 * sz * ((int64_t)n + 1);
+        if (h->tensor && sz >= 2 * NB) {
+            // Same two products on the tensor cores.  S1 holds K-major copies of the left operands at
+            // their own coordinates (B, then A^-1), S2 the transposed right operands (C^-T, then T^T).
+            SplitBatch sb; sb.nbatch = np; sb.src_bstride = sb.dst_bstride = bstride;
+            SplitBatch sbt = sb; sbt.cols_last = tail;                 // blocks with `tail` columns
+            SplitBatch sbc = sb; sbc.rows_last = tail; sbc.cols_last = tail;
+            CU(launch_split(H + sz, n, S1h + sz, S1l + sz, n, (int)sz, (int)sz, false, SPLIT_ALL, 1.f, s, sbt));
+            h->launches++;
+            CU(launch_split(H + sz * n + sz, n, S2h + sz * n + sz, S2l + sz * n + sz, n, (int)sz, (int)sz, true,
+                            SPLIT_UPPER, 1.f, s, sbc));
+            h->launches++;
+            TcGemmArgs g1 = tc_args(T + sz, n, (int)sz, (int)sz, (int)sz, 1.f, 0.f, TC_TRI_RIGHT, TC_MASK_NONE, h->hd);
+            g1.nbatch = np; g1.c_bstride = bstride; g1.N_last = tail; g1.K_last = tail;
+            g1.a_row0 = 0; g1.a_row_bs = (int)(2 * sz); g1.a_k0 = (int)sz; g1.a_k_bs = (int)(2 * sz);
+            g1.b_row0 = (int)sz; g1.b_row_bs = (int)(2 * sz); g1.b_k0 = (int)sz; g1.b_k_bs = (int)(2 * sz);
+            CU(launch_tc_gemm(inv_maps, g1, h->num_sms, s));
+            h->launches++;
+            CU(launch_split(H, n, S1h, S1l, n, (int)sz, (int)sz, false, SPLIT_UPPER, 1.f, s, sb));
+            h->launches++;
+            CU(launch_split(T + sz, n, S2h + sz * n, S2l + sz * n, n, (int)sz, (int)sz, true, SPLIT_ALL, 1.f, s, sbt));
+            h->launches++;
+            TcGemmArgs g2 = tc_args(H + sz, n, (int)sz, (int)sz, (int)sz, -1.f, 0.f, TC_TRI_LEFT, TC_MASK_NONE, h->hd);
+            g2.nbatch = np; g2.c_bstride = bstride; g2.N_last = tail;
+            g2.a_row0 = 0; g2.a_row_bs = (int)(2 * sz); g2.a_k0 = 0; g2.a_k_bs = (int)(2 * sz);
+            g2.b_row0 = (int)sz; g2.b_row_bs = (int)(2 * sz); g2.b_k0 = 0; g2.b_k_bs = (int)(2 * sz);
+            CU(launch_tc_gemm(inv_maps, g2, h->num_sms, s));
+            h->launches++;
+            continue;
+        }
         // T = B * C^-1
         GemmProblem p1 = make_problem(make_operand(H + sz, n, 1),
                                       make_operand(H + sz * n + sz, 1, n), T + sz, n,
@@ -634,9 +681,6 @@ gptaq_status_t gptaq_factor(gptaq_handle_t h, float damp, gptaq_stream_t stream)
     }
     if (h->tensor) {
         // operand copies of U for the products that follow: S1 = split(U), S2 = split(U^T)
-        WsLayout w = ws_layout(h->n, 0, 32);
-        float *S1h = reinterpret_cast<float *>(h->ws + w.s_off[0]), *S1l = reinterpret_cast<float *>(h->ws + w.s_off[1]);
-        float *S2h = reinterpret_cast<float *>(h->ws + w.s_off[2]), *S2l = reinterpret_cast<float *>(h->ws + w.s_off[3]);
         CU(launch_split(H, n, S1h, S1l, n, n, n, false, SPLIT_UPPER, 1.f, s));
         h->launches++;
         CU(launch_split(H, n, S2h, S2l, n, n, n, true, SPLIT_UPPER, 1.f, s));

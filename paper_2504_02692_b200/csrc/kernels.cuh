@@ -81,213 +81,387 @@ __global__ void __launch_bounds__(256) scale_damp_kernel(float *H, int n, const 
 // ---------------------------------------------------------------------------
 // One panel step of the reverse Cholesky  H_d = R R^T  (R upper), block column
 // [b0, b0 + NB):
-//   1. factor the NB x NB diagonal block from its last row/column upwards and invert the
-//      factor, both in shared memory (32-wide sub-blocks: one warp factors and inverts a
-//      32 x 32 block in registers, all warps apply it);
-//   2. rows above the block:  R[0:b0, blk] = A[0:b0, blk] * inv(R_pp)^T, written back in
-//      place and, if asked for, as TF32 hi/lo parts for the tensor-core rank-NB update.
-// Every CTA repeats step 1 (it is short and the other SMs would idle) and then takes row
-// tiles of step 2; CTA 0 stores inv(R_pp).  R_pp itself is not stored: nothing reads it.
+//   1. factor the NB x NB diagonal block from its last row/column upwards in shared memory,
+//      32 columns at a time: one warp factors the 32 x 32 diagonal sub-block in registers
+//      (lane = row, shuffles), the rows above it are solved against the sub-block one thread
+//      per row, and the leading part receives the rank-32 update;
+//   2. rows above the block:  R[0:b0, blk] = A[0:b0, blk] * R_pp^-T  by back substitution,
+//      one thread per row with the row in registers (R_pp is read from shared memory as
+//      broadcasts); written back in place and, if asked for, as TF32 hi/lo parts for the
+//      tensor-core rank-NB update.
+// Every CTA repeats step 1 (it is short and the other SMs would idle) and then takes a
+// slab of rows of step 2; CTA 0 stores R_pp for invert_diag_blocks_kernel.
 // Rows/columns beyond n are padded with the identity.
 // ---------------------------------------------------------------------------
 constexpr int NB = 128;
-constexpr int FP_THREADS = 1024;
+constexpr int FP_THREADS = 256;
+constexpr int FP_WARPS = FP_THREADS / 32;
 constexpr int FP_LD = NB + 4;
-constexpr size_t FP_SMEM = (2 * NB * FP_LD + 32 + 2 * 32 * 33) * sizeof(float);
+constexpr size_t FP_SMEM = (2 * NB * FP_LD + 32 * FP_LD + NB) * sizeof(float);
 
 struct FactorPanelArgs {
     float *H; int n; int b0;
-    float *Rinv;               // NB x NB (ld NB): inverse of the diagonal factor
+    float *Rdiag;              // NB x NB (ld NB): the diagonal factor R_pp (upper, zeros below)
     float *pan_hi, *pan_lo;    // nullptr, or [n][NB]: TF32 parts of the panel rows
+    int rows_per_cta;          // slab of step 2, a multiple of NB
     StateHeader *hd;
 };
 
+template <int K, int LEN>
+struct SolveRowStep {
+    static __device__ __forceinline__ void run(float (&a)[LEN], const float *Rt, int ld, const float *dinv) {
+        const float x = a[K] * dinv[K];
+        a[K] = x;
+        const float *col = Rt + K * ld;
+#pragma unroll
+        for (int j4 = 0; j4 < (K + 3) / 4; ++j4) {
+            const float4 r = *reinterpret_cast<const float4 *>(col + 4 * j4);
+            if (4 * j4 + 0 < K) a[4 * j4 + 0] = fmaf(-x, r.x, a[4 * j4 + 0]);
+            if (4 * j4 + 1 < K) a[4 * j4 + 1] = fmaf(-x, r.y, a[4 * j4 + 1]);
+            if (4 * j4 + 2 < K) a[4 * j4 + 2] = fmaf(-x, r.z, a[4 * j4 + 2]);
+            if (4 * j4 + 3 < K) a[4 * j4 + 3] = fmaf(-x, r.w, a[4 * j4 + 3]);
+        }
+        SolveRowStep<K - 1, LEN>::run(a, Rt, ld, dinv);
+    }
+};
+template <int LEN>
+struct SolveRowStep<-1, LEN> {
+    static __device__ __forceinline__ void run(float (&)[LEN], const float *, int, const float *) {}
+};
+template <int LEN>
+__device__ __forceinline__ void solve_row(float (&a)[LEN], const float *Rt, int ld, const float *dinv) {
+    SolveRowStep<LEN - 1, LEN>::run(a, Rt, ld, dinv);
+}
+
+// One column step (K, then K - 1, ... 0) of the 32 x 32 reverse Cholesky held one row per lane.
+// `piv` is the pivot of this step, already broadcast: the dependent chain from one pivot to the
+// next runs through lane K - 1 alone (its own c), the other lanes' updates overlap with it.
+template <int K>
+struct Chol32Step {
+    static __device__ __forceinline__ void run(float (&d)[32], float piv, int lane, float *dinv,
+                                               StateHeader *hd, bool report, int col0) {
+        if (!(piv > 0.f) || !isfinite(piv)) {
+            if (lane == 0 && report) record_status(hd, ST_NOT_SPD, col0 + K);
+            piv = 1.f;
+        }
+        // 1/sqrt(piv): hardware estimate plus one Newton step (to about one ulp)
+        float rinv = rsqrtf(piv);
+        rinv = rinv * fmaf(-0.5f * piv, rinv * rinv, 1.5f);
+        const float c = lane < K ? d[K] * rinv : 0.f;
+        d[K] = lane < K ? c : (lane == K ? piv * rinv : 0.f);
+        if (lane == K) dinv[K] = rinv;
+        float next = 0.f;
+        if (K > 0) {
+            next = __shfl_sync(0xffffffffu, fmaf(-c, c, d[K - 1]), K - 1);
+#pragma unroll
+            for (int j = K - 1; j >= 0; --j) d[j] = fmaf(-c, __shfl_sync(0xffffffffu, c, j), d[j]);
+        }
+        Chol32Step<K - 1>::run(d, next, lane, dinv, hd, report, col0);
+    }
+};
+template <>
+struct Chol32Step<-1> {
+    static __device__ __forceinline__ void run(float (&)[32], float, int, float *, StateHeader *, bool, int) {}
+};
+
+// C[0:128, 0:o] -= Xt^T * Rt  with Xt[k][row] (32 x 128) and Rt[k][j] (32 x o), both in shared
+// memory with leading dimension FP_LD; C row-major with leading dimension FP_LD.  4 x 8 outputs
+// per thread, all threads of the CTA.
+__device__ __forceinline__ void panel_rank32_update(float (*C)[FP_LD], const float (*Xt)[FP_LD],
+                                                    const float (*Rt)[FP_LD], int o, int tid) {
+    const int tiles_j = o / 8;
+    for (int t = tid; t < 32 * tiles_j; t += FP_THREADS) {
+        const int ti = t / tiles_j, tj = t - ti * tiles_j;
+        float acc[4][8];
+#pragma unroll
+        for (int e = 0; e < 4; ++e)
+#pragma unroll
+            for (int f = 0; f < 8; ++f) acc[e][f] = 0.f;
+#pragma unroll 4
+        for (int k = 0; k < 32; ++k) {
+            const float4 xa = *reinterpret_cast<const float4 *>(&Xt[k][4 * ti]);
+            const float4 r0 = *reinterpret_cast<const float4 *>(&Rt[k][8 * tj]);
+            const float4 r1 = *reinterpret_cast<const float4 *>(&Rt[k][8 * tj + 4]);
+            const float av[4] = {xa.x, xa.y, xa.z, xa.w};
+            const float bv[8] = {r0.x, r0.y, r0.z, r0.w, r1.x, r1.y, r1.z, r1.w};
+#pragma unroll
+            for (int e = 0; e < 4; ++e)
+#pragma unroll
+                for (int f = 0; f < 8; ++f) acc[e][f] = fmaf(av[e], bv[f], acc[e][f]);
+        }
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+            float4 *c0 = reinterpret_cast<float4 *>(&C[4 * ti + e][8 * tj]);
+            float4 v0 = c0[0], v1 = c0[1];
+            v0.x -= acc[e][0]; v0.y -= acc[e][1]; v0.z -= acc[e][2]; v0.w -= acc[e][3];
+            v1.x -= acc[e][4]; v1.y -= acc[e][5]; v1.z -= acc[e][6]; v1.w -= acc[e][7];
+            c0[0] = v0; c0[1] = v1;
+        }
+    }
+}
+
 __global__ void __launch_bounds__(FP_THREADS, 1) factor_panel_kernel(FactorPanelArgs a) {
-    extern __shared__ float smem_f[];
+    extern __shared__ __align__(16) float smem_f[];
+    // S: upper part = the working block, then R; lower part = R^T as it is produced
     float (*S)[FP_LD] = reinterpret_cast<float (*)[FP_LD]>(smem_f);
-    float (*X)[FP_LD] = reinterpret_cast<float (*)[FP_LD]>(smem_f + NB * FP_LD);
-    float *colbuf = smem_f + 2 * NB * FP_LD;
-    float (*T32)[32][33] = reinterpret_cast<float (*)[32][33]>(colbuf + 32);
+    float (*At)[FP_LD] = reinterpret_cast<float (*)[FP_LD]>(smem_f + NB * FP_LD);         // step 2: a tile of panel rows
+    float (*Pt)[FP_LD] = reinterpret_cast<float (*)[FP_LD]>(smem_f + 2 * NB * FP_LD);     // Pt[k][i]: 32 solved columns, transposed
+    float *dinv = smem_f + 2 * NB * FP_LD + 32 * FP_LD;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int n = a.n, b0 = a.b0;
     const int nv = min(NB, n - b0);
+    const bool vec = (n & 3) == 0 && (reinterpret_cast<uintptr_t>(a.H) & 15) == 0 && nv == NB;
 
-    for (int i = warp; i < NB; i += 32)
-        for (int j = lane; j < NB; j += 32) {
-            float v;
-            if (i < nv && j < nv) {
-                const int lo = min(i, j), hi = max(i, j);
-                v = a.H[(int64_t)(b0 + lo) * n + (b0 + hi)];
-            } else {
-                v = (i == j) ? 1.f : 0.f;
-            }
-            S[i][j] = v;
-            X[i][j] = 0.f;
+    // the block, read along rows (all loads in flight before the first store); only j >= i is used
+    if (vec) {
+        float4 v[NB * NB / 4 / FP_THREADS];
+#pragma unroll
+        for (int it = 0; it < NB * NB / 4 / FP_THREADS; ++it) {
+            const int idx = tid + it * FP_THREADS, i = idx >> 5, j4 = idx & 31;
+            v[it] = *reinterpret_cast<const float4 *>(a.H + (int64_t)(b0 + i) * n + b0 + 4 * j4);
         }
+#pragma unroll
+        for (int it = 0; it < NB * NB / 4 / FP_THREADS; ++it) {
+            const int idx = tid + it * FP_THREADS, i = idx >> 5, j4 = idx & 31;
+            *reinterpret_cast<float4 *>(&S[i][4 * j4]) = v[it];
+        }
+    } else {
+        for (int i = warp; i < NB; i += FP_WARPS) {
+            const float *src = a.H + (int64_t)(b0 + i) * n + b0;
+            for (int j = lane; j < NB; j += 32) {
+                float v = (i == j) ? 1.f : 0.f;
+                if (i < nv && j < nv && j >= i) v = src[j];
+                S[i][j] = v;
+            }
+        }
+    }
     __syncthreads();
 
     for (int sb = NB / 32 - 1; sb >= 0; --sb) {
         const int o = 32 * sb;
         if (warp == 0) {
-            // ---- 32 x 32 reverse Cholesky, lane = row, then its inverse, lane = column
+            // ---- 32 x 32 reverse Cholesky in registers, lane = row
             float d[32];
 #pragma unroll
-            for (int j = 0; j < 32; ++j) d[j] = S[o + lane][o + j];
+            for (int j = 0; j < 32; ++j) d[j] = (j >= lane) ? S[o + lane][o + j] : S[o + j][o + lane];
+            Chol32Step<31>::run(d, __shfl_sync(0xffffffffu, d[31], 31), lane, dinv + o, a.hd, blockIdx.x == 0, b0 + o);
+            // R_ss to the upper part, its transpose to the lower part
 #pragma unroll
-            for (int k = 31; k >= 0; --k) {
-                float piv = __shfl_sync(0xffffffffu, d[k], k);
-                if (!(piv > 0.f) || !isfinite(piv)) {
-                    if (lane == 0 && blockIdx.x == 0) record_status(a.hd, ST_NOT_SPD, b0 + o + k);
-                    piv = 1.f;
-                }
-                const float r = sqrtf(piv);
-                const float c = lane < k ? d[k] / r : 0.f;
-                d[k] = lane < k ? c : (lane == k ? r : 0.f);
-                colbuf[lane] = c;
-                __syncwarp();
-#pragma unroll
-                for (int j = 0; j < k; ++j) d[j] = fmaf(-c, colbuf[j], d[j]);
-                __syncwarp();
-            }
-#pragma unroll
-            for (int j = 0; j < 32; ++j) S[o + lane][o + j] = j >= lane ? d[j] : 0.f;
-            __syncwarp();
+            for (int j = 0; j < 32; ++j)
+                if (j >= lane) { S[o + lane][o + j] = d[j]; S[o + j][o + lane] = d[j]; }
+        }
+        __syncthreads();
+        // ---- rows above: x R_ss^T = S[i, sub], one thread per row; results go to the upper part,
+        //      to the lower part (transposed) and to Pt for the update
+        if (tid < o) {
+            const int i = tid;
             float x[32];
 #pragma unroll
-            for (int i = 31; i >= 0; --i) {
-                float sum = (i == lane) ? 1.f : 0.f;
+            for (int k = 0; k < 32; ++k) x[k] = S[i][o + k];
+            solve_row<32>(x, &S[o][o], FP_LD, dinv + o);
 #pragma unroll
-                for (int k = i + 1; k < 32; ++k) sum = fmaf(-S[o + i][o + k], x[k], sum);
-                x[i] = i <= lane ? sum / S[o + i][o + i] : 0.f;
+            for (int k = 0; k < 32; ++k) { S[i][o + k] = x[k]; S[o + k][i] = x[k]; Pt[k][i] = x[k]; }
+        }
+        __syncthreads();
+        // ---- leading part: S[i][j] -= R[i, sub] . R[j, sub] for i <= j < o, 4 x 4 per thread
+        {
+            const int q = o / 4;                    // 4 x 4 tiles per side
+            for (int t = tid; t < q * q; t += FP_THREADS) {
+                const int ti = t / q, tj = t - ti * q;
+                if (tj < ti) continue;
+                float acc[4][4];
+#pragma unroll
+                for (int e = 0; e < 4; ++e)
+#pragma unroll
+                    for (int f = 0; f < 4; ++f) acc[e][f] = 0.f;
+#pragma unroll 8
+                for (int k = 0; k < 32; ++k) {
+                    const float4 ri = *reinterpret_cast<const float4 *>(&Pt[k][4 * ti]);
+                    const float4 rj = *reinterpret_cast<const float4 *>(&Pt[k][4 * tj]);
+                    const float av[4] = {ri.x, ri.y, ri.z, ri.w}, bv[4] = {rj.x, rj.y, rj.z, rj.w};
+#pragma unroll
+                    for (int e = 0; e < 4; ++e)
+#pragma unroll
+                        for (int f = 0; f < 4; ++f) acc[e][f] = fmaf(av[e], bv[f], acc[e][f]);
+                }
+#pragma unroll
+                for (int e = 0; e < 4; ++e)
+#pragma unroll
+                    for (int f = 0; f < 4; ++f)
+                        if (4 * tj + f >= 4 * ti + e) S[4 * ti + e][4 * tj + f] -= acc[e][f];
             }
-#pragma unroll
-            for (int i = 0; i < 32; ++i) X[o + i][o + lane] = x[i];
-        }
-        __syncthreads();
-        // ---- rows above: R[i, sub] = S[i, sub] * inv(R_ss)^T   (one warp per row, in place)
-        for (int i = warp; i < o; i += 32) {
-            float acc = 0.f;
-#pragma unroll 8
-            for (int k = 0; k < 32; ++k) acc = fmaf(S[i][o + k], X[o + lane][o + k], acc);
-            __syncwarp();
-            S[i][o + lane] = acc;
-        }
-        __syncthreads();
-        // ---- leading part: S[i][j] -= R[i, sub] . R[j, sub]  (kept symmetric)
-        for (int idx = tid; idx < o * o; idx += FP_THREADS) {
-            const int i = idx / o, j = idx - i * o;
-            if (j < i) continue;
-            float acc = 0.f;
-#pragma unroll 8
-            for (int k = 0; k < 32; ++k) acc = fmaf(S[i][o + k], S[j][o + k], acc);
-            const float v = S[i][j] - acc;
-            S[i][j] = v;
-            S[j][i] = v;
         }
         __syncthreads();
     }
 
-    // ---- off-diagonal blocks of X = R^-1:  X12 = -X11 (R12 X22), 32 -> 64 -> 128
-    for (int idx = tid; idx < 2 * 1024; idx += FP_THREADS) {
-        const int pr = idx >> 10, i = (idx >> 5) & 31, j = idx & 31;
-        const int oa = 64 * pr, oc = oa + 32;
-        float acc = 0.f;
-        for (int k = 0; k <= j; ++k) acc = fmaf(S[oa + i][oc + k], X[oc + k][oc + j], acc);
-        T32[pr][i][j] = acc;
-    }
-    __syncthreads();
-    for (int idx = tid; idx < 2 * 1024; idx += FP_THREADS) {
-        const int pr = idx >> 10, i = (idx >> 5) & 31, j = idx & 31;
-        const int oa = 64 * pr, oc = oa + 32;
-        float acc = 0.f;
-        for (int k = i; k < 32; ++k) acc = fmaf(X[oa + i][oa + k], T32[pr][k][j], acc);
-        X[oa + i][oc + j] = -acc;
-    }
-    __syncthreads();
-    // T64 = R[0:64, 64:128] X[64:128, 64:128], parked in the (still unused) lower-left of X
-    for (int idx = tid; idx < 64 * 64; idx += FP_THREADS) {
-        const int i = idx >> 6, j = idx & 63;
-        float acc = 0.f;
-        for (int k = 0; k <= j; ++k) acc = fmaf(S[i][64 + k], X[64 + k][64 + j], acc);
-        X[64 + i][j] = acc;
-    }
-    __syncthreads();
-    for (int idx = tid; idx < 64 * 64; idx += FP_THREADS) {
-        const int i = idx >> 6, j = idx & 63;
-        float acc = 0.f;
-        for (int k = i; k < 64; ++k) acc = fmaf(X[i][k], X[64 + k][j], acc);
-        X[i][64 + j] = -acc;
-    }
-    __syncthreads();
-    for (int idx = tid; idx < 64 * 64; idx += FP_THREADS) X[64 + (idx >> 6)][idx & 63] = 0.f;
-    __syncthreads();
     if (blockIdx.x == 0)
-        for (int idx = tid; idx < NB * NB; idx += FP_THREADS) a.Rinv[idx] = X[idx >> 7][idx & 127];
+        for (int idx = tid; idx < NB * NB; idx += FP_THREADS) {
+            const int i = idx >> 7, j = idx & 127;
+            a.Rdiag[idx] = j >= i ? S[i][j] : 0.f;
+        }
     if (b0 == 0) return;
 
-    // ---- X <- X^T in place, so that a thread reads four consecutive columns of inv(R_pp)^T at once
-    for (int idx = tid; idx < NB * NB; idx += FP_THREADS) {
-        const int i = idx >> 7, j = idx & 127;
-        if (j > i) { const float u = X[i][j]; X[i][j] = X[j][i]; X[j][i] = u; }
-    }
-    // (the first tile's load below ends with a barrier)
-
-    const int ntiles = b0 / NB;              // b0 is a multiple of NB
-    const int ty = tid >> 5, tx = tid & 31;  // rows 4 ty .. 4 ty + 3, columns 4 tx .. 4 tx + 3
-    const bool vec = (n & 3) == 0 && (reinterpret_cast<uintptr_t>(a.H) & 15) == 0 && nv == NB;
-    for (int rt = blockIdx.x; rt < ntiles; rt += gridDim.x) {
-        const int r0 = rt * NB;
-        __syncthreads();                     // previous tile's reads of S are done
-        for (int i = warp; i < NB; i += 32) {
-            const float *src = a.H + (int64_t)(r0 + i) * n + b0;
-            for (int k = lane; k < NB; k += 32) S[i][k] = k < nv ? src[k] : 0.f;
+    // ---- step 2: rows [r_begin, r_end) of the panel in tiles of NB rows: a blocked triangular
+    //      solve, 32 columns at a time (one thread per row), then a rank-32 update of the
+    //      columns to the left (all threads)
+    const int r_begin = blockIdx.x * a.rows_per_cta;
+    const int r_end = min(b0, r_begin + a.rows_per_cta);
+    for (int r0 = r_begin; r0 < r_end; r0 += NB) {        // b0 and the slabs are multiples of NB
+        if (vec) {
+            float4 v[NB * NB / 4 / FP_THREADS];
+#pragma unroll
+            for (int it = 0; it < NB * NB / 4 / FP_THREADS; ++it) {
+                const int idx = tid + it * FP_THREADS, i = idx >> 5, j4 = idx & 31;
+                v[it] = *reinterpret_cast<const float4 *>(a.H + (int64_t)(r0 + i) * n + b0 + 4 * j4);
+            }
+#pragma unroll
+            for (int it = 0; it < NB * NB / 4 / FP_THREADS; ++it) {
+                const int idx = tid + it * FP_THREADS, i = idx >> 5, j4 = idx & 31;
+                *reinterpret_cast<float4 *>(&At[i][4 * j4]) = v[it];
+            }
+        } else {
+            for (int i = warp; i < NB; i += FP_WARPS) {
+                const float *src = a.H + (int64_t)(r0 + i) * n + b0;
+                for (int k = lane; k < NB; k += 32) At[i][k] = k < nv ? src[k] : 0.f;
+            }
         }
         __syncthreads();
-        float acc[4][4];
+        for (int sb = NB / 32 - 1; sb >= 0; --sb) {
+            const int o = 32 * sb;
+            if (tid < NB) {
+                float x[32];
 #pragma unroll
-        for (int e = 0; e < 4; ++e)
+                for (int k = 0; k < 32; ++k) x[k] = At[tid][o + k];
+                solve_row<32>(x, &S[o][o], FP_LD, dinv + o);
 #pragma unroll
-            for (int f = 0; f < 4; ++f) acc[e][f] = 0.f;
-#pragma unroll 4
-        for (int k = 0; k < NB; ++k) {
-            const float4 b = *reinterpret_cast<const float4 *>(&X[k][4 * tx]);
-            float av[4];
-#pragma unroll
-            for (int e = 0; e < 4; ++e) av[e] = S[4 * ty + e][k];
-#pragma unroll
-            for (int e = 0; e < 4; ++e) {
-                acc[e][0] = fmaf(av[e], b.x, acc[e][0]); acc[e][1] = fmaf(av[e], b.y, acc[e][1]);
-                acc[e][2] = fmaf(av[e], b.z, acc[e][2]); acc[e][3] = fmaf(av[e], b.w, acc[e][3]);
+                for (int k = 0; k < 32; ++k) { At[tid][o + k] = x[k]; Pt[k][tid] = x[k]; }
+            }
+            __syncthreads();
+            if (o > 0) {
+                panel_rank32_update(At, Pt, reinterpret_cast<const float (*)[FP_LD]>(&S[o][0]), o, tid);
+                __syncthreads();
             }
         }
+        // store the tile (and its TF32 parts)
 #pragma unroll
-        for (int e = 0; e < 4; ++e) {
-            const int row = r0 + 4 * ty + e;
-            float *dst = a.H + (int64_t)row * n + b0 + 4 * tx;
+        for (int it = 0; it < NB * NB / 4 / FP_THREADS; ++it) {
+            const int idx = tid + it * FP_THREADS, i = idx >> 5, j4 = idx & 31;
+            const float4 v = *reinterpret_cast<const float4 *>(&At[i][4 * j4]);
+            float *dst = a.H + (int64_t)(r0 + i) * n + b0 + 4 * j4;
             if (vec) {
-                *reinterpret_cast<float4 *>(dst) = make_float4(acc[e][0], acc[e][1], acc[e][2], acc[e][3]);
+                *reinterpret_cast<float4 *>(dst) = v;
             } else {
-#pragma unroll
-                for (int f = 0; f < 4; ++f) if (4 * tx + f < nv) dst[f] = acc[e][f];
+                if (4 * j4 + 0 < nv) dst[0] = v.x;
+                if (4 * j4 + 1 < nv) dst[1] = v.y;
+                if (4 * j4 + 2 < nv) dst[2] = v.z;
+                if (4 * j4 + 3 < nv) dst[3] = v.w;
             }
             if (a.pan_hi) {
+                const float xs[4] = {v.x, v.y, v.z, v.w};
                 float hv[4], lv[4];
 #pragma unroll
-                for (int f = 0; f < 4; ++f) { hv[f] = tf32_rn(acc[e][f]); lv[f] = tf32_rn(acc[e][f] - hv[f]); }
-                *reinterpret_cast<float4 *>(a.pan_hi + (int64_t)row * NB + 4 * tx) = make_float4(hv[0], hv[1], hv[2], hv[3]);
-                *reinterpret_cast<float4 *>(a.pan_lo + (int64_t)row * NB + 4 * tx) = make_float4(lv[0], lv[1], lv[2], lv[3]);
+                for (int f = 0; f < 4; ++f) { hv[f] = tf32_rn(xs[f]); lv[f] = tf32_rn(xs[f] - hv[f]); }
+                *reinterpret_cast<float4 *>(a.pan_hi + (int64_t)(r0 + i) * NB + 4 * j4) = make_float4(hv[0], hv[1], hv[2], hv[3]);
+                *reinterpret_cast<float4 *>(a.pan_lo + (int64_t)(r0 + i) * NB + 4 * j4) = make_float4(lv[0], lv[1], lv[2], lv[3]);
             }
         }
+        __syncthreads();
     }
 }
 
-// Copies the inverted diagonal blocks (NB x NB each) onto the diagonal of H.
-__global__ void __launch_bounds__(256) place_diag_inverse_kernel(float *H, int n, const float *Rinv) {
-    int b0 = blockIdx.x * NB;
-    const float *src = Rinv + (int64_t)blockIdx.x * NB * NB;
-    for (int e = threadIdx.x; e < NB * NB; e += 256) {
-        int i = e / NB, j = e % NB;
-        if (b0 + i < n && b0 + j < n) H[(int64_t)(b0 + i) * n + (b0 + j)] = src[e];
+// ---------------------------------------------------------------------------
+// Inverts every NB x NB diagonal factor R_pp (one CTA each) and stores the inverse on the
+// diagonal of H (strict lower part of the block zero): the starting point of U = R^-1.
+// 32 x 32 diagonal sub-blocks by back substitution (one warp each, lane = column), then
+// X12 = -X11 (R12 X22) for 32 -> 64 -> 128.
+// ---------------------------------------------------------------------------
+constexpr int ID_THREADS = 512;
+constexpr int ID_LD = NB + 1;
+constexpr size_t ID_SMEM = (2 * NB * ID_LD + 2 * 32 * 33) * sizeof(float);
+
+__global__ void __launch_bounds__(ID_THREADS, 1) invert_diag_blocks_kernel(float *H, int n, const float *Rdiag) {
+    extern __shared__ __align__(16) float smem_f[];
+    float (*S)[ID_LD] = reinterpret_cast<float (*)[ID_LD]>(smem_f);
+    float (*X)[ID_LD] = reinterpret_cast<float (*)[ID_LD]>(smem_f + NB * ID_LD);
+    float (*T32)[32][33] = reinterpret_cast<float (*)[32][33]>(smem_f + 2 * NB * ID_LD);
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int b0 = blockIdx.x * NB;
+    const float *src = Rdiag + (int64_t)blockIdx.x * NB * NB;
+    for (int idx = tid; idx < NB * NB; idx += ID_THREADS) {
+        S[idx >> 7][idx & 127] = src[idx];
+        X[idx >> 7][idx & 127] = 0.f;
+    }
+    __syncthreads();
+    if (warp < NB / 32) {
+        const int o = 32 * warp;
+        float x[32];
+#pragma unroll
+        for (int i = 0; i < 32; ++i) x[i] = (i == lane) ? 1.f : 0.f;
+#pragma unroll
+        for (int i = 31; i >= 0; --i) {
+            x[i] = x[i] / S[o + i][o + i];
+#pragma unroll
+            for (int i2 = 0; i2 < i; ++i2) x[i2] = fmaf(-S[o + i2][o + i], x[i], x[i2]);
+        }
+#pragma unroll
+        for (int i = 0; i < 32; ++i) X[o + i][o + lane] = x[i];
+    }
+    __syncthreads();
+    // (the triangular operands carry explicit zeros, so full-length sums are exact)
+    for (int idx = tid; idx < 2 * 1024; idx += ID_THREADS) {
+        const int pr = idx >> 10, i = (idx >> 5) & 31, j = idx & 31;
+        const int oa = 64 * pr, oc = oa + 32;
+        float s0 = 0.f, s1 = 0.f;
+#pragma unroll 8
+        for (int k = 0; k < 32; k += 2) {
+            s0 = fmaf(S[oa + i][oc + k], X[oc + k][oc + j], s0);
+            s1 = fmaf(S[oa + i][oc + k + 1], X[oc + k + 1][oc + j], s1);
+        }
+        T32[pr][i][j] = s0 + s1;
+    }
+    __syncthreads();
+    for (int idx = tid; idx < 2 * 1024; idx += ID_THREADS) {
+        const int pr = idx >> 10, i = (idx >> 5) & 31, j = idx & 31;
+        const int oa = 64 * pr, oc = oa + 32;
+        float s0 = 0.f, s1 = 0.f;
+#pragma unroll 8
+        for (int k = 0; k < 32; k += 2) {
+            s0 = fmaf(X[oa + i][oa + k], T32[pr][k][j], s0);
+            s1 = fmaf(X[oa + i][oa + k + 1], T32[pr][k + 1][j], s1);
+        }
+        X[oa + i][oc + j] = -(s0 + s1);
+    }
+    __syncthreads();
+    // T64 = R[0:64, 64:128] X[64:128, 64:128], parked in the (still unused) lower-left of X
+    for (int idx = tid; idx < 64 * 64; idx += ID_THREADS) {
+        const int i = idx >> 6, j = idx & 63;
+        float s0 = 0.f, s1 = 0.f, s2 = 0.f, s3 = 0.f;
+#pragma unroll 4
+        for (int k = 0; k < 64; k += 4) {
+            s0 = fmaf(S[i][64 + k], X[64 + k][64 + j], s0);
+            s1 = fmaf(S[i][64 + k + 1], X[64 + k + 1][64 + j], s1);
+            s2 = fmaf(S[i][64 + k + 2], X[64 + k + 2][64 + j], s2);
+            s3 = fmaf(S[i][64 + k + 3], X[64 + k + 3][64 + j], s3);
+        }
+        X[64 + i][j] = (s0 + s1) + (s2 + s3);
+    }
+    __syncthreads();
+    for (int idx = tid; idx < 64 * 64; idx += ID_THREADS) {
+        const int i = idx >> 6, j = idx & 63;
+        float s0 = 0.f, s1 = 0.f, s2 = 0.f, s3 = 0.f;
+#pragma unroll 4
+        for (int k = 0; k < 64; k += 4) {
+            s0 = fmaf(X[i][k], X[64 + k][j], s0);
+            s1 = fmaf(X[i][k + 1], X[64 + k + 1][j], s1);
+            s2 = fmaf(X[i][k + 2], X[64 + k + 2][j], s2);
+            s3 = fmaf(X[i][k + 3], X[64 + k + 3][j], s3);
+        }
+        X[i][64 + j] = -((s0 + s1) + (s2 + s3));
+    }
+    __syncthreads();
+    for (int idx = tid; idx < NB * NB; idx += ID_THREADS) {
+        const int i = idx >> 7, j = idx & 127;
+        if (b0 + i < n && b0 + j < n) H[(int64_t)(b0 + i) * n + (b0 + j)] = (j >= i) ? X[i][j] : 0.f;
     }
 }
 
