@@ -346,6 +346,9 @@ gptaq_status_t quantize_core(const QuantizeTarget &t, void *d_W, int w_dtype, in
     nw = std::max(1, std::min(32, nw));
     const unsigned cl_grid = (unsigned)((m + nw - 1) / nw);
     const int T = blocksize / 32;
+    // rows per CTA of the block kernel: enough CTAs for every SM, at most 128 rows each
+    const int cb_rows = 32 * std::max(1, std::min(4, (int)((m + 32 * (int64_t)t.num_sms - 1) / (32 * (int64_t)t.num_sms))));
+    const unsigned cb_grid = (unsigned)((m + cb_rows - 1) / cb_rows);
     const size_t cl_smem = 2 * (size_t)blocksize * blocksize * sizeof(float);
 
     const bool tensor = t.EW_lo != nullptr;
@@ -361,7 +364,10 @@ gptaq_status_t quantize_core(const QuantizeTarget &t, void *d_W, int w_dtype, in
         a.i0 = i0; a.bw = std::min(blocksize, n - i0);
         a.bits = bits; a.group = group; a.sym = sym;
         a.codes = d_codes; a.scales = d_scales; a.zeros = d_zeros; a.G = G; a.EW = EW; a.EW_lo = t.EW_lo; a.hd = t.hd;
-        if (T == 4) column_loop_kernel<4><<<cl_grid, nw * 32, cl_smem, s>>>(a);
+        const bool fast = a.bw == blocksize && (group <= 0 || (group % 32) == 0) && (i0 % 4) == 0 &&
+                          (reinterpret_cast<uintptr_t>(t.dead) & 3) == 0;
+        if (fast) column_block_kernel<<<cb_grid, CB_THREADS, column_block_smem(cb_rows), s>>>(a, cb_rows, blocksize);
+        else if (T == 4) column_loop_kernel<4><<<cl_grid, nw * 32, cl_smem, s>>>(a);
         else if (T == 2) column_loop_kernel<2><<<cl_grid, nw * 32, cl_smem, s>>>(a);
         else column_loop_kernel<1><<<cl_grid, nw * 32, cl_smem, s>>>(a);
         QLAUNCHED();
@@ -439,6 +445,9 @@ cudaError_t static_scratch_for_current_device(StaticScratch **out) {
         e = cudaFuncSetAttribute(column_loop_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                  2 * 64 * 64 * (int)sizeof(float));
         if (e != cudaSuccess) return e;
+        e = cudaFuncSetAttribute(column_block_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 (int)column_block_smem(128));
+        if (e != cudaSuccess) return e;
         sc.base = static_cast<uint8_t *>(ptr);
         sc.ready = true;
     }
@@ -503,6 +512,9 @@ gptaq_status_t gptaq_create(gptaq_handle_t *out, int64_t n, void *d_state, size_
     if (e == cudaSuccess)
         e = cudaFuncSetAttribute(column_loop_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                  2 * 64 * 64 * (int)sizeof(float));
+    if (e == cudaSuccess)
+        e = cudaFuncSetAttribute(column_block_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 (int)column_block_smem(128));
     if (e != cudaSuccess) {
         delete h;
         return GPTAQ_ERR_CUDA;

@@ -604,7 +604,7 @@ __global__ void __launch_bounds__(1024) column_loop_kernel(ColumnLoopArgs a) {
             const float wj = __shfl_sync(0xffffffffu, w[t], jj);
             float cq = fminf(fmaxf(rintf(wj / scale) + zero, 0.f), maxq);
             const float q = scale * (cq - zero);
-            const float ne = (q - wj) / Us[j][j];   // -(w - q) / U_jj
+            const float ne = (q - wj) * (1.f / Us[j][j]);   // -(w - q) / U_jj
             if (lane == jj) { w[t] = q; nerr[t] = ne; pre[t] = wj; code[t] = (int)cq; }
 #pragma unroll
             for (int t2 = 0; t2 < T; ++t2) {
@@ -637,6 +637,216 @@ __global__ void __launch_bounds__(1024) column_loop_kernel(ColumnLoopArgs a) {
         }
     }
     if (bad) record_status(a.hd, ST_NONFINITE, row);
+}
+
+// ---------------------------------------------------------------------------
+// Column loop over one full lazy-batch block [i0, i0 + B), B in {32, 64, 128}, for grids per
+// output channel or per group of a multiple of 32 columns.  One CTA owns `rows` weight rows
+// (a multiple of 32); their block lives in shared memory.  The block is processed 32 columns
+// at a time:
+//   - one thread per row takes the 32 columns into registers and runs the sequential part
+//     (quantize column k, scaled error, rank-1 update of the later columns of the 32) with
+//     the rows k of U and P read from shared memory as broadcasts;
+//   - all threads then apply the 32 columns' errors and pre-quantization values to the rest
+//     of the block, a (rows x 64) x (64 x rest) product out of shared memory.
+// Same outputs as column_loop_kernel.
+// ---------------------------------------------------------------------------
+constexpr int CB_THREADS = 256;
+constexpr int CB_LD = 128 + 4;
+
+__host__ __device__ inline size_t column_block_smem(int rows) {
+    return ((size_t)rows * CB_LD + 2 * 32 * CB_LD + 64 * (rows + 4) + 32) * sizeof(float);
+}
+
+template <int K>
+struct QuantStep {
+    // x: the row's 32 columns (already-updated weights in, dequantized values out)
+    static __device__ __forceinline__ void run(float (&x)[32], float (&nerr)[32], float (&pre)[32], uint32_t (&code)[8],
+                                               const float *Us, const float *Ps, const float *udinv,
+                                               float scale, float zero, float maxq) {
+        const float w = x[K];
+        const float cq = fminf(fmaxf(rintf(w / scale) + zero, 0.f), maxq);
+        const float q = scale * (cq - zero);
+        const float ne = (q - w) * udinv[K];           // -(w - q) / U_kk
+        x[K] = q; nerr[K] = ne; pre[K] = w;
+        code[K >> 2] |= (uint32_t)cq << (8 * (K & 3));
+        const float *ur = Us + K * CB_LD, *pr = Ps + K * CB_LD;
+#pragma unroll
+        for (int j4 = (K + 1) / 4; j4 < 8; ++j4) {
+            const float4 u = *reinterpret_cast<const float4 *>(ur + 4 * j4);
+            const float4 p = *reinterpret_cast<const float4 *>(pr + 4 * j4);
+            if (4 * j4 + 0 > K) x[4 * j4 + 0] = fmaf(w, p.x, fmaf(ne, u.x, x[4 * j4 + 0]));
+            if (4 * j4 + 1 > K) x[4 * j4 + 1] = fmaf(w, p.y, fmaf(ne, u.y, x[4 * j4 + 1]));
+            if (4 * j4 + 2 > K) x[4 * j4 + 2] = fmaf(w, p.z, fmaf(ne, u.z, x[4 * j4 + 2]));
+            if (4 * j4 + 3 > K) x[4 * j4 + 3] = fmaf(w, p.w, fmaf(ne, u.w, x[4 * j4 + 3]));
+        }
+        QuantStep<K + 1>::run(x, nerr, pre, code, Us, Ps, udinv, scale, zero, maxq);
+    }
+};
+template <>
+struct QuantStep<32> {
+    static __device__ __forceinline__ void run(float (&)[32], float (&)[32], float (&)[32], uint32_t (&)[8],
+                                               const float *, const float *, const float *, float, float, float) {}
+};
+
+__global__ void __launch_bounds__(CB_THREADS, 1) column_block_kernel(ColumnLoopArgs a, int rows, int B) {
+    extern __shared__ __align__(16) float smem_f[];
+    float (*Wt)[CB_LD] = reinterpret_cast<float (*)[CB_LD]>(smem_f);                       // [rows][B]
+    float (*Us)[CB_LD] = reinterpret_cast<float (*)[CB_LD]>(smem_f + rows * CB_LD);        // rows o..o+31 of U, block columns
+    float (*Ps)[CB_LD] = Us + 32;
+    float *St = smem_f + rows * CB_LD + 2 * 32 * CB_LD;                                    // [64][rows + 4]: -Err, then Wpre
+    const int sld = rows + 4;
+    float *udinv = St + 64 * sld;
+    const int tid = threadIdx.x;
+    const int n = a.n, i0 = a.i0;
+    const int row0 = blockIdx.x * rows;
+    const int nrows = min(rows, a.m - row0);
+    const int bq = B / 4;
+
+    // the block of W (dead inputs read as zero), along rows
+    for (int idx = tid; idx < rows * bq; idx += CB_THREADS) {
+        const int r = idx / bq, c4 = idx - r * bq;
+        float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (r < nrows) {
+            const float *src = a.W + (int64_t)(row0 + r) * a.ldw + i0 + 4 * c4;
+            if ((reinterpret_cast<uintptr_t>(src) & 15) == 0) v = *reinterpret_cast<const float4 *>(src);
+            else { v.x = src[0]; v.y = src[1]; v.z = src[2]; v.w = src[3]; }
+            const uchar4 dd = *reinterpret_cast<const uchar4 *>(a.dead + i0 + 4 * c4);
+            if (dd.x) v.x = 0.f;
+            if (dd.y) v.y = 0.f;
+            if (dd.z) v.z = 0.f;
+            if (dd.w) v.w = 0.f;
+        }
+        *reinterpret_cast<float4 *>(&Wt[r][4 * c4]) = v;
+    }
+
+    const float maxq = (float)((1 << a.bits) - 1);
+    float scale = 1.f, zero = 0.f;
+    const bool owner = tid < nrows;
+    const int row = row0 + tid;
+    if (a.group <= 0 && owner) { scale = a.scales[row]; zero = a.zeros[row]; }
+
+    for (int o = 0; o < B; o += 32) {
+        __syncthreads();        // the block is current; Us / Ps / St are free
+        for (int idx = tid; idx < 32 * bq; idx += CB_THREADS) {
+            const int k = idx / bq, c4 = idx - k * bq;
+            const int64_t off = (int64_t)(i0 + o + k) * n + i0 + 4 * c4;
+            float4 u, p;
+            if ((n & 3) == 0) {
+                u = *reinterpret_cast<const float4 *>(a.U + off);
+                p = *reinterpret_cast<const float4 *>(a.P + off);
+            } else {
+                u = make_float4(a.U[off], a.U[off + 1], a.U[off + 2], a.U[off + 3]);
+                p = make_float4(a.P[off], a.P[off + 1], a.P[off + 2], a.P[off + 3]);
+            }
+            *reinterpret_cast<float4 *>(&Us[k][4 * c4]) = u;
+            *reinterpret_cast<float4 *>(&Ps[k][4 * c4]) = p;
+        }
+        if (tid < 32) udinv[tid] = 1.f / a.U[(int64_t)(i0 + o + tid) * n + i0 + o + tid];
+        __syncthreads();
+        if (owner) {
+            if (a.group > 0 && ((i0 + o) % a.group) == 0) {
+                // grid of the group that starts here, from the current values
+                float lo = 0.f, hi = 0.f, am = 0.f;
+                const int gend = min(o + a.group, B);
+                for (int c = o; c < gend; ++c) {
+                    const float v = Wt[tid][c];
+                    lo = fminf(lo, v); hi = fmaxf(hi, v); am = fmaxf(am, fabsf(v));
+                }
+                make_grid(lo, hi, am, a.bits, a.sym, scale, zero);
+                const int g = (i0 + o) / a.group;
+                a.scales[(int64_t)row * a.G + g] = scale;
+                a.zeros[(int64_t)row * a.G + g] = zero;
+            }
+            float x[32], nerr[32], pre[32];
+            uint32_t code[8];
+#pragma unroll
+            for (int k4 = 0; k4 < 8; ++k4) {
+                const float4 v = *reinterpret_cast<const float4 *>(&Wt[tid][o + 4 * k4]);
+                x[4 * k4] = v.x; x[4 * k4 + 1] = v.y; x[4 * k4 + 2] = v.z; x[4 * k4 + 3] = v.w;
+                code[k4] = 0u;
+            }
+            QuantStep<0>::run(x, nerr, pre, code, &Us[0][o], &Ps[0][o], udinv, scale, zero, maxq);
+            uint8_t *crow = a.codes + (int64_t)row * n + i0 + o;
+            if ((reinterpret_cast<uintptr_t>(crow) & 15) == 0) {
+                *reinterpret_cast<uint4 *>(crow) = make_uint4(code[0], code[1], code[2], code[3]);
+                *reinterpret_cast<uint4 *>(crow + 16) = make_uint4(code[4], code[5], code[6], code[7]);
+            } else {
+#pragma unroll
+                for (int k = 0; k < 32; ++k) crow[k] = (uint8_t)(code[k >> 2] >> (8 * (k & 3)));
+            }
+            float *ew = a.EW + (int64_t)row * (2 * B) + o;
+            float *ewl = a.EW_lo ? a.EW_lo + (int64_t)row * (2 * B) + o : nullptr;
+#pragma unroll
+            for (int k4 = 0; k4 < 8; ++k4) {
+                *reinterpret_cast<float4 *>(&Wt[tid][o + 4 * k4]) = make_float4(x[4 * k4], x[4 * k4 + 1], x[4 * k4 + 2], x[4 * k4 + 3]);
+                float e4[4] = {nerr[4 * k4], nerr[4 * k4 + 1], nerr[4 * k4 + 2], nerr[4 * k4 + 3]};
+                float p4[4] = {pre[4 * k4], pre[4 * k4 + 1], pre[4 * k4 + 2], pre[4 * k4 + 3]};
+                if (ewl) {
+                    float el[4], pl[4];
+#pragma unroll
+                    for (int f = 0; f < 4; ++f) {
+                        const float eh = tf32_rn(e4[f]), ph = tf32_rn(p4[f]);
+                        el[f] = tf32_rn(e4[f] - eh); pl[f] = tf32_rn(p4[f] - ph);
+                        e4[f] = eh; p4[f] = ph;
+                    }
+                    *reinterpret_cast<float4 *>(ewl + 4 * k4) = make_float4(el[0], el[1], el[2], el[3]);
+                    *reinterpret_cast<float4 *>(ewl + B + 4 * k4) = make_float4(pl[0], pl[1], pl[2], pl[3]);
+                }
+                *reinterpret_cast<float4 *>(ew + 4 * k4) = make_float4(e4[0], e4[1], e4[2], e4[3]);
+                *reinterpret_cast<float4 *>(ew + B + 4 * k4) = make_float4(p4[0], p4[1], p4[2], p4[3]);
+            }
+#pragma unroll
+            for (int k = 0; k < 32; ++k) { St[k * sld + tid] = nerr[k]; St[(32 + k) * sld + tid] = pre[k]; }
+        } else if (tid < rows) {
+#pragma unroll
+            for (int k = 0; k < 64; ++k) St[k * sld + tid] = 0.f;
+        }
+        __syncthreads();
+        // rest of the block: Wt[:, c] += sum_k (-Err)[:, k] U[o + k][c] + Wpre[:, k] P[o + k][c], c >= o + 32
+        const int c_begin = o + 32;
+        if (c_begin < B) {
+            const int tr = rows / 4, tc = (B - c_begin) / 4;
+            for (int t = tid; t < tr * tc; t += CB_THREADS) {
+                const int tj = t / tr, ti = t - tj * tr;            // consecutive threads: consecutive row tiles
+                const int c0 = c_begin + 4 * tj;
+                float acc[4][4];
+#pragma unroll
+                for (int e = 0; e < 4; ++e)
+#pragma unroll
+                    for (int f = 0; f < 4; ++f) acc[e][f] = 0.f;
+#pragma unroll 4
+                for (int k = 0; k < 64; ++k) {
+                    const float4 av4 = *reinterpret_cast<const float4 *>(St + k * sld + 4 * ti);
+                    const float4 bv4 = *reinterpret_cast<const float4 *>(k < 32 ? &Us[k][c0] : &Ps[k - 32][c0]);
+                    const float av[4] = {av4.x, av4.y, av4.z, av4.w}, bv[4] = {bv4.x, bv4.y, bv4.z, bv4.w};
+#pragma unroll
+                    for (int e = 0; e < 4; ++e)
+#pragma unroll
+                        for (int f = 0; f < 4; ++f) acc[e][f] = fmaf(av[e], bv[f], acc[e][f]);
+                }
+#pragma unroll
+                for (int e = 0; e < 4; ++e) {
+                    float4 *cp = reinterpret_cast<float4 *>(&Wt[4 * ti + e][c0]);
+                    float4 v = *cp;
+                    v.x += acc[e][0]; v.y += acc[e][1]; v.z += acc[e][2]; v.w += acc[e][3];
+                    *cp = v;
+                }
+            }
+        }
+    }
+    __syncthreads();
+    // dequantized block back to W
+    bool bad = false;
+    for (int idx = tid; idx < nrows * bq; idx += CB_THREADS) {
+        const int r = idx / bq, c4 = idx - r * bq;
+        const float4 v = *reinterpret_cast<const float4 *>(&Wt[r][4 * c4]);
+        bad |= !isfinite(v.x) || !isfinite(v.y) || !isfinite(v.z) || !isfinite(v.w);
+        float *dst = a.W + (int64_t)(row0 + r) * a.ldw + i0 + 4 * c4;
+        if ((reinterpret_cast<uintptr_t>(dst) & 15) == 0) *reinterpret_cast<float4 *>(dst) = v;
+        else { dst[0] = v.x; dst[1] = v.y; dst[2] = v.z; dst[3] = v.w; }
+        if (bad) record_status(a.hd, ST_NONFINITE, row0 + r);
+    }
 }
 
 __global__ void __launch_bounds__(256) bf16_to_f32_kernel(const __nv_bfloat16 *src, int64_t lds,
