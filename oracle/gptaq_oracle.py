@@ -126,6 +126,25 @@ def build_P_rowwise(D_sum: np.ndarray, tokens: int, U: np.ndarray, alpha: float)
     return alpha * P
 
 
+def build_P_rows(D_rows: np.ndarray, rows, tokens: int, U: np.ndarray, alpha: float,
+                 chunk: int = 2048) -> np.ndarray:
+    """Rows ``rows`` of P by Theorem 4.2, ``P[q, :] = alpha * ((D[q, :] U^T) .* [a > q]) U``, from the
+    matching rows ``D_rows`` of the raw sum dXX^T.  For layers whose n x n matrices are too large
+    to hold several float64 copies of: ``U`` may be float32 and is widened a block of rows at a
+    time."""
+    D_rows = np.asarray(D_rows, dtype=F64) / float(max(tokens, 1))
+    rows = np.asarray(rows)
+    n = U.shape[0]
+    O = np.zeros((len(rows), n), F64)
+    for a0 in range(0, n, chunk):
+        O[:, a0:a0 + chunk] = D_rows @ np.asarray(U[a0:a0 + chunk], dtype=F64).T
+    O *= (np.arange(n)[None, :] > rows[:, None])
+    P = np.zeros((len(rows), n), F64)
+    for k0 in range(0, n, chunk):
+        P += O[:, k0:k0 + chunk] @ np.asarray(U[k0:k0 + chunk], dtype=F64)
+    return alpha * P
+
+
 # --------------------------------------------------------------------------
 # quant(.)  (Section 3.1; setup of Section 5): min/max grid, round half even
 # --------------------------------------------------------------------------
@@ -271,6 +290,25 @@ def objective(W: np.ndarray, Wq: np.ndarray, st: Stats) -> float:
     t2 = float(np.sum((dW @ st.D.T) * W))
     t3 = float(np.sum((W @ st.G) * W)) if st.G is not None else 0.0
     return t1 - 2.0 * t2 + t3
+
+
+def objective_terms_chunked(W, Wq, H_upper: np.ndarray, D: np.ndarray, chunk: int = 2048) -> float:
+    """The W^-dependent part of J, ``tr(dW H dW^T) - 2 tr(dW D^T W^T)``, for (a few rows of) W, from
+    sums that may be float32 and of which H only needs a valid upper triangle: H and D are widened
+    a block of rows at a time, H is completed by symmetry."""
+    W = np.asarray(W, F64)
+    dW = np.asarray(Wq, F64) - W
+    n = W.shape[1]
+    t1 = 0.0
+    t2 = 0.0
+    for a0 in range(0, n, chunk):
+        a1 = min(a0 + chunk, n)
+        Hc = np.triu(np.asarray(H_upper[a0:a1], dtype=F64), k=a0)      # rows a0..a1 of triu(H)
+        left = dW[:, a0:a1] @ Hc                                      # sum_{a in chunk} dW[a] H[a, b], b >= a
+        diag = np.einsum("ra,a,ra->", dW[:, a0:a1], np.diagonal(Hc, offset=a0).copy(), dW[:, a0:a1])
+        t1 += 2.0 * float(np.sum(left * dW)) - float(diag)
+        t2 += float(np.sum((dW @ np.asarray(D[a0:a1], dtype=F64).T) * W[:, a0:a1]))
+    return t1 - 2.0 * t2
 
 
 def objective_direct(W, Wq, X_tm, Xfp_tm) -> float:

@@ -1,0 +1,213 @@
+"""CUDA path vs float64 oracle at the full sizes of the benchmark configurations, in the launch
+configuration bench.py times (token batches generated on the device, streamed through
+gptaq_accumulate, recommended statistics arithmetic).
+
+cfg2 (n = 4096) is compared end to end: the oracle accumulates all 262,144 tokens in float64.
+cfg3 (n = 14,336) and cfg5 (n = 53,248) are too large for that (2e14 / 1.5e15 float64 flops);
+there the oracle checks sampled outputs it can compute one by one and properties that hold at
+any size, stage by stage:
+  statistics   sampled entries H[i, j], dXX^T[i, j] against float64 sums over all tokens;
+  factor       U upper with positive diagonal and  u_i H_d u_j^T = delta_ij  for sampled rows
+               (H_d from the device's own H, widened to float64): orthonormality of the rows of
+               U in the H_d inner product is the definition of the factor, and its defect is
+               twice the relative error of U;
+  P            sampled rows against Theorem 4.2 evaluated in float64 from the device's D and U;
+  loop         sampled rows of W replayed in follow mode and free-running from the device's U
+               and P (rows are independent), with the flip accounting and the objective bound.
+"""
+import time
+
+import numpy as np
+import pytest
+import torch
+
+import paper_2504_02692_b200 as g
+import workloads as wl
+from oracle import gptaq_oracle as orc
+from tests import helpers as hp
+
+pytestmark = pytest.mark.gpu
+
+
+def _run_device_layer(cfg, sample_cols=None, keep_batches=False, W_rows=None):
+    """Streams the layer's token batches through gptaq_accumulate.  On the host, in float64:
+    the oracle's sums restricted to ``sample_cols`` (``sub``), or over all channels (``full``),
+    and ``resid`` = ||W_rows (X~ - X)||_F^2, the part of the objective that no quantizer changes."""
+    torch.cuda.empty_cache()
+    dev = "cuda"
+    st = g.LayerState(cfg.n, cfg.m, cfg.batch_tokens, cfg.blocksize, dev, total_tokens=cfg.tokens)
+    sub = orc.new_stats(len(sample_cols), True) if sample_cols is not None else None
+    full = orc.new_stats(cfg.n, True) if keep_batches else None
+    idx = torch.as_tensor(sample_cols, device=dev) if sample_cols is not None else None
+    resid = 0.0
+    for b in range(cfg.n_batches):
+        X, Xfp = wl.make_batch(cfg, b, dev)
+        g.gptaq_accumulate(st.handle, X, Xfp)
+        if sub is not None:
+            orc.accumulate(sub, X[:, idx].cpu().numpy(), Xfp[:, idx].cpu().numpy())
+        if full is not None:
+            orc.accumulate(full, X.cpu().numpy(), Xfp.cpu().numpy())
+        if W_rows is not None:
+            Xh, Xfh = X.cpu().numpy(), Xfp.cpu().numpy()
+            for t0 in range(0, Xh.shape[0], 2048):
+                dX = Xfh[t0:t0 + 2048].astype(np.float64) - Xh[t0:t0 + 2048].astype(np.float64)
+                resid += float(np.sum((dX @ W_rows.T) ** 2))
+        del X, Xfp
+    assert g.gptaq_sync_status(st.handle)[0] == g.GPTAQ_OK
+    return st, sub, full, resid
+
+
+def _quantize_on_device(cfg, st, W):
+    dev = "cuda"
+    G = hp.n_groups(cfg.n, cfg.group)
+    codes = torch.empty((cfg.m, cfg.n), dtype=torch.uint8, device=dev)
+    scales = torch.empty((cfg.m, G), dtype=torch.float32, device=dev)
+    zeros = torch.empty((cfg.m, G), dtype=torch.float32, device=dev)
+    Wq = torch.empty((cfg.m, cfg.n), dtype=torch.float32, device=dev)
+    Wd = W.to(torch.bfloat16) if cfg.w_bf16 else W
+    g.gptaq_quantize(st.handle, Wd, cfg.bits, cfg.group, cfg.sym, cfg.blocksize, codes, scales, zeros, Wq)
+    status = g.gptaq_sync_status(st.handle)
+    assert status[0] == g.GPTAQ_OK, status
+    return codes, scales, zeros, Wq
+
+
+def _check_rows(cfg, W_rows, U, P, codes, scales, zeros, Wq_rows, objective):
+    """Follow-mode code check and objective values on the sampled rows; ``objective(Wq)`` returns J
+    for these rows."""
+    dead = np.zeros(cfg.n, bool)
+    rep = orc.follow(W_rows, U, P, dead, cfg.bits, cfg.group, cfg.sym, codes, scales, zeros, band=hp.TOL_FLIP_BAND)
+    assert rep.disallowed == 0, rep
+    assert rep.allowed <= hp.TOL_FLIP_RATE * rep.total, rep
+    assert rep.grid_rel_err <= 5e-5 and rep.zero_mismatch == 0, rep
+    res = orc.quantize(W_rows, U, P, dead, cfg.bits, cfg.group, cfg.sym)
+    rtn = orc.quantize(W_rows, U, None, dead, cfg.bits, cfg.group, cfg.sym, update=False)
+    J_gpu, J_orc, J_rtn = objective(Wq_rows), objective(res.Wq), objective(rtn.Wq)
+    assert abs(J_gpu - J_orc) <= hp.TOL_OBJECTIVE * J_orc, (J_gpu, J_orc)
+    assert J_gpu <= J_rtn, (J_gpu, J_rtn)
+    return rep, J_gpu, J_orc, J_rtn, float(np.mean(codes != res.codes))
+
+
+def _rows_to_host(rows, codes, scales, zeros, Wq):
+    r_t = torch.as_tensor(rows, device="cuda")
+    return (codes[r_t].cpu().numpy(), scales[r_t].cpu().numpy().astype(np.float64),
+            zeros[r_t].cpu().numpy().astype(np.float64), Wq[r_t].cpu().numpy().astype(np.float64))
+
+
+def test_cfg2_full_size_end_to_end():
+    cfg = wl.CONFIGS["cfg2"]
+    t0 = time.time()
+    st, _, full, _ = _run_device_layer(cfg, keep_batches=True)
+    H = st.H().cpu().numpy().astype(np.float64)
+    D = st.D().cpu().numpy().astype(np.float64)
+    iu = np.triu_indices(cfg.n)
+    d = np.sqrt(np.diag(full.H))
+    dd = np.sqrt(np.diag(full.G))
+    # entries carry the operand rounding (2^-11 per fp16 factor) times the root of the two diagonals
+    assert (np.abs(H - full.H)[iu] / np.outer(d, d)[iu]).max() < 2.0 ** -10
+    assert (np.abs(D - full.D) / np.outer(dd, d)).max() < 2.0 ** -10
+    del H, D
+    g.gptaq_factor(st.handle, cfg.damp)
+    g.gptaq_build_P(st.handle, cfg.alpha)
+    Ug = st.H().cpu().numpy().astype(np.float64)
+    Pg = st.D().cpu().numpy().astype(np.float64)
+    U, dead = orc.factor(full.H, full.tokens, cfg.damp)
+    P = orc.build_P(full.D, full.tokens, U, cfg.alpha)
+    assert not dead.any()
+    U_rel = hp.rel_fro(np.triu(Ug), U)
+    P_rel = hp.rel_fro(np.triu(Pg, 1), P)
+    assert U_rel <= hp.TOL_FACTOR, U_rel
+    assert np.abs(np.tril(Ug, -1)).max() == 0.0 and np.abs(np.tril(Pg)).max() == 0.0
+    assert P_rel <= 5e-3, P_rel          # P inherits the fp16 rounding of dXX^T (2^-11 per factor)
+    W = wl.make_weight(cfg, "cuda")
+    codes, scales, zeros, Wq = _quantize_on_device(cfg, st, W)
+    rows = np.sort(np.random.default_rng(1).choice(cfg.m, 96, replace=False))
+    W_rows = W[torch.as_tensor(rows, device="cuda")].cpu().numpy().astype(np.float64)
+    rep, J_gpu, J_orc, J_rtn, free = _check_rows(
+        cfg, W_rows, U, P, *_rows_to_host(rows, codes, scales, zeros, Wq),
+        lambda q: orc.objective(W_rows, q, full))
+    print(f"cfg2 full size: U rel {U_rel:.2e}, P rel {P_rel:.2e}, flips {rep.mismatches}/{rep.total} "
+          f"(excused {rep.allowed}), free-running mismatch {free:.2e}, J gpu/oracle/rtn {J_gpu:.6g}/{J_orc:.6g}/{J_rtn:.6g}, "
+          f"{time.time() - t0:.0f} s")
+    st.close()
+
+
+def _upper_quadratic(H_upper_f32, Y, lam, inv_tokens, chunk=2048):
+    """Y (H / tokens + lam I) Y^T in float64 from a float32 matrix whose upper triangle holds H."""
+    n = H_upper_f32.shape[0]
+    HY = np.zeros((n, Y.shape[0]))
+    for a0 in range(0, n, chunk):
+        a1 = min(a0 + chunk, n)
+        Hc = np.triu(H_upper_f32[a0:a1].astype(np.float64), k=a0)
+        HY[a0:a1] += Hc @ Y.T                                  # rows a, columns b >= a
+        HY += np.triu(Hc, k=a0 + 1).T @ Y[:, a0:a1].T          # mirrored strictly-upper part
+    return Y @ (HY * inv_tokens) + lam * (Y @ Y.T)
+
+
+@pytest.mark.parametrize("name,n_rows,n_cols", [("cfg3", 32, 48), ("cfg5", 8, 40)])
+def test_large_configs_sampled_parity(name, n_rows, n_cols):
+    cfg = wl.CONFIGS[name]
+    t0 = time.time()
+    rng = np.random.default_rng(7)
+    cols = np.sort(rng.choice(cfg.n, n_cols, replace=False))
+    rows = np.sort(rng.choice(cfg.m, n_rows, replace=False))
+    W = wl.make_weight(cfg, "cuda")
+    W_rows = W[torch.as_tensor(rows, device="cuda")].cpu().numpy().astype(np.float64)
+    del W
+    st, sub, _, resid = _run_device_layer(cfg, sample_cols=cols, W_rows=W_rows)
+    split = g.gptaq_recommended_stats_precision(cfg.n, cfg.tokens) == g.GPTAQ_STATS_FP16_SPLIT_TENSOR
+    # ---- statistics: sampled entries against float64 sums over all tokens; the error of an entry
+    # is bounded by the operand rounding (2^-11 per fp16 factor) times the root of the two diagonals
+    c_t = torch.as_tensor(cols, device="cuda")
+    Hs = st.H()[c_t][:, c_t].cpu().numpy().astype(np.float64)
+    Ds = st.D()[c_t][:, c_t].cpu().numpy().astype(np.float64)
+    d = np.sqrt(np.diag(sub.H))
+    dd = np.sqrt(np.diag(sub.G))
+    iu = np.triu_indices(n_cols)
+    errH = (np.abs(Hs - sub.H)[iu] / np.outer(d, d)[iu]).max()
+    assert errH < (1e-5 if split else 2.0 ** -10), errH
+    errD = (np.abs(Ds - sub.D) / np.outer(dd, d)).max()
+    assert errD < 2.0 ** -10, errD
+    tokens = cfg.tokens
+    H_host = st.H().cpu().numpy()                              # float32, upper triangle valid
+    D_host = st.D().cpu().numpy()
+    diagH = np.diagonal(H_host).astype(np.float64)
+    assert (diagH > 0).all()
+    lam = cfg.damp * float(np.mean(diagH / tokens))
+    # ---- factor
+    g.gptaq_factor(st.handle, cfg.damp)
+    assert g.gptaq_sync_status(st.handle)[0] == g.GPTAQ_OK
+    Ud = st.H()
+    for r0 in range(0, cfg.n, 4096):                          # strict lower triangle is zero
+        blk = Ud[r0:r0 + 4096, :r0 + 4096]
+        assert float(torch.tril(blk, diagonal=r0 - 1).abs().max()) == 0.0
+    assert float(torch.diagonal(Ud).min()) > 0.0
+    U_host = Ud.cpu().numpy()
+    urows = np.sort(rng.choice(cfg.n, 12, replace=False))
+    urows[0], urows[-1] = 0, cfg.n - 1
+    Gm = _upper_quadratic(H_host, U_host[urows].astype(np.float64), lam, 1.0 / tokens)
+    defect = np.abs(Gm - np.eye(len(urows))).max()
+    assert defect <= 2 * hp.TOL_FACTOR, defect
+    # ---- P: sampled rows against Theorem 4.2 in float64
+    g.gptaq_build_P(st.handle, cfg.alpha)
+    assert g.gptaq_sync_status(st.handle)[0] == g.GPTAQ_OK
+    Pd = st.D()
+    for r0 in range(0, cfg.n, 4096):                          # lower triangle and diagonal are zero
+        blk = Pd[r0:r0 + 4096, :r0 + 4096]
+        assert float(torch.tril(blk, diagonal=r0).abs().max()) == 0.0
+    P_host = Pd.cpu().numpy()
+    prow = np.sort(rng.choice(cfg.n - 1, 6, replace=False))
+    prow[0] = 0
+    P_want = orc.build_P_rows(D_host[prow], prow, tokens, U_host, cfg.alpha)
+    P_err = np.linalg.norm(P_host[prow] - P_want) / np.linalg.norm(P_want)
+    assert P_err <= 1e-4, P_err
+    # ---- loop: sampled rows
+    W = wl.make_weight(cfg, "cuda")
+    codes, scales, zeros, Wq = _quantize_on_device(cfg, st, W)
+    del W
+    rep, J_gpu, J_orc, J_rtn, free = _check_rows(
+        cfg, W_rows, U_host, P_host, *_rows_to_host(rows, codes, scales, zeros, Wq),
+        lambda q: orc.objective_terms_chunked(W_rows, q, H_host, D_host) + resid)
+    print(f"{name} full size: H err {errH:.2e}, D err {errD:.2e}, U defect {defect:.2e}, P rows rel {P_err:.2e}, "
+          f"flips {rep.mismatches}/{rep.total} (excused {rep.allowed}), free-running mismatch {free:.2e}, "
+          f"J gpu/oracle/rtn {J_gpu:.6g}/{J_orc:.6g}/{J_rtn:.6g}, {time.time() - t0:.0f} s")
+    st.close()

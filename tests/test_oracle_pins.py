@@ -125,6 +125,24 @@ def test_theorem_4_2_three_ways():
     assert np.allclose(orc.build_P(st.D, st.tokens, U, 0.25), 0.25 * P)
 
 
+def test_row_restricted_P_and_chunked_objective_agree_with_the_full_forms():
+    W, X, Xfp = tiny(n=37, m=6)
+    st = stats_of(X, Xfp)
+    U, dead = orc.factor(st.H, st.tokens, 0.01)
+    P = orc.build_P(st.D, st.tokens, U, 0.6)
+    rows = np.array([0, 5, 17, 35, 36])
+    for chunk in (8, 64):
+        Pr = orc.build_P_rows(st.D[rows], rows, st.tokens, U.astype(np.float32), 0.6, chunk)
+        assert np.allclose(Pr, P[rows], atol=1e-6 * np.abs(P).max())
+        assert np.allclose(orc.build_P_rows(st.D[rows], rows, st.tokens, U, 0.6, chunk), P[rows], atol=1e-13)
+    Wq = W + 0.01 * np.random.default_rng(2).standard_normal(W.shape)
+    st0 = orc.Stats(st.n, st.H, st.D, None, st.tokens)
+    want = orc.objective(W, Wq, st0)
+    Hup = np.triu(st.H) + np.tril(np.full_like(st.H, 1e30), -1)     # the lower triangle must not be read
+    for chunk in (5, 16, 100):
+        assert abs(orc.objective_terms_chunked(W, Wq, Hup, st.D, chunk) - want) < 1e-10 * abs(want)
+
+
 def test_P_closed_forms():
     r = np.random.default_rng(3)
     n = 10
