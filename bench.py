@@ -31,6 +31,11 @@ import workloads as wl  # noqa: E402
 
 METRIC = "ms per layer (GPTAQ solve: accumulate + factor + P + quantize)"
 
+# dram__bytes_read.sum + dram__bytes_write.sum of one stats_umma_kernel launch (one token batch), from
+# the ncu capture summarised in profiles/stats_umma_kernel_cfg2_batch.md; keyed by (workload, statistics
+# arithmetic).  Entries are dropped when the kernel changes.
+STATS_KERNEL_TRAFFIC = {("cfg2", 0): 656.8e6}
+
 
 def peaks():
     p = os.path.join(ROOT, "MEASURED_PEAKS.json")
@@ -58,7 +63,7 @@ class ClockSampler:
                 self.rows.append([c.strip() for c in out.strip().split(",")])
             except Exception:
                 pass
-            self.stop.wait(0.2)
+            self.stop.wait(0.1)
 
     def __enter__(self):
         self.th = threading.Thread(target=self._run, daemon=True)
@@ -298,7 +303,7 @@ def run_ours(args, cfg):
                       "layer_quantize": fac_ms + p_ms + q_ms},
         "accumulate_tflops": achieved,
         "roofline": {"kernel": "gptaq_accumulate (one token batch)", "bound": "tensor", "achieved": achieved,
-                     "peak": peak, "unit": "TFLOP/s", "frac": achieved / peak, "traffic": None,
+                     "peak": peak, "unit": "TFLOP/s", "frac": achieved / peak, "traffic": STATS_KERNEL_TRAFFIC.get((cfg.name, prec)),
                      "peak_source": pk["source"] + " bf16 cuBLAS, sustained",
                      "algorithmic_flops_per_launch": flops_call},
         "cpu_baseline": cpu, "e2e": e2e, "gpu_launches": launches, "clocks": clk.summary(),
@@ -311,12 +316,12 @@ def run_ours(args, cfg):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=5)
+    ap.add_argument("--steps", type=int, default=40)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="cfg2", choices=sorted(wl.CONFIGS))
-    ap.add_argument("--ref-tokens", type=int, default=1024)
-    ap.add_argument("--ref-rows", type=int, default=32)
+    ap.add_argument("--ref-tokens", type=int, default=8192)
+    ap.add_argument("--ref-rows", type=int, default=512)
     ap.add_argument("--batches", type=int, default=0,
                     help="profiler captures only: keep this many token batches (the line is marked truncated)")
     ap.add_argument("--no-e2e", action="store_true")
