@@ -146,6 +146,27 @@ def run_reference(args, cfg):
     print(json.dumps(line), flush=True)
 
 
+# --------------------------------------------------------------------------- multi-rank plumbing
+def rank_config(cfg: wl.LayerConfig, rank: int) -> wl.LayerConfig:
+    """Every rank solves its own layer of the same shape: same recipe, seed shifted by the rank."""
+    return wl.scaled(cfg, seed=cfg.seed + rank)
+
+
+def max_over_ranks(ms: float, world: int, device) -> float:
+    """Largest per-rank time (one all-reduce of a scalar; the only collective, outside the timed region)."""
+    if world <= 1:
+        return ms
+    import torch.distributed as dist
+    t = torch.tensor([ms], device=device, dtype=torch.float64)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def per_layer_ms(ms_step: float, world: int) -> float:
+    """One step solves `world` independent layers at once: time per layer of the whole job."""
+    return ms_step / world
+
+
 # --------------------------------------------------------------------------- CUDA leg
 def run_ours(args, cfg):
     import paper_2504_02692_b200 as g
@@ -166,7 +187,7 @@ def run_ours(args, cfg):
     pk = peaks()
 
     # inputs resident in HBM before the timed region (each rank its own layer: seed = rank)
-    cfg_r = wl.scaled(cfg, seed=cfg.seed + rank)
+    cfg_r = rank_config(cfg, rank)
     batches = [wl.make_batch(cfg_r, b, dev) for b in range(cfg.n_batches)]
     W0 = wl.make_weight(cfg_r, dev)
     if cfg.w_bf16:
@@ -232,12 +253,9 @@ def run_ours(args, cfg):
         sync_all()
     launches = g.gptaq_launch_count(h) - l0
     ms_total = t_beg.elapsed_time(t_end)
-    if world > 1:
-        t = torch.tensor([ms_total], device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms_total = float(t.item())
+    ms_total = max_over_ranks(ms_total, world, dev)
     ms_step = ms_total / args.steps
-    ms_layer = ms_step / world           # `world` independent layers per step
+    ms_layer = per_layer_ms(ms_step, world)
 
     acc_ms = [a.elapsed_time(b) for m in marks for (a, b) in m[0]]
     acc_call_ms = sum(acc_ms) / len(acc_ms)
@@ -278,13 +296,10 @@ def run_ours(args, cfg):
         b.record(stream)
         sync_all()
         ems = a.elapsed_time(b) / ke
-        if world > 1:
-            t = torch.tensor([ems], device=dev)
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            ems = float(t.item())
+        ems = max_over_ranks(ems, world, dev)
         h2d = sum(x.numel() * 4 * 2 for x, _ in hb) + hW.numel() * 4
         d2h = hcodes.numel() + (hs.numel() + hz.numel()) * 4
-        e2e = {"value": ems / world, "unit": "ms", "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h}
+        e2e = {"value": per_layer_ms(ems, world), "unit": "ms", "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h}
 
     if rank != 0:
         return
