@@ -223,11 +223,17 @@ cudaError_t launch_split(const float *src, int64_t lds, float *hi, float *lo, in
     return cudaGetLastError();
 }
 
-// Largest token chunk (multiple of 64) whose two fp16 operand copies fit the workspace.
+// Scratch of the statistics kernel's K-split tail: at most one 128 x 256 partial tile per SM.
+size_t stats_scratch_bytes(int num_sms) { return round_up((size_t)num_sms * UBM * UBN * sizeof(float), ALIGN); }
+constexpr int MAX_SMS_FOR_SIZING = 256;
+
+// Largest token chunk (multiple of 64) whose fp16 operand copies fit the workspace next to that scratch.
 int64_t tc_chunk_tokens(const gptaq_ctx *h) {
     const int nbuf = h->stats_precision == GPTAQ_STATS_FP16_SPLIT_TENSOR ? 3 : 2;
     int64_t per_token = nbuf * h->n * 2;   // X^T, dX^T (and the low part of X^T), fp16
-    int64_t cap = (int64_t)(h->ws_bytes / (size_t)per_token);
+    const size_t reserve = stats_scratch_bytes(h->num_sms);
+    if (h->ws_bytes <= reserve) return 0;
+    int64_t cap = (int64_t)((h->ws_bytes - reserve) / (size_t)per_token);
     cap = cap / UBK * UBK;
     return std::min<int64_t>(cap, 1 << 20);
 }
@@ -270,9 +276,27 @@ gptaq_status_t accumulate_tc(gptaq_ctx *h, const float *X, const float *Xfp, int
         }
         StatsGemmArgs ga;
         ga.H = h->H; ga.D = h->D; ga.n = n; ga.kblocks = kp / UBK; ga.nseg_h = split ? 3 : 1; ga.amax = h->hd->amax; ga.hd = h->hd;
-        const int grid = (int)std::min<int64_t>(ntiles, h->num_sms);
-        stats_umma_kernel<<<grid, UMMA_THREADS, UMMA_SMEM, s>>>(mXa, mDa, mXb, mLa, mLb, ga);
+        // the last, partial wave of tiles is cut along K so that every SM has work
+        ga.ntiles = (int)ntiles;
+        ga.full_tiles = (int)(ntiles / h->num_sms) * h->num_sms;
+        ga.ksplit = 1;
+        const int cut = (int)ntiles - ga.full_tiles;
+        if (cut > 0) {
+            const int by_sms = h->num_sms / cut, by_k = ga.kblocks / (2 * UCHUNK);
+            ga.ksplit = std::max(1, std::min(std::min(by_sms, by_k), 8));
+        }
+        if (ga.ksplit == 1) ga.full_tiles = (int)ntiles;
+        // scratch behind the operand copies (one partial tile per SM at most)
+        const size_t opbytes = round_up((size_t)(split ? 3 : 2) * n * kp * 2, ALIGN);
+        ga.scratch = reinterpret_cast<float *>(h->ws + opbytes);
+        const int nitems = ga.full_tiles + ((int)ntiles - ga.full_tiles) * ga.ksplit;
+        const int sgrid = std::min(nitems, h->num_sms);
+        stats_umma_kernel<<<sgrid, UMMA_THREADS, UMMA_SMEM, s>>>(mXa, mDa, mXb, mLa, mLb, ga);
         LAUNCHED();
+        if (ga.ksplit > 1) {
+            stats_fixup_kernel<<<dim3((unsigned)((int)ntiles - ga.full_tiles), FIXUP_SLABS), 256, 0, s>>>(ga);
+            LAUNCHED();
+        }
     }
     h->tokens += tokens;
     return GPTAQ_OK;
@@ -468,7 +492,7 @@ size_t gptaq_workspace_bytes(int64_t n, int64_t m_max, int64_t max_batch_tokens,
     if (n <= 0 || m_max < 0 || max_batch_tokens < 0 || !valid_block(blocksize)) return 0;
     // the fp16 operand copies of one token batch share the space of the later steps' scratch
     size_t kp = round_up((size_t)max_batch_tokens, (size_t)UBK);
-    size_t xt = round_up(3 * (size_t)n * kp * 2, ALIGN);
+    size_t xt = round_up(3 * (size_t)n * kp * 2, ALIGN) + stats_scratch_bytes(MAX_SMS_FOR_SIZING);
     return std::max(ws_layout(n, m_max, blocksize).total, xt);
 }
 

@@ -246,29 +246,64 @@ struct StatsGemmArgs {
     int nseg_h;              // 1: H = hi hi^T;  3: H = hi hi^T + hi lo^T + lo hi^T (split operands)
     const unsigned *amax;    // scales are recomputed from the recorded maxima
     StateHeader *hd;
+    // Work items: tiles [0, full_tiles) are whole tiles; each of the remaining `ntiles - full_tiles`
+    // tiles (the last, partial wave) is cut along K into `ksplit` items so that every SM has work.
+    // Item 0 of a cut tile adds into the sums like a whole tile; items c > 0 store their partial
+    // result at scratch[((tile - full_tiles) * (ksplit - 1) + c - 1) * UBM * UBN] and
+    // stats_fixup_kernel adds those in a fixed order (the result does not depend on timing).
+    int ntiles, full_tiles, ksplit;
+    float *scratch;
 };
 
 // Tile enumeration shared by all roles: row-major over (row tile, column tile);
 // rows [0, TM) belong to H (tiles entirely below the diagonal are not
 // enumerated), rows [TM, 2 TM) to dXX^T.
 struct TileIter {
-    int TM, TN, r, tn, left;      // left: tiles still to skip before the next one of this CTA
-    __device__ TileIter(int n, int first) : TM((n + UBM - 1) / UBM), TN((n + UBN - 1) / UBN), r(0), tn(0), left(first) {
+    int TM, TN, r, tn, ord;       // ord: ordinal of the current tile (r, tn)
+    __device__ TileIter(int n) : TM((n + UBM - 1) / UBM), TN((n + UBN - 1) / UBN), r(0), tn(0), ord(0) {
         tn = first_tn(0);
     }
     __device__ int first_tn(int row) const { return row < TM ? (row * UBM) / UBN : 0; }
-    // Advances to the tile `left` positions ahead; false when the list is exhausted.
-    __device__ bool seek() {
+    // Advances to the tile with ordinal `target` >= ord; false when the list is exhausted.
+    __device__ bool seek_to(int target) {
+        int left = target - ord;
         while (r < 2 * TM) {
             int avail = TN - tn;
-            if (left < avail) { tn += left; left = 0; return true; }
+            if (left < avail) { tn += left; ord = target; return true; }
             left -= avail;
+            ord += avail;
             ++r;
             tn = first_tn(r);
         }
         return false;
     }
 };
+
+// One work item of a CTA: a tile and a range of its K-blocks (all segments concatenated).
+struct StatsItem {
+    int g0, g1;          // K-block range
+    int part;            // 0: adds into H / dXX^T;  c > 0: partial result number c of a cut tile
+    int cut_index;       // index of the cut tile among the cut tiles
+};
+
+__device__ __forceinline__ bool stats_item(const StatsGemmArgs &a, int w, TileIter &it, StatsItem &item) {
+    const int nitems = a.full_tiles + (a.ntiles - a.full_tiles) * a.ksplit;
+    if (w >= nitems) return false;
+    int tile = w, part = 0, parts = 1;
+    if (w >= a.full_tiles) {
+        const int e = w - a.full_tiles;
+        tile = a.full_tiles + e / a.ksplit;
+        part = e - (e / a.ksplit) * a.ksplit;
+        parts = a.ksplit;
+    }
+    if (!it.seek_to(tile)) return false;
+    const int kb_total = (it.r >= it.TM) ? a.kblocks : a.kblocks * a.nseg_h;
+    item.g0 = (int)((long long)kb_total * part / parts);
+    item.g1 = (int)((long long)kb_total * (part + 1) / parts);
+    item.part = part;
+    item.cut_index = tile - a.full_tiles;
+    return true;
+}
 
 // Accumulation chains in tensor memory are kept short: the tensor core truncates
 // its fp32 accumulator once per MMA, which biases a long sum of like-signed
@@ -316,28 +351,26 @@ stats_umma_kernel(const __grid_constant__ CUtensorMap mapXa, const __grid_consta
     if (warp == 0) {
         // ------------------------------------------------------------ TMA producer
         if (lane == 0) {
-            TileIter it(a.n, blockIdx.x);
+            TileIter it(a.n);
+            StatsItem item;
             uint32_t stage = 0, phase = 0;
             int issued = 0;
             bool ok = true;
-            while (ok && it.seek()) {
+            for (int w = blockIdx.x; ok && stats_item(a, w, it, item); w += gridDim.x) {
                 const bool isD = it.r >= it.TM;
                 const int row0 = (isD ? it.r - it.TM : it.r) * UBM, col0 = it.tn * UBN;
-                const int nseg = isD ? 1 : a.nseg_h;
-                for (int seg = 0; seg < nseg && ok; ++seg) {
+                for (int g = item.g0; g < item.g1; ++g) {
+                    const int seg = g / KB, kb = g - seg * KB;
                     const CUtensorMap *mapA = isD ? &mapDa : (seg == 2 ? &mapLa : &mapXa);
                     const CUtensorMap *mapB = (seg == 1) ? &mapLb : &mapXb;
-                    for (int kb = 0; kb < KB; ++kb) {
-                        if (!mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag)) { ok = false; break; }
-                        const uint32_t sa = base + stage * USTAGE_BYTES, sb = sa + UA_BYTES;
-                        mbar_expect_tx(full_bar(stage), USTAGE_BYTES);
-                        tma_load_2d(sa, mapA, kb * UBK, row0, full_bar(stage));
-                        tma_load_2d(sb, mapB, kb * UBK, col0, full_bar(stage));
-                        ++issued;
-                        if (++stage == USTAGES) { stage = 0; phase ^= 1u; }
-                    }
+                    if (!mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag)) { ok = false; break; }
+                    const uint32_t sa = base + stage * USTAGE_BYTES, sb = sa + UA_BYTES;
+                    mbar_expect_tx(full_bar(stage), USTAGE_BYTES);
+                    tma_load_2d(sa, mapA, kb * UBK, row0, full_bar(stage));
+                    tma_load_2d(sb, mapB, kb * UBK, col0, full_bar(stage));
+                    ++issued;
+                    if (++stage == USTAGES) { stage = 0; phase ^= 1u; }
                 }
-                it.left = gridDim.x;
             }
             if (!ok) {
                 // give copies that are still in flight time to land before the CTA exits
@@ -348,17 +381,17 @@ stats_umma_kernel(const __grid_constant__ CUtensorMap mapXa, const __grid_consta
     } else if (warp == 1) {
         // ------------------------------------------------------------ MMA issuer
         if (lane == 0) {
-            TileIter it(a.n, blockIdx.x);
+            TileIter it(a.n);
+            StatsItem item;
             uint32_t stage = 0, phase = 0, ccount = 0;     // ccount: chunks issued so far
             bool ok = true;
-            while (ok && it.seek()) {
-                const int kb_total = (it.r >= it.TM) ? KB : KB * a.nseg_h;
-                for (int kb0 = 0; kb0 < kb_total && ok; kb0 += UCHUNK) {
+            for (int w = blockIdx.x; ok && stats_item(a, w, it, item); w += gridDim.x) {
+                for (int kb0 = item.g0; kb0 < item.g1 && ok; kb0 += UCHUNK) {
                     const uint32_t buf = ccount & 1u, cphase = (ccount >> 1) & 1u;
                     if (!mbar_wait(tempty_bar(buf), cphase ^ 1u, abort_flag)) { ok = false; break; }
                     tc_fence_after();
                     const uint32_t d_tmem = tmem_base + buf * UBN;
-                    const int kb1 = min(kb0 + UCHUNK, kb_total);
+                    const int kb1 = min(kb0 + UCHUNK, item.g1);
                     for (int kb = kb0; kb < kb1; ++kb) {
                         if (!mbar_wait(full_bar(stage), phase, abort_flag)) { ok = false; break; }
                         tc_fence_after();
@@ -375,25 +408,24 @@ stats_umma_kernel(const __grid_constant__ CUtensorMap mapXa, const __grid_consta
                     umma_commit(tfull_bar(buf));
                     ++ccount;
                 }
-                it.left = gridDim.x;
             }
         }
     } else {
         // ------------------------------------------------------------ epilogue (warps 2..9)
         const int quarter = warp & 3;                 // TMEM lanes 32 * quarter .. + 31
         const int half = (warp - 2) >> 2;             // columns [128 * half, 128 * half + 128)
-        TileIter it(a.n, blockIdx.x);
+        TileIter it(a.n);
+        StatsItem item;
         uint32_t ccount = 0;
         bool ok = true;
         const float sx = pick_scale(__uint_as_float(a.amax[0]));
         const float sd = pick_scale(__uint_as_float(a.amax[1]));
         float acc[UBN / 2];
-        while (ok && it.seek()) {
+        for (int w = blockIdx.x; ok && stats_item(a, w, it, item); w += gridDim.x) {
             const bool isD = it.r >= it.TM;
-            const int kb_total = isD ? KB : KB * a.nseg_h;
 #pragma unroll
             for (int i = 0; i < UBN / 2; ++i) acc[i] = 0.f;
-            for (int kb0 = 0; kb0 < kb_total; kb0 += UCHUNK) {
+            for (int kb0 = item.g0; kb0 < item.g1; kb0 += UCHUNK) {
                 const uint32_t buf = ccount & 1u, cphase = (ccount >> 1) & 1u;
                 if (!mbar_wait(tfull_bar(buf), cphase, abort_flag)) { ok = false; break; }
                 tc_fence_after();
@@ -412,10 +444,20 @@ stats_umma_kernel(const __grid_constant__ CUtensorMap mapXa, const __grid_consta
                 ++ccount;
             }
             if (!ok) break;
+            const float inv = 1.f / (sx * (isD ? sd : sx));
+            if (item.part > 0) {
+                // partial result of a cut tile: plain stores into its slot, all 128 x 256 entries
+                float *sp = a.scratch + ((int64_t)item.cut_index * (a.ksplit - 1) + item.part - 1) * (UBM * UBN) +
+                            (quarter * 32 + lane) * UBN + half * (UBN / 2);
+#pragma unroll
+                for (int q = 0; q < UBN / 2 / 4; ++q)
+                    *reinterpret_cast<float4 *>(sp + 4 * q) = make_float4(acc[4 * q + 0] * inv, acc[4 * q + 1] * inv,
+                                                                         acc[4 * q + 2] * inv, acc[4 * q + 3] * inv);
+                continue;
+            }
             const int row = (isD ? it.r - it.TM : it.r) * UBM + quarter * 32 + lane;
             const int col0 = it.tn * UBN + half * (UBN / 2);
             float *C = isD ? a.D : a.H;
-            const float inv = 1.f / (sx * (isD ? sd : sx));
             if (row < a.n) {
                 float *cp = C + (int64_t)row * a.n + col0;
                 if (col0 + UBN / 2 <= a.n && (reinterpret_cast<uintptr_t>(cp) & 15) == 0) {
@@ -432,7 +474,6 @@ stats_umma_kernel(const __grid_constant__ CUtensorMap mapXa, const __grid_consta
                         if (col0 + q < a.n) cp[q] = fmaf(acc[q], inv, cp[q]);
                 }
             }
-            it.left = gridDim.x;
         }
     }
 
@@ -442,6 +483,42 @@ stats_umma_kernel(const __grid_constant__ CUtensorMap mapXa, const __grid_consta
     if (warp == 1) {
         tc_fence_after();
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(512u) : "memory");
+    }
+}
+
+// Adds the partial results of the cut tiles (see StatsGemmArgs) into H / dXX^T, partial 1 first, then 2, ...:
+// one CTA per cut tile, after stats_umma_kernel of the same batch.
+constexpr int FIXUP_SLABS = 16;     // CTAs per cut tile, UBM / FIXUP_SLABS rows each
+__global__ void __launch_bounds__(256) stats_fixup_kernel(StatsGemmArgs a) {
+    TileIter it(a.n);
+    if (!it.seek_to(a.full_tiles + blockIdx.x)) return;
+    const bool isD = it.r >= it.TM;
+    const int row0 = (isD ? it.r - it.TM : it.r) * UBM, col0 = it.tn * UBN;
+    float *C = isD ? a.D : a.H;
+    const float *sp = a.scratch + (int64_t)blockIdx.x * (a.ksplit - 1) * (UBM * UBN);
+    constexpr int ROWS = UBM / FIXUP_SLABS;
+    const bool vec = (a.n & 3) == 0 && (reinterpret_cast<uintptr_t>(C) & 15) == 0;
+#pragma unroll
+    for (int it4 = 0; it4 < ROWS * UBN / 4 / 256; ++it4) {
+        const int e4 = threadIdx.x + it4 * 256;
+        const int i = blockIdx.y * ROWS + e4 / (UBN / 4), j = (e4 % (UBN / 4)) * 4;
+        if (row0 + i >= a.n || col0 + j >= a.n) continue;
+        float *cp = C + (int64_t)(row0 + i) * a.n + col0 + j;
+        const float *pp = sp + i * UBN + j;
+        if (vec && col0 + j + 3 < a.n) {
+            float4 v = *reinterpret_cast<const float4 *>(cp);
+            for (int c = 0; c < a.ksplit - 1; ++c) {
+                const float4 p = *reinterpret_cast<const float4 *>(pp + (int64_t)c * (UBM * UBN));
+                v.x += p.x; v.y += p.y; v.z += p.z; v.w += p.w;
+            }
+            *reinterpret_cast<float4 *>(cp) = v;
+        } else {
+            for (int f = 0; f < 4 && col0 + j + f < a.n; ++f) {
+                float v = cp[f];
+                for (int c = 0; c < a.ksplit - 1; ++c) v += pp[(int64_t)c * (UBM * UBN) + f];
+                cp[f] = v;
+            }
+        }
     }
 }
 
