@@ -100,6 +100,15 @@ gptaq_status_t gptaq_destroy(gptaq_handle_t h);
 gptaq_status_t gptaq_accumulate(gptaq_handle_t h, const float *d_X, const float *d_Xfp,
                                 int64_t tokens, int64_t ld, gptaq_stream_t stream);
 
+/* gptaq_accumulate converts the batch on `stream` and may run the product itself on a stream
+ * of the handle's own, so that the conversion of the next batch overlaps it.  Every other call
+ * that takes the handle and a stream (reset, factor, sync_status) first orders its stream after
+ * that work.  A caller that wants to read the sums through gptaq_H / gptaq_D on `stream` right
+ * after gptaq_accumulate, or to time the accumulation with events on `stream`, calls
+ * gptaq_flush: it makes `stream` wait (on the device, not on the host) for the pending
+ * products. */
+gptaq_status_t gptaq_flush(gptaq_handle_t h, gptaq_stream_t stream);
+
 /* Same with HOST inputs (pinned memory for asynchronous copies): copies the
  * batch into d_stage (device, >= 2 * tokens * n * 4 bytes) on `stream`, then
  * accumulates from there. */

@@ -40,6 +40,7 @@ SIGNATURES = {
     "gptaq_reset": (_int, [_vp, _vp]),
     "gptaq_destroy": (_int, [_vp]),
     "gptaq_accumulate": (_int, [_vp, _vp, _vp, _i64, _i64, _vp]),
+    "gptaq_flush": (_int, [_vp, _vp]),
     "gptaq_accumulate_host": (_int, [_vp, _vp, _vp, _i64, _i64, _vp, _sz, _vp]),
     "gptaq_factor": (_int, [_vp, _f, _vp]),
     "gptaq_build_P": (_int, [_vp, _f, _vp]),
@@ -161,6 +162,11 @@ def gptaq_accumulate(h, d_X: torch.Tensor, d_Xfp: torch.Tensor, stream=None):
     ld = d_X.stride(0) if tokens > 1 else max(d_X.shape[1], 1)
     st = load_library().gptaq_accumulate(h, _ptr(d_X), _ptr(d_Xfp), tokens, ld, _stream(stream))
     _check(st, "gptaq_accumulate", h)
+
+
+def gptaq_flush(h, stream=None):
+    """Orders ``stream`` after the statistics products that gptaq_accumulate left running."""
+    _check(load_library().gptaq_flush(h, _stream(stream)), "gptaq_flush", h)
 
 
 def gptaq_accumulate_host(h, h_X: torch.Tensor, h_Xfp: torch.Tensor, d_stage: torch.Tensor, stream=None):
@@ -313,11 +319,13 @@ class LayerState:
         return self.state[off:off + nbytes].view(torch.float32).view(self.n, self.n)
 
     def H(self) -> torch.Tensor:
-        """View of H (before factor) / U (after), ``[n, n]`` float32."""
+        """View of H (before factor) / U (after), ``[n, n]`` float32, current on torch's stream."""
+        gptaq_flush(self.handle)
         return self._view(gptaq_H_ptr(self.handle))
 
     def D(self) -> torch.Tensor:
-        """View of dXX^T (before build_P) / P (after)."""
+        """View of dXX^T (before build_P) / P (after), current on torch's stream."""
+        gptaq_flush(self.handle)
         return self._view(gptaq_D_ptr(self.handle))
 
     def close(self):

@@ -43,6 +43,13 @@ struct gptaq_ctx {
     int64_t launches;
     int stats_precision;   // GPTAQ_STATS_*
     bool tensor;           // float32-grade tensor-core GEMMs for factor / P / trailing update
+    // Statistics pipeline: the conversion of a token batch runs on the caller's stream, the
+    // tensor-core product on `gemm_stream`, so that the (memory-bound) conversion of the next
+    // batch overlaps the (tensor-bound) product of this one.  Two operand buffers alternate.
+    cudaStream_t gemm_stream;
+    cudaEvent_t conv_done[2], gemm_done[2];
+    bool gemm_pending[2];
+    int next_buf;
     std::string cuda_error;
 };
 
@@ -230,10 +237,10 @@ constexpr int MAX_SMS_FOR_SIZING = 256;
 // Largest token chunk (multiple of 64) whose fp16 operand copies fit the workspace next to that scratch.
 int64_t tc_chunk_tokens(const gptaq_ctx *h) {
     const int nbuf = h->stats_precision == GPTAQ_STATS_FP16_SPLIT_TENSOR ? 3 : 2;
-    int64_t per_token = nbuf * h->n * 2;   // X^T, dX^T (and the low part of X^T), fp16
+    int64_t per_token = 2 * nbuf * h->n * 2;   // two buffers of X^T, dX^T (and the low part of X^T), fp16
     const size_t reserve = stats_scratch_bytes(h->num_sms);
-    if (h->ws_bytes <= reserve) return 0;
-    int64_t cap = (int64_t)((h->ws_bytes - reserve) / (size_t)per_token);
+    if (h->ws_bytes <= reserve + 2 * ALIGN) return 0;
+    int64_t cap = (int64_t)((h->ws_bytes - reserve - 2 * ALIGN) / (size_t)per_token);
     cap = cap / UBK * UBK;
     return std::min<int64_t>(cap, 1 << 20);
 }
@@ -241,6 +248,16 @@ int64_t tc_chunk_tokens(const gptaq_ctx *h) {
 bool tc_eligible(const gptaq_ctx *h) {
     return h->stats_precision != GPTAQ_STATS_FP32 && h->n >= UBN && tc_chunk_tokens(h) >= UBK &&
            encode_tiled_fn() != nullptr;
+}
+
+// Orders `s` after every statistics product still running on the internal stream.
+gptaq_status_t join_statistics(gptaq_ctx *h, cudaStream_t s) {
+    for (int i = 0; i < 2; ++i)
+        if (h->gemm_pending[i]) {
+            CU(cudaStreamWaitEvent(s, h->gemm_done[i], 0));
+            h->gemm_pending[i] = false;
+        }
+    return GPTAQ_OK;
 }
 
 gptaq_status_t accumulate_tc(gptaq_ctx *h, const float *X, const float *Xfp, int64_t tokens, int64_t ld,
@@ -253,19 +270,31 @@ gptaq_status_t accumulate_tc(gptaq_ctx *h, const float *X, const float *Xfp, int
     for (int64_t t0 = 0; t0 < tokens; t0 += chunk) {
         const int tk = (int)std::min<int64_t>(chunk, tokens - t0);
         const int kp = (tk + UBK - 1) / UBK * UBK;
-        __half *Xt = reinterpret_cast<__half *>(h->ws);
-        __half *dXt = Xt + (size_t)n * kp;
         const bool split = h->stats_precision == GPTAQ_STATS_FP16_SPLIT_TENSOR;
+        const int buf = h->next_buf;
+        h->next_buf ^= 1;
+        const size_t buf_bytes = round_up((size_t)(split ? 3 : 2) * n * (size_t)(chunk) * 2, ALIGN);
+        __half *Xt = reinterpret_cast<__half *>(h->ws + (size_t)buf * buf_bytes);
+        __half *dXt = Xt + (size_t)n * kp;
         __half *Xlo = split ? dXt + (size_t)n * kp : nullptr;
-        CU(cudaMemsetAsync(h->hd->amax, 0, 2 * sizeof(unsigned), s));
+        unsigned *amax = h->hd->amax[buf];
+        cudaStream_t gs = h->gemm_stream;
+        // this buffer was last read by the product issued two chunks ago
+        if (h->gemm_pending[buf]) {
+            CU(cudaStreamWaitEvent(s, h->gemm_done[buf], 0));
+            h->gemm_pending[buf] = false;
+        }
+        CU(cudaMemsetAsync(amax, 0, 2 * sizeof(unsigned), s));
         ConvertArgs ca;
         ca.X = X + t0 * ld; ca.Xfp = Xfp + t0 * ld; ca.ld = ld; ca.tokens = tk; ca.n = n; ca.kp = kp;
-        ca.Xt = Xt; ca.dXt = dXt; ca.Xlo = Xlo; ca.amax = h->hd->amax;
+        ca.Xt = Xt; ca.dXt = dXt; ca.Xlo = Xlo; ca.amax = amax;
         dim3 cgrid(kp / 64, (n + 63) / 64);
         convert_transpose_kernel<0><<<cgrid, 256, 0, s>>>(ca);
         LAUNCHED();
         convert_transpose_kernel<1><<<cgrid, 256, 0, s>>>(ca);
         LAUNCHED();
+        CU(cudaEventRecord(h->conv_done[buf], s));
+        CU(cudaStreamWaitEvent(gs, h->conv_done[buf], 0));
         CUtensorMap mXa, mDa, mXb, mLa, mLb;
         const __half *lo = split ? Xlo : Xt;    // unused maps still have to be valid
         if (!make_kmajor_map(&mXa, Xt, n, kp, UBM) || !make_kmajor_map(&mDa, dXt, n, kp, UBM) ||
@@ -275,7 +304,7 @@ gptaq_status_t accumulate_tc(gptaq_ctx *h, const float *X, const float *Xfp, int
             return GPTAQ_ERR_CUDA;
         }
         StatsGemmArgs ga;
-        ga.H = h->H; ga.D = h->D; ga.n = n; ga.kblocks = kp / UBK; ga.nseg_h = split ? 3 : 1; ga.amax = h->hd->amax; ga.hd = h->hd;
+        ga.H = h->H; ga.D = h->D; ga.n = n; ga.kblocks = kp / UBK; ga.nseg_h = split ? 3 : 1; ga.amax = amax; ga.hd = h->hd;
         // the last, partial wave of tiles is cut along K so that every SM has work
         ga.ntiles = (int)ntiles;
         ga.full_tiles = (int)(ntiles / h->num_sms) * h->num_sms;
@@ -286,17 +315,19 @@ gptaq_status_t accumulate_tc(gptaq_ctx *h, const float *X, const float *Xfp, int
             ga.ksplit = std::max(1, std::min(std::min(by_sms, by_k), 8));
         }
         if (ga.ksplit == 1) ga.full_tiles = (int)ntiles;
-        // scratch behind the operand copies (one partial tile per SM at most)
-        const size_t opbytes = round_up((size_t)(split ? 3 : 2) * n * kp * 2, ALIGN);
-        ga.scratch = reinterpret_cast<float *>(h->ws + opbytes);
+        // scratch behind the two operand buffers (one partial tile per SM at most; the products run
+        // one after the other on the internal stream, so one scratch serves both buffers)
+        ga.scratch = reinterpret_cast<float *>(h->ws + 2 * buf_bytes);
         const int nitems = ga.full_tiles + ((int)ntiles - ga.full_tiles) * ga.ksplit;
         const int sgrid = std::min(nitems, h->num_sms);
-        stats_umma_kernel<<<sgrid, UMMA_THREADS, UMMA_SMEM, s>>>(mXa, mDa, mXb, mLa, mLb, ga);
+        stats_umma_kernel<<<sgrid, UMMA_THREADS, UMMA_SMEM, gs>>>(mXa, mDa, mXb, mLa, mLb, ga);
         LAUNCHED();
         if (ga.ksplit > 1) {
-            stats_fixup_kernel<<<dim3((unsigned)((int)ntiles - ga.full_tiles), FIXUP_SLABS), 256, 0, s>>>(ga);
+            stats_fixup_kernel<<<dim3((unsigned)((int)ntiles - ga.full_tiles), FIXUP_SLABS), 256, 0, gs>>>(ga);
             LAUNCHED();
         }
+        CU(cudaEventRecord(h->gemm_done[buf], gs));
+        h->gemm_pending[buf] = true;
     }
     h->tokens += tokens;
     return GPTAQ_OK;
@@ -492,7 +523,7 @@ size_t gptaq_workspace_bytes(int64_t n, int64_t m_max, int64_t max_batch_tokens,
     if (n <= 0 || m_max < 0 || max_batch_tokens < 0 || !valid_block(blocksize)) return 0;
     // the fp16 operand copies of one token batch share the space of the later steps' scratch
     size_t kp = round_up((size_t)max_batch_tokens, (size_t)UBK);
-    size_t xt = round_up(3 * (size_t)n * kp * 2, ALIGN) + stats_scratch_bytes(MAX_SMS_FOR_SIZING);
+    size_t xt = 2 * round_up(3 * (size_t)n * kp * 2, ALIGN) + stats_scratch_bytes(MAX_SMS_FOR_SIZING);
     return std::max(ws_layout(n, m_max, blocksize).total, xt);
 }
 
@@ -533,6 +564,14 @@ gptaq_status_t gptaq_create(gptaq_handle_t *out, int64_t n, void *d_state, size_
         e = cudaFuncSetAttribute(stats_umma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)UMMA_SMEM);
     if (e == cudaSuccess)
         e = cudaFuncSetAttribute(tc_gemm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)TC_SMEM);
+    // the conversion of the next batch shares the SMs with the running product: both kernels ask for
+    // the largest shared-memory carve-out, so that a conversion CTA fits beside a product CTA
+    if (e == cudaSuccess)
+        e = cudaFuncSetAttribute(stats_umma_kernel, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared);
+    if (e == cudaSuccess)
+        e = cudaFuncSetAttribute(convert_transpose_kernel<0>, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared);
+    if (e == cudaSuccess)
+        e = cudaFuncSetAttribute(convert_transpose_kernel<1>, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared);
     if (e == cudaSuccess)
         e = cudaFuncSetAttribute(column_loop_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                  2 * 64 * 64 * (int)sizeof(float));
@@ -543,9 +582,21 @@ gptaq_status_t gptaq_create(gptaq_handle_t *out, int64_t n, void *d_state, size_
         delete h;
         return GPTAQ_ERR_CUDA;
     }
+    h->gemm_stream = nullptr;
+    h->next_buf = 0;
+    for (int i = 0; i < 2; ++i) { h->conv_done[i] = h->gemm_done[i] = nullptr; h->gemm_pending[i] = false; }
+    e = cudaStreamCreateWithFlags(&h->gemm_stream, cudaStreamNonBlocking);
+    for (int i = 0; i < 2 && e == cudaSuccess; ++i) {
+        e = cudaEventCreateWithFlags(&h->conv_done[i], cudaEventDisableTiming);
+        if (e == cudaSuccess) e = cudaEventCreateWithFlags(&h->gemm_done[i], cudaEventDisableTiming);
+    }
+    if (e != cudaSuccess) {
+        gptaq_destroy(h);
+        return GPTAQ_ERR_CUDA;
+    }
     gptaq_status_t st = gptaq_reset(h, stream);
     if (st != GPTAQ_OK) {
-        delete h;
+        gptaq_destroy(h);
         return st;
     }
     *out = h;
@@ -555,6 +606,7 @@ gptaq_status_t gptaq_create(gptaq_handle_t *out, int64_t n, void *d_state, size_
 gptaq_status_t gptaq_reset(gptaq_handle_t h, gptaq_stream_t stream) {
     if (!h) return GPTAQ_ERR_INVALID_ARG;
     Layout l = state_layout(h->n);
+    OK(join_statistics(h, static_cast<cudaStream_t>(stream)));
     CU(cudaMemsetAsync(h->state, 0, l.total, static_cast<cudaStream_t>(stream)));
     h->stage = STAGE_ACCUM;
     h->tokens = 0;
@@ -563,6 +615,14 @@ gptaq_status_t gptaq_reset(gptaq_handle_t h, gptaq_stream_t stream) {
 
 gptaq_status_t gptaq_destroy(gptaq_handle_t h) {
     if (!h) return GPTAQ_ERR_INVALID_ARG;
+    if (h->gemm_stream) {
+        cudaStreamSynchronize(h->gemm_stream);
+        cudaStreamDestroy(h->gemm_stream);
+    }
+    for (int i = 0; i < 2; ++i) {
+        if (h->conv_done[i]) cudaEventDestroy(h->conv_done[i]);
+        if (h->gemm_done[i]) cudaEventDestroy(h->gemm_done[i]);
+    }
     delete h;
     return GPTAQ_OK;
 }
@@ -576,6 +636,7 @@ gptaq_status_t gptaq_accumulate(gptaq_handle_t h, const float *d_X, const float 
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     const int n = (int)h->n;
     if (tc_eligible(h)) return accumulate_tc(h, d_X, d_Xfp, tokens, ld, s);
+    OK(join_statistics(h, s));
     // H (upper tiles) += X X^T
     Operand xa = make_operand(d_X, 1, ld);
     GemmProblem ph = make_problem(xa, xa, h->H, n, n, n, (int)tokens, 1.f, 1.f, GEMM_UPPER_TILES);
@@ -587,6 +648,11 @@ gptaq_status_t gptaq_accumulate(gptaq_handle_t h, const float *d_X, const float 
     OK(gemm(h, pd, true, true, s));
     h->tokens += tokens;
     return GPTAQ_OK;
+}
+
+gptaq_status_t gptaq_flush(gptaq_handle_t h, gptaq_stream_t stream) {
+    if (!h) return GPTAQ_ERR_INVALID_ARG;
+    return join_statistics(h, static_cast<cudaStream_t>(stream));
 }
 
 gptaq_status_t gptaq_accumulate_host(gptaq_handle_t h, const float *h_X, const float *h_Xfp,
@@ -613,6 +679,7 @@ gptaq_status_t gptaq_factor(gptaq_handle_t h, float damp, gptaq_stream_t stream)
     if (!h || !(damp >= 0.f) || !std::isfinite(damp)) return GPTAQ_ERR_INVALID_ARG;
     if (h->stage != STAGE_ACCUM || h->tokens <= 0) return GPTAQ_ERR_BAD_STATE;
     cudaStream_t s = static_cast<cudaStream_t>(stream);
+    OK(join_statistics(h, s));
     const int n = (int)h->n;
     const int nb = (n + NB - 1) / NB;
     WsLayout wl = ws_layout(h->n, 0, 32);
@@ -873,6 +940,7 @@ gptaq_status_t gptaq_quantize_static(const float *d_U, const float *d_P, int64_t
 gptaq_status_t gptaq_sync_status(gptaq_handle_t h, int64_t *info, gptaq_stream_t stream) {
     if (!h) return GPTAQ_ERR_INVALID_ARG;
     cudaStream_t s = static_cast<cudaStream_t>(stream);
+    OK(join_statistics(h, s));
     StateHeader hd;
     CU(cudaMemcpyAsync(&hd, h->hd, sizeof(hd), cudaMemcpyDeviceToHost, s));
     CU(cudaStreamSynchronize(s));

@@ -14,8 +14,8 @@ struct StateHeader {
     long long info;      // index that goes with it
     float lambda;        // damp * mean(diag H / tokens)
     float inv_tokens;
-    unsigned amax[2];    // bit patterns of max|X| and max|X~ - X| of the batch being converted
-    int pad1[24];
+    unsigned amax[2][2]; // per operand buffer: bit patterns of max|X| and max|X~ - X| of the batch converted into it
+    int pad1[22];
 };
 static_assert(sizeof(StateHeader) == 128, "header size");
 
