@@ -70,7 +70,10 @@ __device__ __forceinline__ void tc_decode(const TcGemmArgs &a, int t, TcTile &ti
     const int per = TM * TN;
     ti.z = t / per;
     const int rem = t - ti.z * per;
-    const int tm = rem / TN, tn = rem - tm * TN;
+    // row tile fastest: the tiles a CTA meets as it strides through the list then cover all column
+    // tiles, i.e. all lengths of the triangular K ranges, evenly (column-tile-fastest order gives
+    // every CTA the same few column tiles again and again: up to 2x imbalance)
+    const int tn = rem / TM, tm = rem - tn * TM;
     ti.i0 = tm * TBM; ti.j0 = tn * TBN;
     const bool last = ti.z == a.nbatch - 1;
     ti.Mz = (last && a.M_last) ? a.M_last : a.M;
