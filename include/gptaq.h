@@ -214,6 +214,15 @@ gptaq_status_t gptaq_set_stats_precision(gptaq_handle_t h, int precision);
  * layer of width n calibrated on total_tokens tokens. */
 int gptaq_recommended_stats_precision(int64_t n, int64_t total_tokens);
 
+/* Ablation switches of the weight update (Section 5.3, Table "ablation"): which of the two terms of
+ * Eq. "divided update" later gptaq_quantize calls on this handle apply.
+ *   GPTAQ_TERM_ERR    the quantization-error term  -(w_q - q_q)/U_qq * U[q, :]   (GPTQ's update)
+ *   GPTAQ_TERM_ASYM   the asymmetry term           w_q * P[q, :]
+ * Both (default) = GPTAQ; ERR alone = GPTQ; ASYM alone = the paper's GPTAQ'; none = round to
+ * nearest on the same grids. */
+enum { GPTAQ_TERM_ERR = 1, GPTAQ_TERM_ASYM = 2 };
+gptaq_status_t gptaq_set_update_terms(gptaq_handle_t h, int terms);
+
 /* Number of kernels this handle has launched since create (bookkeeping for benchmarks). */
 int64_t gptaq_launch_count(gptaq_handle_t h);
 

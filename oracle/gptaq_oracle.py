@@ -194,12 +194,13 @@ def _ngroups(n: int, group: int) -> int:
 
 def quantize(W: np.ndarray, U: np.ndarray, P: np.ndarray | None, dead: np.ndarray | None,
              bits: int, group: int, sym: bool, update: bool = True,
-             keep_pre: bool = False) -> QuantResult:
+             keep_pre: bool = False, error_term: bool = True) -> QuantResult:
     """Unblocked column loop (Eq. "divided update"), all rows at once.
 
     For column j: quantize the current column, e = (w - q) / U[j, j], then
     W[:, j+1:] += -e U[j, j+1:] + w P[j, j+1:], w being the value of column j
     just before it was quantized.  ``P = None`` drops the second term (GPTQ);
+    ``error_term = False`` drops the first (the ablation's GPTAQ');
     ``update = False`` drops both (round to nearest).
     """
     W = np.array(W, dtype=F64)
@@ -227,8 +228,9 @@ def quantize(W: np.ndarray, U: np.ndarray, P: np.ndarray | None, dead: np.ndarra
         if keep_pre:
             pre[:, j] = w / s
         if update and j + 1 < n:
-            e = (w - q) / U[j, j]
-            W[:, j + 1:] -= np.outer(e, U[j, j + 1:])
+            if error_term:
+                e = (w - q) / U[j, j]
+                W[:, j + 1:] -= np.outer(e, U[j, j + 1:])
             if P is not None:
                 W[:, j + 1:] += np.outer(w, P[j, j + 1:])
     return QuantResult(codes, scales, zeros, Wq, pre)
@@ -336,7 +338,7 @@ class FollowReport:
 def follow(W: np.ndarray, U: np.ndarray, P: np.ndarray | None, dead,
            bits: int, group: int, sym: bool,
            cand_codes: np.ndarray, cand_scales: np.ndarray, cand_zeros: np.ndarray,
-           band: float = 1e-4) -> FollowReport:
+           band: float = 1e-4, error_term: bool = True) -> FollowReport:
     W = np.array(W, dtype=F64)
     m, n = W.shape
     if dead is not None and dead.any():
@@ -379,8 +381,9 @@ def follow(W: np.ndarray, U: np.ndarray, P: np.ndarray | None, dead,
             worst = max(worst, float(frac.max()))
         q = dequant(got, s, z)
         if j + 1 < n:
-            e = (w - q) / U[j, j]
-            W[:, j + 1:] -= np.outer(e, U[j, j + 1:])
+            if error_term:
+                e = (w - q) / U[j, j]
+                W[:, j + 1:] -= np.outer(e, U[j, j + 1:])
             if P is not None:
                 W[:, j + 1:] += np.outer(w, P[j, j + 1:])
     return FollowReport(m * n, mism, allowed, disallowed, worst, grid_err, zero_mis)

@@ -29,6 +29,8 @@ GPTAQ_W_BF16 = 1
 GPTAQ_STATS_FP16_TENSOR = 0
 GPTAQ_STATS_FP32 = 1
 GPTAQ_STATS_FP16_SPLIT_TENSOR = 2
+GPTAQ_TERM_ERR = 1
+GPTAQ_TERM_ASYM = 2
 
 _vp, _i64, _int, _sz, _f = C.c_void_p, C.c_int64, C.c_int, C.c_size_t, C.c_float
 
@@ -55,6 +57,7 @@ SIGNATURES = {
     "gptaq_tokens": (_i64, [_vp]),
     "gptaq_set_tokens": (_int, [_vp, _i64]),
     "gptaq_set_stats_precision": (_int, [_vp, _int]),
+    "gptaq_set_update_terms": (_int, [_vp, _int]),
     "gptaq_recommended_stats_precision": (_int, [_i64, _i64]),
     "gptaq_launch_count": (_i64, [_vp]),
     "gptaq_status_string": (C.c_char_p, [_int]),
@@ -273,6 +276,11 @@ def gptaq_set_tokens(h, tokens: int):
 
 def gptaq_set_stats_precision(h, precision: int):
     _check(load_library().gptaq_set_stats_precision(h, precision), "gptaq_set_stats_precision", h)
+
+
+def gptaq_set_update_terms(h, terms: int):
+    """Ablation switches: ``GPTAQ_TERM_ERR | GPTAQ_TERM_ASYM`` (default) = GPTAQ, ERR = GPTQ, ASYM = GPTAQ', 0 = RTN."""
+    _check(load_library().gptaq_set_update_terms(h, terms), "gptaq_set_update_terms", h)
 
 
 def gptaq_recommended_stats_precision(n: int, total_tokens: int) -> int:

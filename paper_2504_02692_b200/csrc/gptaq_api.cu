@@ -43,6 +43,7 @@ struct gptaq_ctx {
     int64_t launches;
     int stats_precision;   // GPTAQ_STATS_*
     bool tensor;           // float32-grade tensor-core GEMMs for factor / P / trailing update
+    int terms;             // GPTAQ_TERM_* switches of gptaq_quantize
     // Statistics pipeline: the conversion of a token batch runs on the caller's stream, the
     // tensor-core product on `gemm_stream`, so that the (memory-bound) conversion of the next
     // batch overlaps the (tensor-bound) product of this one.  Two operand buffers alternate.
@@ -348,6 +349,7 @@ struct QuantizeTarget {
     // the low part of [-Err | Wpre]; all null on the plain-FMA path
     const float *UT_hi, *UT_lo, *PT_hi, *PT_lo;
     float *EW_lo;
+    int terms = GPTAQ_TERM_ERR | GPTAQ_TERM_ASYM;   // which terms of the weight update are applied
 };
 
 gptaq_status_t check_quantize_args(int64_t n, const void *d_W, int w_dtype, int64_t m, int64_t ldw, int bits,
@@ -419,6 +421,7 @@ gptaq_status_t quantize_core(const QuantizeTarget &t, void *d_W, int w_dtype, in
         a.i0 = i0; a.bw = std::min(blocksize, n - i0);
         a.bits = bits; a.group = group; a.sym = sym;
         a.codes = d_codes; a.scales = d_scales; a.zeros = d_zeros; a.G = G; a.EW = EW; a.EW_lo = t.EW_lo; a.hd = t.hd;
+        a.err_scale = (t.terms & GPTAQ_TERM_ERR) ? 1.f : 0.f; a.asym_scale = (t.terms & GPTAQ_TERM_ASYM) ? 1.f : 0.f;
         const bool fast = a.bw == blocksize && (group <= 0 || (group % 32) == 0) && (i0 % 4) == 0 &&
                           (reinterpret_cast<uintptr_t>(t.dead) & 3) == 0;
         if (fast) column_block_kernel<<<cb_grid, CB_THREADS, column_block_smem(cb_rows), s>>>(a, cb_rows, blocksize);
@@ -551,6 +554,7 @@ gptaq_status_t gptaq_create(gptaq_handle_t *out, int64_t n, void *d_state, size_
     h->launches = 0;
     h->stats_precision = GPTAQ_STATS_FP16_SPLIT_TENSOR;
     h->tensor = tc_shape_ok(n) && encode_tiled_fn() != nullptr;
+    h->terms = GPTAQ_TERM_ERR | GPTAQ_TERM_ASYM;
     cudaError_t e = cudaGetDevice(&h->device);
     if (e == cudaSuccess) e = cudaDeviceGetAttribute(&h->num_sms, cudaDevAttrMultiProcessorCount, h->device);
     if (e == cudaSuccess)
@@ -850,6 +854,7 @@ gptaq_status_t gptaq_quantize(gptaq_handle_t h, void *d_W, int w_dtype, int64_t 
     t.n = (int)h->n; t.U = h->H; t.P = h->D; t.dead = h->dead; t.hd = h->hd;
     t.EW = reinterpret_cast<float *>(h->ws + wl.ew_off);
     t.num_sms = h->num_sms;
+    t.terms = h->terms;
     t.UT_hi = t.UT_lo = t.PT_hi = t.PT_lo = nullptr; t.EW_lo = nullptr;
     if (h->tensor) {
         t.UT_hi = reinterpret_cast<float *>(h->ws + wl.s_off[2]); t.UT_lo = reinterpret_cast<float *>(h->ws + wl.s_off[3]);
@@ -966,6 +971,13 @@ gptaq_status_t gptaq_set_stats_precision(gptaq_handle_t h, int precision) {
         return GPTAQ_ERR_UNSUPPORTED;
     if (h->stage != STAGE_ACCUM) return GPTAQ_ERR_BAD_STATE;
     h->stats_precision = precision;
+    return GPTAQ_OK;
+}
+
+gptaq_status_t gptaq_set_update_terms(gptaq_handle_t h, int terms) {
+    if (!h) return GPTAQ_ERR_INVALID_ARG;
+    if (terms & ~(GPTAQ_TERM_ERR | GPTAQ_TERM_ASYM)) return GPTAQ_ERR_UNSUPPORTED;
+    h->terms = terms;
     return GPTAQ_OK;
 }
 

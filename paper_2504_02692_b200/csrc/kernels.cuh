@@ -530,6 +530,7 @@ struct ColumnLoopArgs {
     float *EW;                 // m x (2 * 32 * T): [-Err | Wpre]
     float *EW_lo;              // nullptr, or: EW receives the TF32 value of each entry and EW_lo the remainder
     StateHeader *hd;
+    float err_scale, asym_scale;   // 1 or 0: switches of the two terms of the weight update (ablation)
 };
 
 template <int T>
@@ -604,13 +605,14 @@ __global__ void __launch_bounds__(1024) column_loop_kernel(ColumnLoopArgs a) {
             const float wj = __shfl_sync(0xffffffffu, w[t], jj);
             float cq = fminf(fmaxf(rintf(wj / scale) + zero, 0.f), maxq);
             const float q = scale * (cq - zero);
-            const float ne = (q - wj) * (1.f / Us[j][j]);   // -(w - q) / U_jj
-            if (lane == jj) { w[t] = q; nerr[t] = ne; pre[t] = wj; code[t] = (int)cq; }
+            const float ne = a.err_scale * ((q - wj) * (1.f / Us[j][j]));   // -(w - q) / U_jj
+            const float wp = a.asym_scale * wj;
+            if (lane == jj) { w[t] = q; nerr[t] = ne; pre[t] = wp; code[t] = (int)cq; }
 #pragma unroll
             for (int t2 = 0; t2 < T; ++t2) {
                 if (t2 < t) continue;
                 int c = lane + 32 * t2;
-                if (c > j) w[t2] = fmaf(wj, Ps[j][c], fmaf(ne, Us[j][c], w[t2]));
+                if (c > j) w[t2] = fmaf(wp, Ps[j][c], fmaf(ne, Us[j][c], w[t2]));
             }
         }
     }
@@ -663,11 +665,12 @@ struct QuantStep {
     // x: the row's 32 columns (already-updated weights in, dequantized values out)
     static __device__ __forceinline__ void run(float (&x)[32], float (&nerr)[32], float (&pre)[32], uint32_t (&code)[8],
                                                const float *Us, const float *Ps, const float *udinv,
-                                               float scale, float zero, float maxq) {
-        const float w = x[K];
-        const float cq = fminf(fmaxf(rintf(w / scale) + zero, 0.f), maxq);
+                                               float scale, float zero, float maxq, float err_scale, float asym_scale) {
+        const float w0 = x[K];
+        const float cq = fminf(fmaxf(rintf(w0 / scale) + zero, 0.f), maxq);
         const float q = scale * (cq - zero);
-        const float ne = (q - w) * udinv[K];           // -(w - q) / U_kk
+        const float ne = err_scale * ((q - w0) * udinv[K]);           // -(w - q) / U_kk
+        const float w = asym_scale * w0;
         x[K] = q; nerr[K] = ne; pre[K] = w;
         code[K >> 2] |= (uint32_t)cq << (8 * (K & 3));
         const float *ur = Us + K * CB_LD, *pr = Ps + K * CB_LD;
@@ -680,13 +683,13 @@ struct QuantStep {
             if (4 * j4 + 2 > K) x[4 * j4 + 2] = fmaf(w, p.z, fmaf(ne, u.z, x[4 * j4 + 2]));
             if (4 * j4 + 3 > K) x[4 * j4 + 3] = fmaf(w, p.w, fmaf(ne, u.w, x[4 * j4 + 3]));
         }
-        QuantStep<K + 1>::run(x, nerr, pre, code, Us, Ps, udinv, scale, zero, maxq);
+        QuantStep<K + 1>::run(x, nerr, pre, code, Us, Ps, udinv, scale, zero, maxq, err_scale, asym_scale);
     }
 };
 template <>
 struct QuantStep<32> {
     static __device__ __forceinline__ void run(float (&)[32], float (&)[32], float (&)[32], uint32_t (&)[8],
-                                               const float *, const float *, const float *, float, float, float) {}
+                                               const float *, const float *, const float *, float, float, float, float, float) {}
 };
 
 __global__ void __launch_bounds__(CB_THREADS, 1) column_block_kernel(ColumnLoopArgs a, int rows, int B) {
@@ -766,7 +769,7 @@ __global__ void __launch_bounds__(CB_THREADS, 1) column_block_kernel(ColumnLoopA
                 x[4 * k4] = v.x; x[4 * k4 + 1] = v.y; x[4 * k4 + 2] = v.z; x[4 * k4 + 3] = v.w;
                 code[k4] = 0u;
             }
-            QuantStep<0>::run(x, nerr, pre, code, &Us[0][o], &Ps[0][o], udinv, scale, zero, maxq);
+            QuantStep<0>::run(x, nerr, pre, code, &Us[0][o], &Ps[0][o], udinv, scale, zero, maxq, a.err_scale, a.asym_scale);
             uint8_t *crow = a.codes + (int64_t)row * n + i0 + o;
             if ((reinterpret_cast<uintptr_t>(crow) & 15) == 0) {
                 *reinterpret_cast<uint4 *>(crow) = make_uint4(code[0], code[1], code[2], code[3]);

@@ -129,6 +129,42 @@ def test_shared_state_quantizes_several_matrices_and_in_place():
     st.close()
 
 
+@pytest.mark.parametrize("terms", [0, g.GPTAQ_TERM_ERR, g.GPTAQ_TERM_ASYM])
+@pytest.mark.parametrize("n,group,B", [(160, 0, 32), (640, 128, 128)])
+def test_update_term_switches(terms, n, group, B):
+    """Ablation switches (GPTQ, GPTAQ', RTN) against the oracle with the same terms."""
+    cfg = wl.scaled(wl.CONFIGS["cfg2"], name="terms", n=n, m=48, batch_tokens=1536, n_batches=1, group=group,
+                    blocksize=B, outlier_channels=3, alpha=1.0)
+    bt = batches_of(cfg)
+    W = wl.make_weight(cfg)
+    st = g.LayerState(cfg.n, cfg.m, cfg.batch_tokens, cfg.blocksize, total_tokens=cfg.tokens)
+    for X, Xfp in bt:
+        g.gptaq_accumulate(st.handle, X.cuda(), Xfp.cuda())
+    g.gptaq_factor(st.handle, cfg.damp)
+    g.gptaq_build_P(st.handle, cfg.alpha)
+    with pytest.raises(g.GptaqError):
+        g.gptaq_set_update_terms(st.handle, 4)
+    g.gptaq_set_update_terms(st.handle, terms)
+    G = hp.n_groups(cfg.n, cfg.group)
+    codes = torch.empty((cfg.m, cfg.n), dtype=torch.uint8, device="cuda")
+    sc = torch.empty((cfg.m, G), dtype=torch.float32, device="cuda")
+    zp = torch.empty((cfg.m, G), dtype=torch.float32, device="cuda")
+    g.gptaq_quantize(st.handle, W.cuda(), cfg.bits, cfg.group, cfg.sym, cfg.blocksize, codes, sc, zp, None)
+    assert g.gptaq_sync_status(st.handle)[0] == g.GPTAQ_OK
+    so = hp.oracle_stats(cfg, bt)
+    U, dead = orc.factor(so.H, so.tokens, cfg.damp)
+    P = orc.build_P(so.D, so.tokens, U, cfg.alpha) if terms & g.GPTAQ_TERM_ASYM else None
+    Wn = W.numpy().astype(np.float64)
+    rep = orc.follow(Wn, U, P, dead, cfg.bits, cfg.group, cfg.sym, codes.cpu().numpy(),
+                     sc.cpu().numpy().astype(np.float64), zp.cpu().numpy().astype(np.float64),
+                     band=hp.TOL_FLIP_BAND, error_term=bool(terms & g.GPTAQ_TERM_ERR))
+    assert rep.disallowed == 0 and rep.allowed <= hp.TOL_FLIP_RATE * rep.total, rep
+    if terms == 0:
+        rtn = orc.quantize(Wn, U, None, dead, cfg.bits, cfg.group, cfg.sym, update=False)
+        assert np.mean(codes.cpu().numpy() != rtn.codes) < 1e-3
+    st.close()
+
+
 def test_call_order_empty_inputs_and_bad_arguments():
     n, m = 96, 8
     st = g.LayerState(n, m, 64, 32)

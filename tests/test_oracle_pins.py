@@ -279,6 +279,28 @@ def test_rtn_limit_and_objective_order():
     assert J[1.0] < J["rtn"] and J[0.25] < J["rtn"] and J["gptq"] < J["rtn"]
 
 
+def test_update_terms_are_additive_and_switch_off_to_rtn():
+    """The two terms of Eq. "divided update" are separate additive corrections: after the first
+    column, (both terms) - W = (error term only) - W + (asymmetry term only) - W; with both off the
+    loop is round to nearest."""
+    W, X, Xfp = tiny(n=16, m=5)
+    st = stats_of(X, Xfp)
+    U, dead = orc.factor(st.H, st.tokens, 0.01)
+    P = orc.build_P(st.D, st.tokens, U, 1.0)
+    # one step only: a 2-column problem, the second column shows the update (undo its own rounding
+    # by reading the pre-rounding value)
+    def second_col(P_, err):
+        r = orc.quantize(W[:, :2], U[:2, :2], None if P_ is None else P_[:2, :2], None, 4, 0, False,
+                         keep_pre=True, error_term=err)
+        return r.pre[:, 1] * r.scales[:, 0]
+    both, gptq, ponly = second_col(P, True), second_col(None, True), second_col(P, False)
+    assert np.allclose(both - W[:, 1], (gptq - W[:, 1]) + (ponly - W[:, 1]), atol=1e-14)
+    assert not np.allclose(ponly, W[:, 1]) and not np.allclose(gptq, W[:, 1])
+    rtn = orc.quantize(W, U, None, dead, 4, 0, False, update=False)
+    off = orc.quantize(W, U, None, dead, 4, 0, False, error_term=False)
+    assert np.array_equal(rtn.codes, off.codes)
+
+
 @pytest.mark.parametrize("name", ["cfg1"])
 def test_objective_not_worse_than_rtn_on_config(name):
     cfg = wl.CONFIGS[name]
