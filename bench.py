@@ -204,6 +204,8 @@ def run_ours(args, cfg):
     prec_name = {g.GPTAQ_STATS_FP16_TENSOR: "fp16 operands, fp32 accumulate",
                  g.GPTAQ_STATS_FP16_SPLIT_TENSOR: "fp16 hi+lo split for H, fp32 accumulate"}[prec]
     stream = torch.cuda.current_stream()
+    if args.act_order:
+        g.gptaq_set_act_order(h, True)
 
     def ev():
         return torch.cuda.Event(enable_timing=True)
@@ -307,7 +309,7 @@ def run_ours(args, cfg):
         "vs_baseline": None, "dtype": "f16 x f16 -> f32 (statistics), f32 (solve)", "data": "synthetic",
         "config": dict(wl.describe(cfg), parallelism=f"{world} independent layer(s), one per GPU",
                        l2="inputs (%.1f GB per step) exceed L2" % (2 * cfg.tokens * cfg.n * 4 / 1e9),
-                       statistics=prec_name),
+                       statistics=prec_name, act_order=bool(args.act_order)),
         "stages_ms": {"accumulate": acc_step_ms, "factor": fac_ms, "build_P": p_ms, "quantize": q_ms,
                       "layer_quantize": fac_ms + p_ms + q_ms},
         "accumulate_tflops": achieved,
@@ -333,6 +335,7 @@ def main():
     ap.add_argument("--ref-rows", type=int, default=512)
     ap.add_argument("--batches", type=int, default=0,
                     help="profiler captures only: keep this many token batches (the line is marked truncated)")
+    ap.add_argument("--act-order", action="store_true", help="columns sorted by diag(H) (off in the headline configuration)")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()

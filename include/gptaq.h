@@ -214,6 +214,18 @@ gptaq_status_t gptaq_set_stats_precision(gptaq_handle_t h, int precision);
  * layer of width n calibrated on total_tokens tokens. */
 int gptaq_recommended_stats_precision(int64_t n, int64_t total_tokens);
 
+/* act_order (Section 5, experimental setup: "act_order, which sorts the columns by the Hessian diagonal"):
+ * when enabled (before gptaq_factor), gptaq_factor orders the inputs by decreasing diag(H) (dead inputs
+ * count as 1; ties keep the lower index first), permutes H and dXX^T accordingly, and gptaq_quantize
+ * processes the weight columns in that order.  Outputs: d_codes and d_Wq in the CALLER's column order;
+ * group grids (d_scales / d_zeros, group > 0) belong to groups of `group` consecutive columns of the
+ * SORTED order, i.e. caller column c uses group rank(c) / group, rank being the inverse of gptaq_perm.
+ * gptaq_quantize then needs d_Wq as a second buffer (non-NULL, different from d_W).
+ * gptaq_H / gptaq_D show U and P in sorted order.  Supported for n <= 57344.
+ * gptaq_perm: device array of n int32, sorted position -> caller column; NULL unless enabled and factored. */
+gptaq_status_t gptaq_set_act_order(gptaq_handle_t h, int enable);
+const int32_t *gptaq_perm(gptaq_handle_t h);
+
 /* Ablation switches of the weight update (Section 5.3, Table "ablation"): which of the two terms of
  * Eq. "divided update" later gptaq_quantize calls on this handle apply.
  *   GPTAQ_TERM_ERR    the quantization-error term  -(w_q - q_q)/U_qq * U[q, :]   (GPTQ's update)

@@ -404,6 +404,38 @@ def solve_layer(W, batches, damp, alpha, bits, group, sym, with_gram_of_delta=Tr
     return st, U, P, dead, res
 
 
+# --------------------------------------------------------------------------
+# act_order (Section 5, setup): columns sorted by the Hessian diagonal
+# --------------------------------------------------------------------------
+def act_order_perm(H_sum: np.ndarray, tokens: int) -> np.ndarray:
+    """Sorted position -> column: decreasing diag(H / k), dead inputs counting as 1 (they are set
+    to 1 before sorting), ties keeping the lower index first."""
+    d = np.diag(np.asarray(H_sum, F64)) / float(max(tokens, 1))
+    d = np.where(d == 0.0, 1.0, d)
+    return np.argsort(-d, kind="stable")
+
+
+def solve_act_order(W, H_sum, D_sum, tokens, damp, alpha, bits, group, sym, perm=None):
+    """Algorithm 1 on the layer with its inputs relabelled by ``perm`` (default: act_order_perm):
+    H and dXX^T are permuted on both sides, W on its columns; codes and dequantized weights are
+    returned in the original column order, group grids belong to groups of consecutive columns of
+    the sorted order.  Returns (U, P, dead, result, perm), U / P / dead in sorted order."""
+    W = np.asarray(W, F64)
+    if perm is None:
+        perm = act_order_perm(H_sum, tokens)
+    perm = np.asarray(perm)
+    Hp = np.asarray(H_sum, F64)[np.ix_(perm, perm)]
+    Dp = np.asarray(D_sum, F64)[np.ix_(perm, perm)]
+    U, dead = factor(Hp, tokens, damp)
+    P = build_P(Dp, tokens, U, alpha)
+    res = quantize(W[:, perm], U, P, dead, bits, group, sym)
+    codes = np.empty_like(res.codes)
+    Wq = np.empty_like(res.Wq)
+    codes[:, perm] = res.codes
+    Wq[:, perm] = res.Wq
+    return U, P, dead, QuantResult(codes, res.scales, res.zeros, Wq), perm
+
+
 def working_set_elements(m: int, n: int, blocksize: int, asymmetric: bool) -> dict:
     """Matrix dimensions held during the loop (appendix memory table):
     W, H (then L), Q, E for GPTQ; GPTAQ adds dXX^T (then P).  The table lists

@@ -58,6 +58,8 @@ SIGNATURES = {
     "gptaq_set_tokens": (_int, [_vp, _i64]),
     "gptaq_set_stats_precision": (_int, [_vp, _int]),
     "gptaq_set_update_terms": (_int, [_vp, _int]),
+    "gptaq_set_act_order": (_int, [_vp, _int]),
+    "gptaq_perm": (_vp, [_vp]),
     "gptaq_recommended_stats_precision": (_int, [_i64, _i64]),
     "gptaq_launch_count": (_i64, [_vp]),
     "gptaq_status_string": (C.c_char_p, [_int]),
@@ -278,6 +280,15 @@ def gptaq_set_stats_precision(h, precision: int):
     _check(load_library().gptaq_set_stats_precision(h, precision), "gptaq_set_stats_precision", h)
 
 
+def gptaq_set_act_order(h, enable: bool):
+    """Columns processed in order of decreasing diag(H); set before gptaq_factor."""
+    _check(load_library().gptaq_set_act_order(h, int(bool(enable))), "gptaq_set_act_order", h)
+
+
+def gptaq_perm_ptr(h) -> int | None:
+    return load_library().gptaq_perm(h)
+
+
 def gptaq_set_update_terms(h, terms: int):
     """Ablation switches: ``GPTAQ_TERM_ERR | GPTAQ_TERM_ASYM`` (default) = GPTAQ, ERR = GPTQ, ASYM = GPTAQ', 0 = RTN."""
     _check(load_library().gptaq_set_update_terms(h, terms), "gptaq_set_update_terms", h)
@@ -335,6 +346,14 @@ class LayerState:
         """View of dXX^T (before build_P) / P (after), current on torch's stream."""
         gptaq_flush(self.handle)
         return self._view(gptaq_D_ptr(self.handle))
+
+    def perm(self) -> torch.Tensor | None:
+        """act_order: int32 ``[n]``, sorted position -> caller column (None unless enabled and factored)."""
+        ptr = gptaq_perm_ptr(self.handle)
+        if not ptr:
+            return None
+        off = ptr - self.state.data_ptr()
+        return self.state[off:off + 4 * self.n].view(torch.int32)
 
     def close(self):
         if self.handle is not None:

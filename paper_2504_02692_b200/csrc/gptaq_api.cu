@@ -24,6 +24,7 @@ constexpr size_t ALIGN = 256;
 inline size_t round_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 
 enum Stage { STAGE_ACCUM = 0, STAGE_FACTORED = 1, STAGE_P = 2 };
+constexpr int64_t ACT_ORDER_MAX_N = 57344;     // a weight row (float32) has to fit the shared memory of one CTA
 
 }  // namespace
 
@@ -37,7 +38,10 @@ struct gptaq_ctx {
     size_t ws_bytes;
     StateHeader *hd;
     float *H, *D;
-    uint8_t *dead;
+    uint8_t *dead;         // dead-input flags in working (possibly sorted) column order
+    uint8_t *dead_raw;     // ... in the caller's column order
+    int *perm;             // act_order: working column c is the caller's column perm[c]
+    bool act_order;
     int stage;
     int64_t tokens;
     int64_t launches;
@@ -57,7 +61,7 @@ struct gptaq_ctx {
 namespace {
 
 struct Layout {
-    size_t h_off, d_off, dead_off, total;
+    size_t h_off, d_off, dead_off, dead_raw_off, perm_off, total;
 };
 
 Layout state_layout(int64_t n) {
@@ -66,7 +70,9 @@ Layout state_layout(int64_t n) {
     l.h_off = ALIGN;
     l.d_off = l.h_off + mat;
     l.dead_off = l.d_off + mat;
-    l.total = l.dead_off + round_up((size_t)n, ALIGN);
+    l.dead_raw_off = l.dead_off + round_up((size_t)n, ALIGN);
+    l.perm_off = l.dead_raw_off + round_up((size_t)n, ALIGN);
+    l.total = l.perm_off + round_up((size_t)n * sizeof(int), ALIGN);
     return l;
 }
 
@@ -350,6 +356,7 @@ struct QuantizeTarget {
     const float *UT_hi, *UT_lo, *PT_hi, *PT_lo;
     float *EW_lo;
     int terms = GPTAQ_TERM_ERR | GPTAQ_TERM_ASYM;   // which terms of the weight update are applied
+    const int *perm = nullptr;                      // act_order: working column c is the caller's column perm[c]
 };
 
 gptaq_status_t check_quantize_args(int64_t n, const void *d_W, int w_dtype, int64_t m, int64_t ldw, int bits,
@@ -380,7 +387,17 @@ gptaq_status_t quantize_core(const QuantizeTarget &t, void *d_W, int w_dtype, in
     float *EW = t.EW;
     float *Wk = static_cast<float *>(d_W);
     int64_t ldk = ldw;
-    if (w_dtype == GPTAQ_W_BF16) {
+    if (t.perm) {
+        // working copy in sorted column order (the caller's d_Wq; checked to be a second buffer)
+        if (w_dtype == GPTAQ_W_BF16)
+            gather_cols_kernel<__nv_bfloat16><<<t.num_sms * 8, 256, 0, s>>>(static_cast<const __nv_bfloat16 *>(d_W), ldw,
+                                                                           d_Wq, n, (int)m, n, t.perm);
+        else
+            gather_cols_kernel<float><<<t.num_sms * 8, 256, 0, s>>>(static_cast<const float *>(d_W), ldw, d_Wq, n,
+                                                                   (int)m, n, t.perm);
+        QLAUNCHED();
+        Wk = d_Wq; ldk = n;
+    } else if (w_dtype == GPTAQ_W_BF16) {
         bf16_to_f32_kernel<<<t.num_sms * 8, 256, 0, s>>>(static_cast<const __nv_bfloat16 *>(d_W), ldw,
                                                         d_Wq, n, (int)m, n);
         QLAUNCHED();
@@ -421,7 +438,7 @@ gptaq_status_t quantize_core(const QuantizeTarget &t, void *d_W, int w_dtype, in
         a.i0 = i0; a.bw = std::min(blocksize, n - i0);
         a.bits = bits; a.group = group; a.sym = sym;
         a.codes = d_codes; a.scales = d_scales; a.zeros = d_zeros; a.G = G; a.EW = EW; a.EW_lo = t.EW_lo; a.hd = t.hd;
-        a.err_scale = (t.terms & GPTAQ_TERM_ERR) ? 1.f : 0.f; a.asym_scale = (t.terms & GPTAQ_TERM_ASYM) ? 1.f : 0.f;
+        a.perm = t.perm; a.err_scale = (t.terms & GPTAQ_TERM_ERR) ? 1.f : 0.f; a.asym_scale = (t.terms & GPTAQ_TERM_ASYM) ? 1.f : 0.f;
         const bool fast = a.bw == blocksize && (group <= 0 || (group % 32) == 0) && (i0 % 4) == 0 &&
                           (reinterpret_cast<uintptr_t>(t.dead) & 3) == 0;
         if (fast) column_block_kernel<<<cb_grid, CB_THREADS, column_block_smem(cb_rows), s>>>(a, cb_rows, blocksize);
@@ -449,6 +466,11 @@ gptaq_status_t quantize_core(const QuantizeTarget &t, void *d_W, int w_dtype, in
             if (*err != cudaSuccess) return GPTAQ_ERR_CUDA;
             ++*launches;
         }
+    }
+    if (t.perm) {
+        // dequantized weights back to the caller's column order
+        unpermute_rows_kernel<<<(unsigned)m, 256, (size_t)n * sizeof(float), s>>>(Wk, ldk, n, t.perm);
+        QLAUNCHED();
     }
     return GPTAQ_OK;
 }
@@ -551,6 +573,9 @@ gptaq_status_t gptaq_create(gptaq_handle_t *out, int64_t n, void *d_state, size_
     h->H = reinterpret_cast<float *>(h->state + l.h_off);
     h->D = reinterpret_cast<float *>(h->state + l.d_off);
     h->dead = reinterpret_cast<uint8_t *>(h->state + l.dead_off);
+    h->dead_raw = reinterpret_cast<uint8_t *>(h->state + l.dead_raw_off);
+    h->perm = reinterpret_cast<int *>(h->state + l.perm_off);
+    h->act_order = false;
     h->launches = 0;
     h->stats_precision = GPTAQ_STATS_FP16_SPLIT_TENSOR;
     h->tensor = tc_shape_ok(n) && encode_tiled_fn() != nullptr;
@@ -582,6 +607,8 @@ gptaq_status_t gptaq_create(gptaq_handle_t *out, int64_t n, void *d_state, size_
     if (e == cudaSuccess)
         e = cudaFuncSetAttribute(column_block_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                  (int)column_block_smem(128));
+    if (e == cudaSuccess)
+        e = cudaFuncSetAttribute(unpermute_rows_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)ACT_ORDER_MAX_N * 4);
     if (e != cudaSuccess) {
         delete h;
         return GPTAQ_ERR_CUDA;
@@ -691,8 +718,22 @@ gptaq_status_t gptaq_factor(gptaq_handle_t h, float damp, gptaq_stream_t stream)
     float *Rinv = reinterpret_cast<float *>(h->ws + wl.rinv_off);
     float *H = h->H;
 
-    diag_stats_kernel<<<1, 1024, 0, s>>>(H, n, (float)(1.0 / (double)h->tokens), damp, h->hd, h->dead);
+    diag_stats_kernel<<<1, 1024, 0, s>>>(H, n, (float)(1.0 / (double)h->tokens), damp, h->hd, h->dead_raw);
     LAUNCHED();
+    if (h->act_order) {
+        // columns in order of decreasing diag(H): H and dXX^T are permuted on both sides, through T
+        rank_desc_kernel<<<(n + 255) / 256, 256, 0, s>>>(H, n, (float)(1.0 / (double)h->tokens), h->dead_raw, h->perm, h->dead);
+        LAUNCHED();
+        const dim3 pg((n + 255) / 256, n);
+        permute_matrix_kernel<<<pg, 256, 0, s>>>(H, T, n, h->perm, 1);
+        LAUNCHED();
+        CU(cudaMemcpyAsync(H, T, (size_t)n * n * sizeof(float), cudaMemcpyDeviceToDevice, s));
+        permute_matrix_kernel<<<pg, 256, 0, s>>>(h->D, T, n, h->perm, 0);
+        LAUNCHED();
+        CU(cudaMemcpyAsync(h->D, T, (size_t)n * n * sizeof(float), cudaMemcpyDeviceToDevice, s));
+    } else {
+        CU(cudaMemcpyAsync(h->dead, h->dead_raw, (size_t)n, cudaMemcpyDeviceToDevice, s));
+    }
     scale_damp_kernel<<<dim3((n + 63) / 64, (n + 63) / 64), 256, 0, s>>>(H, n, h->hd, h->dead);
     LAUNCHED();
 
@@ -848,6 +889,7 @@ gptaq_status_t gptaq_quantize(gptaq_handle_t h, void *d_W, int w_dtype, int64_t 
     gptaq_status_t st = check_quantize_args(h->n, d_W, w_dtype, m, ldw, bits, group, blocksize, d_codes,
                                             d_scales, d_zeros, d_Wq);
     if (st != GPTAQ_OK || m == 0) return st;
+    if (h->act_order && (!d_Wq || d_Wq == d_W)) return GPTAQ_ERR_INVALID_ARG;
     WsLayout wl = ws_layout(h->n, m, blocksize);
     if (h->ws_bytes < wl.total) return GPTAQ_ERR_WORKSPACE;
     QuantizeTarget t;
@@ -855,6 +897,7 @@ gptaq_status_t gptaq_quantize(gptaq_handle_t h, void *d_W, int w_dtype, int64_t 
     t.EW = reinterpret_cast<float *>(h->ws + wl.ew_off);
     t.num_sms = h->num_sms;
     t.terms = h->terms;
+    t.perm = h->act_order ? h->perm : nullptr;
     t.UT_hi = t.UT_lo = t.PT_hi = t.PT_lo = nullptr; t.EW_lo = nullptr;
     if (h->tensor) {
         t.UT_hi = reinterpret_cast<float *>(h->ws + wl.s_off[2]); t.UT_lo = reinterpret_cast<float *>(h->ws + wl.s_off[3]);
@@ -973,6 +1016,16 @@ gptaq_status_t gptaq_set_stats_precision(gptaq_handle_t h, int precision) {
     h->stats_precision = precision;
     return GPTAQ_OK;
 }
+
+gptaq_status_t gptaq_set_act_order(gptaq_handle_t h, int enable) {
+    if (!h) return GPTAQ_ERR_INVALID_ARG;
+    if (h->stage != STAGE_ACCUM) return GPTAQ_ERR_BAD_STATE;
+    if (enable && h->n > ACT_ORDER_MAX_N) return GPTAQ_ERR_UNSUPPORTED;
+    h->act_order = enable != 0;
+    return GPTAQ_OK;
+}
+
+const int32_t *gptaq_perm(gptaq_handle_t h) { return (h && h->act_order && h->stage != STAGE_ACCUM) ? h->perm : nullptr; }
 
 gptaq_status_t gptaq_set_update_terms(gptaq_handle_t h, int terms) {
     if (!h) return GPTAQ_ERR_INVALID_ARG;

@@ -531,6 +531,7 @@ struct ColumnLoopArgs {
     float *EW_lo;              // nullptr, or: EW receives the TF32 value of each entry and EW_lo the remainder
     StateHeader *hd;
     float err_scale, asym_scale;   // 1 or 0: switches of the two terms of the weight update (ablation)
+    const int *perm;               // nullptr, or: working column c is original column perm[c] (codes go there)
 };
 
 template <int T>
@@ -634,7 +635,8 @@ __global__ void __launch_bounds__(1024) column_loop_kernel(ColumnLoopArgs a) {
         }
         if (c < bw) {
             wrow[c] = w[t];
-            crow[c] = (uint8_t)code[t];
+            if (a.perm) a.codes[(int64_t)row * n + a.perm[i0 + c]] = (uint8_t)code[t];
+            else crow[c] = (uint8_t)code[t];
             bad |= !isfinite(w[t]);
         }
     }
@@ -771,7 +773,12 @@ __global__ void __launch_bounds__(CB_THREADS, 1) column_block_kernel(ColumnLoopA
             }
             QuantStep<0>::run(x, nerr, pre, code, &Us[0][o], &Ps[0][o], udinv, scale, zero, maxq, a.err_scale, a.asym_scale);
             uint8_t *crow = a.codes + (int64_t)row * n + i0 + o;
-            if ((reinterpret_cast<uintptr_t>(crow) & 15) == 0) {
+            if (a.perm) {
+                uint8_t *cbase = a.codes + (int64_t)row * n;
+                const int *pp = a.perm + i0 + o;
+#pragma unroll
+                for (int k = 0; k < 32; ++k) cbase[pp[k]] = (uint8_t)(code[k >> 2] >> (8 * (k & 3)));
+            } else if ((reinterpret_cast<uintptr_t>(crow) & 15) == 0) {
                 *reinterpret_cast<uint4 *>(crow) = make_uint4(code[0], code[1], code[2], code[3]);
                 *reinterpret_cast<uint4 *>(crow + 16) = make_uint4(code[4], code[5], code[6], code[7]);
             } else {
@@ -850,6 +857,66 @@ __global__ void __launch_bounds__(CB_THREADS, 1) column_block_kernel(ColumnLoopA
         else { dst[0] = v.x; dst[1] = v.y; dst[2] = v.z; dst[3] = v.w; }
         if (bad) record_status(a.hd, ST_NONFINITE, row0 + r);
     }
+}
+
+// ---------------------------------------------------------------------------
+// act_order: columns sorted by decreasing diag(H).
+// ---------------------------------------------------------------------------
+// perm[rank] = q, rank = number of inputs that sort before q: larger value v (v = 1 for dead
+// inputs, else H_qq / tokens), ties by smaller index (a stable descending sort).  O(n^2) compares.
+__global__ void __launch_bounds__(256) rank_desc_kernel(const float *H, int n, float inv_tokens, const uint8_t *dead,
+                                                        int *perm, uint8_t *dead_perm) {
+    __shared__ float tile[256];
+    const int q = blockIdx.x * 256 + threadIdx.x;
+    const float vq = q < n ? (dead[q] ? 1.f : H[(int64_t)q * n + q] * inv_tokens) : 0.f;
+    int rank = 0;
+    for (int j0 = 0; j0 < n; j0 += 256) {
+        const int j = j0 + threadIdx.x;
+        tile[threadIdx.x] = j < n ? (dead[j] ? 1.f : H[(int64_t)j * n + j] * inv_tokens) : -1.f;
+        __syncthreads();
+        const int lim = min(256, n - j0);
+        for (int t = 0; t < lim; ++t) {
+            const float v = tile[t];
+            rank += (v > vq) || (v == vq && j0 + t < q);
+        }
+        __syncthreads();
+    }
+    if (q < n) { perm[rank] = q; dead_perm[rank] = dead[q]; }
+}
+
+// dst[i][j] = src[perm[i]][perm[j]]; `symmetric_upper`: src holds a symmetric matrix in its upper
+// triangle (element (a, b) is read at (min, max)) and only j >= i is written.
+__global__ void __launch_bounds__(256) permute_matrix_kernel(const float *src, float *dst, int n, const int *perm,
+                                                             int symmetric_upper) {
+    const int j = blockIdx.x * 256 + threadIdx.x;
+    const int i = blockIdx.y;
+    if (j >= n) return;
+    if (symmetric_upper && j < i) return;
+    int a = perm[i], b = perm[j];
+    if (symmetric_upper && a > b) { const int t = a; a = b; b = t; }
+    dst[(int64_t)i * n + j] = src[(int64_t)a * n + b];
+}
+
+// dst[r][c] = src[r][perm[c]] as float32 (src float32 or bf16): the working copy of W in sorted order.
+template <typename T>
+__global__ void __launch_bounds__(256) gather_cols_kernel(const T *src, int64_t lds, float *dst, int64_t ldd, int m, int n,
+                                                          const int *perm) {
+    int64_t idx = (int64_t)blockIdx.x * 256 + threadIdx.x;
+    const int64_t total = (int64_t)m * n;
+    for (; idx < total; idx += (int64_t)gridDim.x * 256) {
+        const int64_t r = idx / n, c = idx % n;
+        dst[r * ldd + c] = (float)src[r * lds + perm[c]];
+    }
+}
+
+// In place, one CTA per row: W[r][perm[c]] <- W[r][c] (back to the original column order); the
+// row is staged in shared memory (n floats).
+__global__ void __launch_bounds__(256) unpermute_rows_kernel(float *W, int64_t ldw, int n, const int *perm) {
+    extern __shared__ float row_s[];
+    float *w = W + (int64_t)blockIdx.x * ldw;
+    for (int c = threadIdx.x; c < n; c += 256) row_s[c] = w[c];
+    __syncthreads();
+    for (int c = threadIdx.x; c < n; c += 256) w[perm[c]] = row_s[c];
 }
 
 __global__ void __launch_bounds__(256) bf16_to_f32_kernel(const __nv_bfloat16 *src, int64_t lds,

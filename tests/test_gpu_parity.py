@@ -165,6 +165,63 @@ def test_update_term_switches(terms, n, group, B):
     st.close()
 
 
+@pytest.mark.parametrize("n,m,group,B,bf16", [(160, 40, 0, 32, False), (200, 24, 32, 64, False),
+                                                (640, 96, 128, 128, False), (768, 64, 0, 128, True)])
+def test_act_order(n, m, group, B, bf16):
+    """Columns sorted by diag(H).  Several orders are valid where two diagonal entries agree to within the
+    rounding of the statistics, so the device's permutation is checked for validity (it sorts the device's own
+    diagonal; against the float64 diagonal only near-ties may be swapped) and then handed to the oracle."""
+    cfg = wl.scaled(wl.CONFIGS["cfg2"], name="act", n=n, m=m, batch_tokens=2048, n_batches=2, group=group,
+                    blocksize=B, outlier_channels=4, w_bf16=bf16)
+    bt = batches_of(cfg)
+    W = wl.make_weight(cfg)
+    st = g.LayerState(cfg.n, cfg.m, cfg.batch_tokens, cfg.blocksize, total_tokens=cfg.tokens)
+    g.gptaq_set_act_order(st.handle, True)
+    assert st.perm() is None
+    for X, Xfp in bt:
+        g.gptaq_accumulate(st.handle, X.cuda(), Xfp.cuda())
+    diag_dev = torch.diagonal(st.H()).cpu().numpy().astype(np.float64)
+    g.gptaq_factor(st.handle, cfg.damp)
+    g.gptaq_build_P(st.handle, cfg.alpha)
+    perm = st.perm().cpu().numpy().astype(np.int64)
+    assert sorted(perm.tolist()) == list(range(n))
+    assert np.all(np.diff(diag_dev[perm]) <= 0)                       # sorts the device's own diagonal
+    so = hp.oracle_stats(cfg, bt)
+    d64 = np.diag(so.H)[perm]
+    assert np.all(np.diff(d64) <= 2.0 ** -9 * d64[:-1])               # only near-ties out of float64 order
+    Ug = st.H().cpu().numpy().astype(np.float64)
+    Pg = st.D().cpu().numpy().astype(np.float64)
+    G = hp.n_groups(cfg.n, cfg.group)
+    codes = torch.empty((m, n), dtype=torch.uint8, device="cuda")
+    sc = torch.empty((m, G), dtype=torch.float32, device="cuda")
+    zp = torch.empty((m, G), dtype=torch.float32, device="cuda")
+    Wq = torch.empty((m, n), dtype=torch.float32, device="cuda")
+    Wd = W.cuda().to(torch.bfloat16) if bf16 else W.cuda()
+    with pytest.raises(g.GptaqError):                                  # needs a second buffer
+        g.gptaq_quantize(st.handle, W.cuda(), cfg.bits, cfg.group, cfg.sym, cfg.blocksize, codes, sc, zp, None)
+    g.gptaq_quantize(st.handle, Wd, cfg.bits, cfg.group, cfg.sym, cfg.blocksize, codes, sc, zp, Wq)
+    assert g.gptaq_sync_status(st.handle)[0] == g.GPTAQ_OK
+    Wn = W.numpy().astype(np.float64)
+    U, P, dead, res, _ = orc.solve_act_order(Wn, so.H, so.D, so.tokens, cfg.damp, cfg.alpha, cfg.bits, cfg.group,
+                                             cfg.sym, perm=perm)
+    assert hp.rel_fro(np.triu(Ug), U) <= hp.TOL_FACTOR
+    assert hp.rel_fro(np.triu(Pg, 1), P) <= 5e-3
+    cg = codes.cpu().numpy()
+    rep = orc.follow(Wn[:, perm], U, P, dead, cfg.bits, cfg.group, cfg.sym, cg[:, perm],
+                     sc.cpu().numpy().astype(np.float64), zp.cpu().numpy().astype(np.float64), band=hp.TOL_FLIP_BAND)
+    assert rep.disallowed == 0 and rep.allowed <= hp.TOL_FLIP_RATE * rep.total, rep
+    assert rep.grid_rel_err <= 5e-5 and rep.zero_mismatch == 0, rep
+    # dequantized weights come back in the caller's column order and match codes and grids
+    gsz = cfg.group if cfg.group > 0 else n
+    scp = np.repeat(sc.cpu().numpy(), gsz, axis=1)[:, :n]
+    zpp = np.repeat(zp.cpu().numpy(), gsz, axis=1)[:, :n]
+    deq_sorted = scp * (cg[:, perm].astype(np.float32) - zpp)
+    assert np.array_equal(Wq.cpu().numpy()[:, perm], deq_sorted.astype(np.float32))
+    J_gpu, J_orc = orc.objective(Wn, Wq.cpu().numpy().astype(np.float64), so), orc.objective(Wn, res.Wq, so)
+    assert abs(J_gpu - J_orc) <= hp.TOL_OBJECTIVE * J_orc
+    st.close()
+
+
 def test_call_order_empty_inputs_and_bad_arguments():
     n, m = 96, 8
     st = g.LayerState(n, m, 64, 32)

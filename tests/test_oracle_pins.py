@@ -348,6 +348,38 @@ def test_row_independence_and_scale_invariance():
     assert np.allclose(P3, P, atol=1e-12)
 
 
+# ---------------------------------------------------------------- act_order
+@pytest.mark.parametrize("group", [0, 8])
+def test_act_order_is_a_relabelling_sorted_by_the_diagonal(group):
+    W, X, Xfp = tiny(n=24, m=6)
+    X = X * np.linspace(0.5, 3.0, 24)[None, ::-1] ** 0.5 * np.random.default_rng(9).uniform(0.9, 1.1, 24)
+    st = stats_of(X, Xfp)
+    perm = orc.act_order_perm(st.H, st.tokens)
+    d = np.diag(st.H)
+    assert sorted(perm.tolist()) == list(range(24)) and np.all(np.diff(d[perm]) <= 0)
+    U, P, dead, res, _ = orc.solve_act_order(W, st.H, st.D, st.tokens, 0.01, 0.5, 4, group, False)
+    # the same as the plain solve of the explicitly relabelled layer
+    stp = stats_of(X[:, perm], Xfp[:, perm])
+    Up, deadp = orc.factor(stp.H, stp.tokens, 0.01)
+    Pp = orc.build_P(stp.D, stp.tokens, Up, 0.5)
+    plain = orc.quantize(W[:, perm], Up, Pp, deadp, 4, group, False)
+    assert np.array_equal(res.codes[:, perm], plain.codes) and np.allclose(res.Wq[:, perm], plain.Wq, atol=1e-12)
+    assert np.allclose(res.scales, plain.scales, atol=1e-14)
+    # invariance: relabelling the inputs beforehand changes nothing (the sorted order is canonical)
+    pi = np.random.default_rng(4).permutation(24)
+    st2 = stats_of(X[:, pi], Xfp[:, pi])
+    _, _, _, res2, perm2 = orc.solve_act_order(W[:, pi], st2.H, st2.D, st2.tokens, 0.01, 0.5, 4, group, False)
+    assert np.array_equal(pi[perm2], perm)
+    back = np.empty_like(res2.codes); back[:, pi] = res2.codes
+    assert np.array_equal(back, res.codes) and np.allclose(res2.scales, res.scales, atol=1e-12)
+    # already sorted input: the identity, and the plain solve
+    st3 = stats_of(X[:, perm], Xfp[:, perm])
+    assert np.array_equal(orc.act_order_perm(st3.H, st3.tokens), np.arange(24))
+    # ties keep the lower index first; dead inputs count as 1
+    Ht = np.diag([2.0, 0.0, 2.0, 0.5, 1.0])
+    assert orc.act_order_perm(Ht, 1).tolist() == [0, 2, 1, 4, 3]
+
+
 # ---------------------------------------------------------------- objective
 def test_objective_identity():
     W, X, Xfp = tiny(n=12, m=4, k=90)
