@@ -222,6 +222,38 @@ def test_act_order(n, m, group, B, bf16):
     st.close()
 
 
+def test_correlated_inputs_stress():
+    """Correlated channels (X <- X A, A = identity + low rank): cond(H_d) grows from ~1e3 (independent
+    channels of the benchmark layers) to ~2e4.  float32 sums and a float32 factorization then carry
+    cond * 1e-8 of relative error into U, which is past the 1e-4 bound of the benchmark layers for any choice of
+    statistics arithmetic (the exact-float32 path included); this test records that, and checks what must
+    hold regardless: a clean status, the loop's parity given the device's own U and P, and the objective."""
+    n = 1024
+    cfg = wl.scaled(wl.CONFIGS["cfg2"], name="stress", n=n, m=128, batch_tokens=4096, n_batches=4, outlier_channels=10)
+    gen = torch.Generator().manual_seed(5)
+    A = torch.eye(n) + 10.0 / n ** 0.5 * (torch.randn(n, 64, generator=gen) @ torch.randn(64, n, generator=gen)) / 8.0
+    bt = [((X @ A).contiguous(), (Xfp @ A).contiguous()) for X, Xfp in batches_of(cfg)]
+    W = wl.make_weight(cfg)
+    run = hp.gpu_layer(cfg, W, bt)
+    assert run.status[0] == g.GPTAQ_OK
+    so = hp.oracle_stats(cfg, bt)
+    U, dead = orc.factor(so.H, so.tokens, cfg.damp)
+    P = orc.build_P(so.D, so.tokens, U, cfg.alpha)
+    Hd, _ = orc.damped_hessian(so.H, so.tokens, cfg.damp)
+    cond = np.linalg.cond(Hd)
+    U_rel = hp.rel_fro(np.triu(run.U), U)
+    assert 5e3 < cond < 1e5 and U_rel < 1e-7 * cond, (cond, U_rel)
+    Wn = W.numpy().astype(np.float64)
+    rep = orc.follow(Wn, np.triu(run.U), np.triu(run.P, 1), dead, cfg.bits, cfg.group, cfg.sym, run.codes, run.scales,
+                     run.zeros, band=hp.TOL_FLIP_BAND)
+    assert rep.disallowed == 0 and rep.allowed <= hp.TOL_FLIP_RATE * rep.total, rep
+    res = orc.quantize(Wn, U, P, dead, cfg.bits, cfg.group, cfg.sym)
+    J_gpu, J_orc = orc.objective(Wn, run.Wq, so), orc.objective(Wn, res.Wq, so)
+    assert abs(J_gpu - J_orc) <= hp.TOL_OBJECTIVE * J_orc, (J_gpu, J_orc)
+    print(f"correlated stress: cond {cond:.2e}, U rel {U_rel:.2e}, J rel {abs(J_gpu - J_orc) / J_orc:.2e}, "
+          f"free-running mismatch {np.mean(run.codes != res.codes):.2e}")
+
+
 def test_call_order_empty_inputs_and_bad_arguments():
     n, m = 96, 8
     st = g.LayerState(n, m, 64, 32)
