@@ -204,6 +204,10 @@ gptaq_status_t gptaq_sync_status(gptaq_handle_t h, int64_t *info, gptaq_stream_t
  * callers that checkpoint the sums: H / U and dXX^T / P share storage. */
 float *gptaq_H(gptaq_handle_t h);
 float *gptaq_D(gptaq_handle_t h);
+/* The same storage under the names of what it holds later: U (Algorithm 1, line 3; NULL before
+ * gptaq_factor) and P (line 4; NULL before gptaq_build_P). */
+const float *gptaq_U(gptaq_handle_t h);
+const float *gptaq_P(gptaq_handle_t h);
 int64_t gptaq_tokens(gptaq_handle_t h);
 /* Sets the token count (for callers that restore checkpointed sums). */
 gptaq_status_t gptaq_set_tokens(gptaq_handle_t h, int64_t tokens);
@@ -237,6 +241,12 @@ gptaq_status_t gptaq_set_update_terms(gptaq_handle_t h, int terms);
 
 /* Number of kernels this handle has launched since create (bookkeeping for benchmarks). */
 int64_t gptaq_launch_count(gptaq_handle_t h);
+
+/* Failure-path self-test: enqueues one warp that waits, with the bounded wait of the tensor-core
+ * kernels, for a barrier that nothing completes; after `seconds` (0 < seconds <= 2, in SM clock
+ * cycles at the nominal clock) it gives up and records GPTAQ_ERR_TIMEOUT (info 2000000) for
+ * gptaq_sync_status.  Nothing traps and the context stays usable; gptaq_reset clears the status. */
+gptaq_status_t gptaq_selftest_bounded_wait(gptaq_handle_t h, double seconds, gptaq_stream_t stream);
 
 const char *gptaq_status_string(gptaq_status_t s);
 /* Text of the last CUDA runtime error seen by this handle ("" if none). */

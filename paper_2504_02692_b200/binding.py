@@ -54,6 +54,9 @@ SIGNATURES = {
     "gptaq_sync_status": (_int, [_vp, C.POINTER(_i64), _vp]),
     "gptaq_H": (_vp, [_vp]),
     "gptaq_D": (_vp, [_vp]),
+    "gptaq_U": (_vp, [_vp]),
+    "gptaq_P": (_vp, [_vp]),
+    "gptaq_selftest_bounded_wait": (_int, [_vp, C.c_double, _vp]),
     "gptaq_tokens": (_i64, [_vp]),
     "gptaq_set_tokens": (_int, [_vp, _i64]),
     "gptaq_set_stats_precision": (_int, [_vp, _int]),
@@ -266,6 +269,11 @@ def gptaq_sync_status(h, stream=None):
     info = _i64(0)
     st = load_library().gptaq_sync_status(h, C.byref(info), _stream(stream))
     return st, info.value
+
+
+def gptaq_selftest_bounded_wait(h, seconds: float, stream=None):
+    """Makes a bounded device-side wait run out on purpose; gptaq_sync_status then reports GPTAQ_ERR_TIMEOUT."""
+    _check(load_library().gptaq_selftest_bounded_wait(h, seconds, _stream(stream)), "gptaq_selftest_bounded_wait", h)
 
 
 def gptaq_tokens(h) -> int:

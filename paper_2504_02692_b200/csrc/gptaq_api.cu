@@ -998,6 +998,18 @@ gptaq_status_t gptaq_sync_status(gptaq_handle_t h, int64_t *info, gptaq_stream_t
 
 float *gptaq_H(gptaq_handle_t h) { return h ? h->H : nullptr; }
 float *gptaq_D(gptaq_handle_t h) { return h ? h->D : nullptr; }
+const float *gptaq_U(gptaq_handle_t h) { return (h && h->stage != STAGE_ACCUM) ? h->H : nullptr; }
+const float *gptaq_P(gptaq_handle_t h) { return (h && h->stage == STAGE_P) ? h->D : nullptr; }
+
+gptaq_status_t gptaq_selftest_bounded_wait(gptaq_handle_t h, double seconds, gptaq_stream_t stream) {
+    if (!h || !(seconds > 0.0) || seconds > 2.0) return GPTAQ_ERR_INVALID_ARG;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    int khz = 0;
+    CU(cudaDeviceGetAttribute(&khz, cudaDevAttrClockRate, h->device));
+    bounded_wait_selftest_kernel<<<1, 32, 0, s>>>(h->hd, (long long)(seconds * 1e3 * (double)khz));
+    LAUNCHED();
+    return GPTAQ_OK;
+}
 int64_t gptaq_tokens(gptaq_handle_t h) { return h ? h->tokens : -1; }
 
 gptaq_status_t gptaq_set_tokens(gptaq_handle_t h, int64_t tokens) {

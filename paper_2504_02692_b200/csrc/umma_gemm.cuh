@@ -184,14 +184,15 @@ __device__ __forceinline__ bool mbar_try(uint32_t bar, uint32_t parity) {
     return ok != 0;
 }
 // Bounded wait: false if the clock limit ran out or another role gave up.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag) {
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag,
+                                          long long limit_cycles = WAIT_LIMIT_CYCLES) {
     if (mbar_try(bar, parity)) return true;
     const long long t0 = clock64();
     for (uint32_t it = 1;; ++it) {
         if (mbar_try(bar, parity)) return true;
         if ((it & 63) == 0) {
             if (*abort_flag) return false;
-            if (clock64() - t0 > WAIT_LIMIT_CYCLES) { *abort_flag = 1; return false; }
+            if (clock64() - t0 > limit_cycles) { *abort_flag = 1; return false; }
         }
     }
 }
@@ -484,6 +485,22 @@ stats_umma_kernel(const __grid_constant__ CUtensorMap mapXa, const __grid_consta
         tc_fence_after();
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(512u) : "memory");
     }
+}
+
+// Exercises the bounded wait on its own: one warp waits for a barrier phase that nothing will ever
+// complete, gives up after `limit_cycles` and records GPTAQ_ERR_TIMEOUT like the GEMM kernels do.
+__global__ void bounded_wait_selftest_kernel(StateHeader *hd, long long limit_cycles) {
+    __shared__ __align__(8) unsigned long long bar;
+    __shared__ int abort_flag;
+    if (threadIdx.x == 0) {
+        mbar_init(smem_u32(&bar), 1);
+        abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    __syncthreads();
+    const bool ok = mbar_wait(smem_u32(&bar), 0u, &abort_flag, limit_cycles);
+    __syncthreads();
+    if (!ok && threadIdx.x == 0) record_status(hd, ST_TIMEOUT, 2000000);
 }
 
 // Adds the partial results of the cut tiles (see StatsGemmArgs) into H / dXX^T, partial 1 first, then 2, ...:

@@ -316,6 +316,27 @@ def test_device_side_conditions_are_reported_not_trapped():
     st.close()
 
 
+def test_bounded_wait_runs_out_and_is_reported():
+    """A wait that nothing satisfies ends by itself with a status, not a hang or a trap."""
+    st = g.LayerState(64, 4, 16, 32)
+    h = st.handle
+    lib = g.load_library()
+    assert not lib.gptaq_U(h) and not lib.gptaq_P(h)
+    g.gptaq_selftest_bounded_wait(h, 0.05)
+    status, info = g.gptaq_sync_status(h)
+    assert status == g.GPTAQ_ERR_TIMEOUT and info == 2000000
+    assert g.gptaq_status_string(status) == "bounded device wait ran out"
+    g.gptaq_reset(h)                                  # clears the status; the context is still usable
+    X = torch.randn(16, 64, device="cuda")
+    g.gptaq_accumulate(h, X, X)
+    g.gptaq_factor(h, 0.01)
+    assert g.gptaq_sync_status(h)[0] == g.GPTAQ_OK
+    assert lib.gptaq_U(h) == g.gptaq_H_ptr(h) and not lib.gptaq_P(h)
+    g.gptaq_build_P(h, 1.0)
+    assert lib.gptaq_P(h) == g.gptaq_D_ptr(h)
+    st.close()
+
+
 def test_dead_inputs():
     cfg = wl.scaled(wl.CONFIGS["cfg1"], n=160, m=24, batch_tokens=500, group=32, blocksize=32)
     W = wl.make_weight(cfg)
