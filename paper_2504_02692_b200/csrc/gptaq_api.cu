@@ -54,6 +54,7 @@ struct gptaq_ctx {
     cudaStream_t gemm_stream;
     cudaEvent_t conv_done[2], gemm_done[2];
     bool gemm_pending[2];
+    bool relayout;         // the operand buffers change size: wait for the products in flight first
     int next_buf;
     std::string cuda_error;
 };
@@ -270,6 +271,10 @@ gptaq_status_t join_statistics(gptaq_ctx *h, cudaStream_t s) {
 gptaq_status_t accumulate_tc(gptaq_ctx *h, const float *X, const float *Xfp, int64_t tokens, int64_t ld,
                              cudaStream_t s) {
     const int n = (int)h->n;
+    if (h->relayout) {
+        OK(join_statistics(h, s));
+        h->relayout = false;
+    }
     const int64_t chunk = tc_chunk_tokens(h);
     const int TM = (n + UBM - 1) / UBM, TN = (n + UBN - 1) / UBN;
     int64_t ntiles = (int64_t)TM * TN;
@@ -614,6 +619,7 @@ gptaq_status_t gptaq_create(gptaq_handle_t *out, int64_t n, void *d_state, size_
         return GPTAQ_ERR_CUDA;
     }
     h->gemm_stream = nullptr;
+    h->relayout = false;
     h->next_buf = 0;
     for (int i = 0; i < 2; ++i) { h->conv_done[i] = h->gemm_done[i] = nullptr; h->gemm_pending[i] = false; }
     e = cudaStreamCreateWithFlags(&h->gemm_stream, cudaStreamNonBlocking);
@@ -1025,6 +1031,7 @@ gptaq_status_t gptaq_set_stats_precision(gptaq_handle_t h, int precision) {
         precision != GPTAQ_STATS_FP16_SPLIT_TENSOR)
         return GPTAQ_ERR_UNSUPPORTED;
     if (h->stage != STAGE_ACCUM) return GPTAQ_ERR_BAD_STATE;
+    if (precision != h->stats_precision) h->relayout = true;
     h->stats_precision = precision;
     return GPTAQ_OK;
 }
