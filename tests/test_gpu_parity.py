@@ -53,6 +53,44 @@ def test_ragged_shapes(n, m, tokens, nb, bits, group, sym, B):
     hp.assert_parity(out)
 
 
+@pytest.mark.parametrize("n,m,B,group,sym,bits", [(576, 70, 64, 64, True, 4), (640, 33, 32, 32, False, 3),
+                                                   (516, 129, 128, 0, False, 4)])
+def test_tensor_path_block_sizes_and_tails(n, m, B, group, sym, bits):
+    """Widths >= 512 (float32-grade tensor-core products) with the smaller lazy-batch blocks, a width that is
+    a multiple of 4 only, and row counts that do not fill the last CTA."""
+    cfg = wl.scaled(wl.CONFIGS["cfg2"], name="tails", n=n, m=m, batch_tokens=1500, n_batches=2, bits=bits, group=group,
+                    sym=sym, blocksize=B, outlier_channels=5)
+    out = hp.check_layer(cfg, wl.make_weight(cfg), batches_of(cfg))
+    hp.assert_parity(out)
+
+
+def test_strided_inputs():
+    """Activations and weights given as views with a leading dimension larger than n."""
+    cfg = wl.scaled(wl.CONFIGS["cfg2"], name="strided", n=512, m=64, batch_tokens=1024, n_batches=2, outlier_channels=5)
+    W = wl.make_weight(cfg)
+    bt = batches_of(cfg)
+    ref = hp.gpu_layer(cfg, W, bt)
+    st = g.LayerState(cfg.n, cfg.m, cfg.batch_tokens, cfg.blocksize, total_tokens=cfg.tokens)
+    for X, Xfp in bt:
+        big = torch.zeros((2, X.shape[0], cfg.n + 12), device="cuda")
+        big[0, :, :cfg.n] = X.cuda(); big[1, :, :cfg.n] = Xfp.cuda()
+        g.gptaq_accumulate(st.handle, big[0, :, :cfg.n], big[1, :, :cfg.n])
+    g.gptaq_factor(st.handle, cfg.damp)
+    g.gptaq_build_P(st.handle, cfg.alpha)
+    Wbig = torch.zeros((cfg.m, cfg.n + 20), device="cuda")
+    Wbig[:, :cfg.n] = W.cuda()
+    G = hp.n_groups(cfg.n, cfg.group)
+    codes = torch.empty((cfg.m, cfg.n), dtype=torch.uint8, device="cuda")
+    sc = torch.empty((cfg.m, G), dtype=torch.float32, device="cuda")
+    zp = torch.empty((cfg.m, G), dtype=torch.float32, device="cuda")
+    g.gptaq_quantize(st.handle, Wbig[:, :cfg.n], cfg.bits, cfg.group, cfg.sym, cfg.blocksize, codes, sc, zp, None)
+    assert g.gptaq_sync_status(st.handle)[0] == g.GPTAQ_OK
+    assert np.array_equal(codes.cpu().numpy(), ref.codes)
+    assert np.array_equal(Wbig[:, :cfg.n].cpu().numpy().astype(np.float64), ref.Wq)      # in place, strided
+    assert float(Wbig[:, cfg.n:].abs().max()) == 0.0                                    # nothing written beyond n
+    st.close()
+
+
 def test_cfg4_shape_row_subset():
     """ViT-shaped layer at full n and tokens; the oracle loop replays a seeded row subset
     (rows are independent)."""
