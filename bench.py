@@ -187,9 +187,20 @@ def run_ours(args, cfg):
     pk = peaks()
 
     # inputs resident in HBM before the timed region (each rank its own layer: seed = rank)
-    cfg_r = rank_config(cfg, rank)
-    batches = [wl.make_batch(cfg_r, b, dev) for b in range(cfg.n_batches)]
-    W0 = wl.make_weight(cfg_r, dev)
+    shard = bool(args.shard_layer) and world > 1
+    if shard:
+        # ONE layer across the ranks: this rank's share of the token batches and of the rows of W
+        from paper_2504_02692_b200 import sharded
+        cfg_r = cfg
+        my_batches = sharded.token_shard(cfg.n_batches, rank, world)
+        r0, r1 = sharded.row_shard(cfg.m, rank, world)
+        batches = [wl.make_batch(cfg_r, b, dev) for b in my_batches]
+        W0 = wl.make_weight(cfg_r, dev)[r0:r1].contiguous()
+        cfg = wl.scaled(cfg, m=r1 - r0)
+    else:
+        cfg_r = rank_config(cfg, rank)
+        batches = [wl.make_batch(cfg_r, b, dev) for b in range(cfg.n_batches)]
+        W0 = wl.make_weight(cfg_r, dev)
     if cfg.w_bf16:
         W0 = W0.to(torch.bfloat16)
     G = 1 if cfg.group <= 0 else (cfg.n + cfg.group - 1) // cfg.group
@@ -215,6 +226,8 @@ def run_ours(args, cfg):
         e0 = ev(); e0.record(stream)
         for X, Xfp in batches:
             g.gptaq_accumulate(h, X, Xfp)
+        if shard:
+            sharded.allreduce_statistics(st)     # the one exchange step: sum of H and dXX^T over the ranks
         g.gptaq_flush(h)            # the products run on the handle's own stream: order `stream` after them
         e1 = ev(); e1.record(stream)
         g.gptaq_factor(h, cfg.damp)
@@ -252,10 +265,10 @@ def run_ours(args, cfg):
     ms_total = t_beg.elapsed_time(t_end)
     ms_total = max_over_ranks(ms_total, world, dev)
     ms_step = ms_total / args.steps
-    ms_layer = per_layer_ms(ms_step, world)
+    ms_layer = ms_step if shard else per_layer_ms(ms_step, world)
 
     acc_step_ms = sum(m[0].elapsed_time(m[1]) for m in marks) / args.steps
-    acc_call_ms = acc_step_ms / cfg.n_batches      # conversion and product of consecutive batches overlap
+    acc_call_ms = acc_step_ms / max(1, len(batches))      # conversion and product of consecutive batches overlap
     fac_ms = sum(m[1].elapsed_time(m[2]) for m in marks) / args.steps
     p_ms = sum(m[2].elapsed_time(m[3]) for m in marks) / args.steps
     q_ms = sum(m[3].elapsed_time(m[4]) for m in marks) / args.steps
@@ -278,6 +291,8 @@ def run_ours(args, cfg):
             g.gptaq_reset(h)
             for X, Xfp in hb:
                 g.gptaq_accumulate_host(h, X, Xfp, stage)
+            if shard:
+                sharded.allreduce_statistics(st)
             g.gptaq_factor(h, cfg.damp)
             g.gptaq_build_P(h, cfg.alpha)
             g.gptaq_quantize_host(h, hW, cfg.bits, cfg.group, cfg.sym, cfg.blocksize, hcodes, hs, hz, stage)
@@ -295,7 +310,7 @@ def run_ours(args, cfg):
         ems = max_over_ranks(ems, world, dev)
         h2d = sum(x.numel() * 4 * 2 for x, _ in hb) + hW.numel() * 4
         d2h = hcodes.numel() + (hs.numel() + hz.numel()) * 4
-        e2e = {"value": per_layer_ms(ems, world), "unit": "ms", "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h}
+        e2e = {"value": ems if shard else per_layer_ms(ems, world), "unit": "ms", "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h}
 
     if rank != 0:
         return
@@ -305,9 +320,10 @@ def run_ours(args, cfg):
         cpu = {"value": v, "unit": "ms", "cores": threads, "kind": "oracle", "sample": desc}
     line = {
         "metric": METRIC, "value": ms_layer, "unit": "ms", "n_gpus": world, "steps": args.steps,
-        "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": False, "scaling": "weak",
+        "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": False, "scaling": "strong" if shard else "weak",
         "vs_baseline": None, "dtype": "f16 x f16 -> f32 (statistics), f32 (solve)", "data": "synthetic",
-        "config": dict(wl.describe(cfg), parallelism=f"{world} independent layer(s), one per GPU",
+        "config": dict(wl.describe(cfg), parallelism=(f"one layer over {world} GPUs: tokens sharded, one all-reduce of H and dXX^T, rows sharded"
+                                    if shard else f"{world} independent layer(s), one per GPU"),
                        l2="inputs (%.1f GB per step) exceed L2" % (2 * cfg.tokens * cfg.n * 4 / 1e9),
                        statistics=prec_name, act_order=bool(args.act_order)),
         "stages_ms": {"accumulate": acc_step_ms, "factor": fac_ms, "build_P": p_ms, "quantize": q_ms,
@@ -335,6 +351,9 @@ def main():
     ap.add_argument("--ref-rows", type=int, default=512)
     ap.add_argument("--batches", type=int, default=0,
                     help="profiler captures only: keep this many token batches (the line is marked truncated)")
+    ap.add_argument("--shard-layer", action="store_true",
+                    help="N > 1: one layer across the ranks (token-sharded statistics, one all-reduce, row-sharded "
+                         "quantize; strong scaling) instead of one independent layer per rank")
     ap.add_argument("--act-order", action="store_true", help="columns sorted by diag(H) (off in the headline configuration)")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")

@@ -63,3 +63,54 @@ def test_reference_arm_under_two_ranks_prints_once():
     line = json.loads(lines0[0])
     assert line["impl"] == "reference" and line["n_gpus"] == 2 and line["cpu_baseline"]["kind"] == "oracle"
     assert line["e2e"]["h2d_bytes_per_step"] == 0 and line["value"] > 0
+
+
+def _shard_worker(rank, world, port, out):
+    os.environ.update(MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port))
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    sys.path.insert(0, ROOT)
+    import numpy as np
+    import workloads as wl
+    from oracle import gptaq_oracle as orc
+    from paper_2504_02692_b200 import sharded
+    cfg = wl.scaled(wl.CONFIGS["cfg1"], n=48, m=70, batch_tokens=64, n_batches=5, group=0, blocksize=32)
+    # this rank's share of the token batches, accumulated by the oracle into plain CPU tensors
+    st = orc.new_stats(cfg.n)
+    for b in sharded.token_shard(cfg.n_batches, rank, world):
+        X, Xfp = wl.make_batch(cfg, b)
+        orc.accumulate(st, X.numpy(), Xfp.numpy())
+    H, D = torch.from_numpy(st.H.astype(np.float32)), torch.from_numpy(st.D.astype(np.float32))
+    total = sharded.allreduce_sums(H, D, st.tokens)
+    full = orc.new_stats(cfg.n)
+    for b in range(cfg.n_batches):
+        X, Xfp = wl.make_batch(cfg, b)
+        orc.accumulate(full, X.numpy(), Xfp.numpy())
+    ok_stats = total == full.tokens and np.allclose(H.numpy(), full.H, rtol=1e-5) and np.allclose(D.numpy(), full.D, rtol=1e-4, atol=1e-3)
+    # row slabs: quantizing a slab gives the slab of the full result (rows are independent)
+    W = wl.make_weight(cfg).numpy().astype(np.float64)
+    U, dead = orc.factor(full.H, full.tokens, cfg.damp)
+    P = orc.build_P(full.D, full.tokens, U, cfg.alpha)
+    r0, r1 = sharded.row_shard(cfg.m, rank, world)
+    mine = orc.quantize(W[r0:r1], U, P, dead, cfg.bits, cfg.group, cfg.sym)
+    whole = orc.quantize(W, U, P, dead, cfg.bits, cfg.group, cfg.sym)
+    ok_rows = np.array_equal(mine.codes, whole.codes[r0:r1])
+    spans = [None] * world
+    dist.all_gather_object(spans, (r0, r1))
+    if rank == 0:
+        json.dump({"ok_stats": bool(ok_stats), "ok_rows": bool(ok_rows), "spans": spans}, open(out, "w"))
+    dist.barrier()
+    dist.destroy_process_group()
+
+
+def test_token_sharded_statistics_and_row_sharded_quantize(tmp_path):
+    """The one exchange step of a layer spread over ranks: all-reduced partial sums equal the full sums, and
+    the row slabs tile the matrix and reproduce the full result."""
+    from paper_2504_02692_b200 import sharded
+    assert [list(sharded.token_shard(5, r, 2)) for r in range(2)] == [[0, 1, 2], [3, 4]]
+    assert [list(sharded.token_shard(3, r, 4)) for r in range(4)] == [[0], [1], [2], []]
+    assert [sharded.row_shard(70, r, 2) for r in range(2)] == [(0, 64), (64, 70)]
+    assert [sharded.row_shard(4096, r, 8) for r in range(8)] == [(512 * r, 512 * r + 512) for r in range(8)]
+    out = str(tmp_path / "shard.json")
+    mp.spawn(_shard_worker, args=(2, _free_port(), out), nprocs=2, join=True)
+    res = json.load(open(out))
+    assert res["ok_stats"] and res["ok_rows"] and res["spans"] == [[0, 64], [64, 70]]
