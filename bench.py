@@ -217,6 +217,8 @@ def run_ours(args, cfg):
     stream = torch.cuda.current_stream()
     if args.act_order:
         g.gptaq_set_act_order(h, True)
+    if args.clip_search > 0:
+        g.gptaq_set_clip_search(h, args.clip_search, 0.2)
 
     def ev():
         return torch.cuda.Event(enable_timing=True)
@@ -325,7 +327,7 @@ def run_ours(args, cfg):
         "config": dict(wl.describe(cfg), parallelism=(f"one layer over {world} GPUs: tokens sharded, one all-reduce of H and dXX^T, rows sharded"
                                     if shard else f"{world} independent layer(s), one per GPU"),
                        l2="inputs (%.1f GB per step) exceed L2" % (2 * cfg.tokens * cfg.n * 4 / 1e9),
-                       statistics=prec_name, act_order=bool(args.act_order)),
+                       statistics=prec_name, act_order=bool(args.act_order), clip_search=args.clip_search),
         "stages_ms": {"accumulate": acc_step_ms, "factor": fac_ms, "build_P": p_ms, "quantize": q_ms,
                       "layer_quantize": fac_ms + p_ms + q_ms},
         "accumulate_tflops": achieved,
@@ -354,6 +356,8 @@ def main():
     ap.add_argument("--shard-layer", action="store_true",
                     help="N > 1: one layer across the ranks (token-sharded statistics, one all-reduce, row-sharded "
                          "quantize; strong scaling) instead of one independent layer per rank")
+    ap.add_argument("--clip-search", type=int, default=0,
+                    help="clipping-range search of the grids with this many candidates (off in the headline configuration)")
     ap.add_argument("--act-order", action="store_true", help="columns sorted by diag(H) (off in the headline configuration)")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")

@@ -230,6 +230,14 @@ int gptaq_recommended_stats_precision(int64_t n, int64_t total_tokens);
 gptaq_status_t gptaq_set_act_order(gptaq_handle_t h, int enable);
 const int32_t *gptaq_perm(gptaq_handle_t h);
 
+/* Clipping-range search of the quantization grids (Section 5, setup: "the weight clipping range is
+ * searched by minimizing mean squared error"; the paper gives no further detail).  With steps > 0 every
+ * grid -- per output channel, or per group at the group's first column -- is chosen among `steps`
+ * candidates that shrink the min/max range by p_k = 1 - k (1 - min_ratio) / steps, k = 0 .. steps - 1:
+ * the candidate with the smallest sum of squared rounding errors over the grid's weights, the widest one
+ * on ties.  steps = 0 (default) is the plain min/max grid; 0 < min_ratio < 1. */
+gptaq_status_t gptaq_set_clip_search(gptaq_handle_t h, int steps, float min_ratio);
+
 /* Ablation switches of the weight update (Section 5.3, Table "ablation"): which of the two terms of
  * Eq. "divided update" later gptaq_quantize calls on this handle apply.
  *   GPTAQ_TERM_ERR    the quantization-error term  -(w_q - q_q)/U_qq * U[q, :]   (GPTQ's update)

@@ -176,6 +176,45 @@ def dequant(code: np.ndarray, scale: np.ndarray, zero: np.ndarray) -> np.ndarray
     return scale * (code - zero)
 
 
+def clip_candidates(w: np.ndarray, bits: int, sym: bool, steps: int, min_ratio: float):
+    """All candidate grids of the clipping-range search (setup of Section 5; the paper only says the
+    range "is searched by minimizing mean squared error"): candidate k shrinks the min/max range by
+    p_k = 1 - k (1 - min_ratio) / steps.  Returns (scales, zeros, errors), each ``[steps, rows]``;
+    errors are the sums of squared rounding errors of ``w`` on the candidate grid."""
+    w = np.asarray(w, dtype=F64)
+    scales, zeros, errs = [], [], []
+    for k in range(steps):
+        p = 1.0 - k * (1.0 - min_ratio) / steps
+        if sym:
+            a = p * np.max(np.abs(w), axis=1)
+            a = np.where(a == 0.0, 1.0, a)
+            s = a / float(2 ** (bits - 1) - 1)
+            z = np.full_like(s, float(2 ** (bits - 1)))
+        else:
+            lo = p * np.minimum(w.min(axis=1), 0.0)
+            hi = p * np.maximum(w.max(axis=1), 0.0)
+            flat = hi == lo
+            s = np.where(flat, 1.0, (hi - lo) / float(2 ** bits - 1))
+            z = np.where(flat, 0.0, np.rint(-lo / s))
+        q = dequant(qcode(w, s[:, None], z[:, None], bits), s[:, None], z[:, None])
+        scales.append(s); zeros.append(z); errs.append(np.sum((q - w) ** 2, axis=1))
+    return np.array(scales), np.array(zeros), np.array(errs)
+
+
+def grid_search(w: np.ndarray, bits: int, sym: bool, steps: int, min_ratio: float):
+    """Per-row grid with the least squared rounding error among the candidates; the widest on ties."""
+    scales, zeros, errs = clip_candidates(w, bits, sym, steps, min_ratio)
+    k = np.argmin(errs, axis=0)                      # first minimum = smallest k = widest range
+    r = np.arange(scales.shape[1])
+    return scales[k, r], zeros[k, r]
+
+
+def _grid_fn(bits, sym, clip):
+    if clip is None or clip[0] <= 0:
+        return lambda blk: grid(blk, bits, sym)
+    return lambda blk: grid_search(blk, bits, sym, clip[0], clip[1])
+
+
 # --------------------------------------------------------------------------
 # Steps 3-4 of Algorithm 1 (lines 6-13): the quantize-and-propagate loop
 # --------------------------------------------------------------------------
@@ -194,7 +233,7 @@ def _ngroups(n: int, group: int) -> int:
 
 def quantize(W: np.ndarray, U: np.ndarray, P: np.ndarray | None, dead: np.ndarray | None,
              bits: int, group: int, sym: bool, update: bool = True,
-             keep_pre: bool = False, error_term: bool = True) -> QuantResult:
+             keep_pre: bool = False, error_term: bool = True, clip=None) -> QuantResult:
     """Unblocked column loop (Eq. "divided update"), all rows at once.
 
     For column j: quantize the current column, e = (w - q) / U[j, j], then
@@ -213,12 +252,13 @@ def quantize(W: np.ndarray, U: np.ndarray, P: np.ndarray | None, dead: np.ndarra
     zeros = np.zeros((m, ng), F64)
     Wq = np.zeros((m, n), F64)
     pre = np.zeros((m, n), F64) if keep_pre else None
+    make = _grid_fn(bits, sym, clip)      # ``clip = (steps, min_ratio)``: clipping-range search of every grid
     if group <= 0:
-        s, z = grid(W, bits, sym)
+        s, z = make(W)
         scales[:, 0], zeros[:, 0] = s, z
     for j in range(n):
         if group > 0 and j % group == 0:
-            s, z = grid(W[:, j:j + group], bits, sym)
+            s, z = make(W[:, j:j + group])
             scales[:, j // group], zeros[:, j // group] = s, z
         w = W[:, j].copy()
         c = qcode(w, s, z, bits)
@@ -338,7 +378,7 @@ class FollowReport:
 def follow(W: np.ndarray, U: np.ndarray, P: np.ndarray | None, dead,
            bits: int, group: int, sym: bool,
            cand_codes: np.ndarray, cand_scales: np.ndarray, cand_zeros: np.ndarray,
-           band: float = 1e-4, error_term: bool = True) -> FollowReport:
+           band: float = 1e-4, error_term: bool = True, clip=None) -> FollowReport:
     W = np.array(W, dtype=F64)
     m, n = W.shape
     if dead is not None and dead.any():
@@ -352,8 +392,21 @@ def follow(W: np.ndarray, U: np.ndarray, P: np.ndarray | None, dead,
 
     def check_grid(block, g):
         nonlocal grid_err, zero_mis
-        s_o, z_o = grid(block, bits, sym)
         s_c, z_c = cand_scales[:, g], cand_zeros[:, g]
+        if clip is not None and clip[0] > 0:
+            # clipping-range search: the candidate's grid must be one of the candidate grids, and its
+            # squared error (in float64) must equal the best one up to rounding: near-ties may fall
+            # either way in float32
+            S, Z, E = clip_candidates(block, bits, sym, clip[0], clip[1])
+            rel = np.abs(S - s_c[None, :]) / S
+            k = np.argmin(rel, axis=0)
+            r = np.arange(S.shape[1])
+            grid_err = max(grid_err, float(np.max(rel[k, r])))
+            best = E.min(axis=0)
+            worse = E[k, r] > best * (1.0 + 1e-5) + 1e-30
+            zero_mis += int(np.sum(worse)) + int(np.sum(Z[k, r] != z_c))
+            return s_c, z_c
+        s_o, z_o = grid(block, bits, sym)
         grid_err = max(grid_err, float(np.max(np.abs(s_c - s_o) / s_o)))
         if not sym:
             lo = np.minimum(block.min(axis=1), 0.0)

@@ -61,6 +61,7 @@ SIGNATURES = {
     "gptaq_set_tokens": (_int, [_vp, _i64]),
     "gptaq_set_stats_precision": (_int, [_vp, _int]),
     "gptaq_set_update_terms": (_int, [_vp, _int]),
+    "gptaq_set_clip_search": (_int, [_vp, _int, _f]),
     "gptaq_set_act_order": (_int, [_vp, _int]),
     "gptaq_perm": (_vp, [_vp]),
     "gptaq_recommended_stats_precision": (_int, [_i64, _i64]),
@@ -295,6 +296,11 @@ def gptaq_set_act_order(h, enable: bool):
 
 def gptaq_perm_ptr(h) -> int | None:
     return load_library().gptaq_perm(h)
+
+
+def gptaq_set_clip_search(h, steps: int, min_ratio: float = 0.2):
+    """Grids chosen by the least squared rounding error among ``steps`` shrunken min/max ranges (0: off)."""
+    _check(load_library().gptaq_set_clip_search(h, steps, min_ratio), "gptaq_set_clip_search", h)
 
 
 def gptaq_set_update_terms(h, terms: int):

@@ -48,6 +48,7 @@ struct gptaq_ctx {
     int stats_precision;   // GPTAQ_STATS_*
     bool tensor;           // float32-grade tensor-core GEMMs for factor / P / trailing update
     int terms;             // GPTAQ_TERM_* switches of gptaq_quantize
+    int clip_steps; float clip_min;   // clipping-range search of the grids
     // Statistics pipeline: the conversion of a token batch runs on the caller's stream, the
     // tensor-core product on `gemm_stream`, so that the (memory-bound) conversion of the next
     // batch overlaps the (tensor-bound) product of this one.  Two operand buffers alternate.
@@ -362,6 +363,7 @@ struct QuantizeTarget {
     float *EW_lo;
     int terms = GPTAQ_TERM_ERR | GPTAQ_TERM_ASYM;   // which terms of the weight update are applied
     const int *perm = nullptr;                      // act_order: working column c is the caller's column perm[c]
+    int clip_steps = 0; float clip_min = 1.f;       // clipping-range search of the grids (0 steps: min/max)
 };
 
 gptaq_status_t check_quantize_args(int64_t n, const void *d_W, int w_dtype, int64_t m, int64_t ldw, int bits,
@@ -417,7 +419,7 @@ gptaq_status_t quantize_core(const QuantizeTarget &t, void *d_W, int w_dtype, in
     const int G = group > 0 ? (n + group - 1) / group : 1;
     if (group <= 0) {
         row_grid_kernel<<<(unsigned)((m + 7) / 8), 256, 0, s>>>(Wk, ldk, (int)m, n, t.dead, bits, sym,
-                                                               d_scales, d_zeros);
+                                                               d_scales, d_zeros, t.clip_steps, t.clip_min);
         QLAUNCHED();
     }
 
@@ -443,7 +445,7 @@ gptaq_status_t quantize_core(const QuantizeTarget &t, void *d_W, int w_dtype, in
         a.i0 = i0; a.bw = std::min(blocksize, n - i0);
         a.bits = bits; a.group = group; a.sym = sym;
         a.codes = d_codes; a.scales = d_scales; a.zeros = d_zeros; a.G = G; a.EW = EW; a.EW_lo = t.EW_lo; a.hd = t.hd;
-        a.perm = t.perm; a.err_scale = (t.terms & GPTAQ_TERM_ERR) ? 1.f : 0.f; a.asym_scale = (t.terms & GPTAQ_TERM_ASYM) ? 1.f : 0.f;
+        a.perm = t.perm; a.clip_steps = t.clip_steps; a.clip_min = t.clip_min; a.err_scale = (t.terms & GPTAQ_TERM_ERR) ? 1.f : 0.f; a.asym_scale = (t.terms & GPTAQ_TERM_ASYM) ? 1.f : 0.f;
         const bool fast = a.bw == blocksize && (group <= 0 || (group % 32) == 0) && (i0 % 4) == 0 &&
                           (reinterpret_cast<uintptr_t>(t.dead) & 3) == 0;
         if (fast) column_block_kernel<<<cb_grid, CB_THREADS, column_block_smem(cb_rows), s>>>(a, cb_rows, blocksize);
@@ -585,6 +587,7 @@ gptaq_status_t gptaq_create(gptaq_handle_t *out, int64_t n, void *d_state, size_
     h->stats_precision = GPTAQ_STATS_FP16_SPLIT_TENSOR;
     h->tensor = tc_shape_ok(n) && encode_tiled_fn() != nullptr;
     h->terms = GPTAQ_TERM_ERR | GPTAQ_TERM_ASYM;
+    h->clip_steps = 0; h->clip_min = 1.f;
     cudaError_t e = cudaGetDevice(&h->device);
     if (e == cudaSuccess) e = cudaDeviceGetAttribute(&h->num_sms, cudaDevAttrMultiProcessorCount, h->device);
     if (e == cudaSuccess)
@@ -904,6 +907,7 @@ gptaq_status_t gptaq_quantize(gptaq_handle_t h, void *d_W, int w_dtype, int64_t 
     t.num_sms = h->num_sms;
     t.terms = h->terms;
     t.perm = h->act_order ? h->perm : nullptr;
+    t.clip_steps = h->clip_steps; t.clip_min = h->clip_min;
     t.UT_hi = t.UT_lo = t.PT_hi = t.PT_lo = nullptr; t.EW_lo = nullptr;
     if (h->tensor) {
         t.UT_hi = reinterpret_cast<float *>(h->ws + wl.s_off[2]); t.UT_lo = reinterpret_cast<float *>(h->ws + wl.s_off[3]);
@@ -1045,6 +1049,15 @@ gptaq_status_t gptaq_set_act_order(gptaq_handle_t h, int enable) {
 }
 
 const int32_t *gptaq_perm(gptaq_handle_t h) { return (h && h->act_order && h->stage != STAGE_ACCUM) ? h->perm : nullptr; }
+
+gptaq_status_t gptaq_set_clip_search(gptaq_handle_t h, int steps, float min_ratio) {
+    if (!h) return GPTAQ_ERR_INVALID_ARG;
+    if (steps < 0 || steps > 1024) return GPTAQ_ERR_UNSUPPORTED;
+    if (steps > 0 && !(min_ratio > 0.f && min_ratio < 1.f)) return GPTAQ_ERR_INVALID_ARG;
+    h->clip_steps = steps;
+    h->clip_min = steps > 0 ? min_ratio : 1.f;
+    return GPTAQ_OK;
+}
 
 gptaq_status_t gptaq_set_update_terms(gptaq_handle_t h, int terms) {
     if (!h) return GPTAQ_ERR_INVALID_ARG;

@@ -485,10 +485,22 @@ __device__ __forceinline__ void make_grid(float lo, float hi, float amax, int bi
     }
 }
 
+// Clipping-range search (setup of Section 5: "the weight clipping range is searched by minimizing mean
+// squared error"): candidate k of `steps` shrinks the min/max range by p_k = 1 - k (1 - min_ratio) / steps;
+// the candidate with the least squared rounding error of the group's weights wins, the widest one on ties.
+__device__ __forceinline__ float clip_ratio(int k, int steps, float min_ratio) {
+    return 1.f - (float)k * ((1.f - min_ratio) / (float)steps);
+}
+__device__ __forceinline__ float rounding_error_sq(float w, float scale, float zero, float maxq) {
+    const float cq = fminf(fmaxf(rintf(w / scale) + zero, 0.f), maxq);
+    const float d = scale * (cq - zero) - w;
+    return d * d;
+}
+
 // Per-channel grids from the original rows (dead inputs count as zero weights).
 __global__ void __launch_bounds__(256) row_grid_kernel(const float *W, int64_t ldw, int m, int n,
                                                        const uint8_t *dead, int bits, int sym,
-                                                       float *scales, float *zeros) {
+                                                       float *scales, float *zeros, int clip_steps, float clip_min) {
     int row = blockIdx.x * 8 + (threadIdx.x >> 5);
     int lane = threadIdx.x & 31;
     if (row >= m) return;
@@ -504,11 +516,23 @@ __global__ void __launch_bounds__(256) row_grid_kernel(const float *W, int64_t l
         hi = fmaxf(hi, __shfl_xor_sync(0xffffffffu, hi, o));
         am = fmaxf(am, __shfl_xor_sync(0xffffffffu, am, o));
     }
-    if (lane == 0) {
-        float s, z;
-        make_grid(lo, hi, am, bits, sym, s, z);
-        scales[row] = s; zeros[row] = z;
+    float s, z;
+    make_grid(lo, hi, am, bits, sym, s, z);
+    if (clip_steps > 0) {
+        const float maxq = (float)((1 << bits) - 1);
+        float best = INFINITY;
+        for (int k = 0; k < clip_steps; ++k) {
+            const float p = clip_ratio(k, clip_steps, clip_min);
+            float sk, zk;
+            make_grid(p * lo, p * hi, p * am, bits, sym, sk, zk);
+            float err = 0.f;
+            for (int c = lane; c < n; c += 32) err += rounding_error_sq(dead[c] ? 0.f : w[c], sk, zk, maxq);
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) err += __shfl_xor_sync(0xffffffffu, err, o);
+            if (err < best) { best = err; s = sk; z = zk; }
+        }
     }
+    if (lane == 0) { scales[row] = s; zeros[row] = z; }
 }
 
 // ---------------------------------------------------------------------------
@@ -532,6 +556,7 @@ struct ColumnLoopArgs {
     StateHeader *hd;
     float err_scale, asym_scale;   // 1 or 0: switches of the two terms of the weight update (ablation)
     const int *perm;               // nullptr, or: working column c is original column perm[c] (codes go there)
+    int clip_steps; float clip_min; // clipping-range search of the group grids (0: plain min/max)
 };
 
 template <int T>
@@ -597,6 +622,23 @@ __global__ void __launch_bounds__(1024) column_loop_kernel(ColumnLoopArgs a) {
                     am = fmaxf(am, __shfl_xor_sync(0xffffffffu, am, o));
                 }
                 make_grid(lo, hi, am, a.bits, a.sym, scale, zero);
+                if (a.clip_steps > 0) {
+                    float best = INFINITY;
+                    for (int k = 0; k < a.clip_steps; ++k) {
+                        const float p = clip_ratio(k, a.clip_steps, a.clip_min);
+                        float sk, zk;
+                        make_grid(p * lo, p * hi, p * am, a.bits, a.sym, sk, zk);
+                        float err = 0.f;
+#pragma unroll
+                        for (int t2 = 0; t2 < T; ++t2) {
+                            int c = lane + 32 * t2;
+                            if (c >= j && c < gend) err += rounding_error_sq(w[t2], sk, zk, maxq);
+                        }
+#pragma unroll
+                        for (int o = 16; o > 0; o >>= 1) err += __shfl_xor_sync(0xffffffffu, err, o);
+                        if (err < best) { best = err; scale = sk; zero = zk; }
+                    }
+                }
                 if (lane == 0) {
                     int g = (i0 + j) / a.group;
                     a.scales[(int64_t)row * a.G + g] = scale;
@@ -749,8 +791,48 @@ __global__ void __launch_bounds__(CB_THREADS, 1) column_block_kernel(ColumnLoopA
         }
         if (tid < 32) udinv[tid] = 1.f / a.U[(int64_t)(i0 + o + tid) * n + i0 + o + tid];
         __syncthreads();
+        const bool group_start = a.group > 0 && ((i0 + o) % a.group) == 0;
+        int best_k = 0;
+        if (group_start && a.clip_steps > 0) {
+            // clipping-range search, all threads: thread = (row, share of the candidates); the shares'
+            // best (error, candidate) pairs meet in St, which is free until the columns are quantized
+            const int ncg = CB_THREADS / rows;
+            const int r = tid % rows, cgi = tid / rows;
+            float *berr = St;
+            int *bk = reinterpret_cast<int *>(St + CB_THREADS);
+            if (cgi < ncg) {
+                float lo = 0.f, hi = 0.f, am = 0.f;
+                const int gend = min(o + a.group, B);
+                for (int c = o; c < gend; ++c) {
+                    const float v = Wt[r][c];
+                    lo = fminf(lo, v); hi = fmaxf(hi, v); am = fmaxf(am, fabsf(v));
+                }
+                float best = INFINITY;
+                int kb = 0;
+                for (int k = cgi; k < a.clip_steps; k += ncg) {
+                    const float p = clip_ratio(k, a.clip_steps, a.clip_min);
+                    float sk, zk;
+                    make_grid(p * lo, p * hi, p * am, a.bits, a.sym, sk, zk);
+                    float err = 0.f;
+                    for (int c = o; c < gend; ++c) err += rounding_error_sq(Wt[r][c], sk, zk, maxq);
+                    if (err < best) { best = err; kb = k; }
+                }
+                berr[cgi * rows + r] = best;
+                bk[cgi * rows + r] = kb;
+            }
+            __syncthreads();
+            if (owner) {
+                float best = INFINITY;
+                for (int c = 0; c < ncg; ++c) {
+                    const float e = berr[c * rows + tid];
+                    const int k = bk[c * rows + tid];
+                    if (e < best || (e == best && k < best_k)) { best = e; best_k = k; }
+                }
+            }
+            __syncthreads();
+        }
         if (owner) {
-            if (a.group > 0 && ((i0 + o) % a.group) == 0) {
+            if (group_start) {
                 // grid of the group that starts here, from the current values
                 float lo = 0.f, hi = 0.f, am = 0.f;
                 const int gend = min(o + a.group, B);
@@ -758,7 +840,8 @@ __global__ void __launch_bounds__(CB_THREADS, 1) column_block_kernel(ColumnLoopA
                     const float v = Wt[tid][c];
                     lo = fminf(lo, v); hi = fmaxf(hi, v); am = fmaxf(am, fabsf(v));
                 }
-                make_grid(lo, hi, am, a.bits, a.sym, scale, zero);
+                const float p = a.clip_steps > 0 ? clip_ratio(best_k, a.clip_steps, a.clip_min) : 1.f;
+                make_grid(p * lo, p * hi, p * am, a.bits, a.sym, scale, zero);
                 const int g = (i0 + o) / a.group;
                 a.scales[(int64_t)row * a.G + g] = scale;
                 a.zeros[(int64_t)row * a.G + g] = zero;

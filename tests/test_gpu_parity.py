@@ -260,6 +260,51 @@ def test_act_order(n, m, group, B, bf16):
     st.close()
 
 
+@pytest.mark.parametrize("n,m,group,B,sym,bits", [(160, 40, 0, 32, False, 3), (200, 24, 8, 32, False, 2),
+                                                   (640, 96, 128, 128, False, 3), (576, 130, 64, 64, True, 3)])
+def test_clip_search(n, m, group, B, sym, bits):
+    """Grids chosen by the clipping-range search.  Which candidate wins is decided by sums of squares that the
+    device takes in float32: where two candidates are within rounding of each other either is valid, so the
+    oracle's follow mode checks that the device's grid IS a candidate and that its float64 error equals the
+    best one up to 1e-5, then replays the codes with it."""
+    cfg = wl.scaled(wl.CONFIGS["cfg2"], name="clip", n=n, m=m, batch_tokens=2048, n_batches=1, group=group,
+                    blocksize=B, sym=sym, bits=bits, outlier_channels=3)
+    bt = batches_of(cfg)
+    W = wl.make_weight(cfg)
+    clip = (24, 0.4)
+    st = g.LayerState(cfg.n, cfg.m, cfg.batch_tokens, cfg.blocksize, total_tokens=cfg.tokens)
+    with pytest.raises(g.GptaqError):
+        g.gptaq_set_clip_search(st.handle, 8, 1.5)
+    g.gptaq_set_clip_search(st.handle, *clip)
+    for X, Xfp in bt:
+        g.gptaq_accumulate(st.handle, X.cuda(), Xfp.cuda())
+    g.gptaq_factor(st.handle, cfg.damp)
+    g.gptaq_build_P(st.handle, cfg.alpha)
+    G = hp.n_groups(cfg.n, cfg.group)
+    codes = torch.empty((m, n), dtype=torch.uint8, device="cuda")
+    sc = torch.empty((m, G), dtype=torch.float32, device="cuda")
+    zp = torch.empty((m, G), dtype=torch.float32, device="cuda")
+    Wq = torch.empty((m, n), dtype=torch.float32, device="cuda")
+    g.gptaq_quantize(st.handle, W.cuda(), cfg.bits, cfg.group, cfg.sym, cfg.blocksize, codes, sc, zp, Wq)
+    assert g.gptaq_sync_status(st.handle)[0] == g.GPTAQ_OK
+    so = hp.oracle_stats(cfg, bt)
+    U, dead = orc.factor(so.H, so.tokens, cfg.damp)
+    P = orc.build_P(so.D, so.tokens, U, cfg.alpha)
+    Wn = W.numpy().astype(np.float64)
+    rep = orc.follow(Wn, U, P, dead, cfg.bits, cfg.group, cfg.sym, codes.cpu().numpy(),
+                     sc.cpu().numpy().astype(np.float64), zp.cpu().numpy().astype(np.float64),
+                     band=hp.TOL_FLIP_BAND, clip=clip)
+    assert rep.disallowed == 0 and rep.allowed <= hp.TOL_FLIP_RATE * rep.total, rep
+    assert rep.grid_rel_err <= 5e-5 and rep.zero_mismatch == 0, rep
+    # the search does change grids on this input, and the objective matches the oracle's
+    plain = orc.quantize(Wn, U, P, dead, cfg.bits, cfg.group, cfg.sym)
+    res = orc.quantize(Wn, U, P, dead, cfg.bits, cfg.group, cfg.sym, clip=clip)
+    assert np.mean(res.scales < plain.scales * (1 - 1e-9)) > 0.05
+    J_gpu, J_orc = orc.objective(Wn, Wq.cpu().numpy().astype(np.float64), so), orc.objective(Wn, res.Wq, so)
+    assert abs(J_gpu - J_orc) <= 5 * hp.TOL_OBJECTIVE * J_orc, (J_gpu, J_orc)
+    st.close()
+
+
 def test_correlated_inputs_stress():
     """Correlated channels (X <- X A, A = identity + low rank): cond(H_d) grows from ~1e3 (independent
     channels of the benchmark layers) to ~2e4.  float32 sums and a float32 factorization then carry

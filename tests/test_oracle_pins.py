@@ -189,6 +189,53 @@ def test_quantizer_exhaustive(bits, sym):
     assert orc.qcode(np.array([0.5, 1.5, 2.5, -0.5]), s1, z1, 4).tolist() == [4.0, 6.0, 6.0, 4.0]
 
 
+def test_clip_search_brute_force():
+    r = np.random.default_rng(11)
+    w = r.standard_normal((7, 19)) * 0.1
+    w[0, 3] = 0.45                      # a mild outlier: somewhere a shrunken range wins
+    w[6] = 0.0
+    steps, mr = 10, 0.3
+    shrunk = 0
+    for bits, sym in ((2, False), (3, False), (3, True)):
+        s, z = orc.grid_search(w, bits, sym, steps, mr)
+        s0, z0 = orc.grid(w, bits, sym)
+        for i in range(7):
+            best = None
+            for k in range(steps):
+                p = 1.0 - k * (1.0 - mr) / steps
+                if sym:
+                    a = p * max(abs(x) for x in w[i]) or 1.0
+                    sk, zk = a / (2 ** (bits - 1) - 1), float(2 ** (bits - 1))
+                else:
+                    lo, hi = p * min(min(w[i]), 0.0), p * max(max(w[i]), 0.0)
+                    sk = (hi - lo) / (2 ** bits - 1) if hi != lo else 1.0
+                    zk = float(np.rint(-lo / sk)) if hi != lo else 0.0
+                err = 0.0
+                for x in w[i]:
+                    c = min(max(float(np.rint(x / sk)) + zk, 0.0), 2.0 ** bits - 1)
+                    err += (sk * (c - zk) - x) ** 2
+                if best is None or err < best[0]:
+                    best = (err, sk, zk)
+            assert abs(s[i] - best[1]) <= 1e-15 * best[1] and z[i] == best[2]
+        # candidate 0 is the plain min/max grid, so the search never does worse than it
+        e_plain = np.sum((orc.dequant(orc.qcode(w, s0[:, None], z0[:, None], bits), s0[:, None], z0[:, None]) - w) ** 2, axis=1)
+        e_best = np.sum((orc.dequant(orc.qcode(w, s[:, None], z[:, None], bits), s[:, None], z[:, None]) - w) ** 2, axis=1)
+        assert np.all(e_best <= e_plain + 1e-18)
+        shrunk += int(np.sum(s < s0 * (1 - 1e-12)))
+    assert shrunk > 0
+    # the loop takes its grids from the search
+    W, X, Xfp = tiny(n=16, m=4)
+    st = stats_of(X, Xfp)
+    U, dead = orc.factor(st.H, st.tokens, 0.01)
+    res = orc.quantize(W, U, None, dead, 3, 8, False, clip=(10, 0.3))
+    s, z = orc.grid_search(W[:, :8], 3, False, 10, 0.3)
+    assert np.array_equal(res.scales[:, 0], s) and np.array_equal(res.zeros[:, 0], z)
+    rep = orc.follow(W, U, None, dead, 3, 8, False, res.codes, res.scales, res.zeros, clip=(10, 0.3))
+    assert rep.mismatches == 0 and rep.zero_mismatch == 0 and rep.grid_rel_err == 0.0
+    bad = res.scales.copy(); bad[2, 1] *= 1.03
+    assert orc.follow(W, U, None, dead, 3, 8, False, res.codes, bad, res.zeros, clip=(10, 0.3)).grid_rel_err > 1e-3
+
+
 # ---------------------------------------------------------------- loop
 def constrained_ls_step(Hd, D, w_q, c, q):
     """min_d  d A d^T - 2 w_q D[q, q:] d^T  s.t. d[0] = c, with A = H_d[q:, q:]
