@@ -320,6 +320,26 @@ def run_ours(args, cfg):
     if world == 1 and not args.no_cpu_baseline:
         v, desc, threads = oracle_sample(cfg, args.ref_tokens, args.ref_rows)
         cpu = {"value": v, "unit": "ms", "cores": threads, "kind": "oracle", "sample": desc}
+    # Per-stage rooflines (algorithmic work / stage time against the bound that applies): the products of
+    # factor, P and the lazy-batch update run as three TF32 tensor-core products, i.e. at most
+    # (bf16 peak / 2) / 3 of useful flops; the column loop is bound by HBM on paper.
+    tf32x3_peak = peak / 2.0 / 3.0
+    n_, m_, B_ = float(cfg.n), float(cfg.m), float(cfg.blocksize)
+    fl_factor, fl_P = 2.0 * n_ ** 3 / 3.0, 2.0 * n_ ** 3 / 3.0
+    fl_trail = 2.0 * m_ * n_ * n_ * max(0.0, 1.0 - B_ / n_)
+    by_loop = 25.0 * m_ * n_ + 8.0 * n_ * B_
+    layer_roofline_ms = (flops_call * len(batches) / (peak * 1e12) + (fl_factor + fl_P + fl_trail) / (tf32x3_peak * 1e12)
+                         + by_loop / (pk["hbm_gbs"] * 1e9)) * 1e3
+    stage_rooflines = {
+        "factor": {"bound": "tensor (3xTF32)", "achieved": fl_factor / (fac_ms * 1e-3) / 1e12, "peak": tf32x3_peak, "unit": "TFLOP/s"},
+        "build_P": {"bound": "tensor (3xTF32)", "achieved": fl_P / (p_ms * 1e-3) / 1e12, "peak": tf32x3_peak, "unit": "TFLOP/s"},
+        "quantize": {"bound": "tensor (3xTF32) + hbm", "trailing_update_tflops_if_alone": fl_trail / (q_ms * 1e-3) / 1e12,
+                     "column_loop_gbs_if_alone": by_loop / (q_ms * 1e-3) / 1e9, "peak_tflops": tf32x3_peak,
+                     "peak_gbs": pk["hbm_gbs"]},
+        "layer": {"roofline_ms": layer_roofline_ms, "measured_ms": ms_step, "frac": layer_roofline_ms / ms_step},
+    }
+    for k in ("factor", "build_P"):
+        stage_rooflines[k]["frac"] = stage_rooflines[k]["achieved"] / tf32x3_peak
     line = {
         "metric": METRIC, "value": ms_layer, "unit": "ms", "n_gpus": world, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": False, "scaling": "strong" if shard else "weak",
@@ -330,7 +350,7 @@ def run_ours(args, cfg):
                        statistics=prec_name, act_order=bool(args.act_order), clip_search=args.clip_search),
         "stages_ms": {"accumulate": acc_step_ms, "factor": fac_ms, "build_P": p_ms, "quantize": q_ms,
                       "layer_quantize": fac_ms + p_ms + q_ms},
-        "accumulate_tflops": achieved,
+        "accumulate_tflops": achieved, "stage_rooflines": stage_rooflines,
         "roofline": {"kernel": "gptaq_accumulate (one token batch)", "bound": "tensor", "achieved": achieved,
                      "peak": peak, "unit": "TFLOP/s", "frac": achieved / peak, "traffic": STATS_KERNEL_TRAFFIC.get((cfg.name, prec)),
                      "peak_source": pk["source"] + " bf16 cuBLAS, sustained",
