@@ -760,8 +760,14 @@ gptaq_status_t gptaq_factor(gptaq_handle_t h, float damp, gptaq_stream_t stream)
         FactorPanelArgs fa;
         fa.H = H; fa.n = n; fa.b0 = b0; fa.Rdiag = Rinv + (size_t)p * NB * NB;
         fa.pan_hi = pan_hi; fa.pan_lo = pan_lo; fa.hd = h->hd;
-        const int fgrid = std::max(1, std::min(b0 / NB, h->num_sms));
-        fa.rows_per_cta = ((b0 + fgrid - 1) / fgrid + NB - 1) / NB * NB;
+        // rows above the block in tiles of 32, 64 or 128 rows: the smallest tile that still gives every
+        // SM at most one tile spreads a short panel over more SMs (the diagonal block is refactored by
+        // every CTA either way)
+        int tr = 32;
+        while (tr < NB && b0 / tr > h->num_sms) tr *= 2;
+        fa.tile_rows = tr;
+        const int fgrid = std::max(1, std::min(b0 / tr, h->num_sms));
+        fa.rows_per_cta = ((b0 + fgrid - 1) / fgrid + tr - 1) / tr * tr;
         factor_panel_kernel<<<fgrid, FP_THREADS, FP_SMEM, s>>>(fa);
         LAUNCHED();
         if (p == 0) break;

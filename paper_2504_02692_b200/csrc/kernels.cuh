@@ -103,7 +103,8 @@ struct FactorPanelArgs {
     float *H; int n; int b0;
     float *Rdiag;              // NB x NB (ld NB): the diagonal factor R_pp (upper, zeros below)
     float *pan_hi, *pan_lo;    // nullptr, or [n][NB]: TF32 parts of the panel rows
-    int rows_per_cta;          // slab of step 2, a multiple of NB
+    int rows_per_cta;          // slab of step 2, a multiple of tile_rows
+    int tile_rows;             // rows of the slab processed at a time: 32, 64 or 128
     StateHeader *hd;
 };
 
@@ -164,13 +165,13 @@ struct Chol32Step<-1> {
     static __device__ __forceinline__ void run(float (&)[32], float, int, float *, StateHeader *, bool, int) {}
 };
 
-// C[0:128, 0:o] -= Xt^T * Rt  with Xt[k][row] (32 x 128) and Rt[k][j] (32 x o), both in shared
+// C[0:rows, 0:o] -= Xt^T * Rt  with Xt[k][row] (32 x rows) and Rt[k][j] (32 x o), both in shared
 // memory with leading dimension FP_LD; C row-major with leading dimension FP_LD.  4 x 8 outputs
 // per thread, all threads of the CTA.
 __device__ __forceinline__ void panel_rank32_update(float (*C)[FP_LD], const float (*Xt)[FP_LD],
-                                                    const float (*Rt)[FP_LD], int o, int tid) {
+                                                    const float (*Rt)[FP_LD], int o, int tid, int rows) {
     const int tiles_j = o / 8;
-    for (int t = tid; t < 32 * tiles_j; t += FP_THREADS) {
+    for (int t = tid; t < (rows / 4) * tiles_j; t += FP_THREADS) {
         const int ti = t / tiles_j, tj = t - ti * tiles_j;
         float acc[4][8];
 #pragma unroll
@@ -306,21 +307,22 @@ __global__ void __launch_bounds__(FP_THREADS, 1) factor_panel_kernel(FactorPanel
     //      columns to the left (all threads)
     const int r_begin = blockIdx.x * a.rows_per_cta;
     const int r_end = min(b0, r_begin + a.rows_per_cta);
-    for (int r0 = r_begin; r0 < r_end; r0 += NB) {        // b0 and the slabs are multiples of NB
+    const int TR = a.tile_rows;
+    for (int r0 = r_begin; r0 < r_end; r0 += TR) {        // b0 and the slabs are multiples of TR
         if (vec) {
             float4 v[NB * NB / 4 / FP_THREADS];
 #pragma unroll
             for (int it = 0; it < NB * NB / 4 / FP_THREADS; ++it) {
                 const int idx = tid + it * FP_THREADS, i = idx >> 5, j4 = idx & 31;
-                v[it] = *reinterpret_cast<const float4 *>(a.H + (int64_t)(r0 + i) * n + b0 + 4 * j4);
+                if (i < TR) v[it] = *reinterpret_cast<const float4 *>(a.H + (int64_t)(r0 + i) * n + b0 + 4 * j4);
             }
 #pragma unroll
             for (int it = 0; it < NB * NB / 4 / FP_THREADS; ++it) {
                 const int idx = tid + it * FP_THREADS, i = idx >> 5, j4 = idx & 31;
-                *reinterpret_cast<float4 *>(&At[i][4 * j4]) = v[it];
+                if (i < TR) *reinterpret_cast<float4 *>(&At[i][4 * j4]) = v[it];
             }
         } else {
-            for (int i = warp; i < NB; i += FP_WARPS) {
+            for (int i = warp; i < TR; i += FP_WARPS) {
                 const float *src = a.H + (int64_t)(r0 + i) * n + b0;
                 for (int k = lane; k < NB; k += 32) At[i][k] = k < nv ? src[k] : 0.f;
             }
@@ -328,7 +330,7 @@ __global__ void __launch_bounds__(FP_THREADS, 1) factor_panel_kernel(FactorPanel
         __syncthreads();
         for (int sb = NB / 32 - 1; sb >= 0; --sb) {
             const int o = 32 * sb;
-            if (tid < NB) {
+            if (tid < TR) {
                 float x[32];
 #pragma unroll
                 for (int k = 0; k < 32; ++k) x[k] = At[tid][o + k];
@@ -338,7 +340,7 @@ __global__ void __launch_bounds__(FP_THREADS, 1) factor_panel_kernel(FactorPanel
             }
             __syncthreads();
             if (o > 0) {
-                panel_rank32_update(At, Pt, reinterpret_cast<const float (*)[FP_LD]>(&S[o][0]), o, tid);
+                panel_rank32_update(At, Pt, reinterpret_cast<const float (*)[FP_LD]>(&S[o][0]), o, tid, TR);
                 __syncthreads();
             }
         }
@@ -346,6 +348,7 @@ __global__ void __launch_bounds__(FP_THREADS, 1) factor_panel_kernel(FactorPanel
 #pragma unroll
         for (int it = 0; it < NB * NB / 4 / FP_THREADS; ++it) {
             const int idx = tid + it * FP_THREADS, i = idx >> 5, j4 = idx & 31;
+            if (i >= TR) continue;
             const float4 v = *reinterpret_cast<const float4 *>(&At[i][4 * j4]);
             float *dst = a.H + (int64_t)(r0 + i) * n + b0 + 4 * j4;
             if (vec) {
