@@ -704,7 +704,7 @@ constexpr int CB_THREADS = 256;
 constexpr int CB_LD = 128 + 4;
 
 __host__ __device__ inline size_t column_block_smem(int rows) {
-    return ((size_t)rows * CB_LD + 2 * 32 * CB_LD + 64 * (rows + 4) + 32) * sizeof(float);
+    return ((size_t)rows * CB_LD + 2 * 2 * 32 * CB_LD + 64 * (rows + 4) + 2 * 32) * sizeof(float);
 }
 
 template <int K>
@@ -742,11 +742,12 @@ struct QuantStep<32> {
 __global__ void __launch_bounds__(CB_THREADS, 1) column_block_kernel(ColumnLoopArgs a, int rows, int B) {
     extern __shared__ __align__(16) float smem_f[];
     float (*Wt)[CB_LD] = reinterpret_cast<float (*)[CB_LD]>(smem_f);                       // [rows][B]
-    float (*Us)[CB_LD] = reinterpret_cast<float (*)[CB_LD]>(smem_f + rows * CB_LD);        // rows o..o+31 of U, block columns
-    float (*Ps)[CB_LD] = Us + 32;
-    float *St = smem_f + rows * CB_LD + 2 * 32 * CB_LD;                                    // [64][rows + 4]: -Err, then Wpre
+    // rows o..o+31 of U and of P (block columns), two buffers: the next 32 rows are fetched while the
+    // current 32 columns are quantized
+    float (*UP)[CB_LD] = reinterpret_cast<float (*)[CB_LD]>(smem_f + rows * CB_LD);        // [2 buffers][U, P][32]
+    float *St = smem_f + rows * CB_LD + 2 * 2 * 32 * CB_LD;                                // [64][rows + 4]: -Err, then Wpre
     const int sld = rows + 4;
-    float *udinv = St + 64 * sld;
+    float *udinv2 = St + 64 * sld;                                                         // [2][32]
     const int tid = threadIdx.x;
     const int n = a.n, i0 = a.i0;
     const int row0 = blockIdx.x * rows;
@@ -776,9 +777,12 @@ __global__ void __launch_bounds__(CB_THREADS, 1) column_block_kernel(ColumnLoopA
     const int row = row0 + tid;
     if (a.group <= 0 && owner) { scale = a.scales[row]; zero = a.zeros[row]; }
 
-    for (int o = 0; o < B; o += 32) {
-        __syncthreads();        // the block is current; Us / Ps / St are free
-        for (int idx = tid; idx < 32 * bq; idx += CB_THREADS) {
+    // rows [o, o + 32) of U and P of this block into buffer `buf`, by `nthr` threads starting at `t0`
+    auto fetch_up = [&](int o, int buf, int t0, int nthr) {
+        float (*Ub)[CB_LD] = UP + buf * 64;
+        float (*Pb)[CB_LD] = Ub + 32;
+        const int t = tid - t0;
+        for (int idx = t; idx < 32 * bq; idx += nthr) {
             const int k = idx / bq, c4 = idx - k * bq;
             const int64_t off = (int64_t)(i0 + o + k) * n + i0 + 4 * c4;
             float4 u, p;
@@ -789,11 +793,19 @@ __global__ void __launch_bounds__(CB_THREADS, 1) column_block_kernel(ColumnLoopA
                 u = make_float4(a.U[off], a.U[off + 1], a.U[off + 2], a.U[off + 3]);
                 p = make_float4(a.P[off], a.P[off + 1], a.P[off + 2], a.P[off + 3]);
             }
-            *reinterpret_cast<float4 *>(&Us[k][4 * c4]) = u;
-            *reinterpret_cast<float4 *>(&Ps[k][4 * c4]) = p;
+            *reinterpret_cast<float4 *>(&Ub[k][4 * c4]) = u;
+            *reinterpret_cast<float4 *>(&Pb[k][4 * c4]) = p;
         }
-        if (tid < 32) udinv[tid] = 1.f / a.U[(int64_t)(i0 + o + tid) * n + i0 + o + tid];
-        __syncthreads();
+        if (t < 32) udinv2[buf * 32 + t] = 1.f / a.U[(int64_t)(i0 + o + t) * n + i0 + o + t];
+    };
+    fetch_up(0, 0, 0, CB_THREADS);
+
+    for (int o = 0; o < B; o += 32) {
+        const int buf = (o >> 5) & 1;
+        float (*Us)[CB_LD] = UP + buf * 64;
+        float (*Ps)[CB_LD] = Us + 32;
+        const float *udinv = udinv2 + buf * 32;
+        __syncthreads();        // the block is current; this buffer of U / P is loaded; St and the other buffer are free
         const bool group_start = a.group > 0 && ((i0 + o) % a.group) == 0;
         int best_k = 0;
         if (group_start && a.clip_steps > 0) {
@@ -834,6 +846,7 @@ __global__ void __launch_bounds__(CB_THREADS, 1) column_block_kernel(ColumnLoopA
             }
             __syncthreads();
         }
+        if (tid >= CB_THREADS / 2 && o + 32 < B) fetch_up(o + 32, buf ^ 1, CB_THREADS / 2, CB_THREADS / 2);
         if (owner) {
             if (group_start) {
                 // grid of the group that starts here, from the current values
