@@ -495,7 +495,7 @@ __device__ __forceinline__ float clip_ratio(int k, int steps, float min_ratio) {
     return 1.f - (float)k * ((1.f - min_ratio) / (float)steps);
 }
 __device__ __forceinline__ float rounding_error_sq(float w, float scale, float zero, float maxq) {
-    const float cq = fminf(fmaxf(rintf(w / scale) + zero, 0.f), maxq);
+    const float cq = fminf(fmaxf(rintf(w * (1.f / scale)) + zero, 0.f), maxq);
     const float d = scale * (cq - zero) - w;
     return d * d;
 }
@@ -649,7 +649,7 @@ __global__ void __launch_bounds__(1024) column_loop_kernel(ColumnLoopArgs a) {
                 }
             }
             const float wj = __shfl_sync(0xffffffffu, w[t], jj);
-            float cq = fminf(fmaxf(rintf(wj / scale) + zero, 0.f), maxq);
+            float cq = fminf(fmaxf(rintf(wj * (1.f / scale)) + zero, 0.f), maxq);
             const float q = scale * (cq - zero);
             const float ne = a.err_scale * ((q - wj) * (1.f / Us[j][j]));   // -(w - q) / U_jj
             const float wp = a.asym_scale * wj;
@@ -712,9 +712,12 @@ struct QuantStep {
     // x: the row's 32 columns (already-updated weights in, dequantized values out)
     static __device__ __forceinline__ void run(float (&x)[32], float (&nerr)[32], float (&pre)[32], uint32_t (&code)[8],
                                                const float *Us, const float *Ps, const float *udinv,
-                                               float scale, float zero, float maxq, float err_scale, float asym_scale) {
+                                               float scale, float inv_scale, float zero, float maxq, float err_scale,
+                                               float asym_scale) {
         const float w0 = x[K];
-        const float cq = fminf(fmaxf(rintf(w0 / scale) + zero, 0.f), maxq);
+        // w / scale as w * (1 / scale): one rounding more (about 1e-7 of a step, far inside the tie band)
+        // for a much shorter dependent chain
+        const float cq = fminf(fmaxf(rintf(w0 * inv_scale) + zero, 0.f), maxq);
         const float q = scale * (cq - zero);
         const float ne = err_scale * ((q - w0) * udinv[K]);           // -(w - q) / U_kk
         const float w = asym_scale * w0;
@@ -730,13 +733,13 @@ struct QuantStep {
             if (4 * j4 + 2 > K) x[4 * j4 + 2] = fmaf(w, p.z, fmaf(ne, u.z, x[4 * j4 + 2]));
             if (4 * j4 + 3 > K) x[4 * j4 + 3] = fmaf(w, p.w, fmaf(ne, u.w, x[4 * j4 + 3]));
         }
-        QuantStep<K + 1>::run(x, nerr, pre, code, Us, Ps, udinv, scale, zero, maxq, err_scale, asym_scale);
+        QuantStep<K + 1>::run(x, nerr, pre, code, Us, Ps, udinv, scale, inv_scale, zero, maxq, err_scale, asym_scale);
     }
 };
 template <>
 struct QuantStep<32> {
     static __device__ __forceinline__ void run(float (&)[32], float (&)[32], float (&)[32], uint32_t (&)[8],
-                                               const float *, const float *, const float *, float, float, float, float, float) {}
+                                               const float *, const float *, const float *, float, float, float, float, float, float) {}
 };
 
 __global__ void __launch_bounds__(CB_THREADS, 1) column_block_kernel(ColumnLoopArgs a, int rows, int B) {
@@ -754,21 +757,32 @@ __global__ void __launch_bounds__(CB_THREADS, 1) column_block_kernel(ColumnLoopA
     const int nrows = min(rows, a.m - row0);
     const int bq = B / 4;
 
-    // the block of W (dead inputs read as zero), along rows
-    for (int idx = tid; idx < rows * bq; idx += CB_THREADS) {
-        const int r = idx / bq, c4 = idx - r * bq;
-        float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
-        if (r < nrows) {
-            const float *src = a.W + (int64_t)(row0 + r) * a.ldw + i0 + 4 * c4;
-            if ((reinterpret_cast<uintptr_t>(src) & 15) == 0) v = *reinterpret_cast<const float4 *>(src);
-            else { v.x = src[0]; v.y = src[1]; v.z = src[2]; v.w = src[3]; }
-            const uchar4 dd = *reinterpret_cast<const uchar4 *>(a.dead + i0 + 4 * c4);
-            if (dd.x) v.x = 0.f;
-            if (dd.y) v.y = 0.f;
-            if (dd.z) v.z = 0.f;
-            if (dd.w) v.w = 0.f;
+    // the block of W (dead inputs read as zero), along rows; four loads in flight per thread
+    for (int base = 0; base < rows * bq; base += 4 * CB_THREADS) {
+        float4 v[4];
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            const int idx = base + u * CB_THREADS + tid;
+            const int r = idx / bq, c4 = idx - r * bq;
+            v[u] = make_float4(0.f, 0.f, 0.f, 0.f);
+            if (idx < rows * bq && r < nrows) {
+                const float *src = a.W + (int64_t)(row0 + r) * a.ldw + i0 + 4 * c4;
+                if ((reinterpret_cast<uintptr_t>(src) & 15) == 0) v[u] = *reinterpret_cast<const float4 *>(src);
+                else { v[u].x = src[0]; v[u].y = src[1]; v[u].z = src[2]; v[u].w = src[3]; }
+            }
         }
-        *reinterpret_cast<float4 *>(&Wt[r][4 * c4]) = v;
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            const int idx = base + u * CB_THREADS + tid;
+            if (idx >= rows * bq) continue;
+            const int r = idx / bq, c4 = idx - r * bq;
+            const uchar4 dd = *reinterpret_cast<const uchar4 *>(a.dead + i0 + 4 * c4);
+            if (dd.x) v[u].x = 0.f;
+            if (dd.y) v[u].y = 0.f;
+            if (dd.z) v[u].z = 0.f;
+            if (dd.w) v[u].w = 0.f;
+            *reinterpret_cast<float4 *>(&Wt[r][4 * c4]) = v[u];
+        }
     }
 
     const float maxq = (float)((1 << a.bits) - 1);
@@ -870,7 +884,7 @@ __global__ void __launch_bounds__(CB_THREADS, 1) column_block_kernel(ColumnLoopA
                 x[4 * k4] = v.x; x[4 * k4 + 1] = v.y; x[4 * k4 + 2] = v.z; x[4 * k4 + 3] = v.w;
                 code[k4] = 0u;
             }
-            QuantStep<0>::run(x, nerr, pre, code, &Us[0][o], &Ps[0][o], udinv, scale, zero, maxq, a.err_scale, a.asym_scale);
+            QuantStep<0>::run(x, nerr, pre, code, &Us[0][o], &Ps[0][o], udinv, scale, 1.f / scale, zero, maxq, a.err_scale, a.asym_scale);
             uint8_t *crow = a.codes + (int64_t)row * n + i0 + o;
             if (a.perm) {
                 uint8_t *cbase = a.codes + (int64_t)row * n;
