@@ -47,6 +47,8 @@ struct gptaq_ctx {
     int64_t launches;
     int stats_precision;   // GPTAQ_STATS_*
     bool tensor;           // float32-grade tensor-core GEMMs for factor / P / trailing update
+    bool f16;              // ... with FP16-split operands where the producer can record their range (n % 8 == 0)
+    bool tf32_copies;      // f16 handles: the TF32 copies of U^T and P^T exist (made on demand by gptaq_quantize)
     int terms;             // GPTAQ_TERM_* switches of gptaq_quantize
     int clip_steps; float clip_min;   // clipping-range search of the grids
     // Statistics pipeline: the conversion of a token batch runs on the caller's stream, the
@@ -87,7 +89,7 @@ struct WsLayout {
     size_t t_off, rinv_off;
     size_t s_off[6];        // split operand matrices (n x n each): S1 hi/lo, S2 hi/lo, S3 hi/lo
     size_t pan_off[2];      // split copy of one factor panel (n x 128), hi/lo
-    size_t ew_off, ew_lo_off, total;
+    size_t ew_off, ew_lo_off, rs_off, total;   // [-Err | Wpre] (m x 2B), its second part, one scale per row
     bool tensor;
 };
 
@@ -104,7 +106,8 @@ WsLayout ws_layout(int64_t n, int64_t m_max, int blocksize) {
     const size_t ew = round_up((size_t)m_max * 2 * (size_t)blocksize * sizeof(float), ALIGN);
     w.ew_off = off;
     w.ew_lo_off = off + ew;
-    w.total = off + (w.tensor ? 2 * ew : ew);
+    w.rs_off = off + (w.tensor ? 2 * ew : ew);
+    w.total = w.rs_off + (w.tensor ? round_up((size_t)m_max * sizeof(float), ALIGN) : 0);
     return w;
 }
 
@@ -187,20 +190,40 @@ bool make_f32_map(CUtensorMap *map, const void *ptr, int64_t rows, int64_t cols,
 
 // A split operand (hi / lo arrays of the same shape) as seen by the tensor-core GEMM.
 struct SplitOperand {
-    const float *hi, *lo;
+    const void *hi, *lo;       // float32 arrays holding TF32 values, or __half arrays (f16)
     int64_t rows, cols, ld;
+    bool f16 = false;
 };
+
+// __half matrix [rows][ld] with `cols` valid K-contiguous elements per row; box = 64 x box_rows.
+bool make_f16_map(CUtensorMap *map, const void *ptr, int64_t rows, int64_t cols, int64_t ld, int box_rows) {
+    EncodeTiledFn fn = encode_tiled_fn();
+    if (!fn) return false;
+    cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
+    cuuint64_t strides[1] = {(cuuint64_t)ld * 2};
+    cuuint32_t box[2] = {(cuuint32_t)(2 * TBK), (cuuint32_t)box_rows};
+    cuuint32_t estr[2] = {1, 1};
+    return fn(map, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 2, const_cast<void *>(ptr), dims, strides, box, estr,
+              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+bool make_operand_map(CUtensorMap *map, const void *ptr, const SplitOperand &o, int box_rows) {
+    return o.f16 ? make_f16_map(map, ptr, o.rows, o.cols, o.ld, box_rows)
+                 : make_f32_map(map, ptr, o.rows, o.cols, o.ld, box_rows);
+}
 
 struct TcMaps {
     CUtensorMap a_hi, a_lo, b_hi, b_lo, b2_hi, b2_lo;
+    bool f16 = false;
 };
 
 bool make_tc_maps(TcMaps *m, const SplitOperand &A, const SplitOperand &B, const SplitOperand *B2) {
     const SplitOperand &b2 = B2 ? *B2 : B;
-    return make_f32_map(&m->a_hi, A.hi, A.rows, A.cols, A.ld, TBM) && make_f32_map(&m->a_lo, A.lo, A.rows, A.cols, A.ld, TBM) &&
-           make_f32_map(&m->b_hi, B.hi, B.rows, B.cols, B.ld, TBN) && make_f32_map(&m->b_lo, B.lo, B.rows, B.cols, B.ld, TBN) &&
-           make_f32_map(&m->b2_hi, b2.hi, b2.rows, b2.cols, b2.ld, TBN) &&
-           make_f32_map(&m->b2_lo, b2.lo, b2.rows, b2.cols, b2.ld, TBN);
+    m->f16 = A.f16;
+    return make_operand_map(&m->a_hi, A.hi, A, TBM) && make_operand_map(&m->a_lo, A.lo, A, TBM) &&
+           make_operand_map(&m->b_hi, B.hi, B, TBN) && make_operand_map(&m->b_lo, B.lo, B, TBN) &&
+           make_operand_map(&m->b2_hi, b2.hi, b2, TBN) && make_operand_map(&m->b2_lo, b2.lo, b2, TBN);
 }
 
 TcGemmArgs tc_args(float *C, int64_t ldc, int M, int N, int K, float alpha, float beta, int mode, int mask,
@@ -212,11 +235,54 @@ TcGemmArgs tc_args(float *C, int64_t ldc, int M, int N, int K, float alpha, floa
     return a;
 }
 
-cudaError_t launch_tc_gemm(const TcMaps &m, const TcGemmArgs &a, int num_sms, cudaStream_t s) {
-    if (a.M <= 0 || a.N <= 0 || a.nbatch <= 0) return cudaSuccess;
+// float32 matrix C [M][ldc] with N valid columns as the target of bulk reductions: box = 32 x 128,
+// 128-byte swizzle (the layout the epilogue writes its staging boxes in).
+bool make_c_map(CUtensorMap *map, float *C, int64_t M, int64_t N, int64_t ldc) {
+    EncodeTiledFn fn = encode_tiled_fn();
+    if (!fn) return false;
+    cuuint64_t dims[2] = {(cuuint64_t)N, (cuuint64_t)M};
+    cuuint64_t strides[1] = {(cuuint64_t)ldc * 4};
+    cuuint32_t box[2] = {32, (cuuint32_t)TBM};
+    cuuint32_t estr[2] = {1, 1};
+    return fn(map, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, C, dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+              CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+cudaError_t launch_tc_gemm(const TcMaps &m, const TcGemmArgs &a_in, int num_sms, cudaStream_t s) {
+    if (a_in.M <= 0 || a_in.N <= 0 || a_in.nbatch <= 0) return cudaSuccess;
+    TcGemmArgs a = a_in;
     const int64_t tiles = (int64_t)a.nbatch * ((a.M + TBM - 1) / TBM) * ((a.N + TBN - 1) / TBN);
     const int grid = (int)std::min<int64_t>(tiles, num_sms);
-    tc_gemm_kernel<<<grid, TC_THREADS, TC_SMEM, s>>>(m.a_hi, m.a_lo, m.b_hi, m.b_lo, m.b2_hi, m.b2_lo, a);
+    // "C += ...": bulk tensor reductions where the target qualifies for a tensor map (16-byte aligned base
+    // and row pitch); scattered per-thread reductions otherwise
+    CUtensorMap mapC = m.a_hi;       // placeholder, not dereferenced unless c_tma is set
+    a.c_tma = 0;
+    if (a.beta == 1.f && a.nbatch == 1 && !a.amax_out && (a.mask == TC_MASK_NONE || a.mask == TC_MASK_UPPER_KEEP) &&
+        (reinterpret_cast<uintptr_t>(a.C) & 15) == 0 && (a.ldc & 3) == 0 && make_c_map(&mapC, a.C, a.M, a.N, a.ldc))
+        a.c_tma = 1;
+    if (m.f16) tc_gemm_kernel<true><<<grid, TC_THREADS, TC_SMEM, s>>>(m.a_hi, m.a_lo, m.b_hi, m.b_lo, m.b2_hi, m.b2_lo, mapC, a);
+    else tc_gemm_kernel<false><<<grid, TC_THREADS, TC_SMEM, s>>>(m.a_hi, m.a_lo, m.b_hi, m.b_lo, m.b2_hi, m.b2_lo, mapC, a);
+    return cudaGetLastError();
+}
+
+// Slots of StateHeader::tc_amax (largest magnitudes of FP16-split operands).
+
+cudaError_t launch_absmax(const float *src, int64_t lds, int rows, int cols, int mask, float scale, unsigned *slot,
+                          int num_sms, cudaStream_t s) {
+    const int grid = std::max(1, std::min(rows, 8 * num_sms));
+    absmax_kernel<<<grid, 256, 0, s>>>(src, lds, rows, cols, mask, scale, slot);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_split16(const float *src, int64_t lds, __half *hi, __half *lo, int64_t ldd, int rows, int cols,
+                           bool transpose, int mask, float scale, const unsigned *amax, cudaStream_t s) {
+    if (rows <= 0 || cols <= 0) return cudaSuccess;
+    Split16Args a;
+    a.src = src; a.lds = lds; a.hi = hi; a.lo = lo; a.ldd = ldd; a.rows = rows; a.cols = cols;
+    a.transpose = transpose ? 1 : 0; a.mask = mask; a.scale = scale; a.amax = amax;
+    dim3 grid((cols + 63) / 64, (rows + 63) / 64, 1);
+    split16_kernel<<<grid, 256, 0, s>>>(a);
     return cudaGetLastError();
 }
 
@@ -361,6 +427,13 @@ struct QuantizeTarget {
     // the low part of [-Err | Wpre]; all null on the plain-FMA path
     const float *UT_hi, *UT_lo, *PT_hi, *PT_lo;
     float *EW_lo;
+    // the same update with FP16-split operands (takes precedence when set): U^T and P^T as fp16 hi / lo
+    // (lo = hi + n * n), each with the scale of its recorded maximum, [-Err | Wpre] as fp16 hi / lo with
+    // one scale per row
+    const __half *UT16 = nullptr, *PT16 = nullptr;
+    __half *EW16 = nullptr;
+    float *row_inv = nullptr;
+    const unsigned *amax_u = nullptr, *amax_p = nullptr;
     int terms = GPTAQ_TERM_ERR | GPTAQ_TERM_ASYM;   // which terms of the weight update are applied
     const int *perm = nullptr;                      // act_order: working column c is the caller's column perm[c]
     int clip_steps = 0; float clip_min = 1.f;       // clipping-range search of the grids (0 steps: min/max)
@@ -432,9 +505,15 @@ gptaq_status_t quantize_core(const QuantizeTarget &t, void *d_W, int w_dtype, in
     const unsigned cb_grid = (unsigned)((m + cb_rows - 1) / cb_rows);
     const size_t cl_smem = 2 * (size_t)blocksize * blocksize * sizeof(float);
 
-    const bool tensor = t.EW_lo != nullptr;
+    const bool tensor16 = t.EW16 != nullptr;
+    const bool tensor = tensor16 || t.EW_lo != nullptr;
     TcMaps maps;
-    if (tensor) {
+    if (tensor16) {
+        const size_t nn = (size_t)n * n, me = (size_t)m * 2 * blocksize;
+        const SplitOperand A{t.EW16, t.EW16 + me, m, 2 * blocksize, 2 * blocksize, true};
+        const SplitOperand B{t.UT16, t.UT16 + nn, n, n, n, true}, B2{t.PT16, t.PT16 + nn, n, n, n, true};
+        if (!make_tc_maps(&maps, A, B, &B2)) { *err = cudaErrorUnknown; return GPTAQ_ERR_CUDA; }
+    } else if (tensor) {
         const SplitOperand A{EW, t.EW_lo, m, 2 * blocksize, 2 * blocksize};
         const SplitOperand B{t.UT_hi, t.UT_lo, n, n, n}, B2{t.PT_hi, t.PT_lo, n, n, n};
         if (!make_tc_maps(&maps, A, B, &B2)) { *err = cudaErrorUnknown; return GPTAQ_ERR_CUDA; }
@@ -444,7 +523,9 @@ gptaq_status_t quantize_core(const QuantizeTarget &t, void *d_W, int w_dtype, in
         a.W = Wk; a.ldw = ldk; a.m = (int)m; a.n = n; a.U = t.U; a.P = t.P; a.dead = t.dead;
         a.i0 = i0; a.bw = std::min(blocksize, n - i0);
         a.bits = bits; a.group = group; a.sym = sym;
-        a.codes = d_codes; a.scales = d_scales; a.zeros = d_zeros; a.G = G; a.EW = EW; a.EW_lo = t.EW_lo; a.hd = t.hd;
+        a.codes = d_codes; a.scales = d_scales; a.zeros = d_zeros; a.G = G; a.EW = EW; a.EW_lo = tensor16 ? nullptr : t.EW_lo; a.hd = t.hd;
+        a.EW16_hi = tensor16 ? t.EW16 : nullptr; a.EW16_lo = tensor16 ? t.EW16 + (size_t)m * 2 * blocksize : nullptr;
+        a.row_inv = t.row_inv; a.amax_u = t.amax_u; a.amax_p = t.amax_p;
         a.perm = t.perm; a.clip_steps = t.clip_steps; a.clip_min = t.clip_min; a.err_scale = (t.terms & GPTAQ_TERM_ERR) ? 1.f : 0.f; a.asym_scale = (t.terms & GPTAQ_TERM_ASYM) ? 1.f : 0.f;
         const bool fast = a.bw == blocksize && (group <= 0 || (group % 32) == 0) && (i0 % 4) == 0 &&
                           (reinterpret_cast<uintptr_t>(t.dead) & 3) == 0;
@@ -459,6 +540,7 @@ gptaq_status_t quantize_core(const QuantizeTarget &t, void *d_W, int w_dtype, in
             // are rows i2.. of U^T (first B contraction steps) and of P^T (the next B)
             TcGemmArgs g = tc_args(Wk + i2, ldk, (int)m, n - i2, 2 * blocksize, 1.f, 1.f, TC_FULL, TC_MASK_NONE, t.hd);
             g.b_row0 = i2; g.b_k0 = i0; g.k_split = blocksize; g.b2_k0 = i0;
+            if (tensor16) { g.row_inv = t.row_inv; g.amax_b = t.amax_u; }
             *err = launch_tc_gemm(maps, g, t.num_sms, s);
             if (*err != cudaSuccess) return GPTAQ_ERR_CUDA;
             ++*launches;
@@ -586,6 +668,7 @@ gptaq_status_t gptaq_create(gptaq_handle_t *out, int64_t n, void *d_state, size_
     h->launches = 0;
     h->stats_precision = GPTAQ_STATS_FP16_SPLIT_TENSOR;
     h->tensor = tc_shape_ok(n) && encode_tiled_fn() != nullptr;
+    h->f16 = h->tensor && (n % 8) == 0;
     h->terms = GPTAQ_TERM_ERR | GPTAQ_TERM_ASYM;
     h->clip_steps = 0; h->clip_min = 1.f;
     cudaError_t e = cudaGetDevice(&h->device);
@@ -600,7 +683,9 @@ gptaq_status_t gptaq_create(gptaq_handle_t *out, int64_t n, void *d_state, size_
     if (e == cudaSuccess)
         e = cudaFuncSetAttribute(stats_umma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)UMMA_SMEM);
     if (e == cudaSuccess)
-        e = cudaFuncSetAttribute(tc_gemm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)TC_SMEM);
+        e = cudaFuncSetAttribute(tc_gemm_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)TC_SMEM);
+    if (e == cudaSuccess)
+        e = cudaFuncSetAttribute(tc_gemm_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)TC_SMEM);
     // the conversion of the next batch shares the SMs with the running product: both kernels ask for
     // the largest shared-memory carve-out, so that a conversion CTA fits beside a product CTA
     if (e == cudaSuccess)
@@ -751,7 +836,7 @@ gptaq_status_t gptaq_factor(gptaq_handle_t h, float damp, gptaq_stream_t stream)
     float *pan_lo = h->tensor ? reinterpret_cast<float *>(h->ws + wl.pan_off[1]) : nullptr;
     TcMaps pan_maps;
     if (h->tensor) {
-        const SplitOperand pan{pan_hi, pan_lo, n, NB, NB};
+        const SplitOperand pan{pan_hi, pan_lo, n, NB, NB, h->f16};
         if (!make_tc_maps(&pan_maps, pan, pan, nullptr)) { h->cuda_error = "cuTensorMapEncodeTiled failed"; return GPTAQ_ERR_CUDA; }
     }
     for (int p = nb - 1; p >= 0; --p) {
@@ -759,7 +844,7 @@ gptaq_status_t gptaq_factor(gptaq_handle_t h, float damp, gptaq_stream_t stream)
         // diagonal block (factor + inverse) and the panel above it: R[0:b0, blk] = A[0:b0, blk] inv(R_pp)^T
         FactorPanelArgs fa;
         fa.H = H; fa.n = n; fa.b0 = b0; fa.Rdiag = Rinv + (size_t)p * NB * NB;
-        fa.pan_hi = pan_hi; fa.pan_lo = pan_lo; fa.hd = h->hd;
+        fa.pan_hi = pan_hi; fa.pan_lo = pan_lo; fa.pan_f16 = h->f16 ? 1 : 0; fa.hd = h->hd;
         // rows above the block in tiles of 32, 64 or 128 rows: the smallest tile that still gives every
         // SM at most one tile spreads a short panel over more SMs (the diagonal block is refactored by
         // every CTA either way)
@@ -774,6 +859,7 @@ gptaq_status_t gptaq_factor(gptaq_handle_t h, float damp, gptaq_stream_t stream)
         // A[0:b0, 0:b0] -= R[0:b0, blk] R[0:b0, blk]^T  (upper part)
         if (h->tensor && b0 >= TC_MIN_N) {
             TcGemmArgs g = tc_args(H, n, b0, b0, NB, -1.f, 1.f, TC_UPPER_TILES, TC_MASK_UPPER_KEEP, h->hd);
+            if (h->f16) g.amax_a = g.amax_b = h->hd->tc_amax + AMAX_PAN;
             CU(launch_tc_gemm(pan_maps, g, h->num_sms, s));
             h->launches++;
         } else {
@@ -842,13 +928,15 @@ gptaq_status_t gptaq_factor(gptaq_handle_t h, float damp, gptaq_stream_t stream)
         p2.batchN_last = tail;
         OK(gemm(h, p2, false, true, s));
     }
-    if (h->tensor) {
+    if (h->tensor && !h->f16) {
         // operand copies of U for the products that follow: S1 = split(U), S2 = split(U^T)
+        // (FP16-split handles make theirs in gptaq_build_P, once the range of U is known)
         CU(launch_split(H, n, S1h, S1l, n, n, n, false, SPLIT_UPPER, 1.f, s));
         h->launches++;
         CU(launch_split(H, n, S2h, S2l, n, n, n, true, SPLIT_UPPER, 1.f, s));
         h->launches++;
     }
+    h->tf32_copies = false;
     h->stage = STAGE_FACTORED;
     return GPTAQ_OK;
 }
@@ -860,6 +948,44 @@ gptaq_status_t gptaq_build_P(gptaq_handle_t h, float alpha, gptaq_stream_t strea
     const int n = (int)h->n;
     WsLayout wl = ws_layout(h->n, 0, 32);
     float *O = reinterpret_cast<float *>(h->ws + wl.t_off);
+    if (h->tensor && h->f16) {
+        // FP16-split operands (half the bytes and twice the MMA rate of the TF32 form): every operand is
+        // scaled by a power of two into the fp16 range, so its largest magnitude is recorded first (by a
+        // reduction kernel for U and dXX^T, by the producing GEMM's epilogue for O and P).
+        // Workspace: S[0] = U^T (kept for gptaq_quantize), S[1] = U, then P^T (kept), S[4] = dXX^T, then O.
+        const size_t nn = (size_t)n * n;
+        __half *UT16 = reinterpret_cast<__half *>(h->ws + wl.s_off[0]);
+        __half *U16 = reinterpret_cast<__half *>(h->ws + wl.s_off[1]);
+        __half *A16 = reinterpret_cast<__half *>(h->ws + wl.s_off[4]);
+        unsigned *am = h->hd->tc_amax;
+        const float inv_tokens = (float)(1.0 / (double)h->tokens);
+        CU(cudaMemsetAsync(am + AMAX_U, 0, 4 * sizeof(unsigned), s));      // slots U, D, O, P
+        CU(launch_absmax(h->H, n, n, n, SPLIT_UPPER, 1.f, am + AMAX_U, h->num_sms, s));
+        CU(launch_absmax(h->D, n, n, n, SPLIT_ALL, inv_tokens, am + AMAX_D, h->num_sms, s));
+        CU(launch_split16(h->H, n, U16, U16 + nn, n, n, n, false, SPLIT_UPPER, 1.f, am + AMAX_U, s));
+        CU(launch_split16(h->H, n, UT16, UT16 + nn, n, n, n, true, SPLIT_UPPER, 1.f, am + AMAX_U, s));
+        CU(launch_split16(h->D, n, A16, A16 + nn, n, n, n, false, SPLIT_ALL, inv_tokens, am + AMAX_D, s));
+        h->launches += 5;
+        const SplitOperand Uop{U16, U16 + nn, n, n, n, true}, UTop{UT16, UT16 + nn, n, n, n, true};
+        const SplitOperand Aop{A16, A16 + nn, n, n, n, true};
+        TcMaps maps;
+        // O = ((dXX^T / tokens) U^T) .* M_U  (contraction over k >= column, U[a][k] = 0 below)
+        if (!make_tc_maps(&maps, Aop, Uop, nullptr)) { h->cuda_error = "cuTensorMapEncodeTiled failed"; return GPTAQ_ERR_CUDA; }
+        TcGemmArgs go = tc_args(O, n, n, n, n, 1.f, 0.f, TC_O, TC_MASK_STRICT_ZERO, h->hd);
+        go.amax_a = am + AMAX_D; go.amax_b = am + AMAX_U; go.amax_out = am + AMAX_O;
+        CU(launch_tc_gemm(maps, go, h->num_sms, s));
+        CU(launch_split16(O, n, A16, A16 + nn, n, n, n, false, SPLIT_STRICT_UPPER, 1.f, am + AMAX_O, s));
+        // P = alpha * O U  (B operand rows are rows of U^T)
+        if (!make_tc_maps(&maps, Aop, UTop, nullptr)) { h->cuda_error = "cuTensorMapEncodeTiled failed"; return GPTAQ_ERR_CUDA; }
+        TcGemmArgs gp = tc_args(h->D, n, n, n, n, alpha, 0.f, TC_P, TC_MASK_STRICT_ZERO, h->hd);
+        gp.amax_a = am + AMAX_O; gp.amax_b = am + AMAX_U; gp.amax_out = am + AMAX_P;
+        CU(launch_tc_gemm(maps, gp, h->num_sms, s));
+        // P^T for the lazy-batch updates of gptaq_quantize, over the copy of U that is no longer needed
+        CU(launch_split16(h->D, n, U16, U16 + nn, n, n, n, true, SPLIT_STRICT_UPPER, 1.f, am + AMAX_P, s));
+        h->launches += 4;
+        h->stage = STAGE_P;
+        return GPTAQ_OK;
+    }
     if (h->tensor) {
         float *S[6];
         for (int i = 0; i < 6; ++i) S[i] = reinterpret_cast<float *>(h->ws + wl.s_off[i]);
@@ -915,9 +1041,29 @@ gptaq_status_t gptaq_quantize(gptaq_handle_t h, void *d_W, int w_dtype, int64_t 
     t.perm = h->act_order ? h->perm : nullptr;
     t.clip_steps = h->clip_steps; t.clip_min = h->clip_min;
     t.UT_hi = t.UT_lo = t.PT_hi = t.PT_lo = nullptr; t.EW_lo = nullptr;
-    if (h->tensor) {
-        t.UT_hi = reinterpret_cast<float *>(h->ws + wl.s_off[2]); t.UT_lo = reinterpret_cast<float *>(h->ws + wl.s_off[3]);
-        t.PT_hi = reinterpret_cast<float *>(h->ws + wl.s_off[4]); t.PT_lo = reinterpret_cast<float *>(h->ws + wl.s_off[5]);
+    // FP16-split trailing update: every block that has columns to its right goes through
+    // column_block_kernel (which writes the row-scaled fp16 operand) and the block is a whole number of
+    // 64-step K-blocks
+    const bool f16 = h->f16 && (blocksize % 64) == 0 && (group <= 0 || (group % 32) == 0) &&
+                     (reinterpret_cast<uintptr_t>(h->dead) & 3) == 0;
+    if (f16) {
+        t.UT16 = reinterpret_cast<const __half *>(h->ws + wl.s_off[0]);
+        t.PT16 = reinterpret_cast<const __half *>(h->ws + wl.s_off[1]);
+        t.EW16 = reinterpret_cast<__half *>(h->ws + wl.ew_lo_off);
+        t.row_inv = reinterpret_cast<float *>(h->ws + wl.rs_off);
+        t.amax_u = h->hd->tc_amax + AMAX_U; t.amax_p = h->hd->tc_amax + AMAX_P;
+    } else if (h->tensor) {
+        float *S[6];
+        for (int i = 0; i < 6; ++i) S[i] = reinterpret_cast<float *>(h->ws + wl.s_off[i]);
+        if (h->f16 && !h->tf32_copies) {
+            const int n = (int)h->n;
+            cudaStream_t s = static_cast<cudaStream_t>(stream);
+            CU(launch_split(h->H, n, S[2], S[3], n, n, n, true, SPLIT_UPPER, 1.f, s));
+            CU(launch_split(h->D, n, S[4], S[5], n, n, n, true, SPLIT_STRICT_UPPER, 1.f, s));
+            h->launches += 2;
+            h->tf32_copies = true;
+        }
+        t.UT_hi = S[2]; t.UT_lo = S[3]; t.PT_hi = S[4]; t.PT_lo = S[5];
         t.EW_lo = reinterpret_cast<float *>(h->ws + wl.ew_lo_off);
     }
     cudaError_t e = cudaSuccess;

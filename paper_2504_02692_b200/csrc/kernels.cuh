@@ -2,6 +2,7 @@
 // Cholesky, the per-column quantize-and-propagate loop, and helpers.
 #pragma once
 #include <cuda_bf16.h>
+#include <cuda_fp16.h>
 #include <cuda_runtime.h>
 #include <stdint.h>
 
@@ -15,11 +16,23 @@ struct StateHeader {
     float lambda;        // damp * mean(diag H / tokens)
     float inv_tokens;
     unsigned amax[2][2]; // per operand buffer: bit patterns of max|X| and max|X~ - X| of the batch converted into it
-    int pad1[22];
+    unsigned tc_amax[8]; // largest magnitudes of FP16-split operands of the float32-grade GEMMs (see tc_gemm.cuh)
+    int pad1[14];
 };
 static_assert(sizeof(StateHeader) == 128, "header size");
 
 constexpr int ST_NOT_SPD = 4, ST_NONFINITE = 5, ST_TIMEOUT = 6;
+
+// Slots of StateHeader::tc_amax: factor panels (an a-priori bound), U, dXX^T / tokens, O, P.
+enum { AMAX_PAN = 0, AMAX_U = 1, AMAX_D = 2, AMAX_O = 3, AMAX_P = 4 };
+
+// Scale of an FP16-split operand: a power of two that puts the largest magnitude into [2^13, 2^14).
+__host__ __device__ __forceinline__ float split_scale(float amax) {
+    if (!(amax > 0.f) || !isfinite(amax)) return 1.f;
+    int e;
+    frexpf(amax, &e);                 // amax = f * 2^e, f in [0.5, 1)
+    return ldexpf(1.f, 14 - e);
+}
 
 // Round to the nearest TF32 value (10 explicit mantissa bits), kept in a float.
 __device__ __forceinline__ float tf32_rn(float x) {
@@ -40,23 +53,35 @@ __global__ void __launch_bounds__(1024) diag_stats_kernel(const float *H, int n,
                                                           float damp, StateHeader *hd,
                                                           uint8_t *dead) {
     __shared__ double red[1024];
+    __shared__ float redmax[1024];
     double s = 0.0;
+    float mx = 0.f;
     for (int q = threadIdx.x; q < n; q += 1024) {
         float d = H[(int64_t)q * n + q];
         if (!isfinite(d)) record_status(hd, ST_NONFINITE, q);
         bool dd = (d == 0.f);
         dead[q] = dd ? 1 : 0;
+        const float v = dd ? 1.f : d * inv_tokens;
         s += dd ? 1.0 : (double)d * (double)inv_tokens;
+        mx = fmaxf(mx, v);
     }
     red[threadIdx.x] = s;
+    redmax[threadIdx.x] = mx;
     __syncthreads();
     for (int w = 512; w > 0; w >>= 1) {
-        if (threadIdx.x < w) red[threadIdx.x] += red[threadIdx.x + w];
+        if (threadIdx.x < w) {
+            red[threadIdx.x] += red[threadIdx.x + w];
+            redmax[threadIdx.x] = fmaxf(redmax[threadIdx.x], redmax[threadIdx.x + w]);
+        }
         __syncthreads();
     }
     if (threadIdx.x == 0) {
-        hd->lambda = (float)((double)damp * red[0] / (double)n);
+        const float lambda = (float)((double)damp * red[0] / (double)n);
+        hd->lambda = lambda;
         hd->inv_tokens = inv_tokens;
+        // every entry of row i of the factor R (H_d = R R^T) is at most sqrt(H_d,ii): the range of the
+        // factor panels is known before they exist
+        hd->tc_amax[AMAX_PAN] = __float_as_uint(sqrtf(redmax[0] + lambda));
     }
 }
 
@@ -103,6 +128,7 @@ struct FactorPanelArgs {
     float *H; int n; int b0;
     float *Rdiag;              // NB x NB (ld NB): the diagonal factor R_pp (upper, zeros below)
     float *pan_hi, *pan_lo;    // nullptr, or [n][NB]: TF32 parts of the panel rows
+    int pan_f16;               // the two arrays hold __half instead: fp16 parts of split_scale(tc_amax[AMAX_PAN]) * row
     int rows_per_cta;          // slab of step 2, a multiple of tile_rows
     int tile_rows;             // rows of the slab processed at a time: 32, 64 or 128
     StateHeader *hd;
@@ -359,7 +385,22 @@ __global__ void __launch_bounds__(FP_THREADS, 1) factor_panel_kernel(FactorPanel
                 if (4 * j4 + 2 < nv) dst[2] = v.z;
                 if (4 * j4 + 3 < nv) dst[3] = v.w;
             }
-            if (a.pan_hi) {
+            if (a.pan_hi && a.pan_f16) {
+                const float sc = split_scale(__uint_as_float(a.hd->tc_amax[AMAX_PAN]));
+                const float xs[4] = {sc * v.x, sc * v.y, sc * v.z, sc * v.w};
+                __half2 hv[2], lv[2];
+#pragma unroll
+                for (int f = 0; f < 2; ++f) {
+                    const __half h0 = __float2half_rn(xs[2 * f]), h1 = __float2half_rn(xs[2 * f + 1]);
+                    hv[f] = __halves2half2(h0, h1);
+                    lv[f] = __halves2half2(__float2half_rn(xs[2 * f] - __half2float(h0)),
+                                           __float2half_rn(xs[2 * f + 1] - __half2float(h1)));
+                }
+                __half *ph = reinterpret_cast<__half *>(a.pan_hi) + (int64_t)(r0 + i) * NB + 4 * j4;
+                __half *pl = reinterpret_cast<__half *>(a.pan_lo) + (int64_t)(r0 + i) * NB + 4 * j4;
+                *reinterpret_cast<uint2 *>(ph) = make_uint2(*reinterpret_cast<uint32_t *>(&hv[0]), *reinterpret_cast<uint32_t *>(&hv[1]));
+                *reinterpret_cast<uint2 *>(pl) = make_uint2(*reinterpret_cast<uint32_t *>(&lv[0]), *reinterpret_cast<uint32_t *>(&lv[1]));
+            } else if (a.pan_hi) {
                 const float xs[4] = {v.x, v.y, v.z, v.w};
                 float hv[4], lv[4];
 #pragma unroll
@@ -556,6 +597,13 @@ struct ColumnLoopArgs {
     int G;
     float *EW;                 // m x (2 * 32 * T): [-Err | Wpre]
     float *EW_lo;              // nullptr, or: EW receives the TF32 value of each entry and EW_lo the remainder
+    // FP16 operand for the tensor-core update (column_block_kernel only; EW_lo is null then), or nullptr:
+    // row i of [-Err | rho * Wpre] times a power of two s_i, as fp16 hi / lo parts, m x (2 * block) each;
+    // row_inv[i] = 1 / s_i.  rho = scale of U^T / scale of P^T (from the two recorded maxima) lets the two
+    // halves of the B operand keep scales of their own.
+    __half *EW16_hi, *EW16_lo;
+    float *row_inv;
+    const unsigned *amax_u, *amax_p;
     StateHeader *hd;
     float err_scale, asym_scale;   // 1 or 0: switches of the two terms of the weight update (ablation)
     const int *perm;               // nullptr, or: working column c is original column perm[c] (codes go there)
@@ -790,6 +838,12 @@ __global__ void __launch_bounds__(CB_THREADS, 1) column_block_kernel(ColumnLoopA
     const bool owner = tid < nrows;
     const int row = row0 + tid;
     if (a.group <= 0 && owner) { scale = a.scales[row]; zero = a.zeros[row]; }
+    const bool f16 = a.EW16_hi != nullptr;
+    float rho = 1.f, rmax = 0.f;
+    if (f16) {
+        const float ap = __uint_as_float(*a.amax_p);
+        rho = ap > 0.f ? split_scale(__uint_as_float(*a.amax_u)) / split_scale(ap) : 0.f;
+    }
 
     // rows [o, o + 32) of U and P of this block into buffer `buf`, by `nthr` threads starting at `t0`
     auto fetch_up = [&](int o, int buf, int t0, int nthr) {
@@ -905,6 +959,13 @@ __global__ void __launch_bounds__(CB_THREADS, 1) column_block_kernel(ColumnLoopA
                 *reinterpret_cast<float4 *>(&Wt[tid][o + 4 * k4]) = make_float4(x[4 * k4], x[4 * k4 + 1], x[4 * k4 + 2], x[4 * k4 + 3]);
                 float e4[4] = {nerr[4 * k4], nerr[4 * k4 + 1], nerr[4 * k4 + 2], nerr[4 * k4 + 3]};
                 float p4[4] = {pre[4 * k4], pre[4 * k4 + 1], pre[4 * k4 + 2], pre[4 * k4 + 3]};
+                if (f16) {
+#pragma unroll
+                    for (int f = 0; f < 4; ++f) {
+                        p4[f] *= rho;
+                        rmax = fmaxf(rmax, fmaxf(fabsf(e4[f]), fabsf(p4[f])));
+                    }
+                }
                 if (ewl) {
                     float el[4], pl[4];
 #pragma unroll
@@ -969,6 +1030,33 @@ __global__ void __launch_bounds__(CB_THREADS, 1) column_block_kernel(ColumnLoopA
         if ((reinterpret_cast<uintptr_t>(dst) & 15) == 0) *reinterpret_cast<float4 *>(dst) = v;
         else { dst[0] = v.x; dst[1] = v.y; dst[2] = v.z; dst[3] = v.w; }
         if (bad) record_status(a.hd, ST_NONFINITE, row0 + r);
+    }
+    if (f16) {
+        // this CTA's rows of [-Err | rho * Wpre], scaled row by row into the fp16 range and split
+        float *srow = St;                       // free since the last rank update
+        if (tid < rows) {
+            const float sc = owner ? split_scale(rmax) : 1.f;
+            srow[tid] = sc;
+            if (owner) a.row_inv[row] = 1.f / sc;
+        }
+        __syncthreads();                        // (also: the rows written above are visible to the whole CTA)
+        const int q = 2 * B / 4;
+        for (int idx = tid; idx < nrows * q; idx += CB_THREADS) {
+            const int r = idx / q, c4 = idx - r * q;
+            const int64_t off = (int64_t)(row0 + r) * (2 * B) + 4 * c4;
+            const float4 v = *reinterpret_cast<const float4 *>(a.EW + off);
+            const float sc = srow[r];
+            const float x[4] = {sc * v.x, sc * v.y, sc * v.z, sc * v.w};
+            __half h[4], l[4];
+#pragma unroll
+            for (int e = 0; e < 4; ++e) { h[e] = __float2half_rn(x[e]); l[e] = __float2half_rn(x[e] - __half2float(h[e])); }
+            const __half2 h01 = __halves2half2(h[0], h[1]), h23 = __halves2half2(h[2], h[3]);
+            const __half2 l01 = __halves2half2(l[0], l[1]), l23 = __halves2half2(l[2], l[3]);
+            *reinterpret_cast<uint2 *>(a.EW16_hi + off) =
+                make_uint2(*reinterpret_cast<const uint32_t *>(&h01), *reinterpret_cast<const uint32_t *>(&h23));
+            *reinterpret_cast<uint2 *>(a.EW16_lo + off) =
+                make_uint2(*reinterpret_cast<const uint32_t *>(&l01), *reinterpret_cast<const uint32_t *>(&l23));
+        }
     }
 }
 

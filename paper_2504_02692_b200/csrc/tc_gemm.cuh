@@ -16,6 +16,12 @@
 // the non-zero part of triangular operands, a B operand that switches to a second matrix
 // after k_split ([U ; P] of the lazy-batch update), and masked stores.
 //
+// The kernel exists for two operand kinds.  TF32: hi / lo are float32 arrays holding TF32 values, no
+// range limits, 32 contraction steps per 128-byte row.  FP16: hi = fp16(s x), lo = fp16(s x - hi) with a
+// power-of-two scale s per operand that puts the largest magnitude at 2^14 (split16_kernel; the scale
+// is recomputed from the recorded maximum wherever it is needed), 64 contraction steps per row and
+// tcgen05.mma.kind::f16: half the operand bytes and twice the MMA rate for the same 22 bits.
+//
 // Every wait on an mbarrier is bounded; see umma_gemm.cuh.
 #pragma once
 #include "umma_gemm.cuh"
@@ -28,7 +34,11 @@ constexpr int TB_BYTES = TBN * TBK * 4;
 constexpr int TSTAGE_BYTES = 2 * TA_BYTES + 2 * TB_BYTES;
 constexpr int TCHUNK = 4;            // K-blocks (of 32) per accumulation chain in tensor memory
 constexpr int TC_THREADS = 64 + 32 * UEPI_WARPS;
-constexpr size_t TC_SMEM = (size_t)TSTAGES * TSTAGE_BYTES + 1024 + 256;
+// staging of the "C += ..." epilogue: per column half one 128 x 32 float32 box (128-byte rows, swizzled),
+// handed to the TMA unit as a bulk reduction
+constexpr int TC_STG_BOX_BYTES = TBM * 32 * 4;
+constexpr int TC_STG_BYTES = 2 * TC_STG_BOX_BYTES;
+constexpr size_t TC_SMEM = (size_t)TSTAGES * TSTAGE_BYTES + TC_STG_BYTES + 1024 + 256;
 
 enum TcMode {
     TC_FULL = 0,
@@ -58,6 +68,12 @@ struct TcGemmArgs {
     float alpha, beta;
     int mode, mask;
     StateHeader *hd;
+    // FP16 operands: bit patterns of the operands' largest magnitudes (the B matrices share one scale);
+    // the result is divided by the two scales.  nullptr for TF32 operands.
+    const unsigned *amax_a, *amax_b;
+    const float *row_inv;            // FP16 operands with one scale per row of A: 1 / scale of row i (amax_a null)
+    unsigned *amax_out;              // if set: receives (atomicMax) the bit pattern of max |C| over what is stored
+    int c_tma;                       // beta == 1, one batch entry: C += through bulk tensor reductions (mapC)
 };
 
 struct TcTile {
@@ -65,7 +81,7 @@ struct TcTile {
     int z, i0, j0, Mz, Nz, kb0, kb1;   // K-block range [kb0, kb1)
 };
 
-__device__ __forceinline__ void tc_decode(const TcGemmArgs &a, int t, TcTile &ti) {
+__device__ __forceinline__ void tc_decode(const TcGemmArgs &a, int t, TcTile &ti, int bk) {
     const int TM = (a.M + TBM - 1) / TBM, TN = (a.N + TBN - 1) / TBN;
     const int per = TM * TN;
     ti.z = t / per;
@@ -92,8 +108,8 @@ __device__ __forceinline__ void tc_decode(const TcGemmArgs &a, int t, TcTile &ti
         case TC_TRI_LEFT: kb = ti.i0; break;
         default: break;
     }
-    ti.kb0 = kb / TBK;
-    ti.kb1 = (ke + TBK - 1) / TBK;
+    ti.kb0 = kb / bk;
+    ti.kb1 = (ke + bk - 1) / bk;
     ti.work = !ti.skip && ti.kb0 < ti.kb1;
 }
 
@@ -108,22 +124,50 @@ __device__ __forceinline__ void umma_tf32(uint32_t d_tmem, uint64_t adesc, uint6
 // kind::tf32 instruction descriptor: TF32 A and B (both K-major), fp32 D, M = 128, N = 256.
 constexpr uint32_t UMMA_IDESC_TF32 = (1u << 4) | (2u << 7) | (2u << 10) | ((TBN >> 3) << 17) | ((TBM >> 4) << 24);
 
+// C[c1 .. , c0 ..] += box in shared memory (float32 add at the memory side, one request per box)
+__device__ __forceinline__ void tma_reduce_add_2d(const CUtensorMap *map, uint32_t src, int c0, int c1) {
+    asm volatile("cp.reduce.async.bulk.tensor.2d.global.shared::cta.add.tile.bulk_group [%0, {%2, %3}], [%1];"
+                 ::"l"(reinterpret_cast<uint64_t>(map)), "r"(src), "r"(c0), "r"(c1) : "memory");
+}
+__device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
+__device__ __forceinline__ void bulk_wait_read0() { asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory"); }
+__device__ __forceinline__ void bulk_wait0() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
+__device__ __forceinline__ void fence_proxy_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+__device__ __forceinline__ void named_bar_sync(int id, int nthreads) {
+    asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(nthreads) : "memory");
+}
+// true for every thread of the named barrier if `flag` is set for any of them
+__device__ __forceinline__ bool named_bar_any(int id, int nthreads, bool flag) {
+    uint32_t r;
+    asm volatile(
+        "{\n\t.reg .pred p, q;\n\t"
+        "setp.ne.b32 p, %1, 0;\n\t"
+        "bar.red.or.pred q, %2, %3, p;\n\t"
+        "selp.b32 %0, 1, 0, q;\n\t}"
+        : "=r"(r) : "r"((uint32_t)flag), "r"(id), "r"(nthreads) : "memory");
+    return r != 0;
+}
+
+template <bool F16>
 __global__ void __launch_bounds__(TC_THREADS, 1)
 tc_gemm_kernel(const __grid_constant__ CUtensorMap mapAhi, const __grid_constant__ CUtensorMap mapAlo,
                const __grid_constant__ CUtensorMap mapBhi, const __grid_constant__ CUtensorMap mapBlo,
                const __grid_constant__ CUtensorMap mapB2hi, const __grid_constant__ CUtensorMap mapB2lo,
-               TcGemmArgs a) {
+               const __grid_constant__ CUtensorMap mapC, TcGemmArgs a) {
+    constexpr int BK = F16 ? 2 * TBK : TBK;        // contraction steps per K-block (one 128-byte row)
+    constexpr int KSTEP = F16 ? 16 : 8;            // contraction steps per MMA (32 bytes)
     extern __shared__ uint8_t smem_raw[];
     const uint32_t raw = smem_u32(smem_raw);
     const uint32_t base = (raw + 1023u) & ~1023u;
     uint8_t *aligned = smem_raw + (base - raw);
-    const uint32_t bar0 = base + TSTAGES * TSTAGE_BYTES;
+    const uint32_t stg0 = base + TSTAGES * TSTAGE_BYTES;
+    const uint32_t bar0 = stg0 + TC_STG_BYTES;
     // barrier slots (8 bytes each): full[2], empty[2], tfull[2], tempty[2]; then tmem slot, abort flag
     auto full_bar = [&](int s) { return bar0 + 8u * s; };
     auto empty_bar = [&](int s) { return bar0 + 8u * (TSTAGES + s); };
     auto tfull_bar = [&](int b) { return bar0 + 8u * (2 * TSTAGES + b); };
     auto tempty_bar = [&](int b) { return bar0 + 8u * (2 * TSTAGES + 2 + b); };
-    volatile uint32_t *tmem_slot = reinterpret_cast<volatile uint32_t *>(aligned + TSTAGES * TSTAGE_BYTES + 8 * (2 * TSTAGES + 4));
+    volatile uint32_t *tmem_slot = reinterpret_cast<volatile uint32_t *>(aligned + TSTAGES * TSTAGE_BYTES + TC_STG_BYTES + 8 * (2 * TSTAGES + 4));
     volatile int *abort_flag = reinterpret_cast<volatile int *>(tmem_slot + 1);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -152,7 +196,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap mapAhi, const __grid_constant
             bool ok = true;
             TcTile ti;
             for (int t = blockIdx.x; t < ntiles && ok; t += gridDim.x) {
-                tc_decode(a, t, ti);
+                tc_decode(a, t, ti, BK);
                 if (!ti.work) continue;
                 const int arow = a.a_row0 + ti.z * a.a_row_bs + ti.i0;
                 const int brow = a.b_row0 + ti.z * a.b_row_bs + ti.j0;
@@ -160,7 +204,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap mapAhi, const __grid_constant
                 for (int kb = ti.kb0; kb < ti.kb1; ++kb) {
                     if (!mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag)) { ok = false; break; }
                     const uint32_t s0 = base + stage * TSTAGE_BYTES;
-                    const int k = kb * TBK;
+                    const int k = kb * BK;
                     const bool second = a.k_split > 0 && k >= a.k_split;
                     mbar_expect_tx(full_bar(stage), TSTAGE_BYTES);
                     tma_load_2d(s0, &mapAhi, ak0 + k, arow, full_bar(stage));
@@ -190,7 +234,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap mapAhi, const __grid_constant
             bool ok = true;
             TcTile ti;
             for (int t = blockIdx.x; t < ntiles && ok; t += gridDim.x) {
-                tc_decode(a, t, ti);
+                tc_decode(a, t, ti, BK);
                 if (!ti.work) continue;
                 for (int kc = ti.kb0; kc < ti.kb1 && ok; kc += TCHUNK) {
                     const uint32_t buf = ccount & 1u, cphase = (ccount >> 1) & 1u;
@@ -206,16 +250,17 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap mapAhi, const __grid_constant
                         const uint64_t bhi = make_kmajor_desc(s0 + 2 * TA_BYTES);
                         const uint64_t blo = make_kmajor_desc(s0 + 2 * TA_BYTES + TB_BYTES);
                         // small terms first, the hi * hi term last
+                        auto mma = [&](uint64_t ad, uint64_t bd, uint32_t accumulate) {
+                            if (F16) umma_f16(d_tmem, ad, bd, UMMA_IDESC_F16, accumulate);
+                            else umma_tf32(d_tmem, ad, bd, UMMA_IDESC_TF32, accumulate);
+                        };
 #pragma unroll
-                        for (int k = 0; k < TBK / 8; ++k)
-                            umma_tf32(d_tmem, alo + (uint64_t)(k * 2), bhi + (uint64_t)(k * 2), UMMA_IDESC_TF32,
-                                      (kb != kc || k != 0) ? 1u : 0u);
+                        for (int k = 0; k < BK / KSTEP; ++k)
+                            mma(alo + (uint64_t)(k * 2), bhi + (uint64_t)(k * 2), (kb != kc || k != 0) ? 1u : 0u);
 #pragma unroll
-                        for (int k = 0; k < TBK / 8; ++k)
-                            umma_tf32(d_tmem, ahi + (uint64_t)(k * 2), blo + (uint64_t)(k * 2), UMMA_IDESC_TF32, 1u);
+                        for (int k = 0; k < BK / KSTEP; ++k) mma(ahi + (uint64_t)(k * 2), blo + (uint64_t)(k * 2), 1u);
 #pragma unroll
-                        for (int k = 0; k < TBK / 8; ++k)
-                            umma_tf32(d_tmem, ahi + (uint64_t)(k * 2), bhi + (uint64_t)(k * 2), UMMA_IDESC_TF32, 1u);
+                        for (int k = 0; k < BK / KSTEP; ++k) mma(ahi + (uint64_t)(k * 2), bhi + (uint64_t)(k * 2), 1u);
                         umma_commit(empty_bar(stage));
                         if (++stage == TSTAGES) { stage = 0; phase ^= 1u; }
                     }
@@ -232,9 +277,15 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap mapAhi, const __grid_constant
         uint32_t ccount = 0;
         bool ok = true;
         float acc[TBN / 2];
+        float out_max = 0.f;
+        float op_scale = 1.f;            // 1 / (scale of A * scale of B), without the per-row part
+        if (F16) {
+            if (a.amax_a) op_scale /= split_scale(__uint_as_float(*a.amax_a));
+            if (a.amax_b) op_scale /= split_scale(__uint_as_float(*a.amax_b));
+        }
         TcTile ti;
         for (int t = blockIdx.x; t < ntiles && ok; t += gridDim.x) {
-            tc_decode(a, t, ti);
+            tc_decode(a, t, ti, BK);
             if (ti.skip && !ti.zero_fill) continue;
 #pragma unroll
             for (int i = 0; i < TBN / 2; ++i) acc[i] = 0.f;
@@ -257,13 +308,51 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap mapAhi, const __grid_constant
                     if (lane == 0) mbar_arrive(tempty_bar(buf));
                     ++ccount;
                 }
-                if (!ok) break;
+                if (!a.c_tma && !ok) break;
             }
             const int row = ti.i0 + quarter * 32 + lane;           // within the batch entry
             const int col0 = ti.j0 + half * (TBN / 2);
+            if (a.c_tma) {
+                // C += alpha * acc through shared memory and bulk tensor reductions: the four warps of a
+                // column half fill one 128 x 32 box at a time (row = TMEM lane, 16-byte chunks swizzled
+                // like the tensor map's 128-byte mode), one thread hands it to the TMA unit.  Rows and
+                // columns beyond the matrix are clipped by the tensor map.
+                if (named_bar_any(1 + half, 128, !ok)) { ok = false; break; }       // a wait gave up: all leave together
+                float alpha = a.alpha;
+                if (F16) alpha *= (a.row_inv && row < ti.Mz) ? op_scale * a.row_inv[row] : op_scale;
+                const bool issuer = quarter == 2 && lane == 0;                       // first warp of the half
+                const int r_in = quarter * 32 + lane;
+                const uint32_t box = stg0 + half * TC_STG_BOX_BYTES;
+#pragma unroll
+                for (int g = 0; g < TBN / 2 / 32; ++g) {
+                    if (col0 + 32 * g >= ti.Nz) break;
+                    if (issuer) bulk_wait_read0();                                   // the box has been read out
+                    named_bar_sync(1 + half, 128);
+#pragma unroll
+                    for (int j = 0; j < 8; ++j) {
+                        float v[4];
+#pragma unroll
+                        for (int e = 0; e < 4; ++e) {
+                            v[e] = alpha * acc[32 * g + 4 * j + e];
+                            if (a.mask == TC_MASK_UPPER_KEEP && col0 + 32 * g + 4 * j + e < row) v[e] = 0.f;
+                        }
+                        const uint32_t dst = box + r_in * 128 + ((j ^ (r_in & 7)) << 4);
+                        asm volatile("st.shared.v4.f32 [%0], {%1, %2, %3, %4};" ::"r"(dst), "f"(v[0]), "f"(v[1]), "f"(v[2]), "f"(v[3]) : "memory");
+                    }
+                    fence_proxy_async_smem();
+                    named_bar_sync(1 + half, 128);
+                    if (issuer) {
+                        tma_reduce_add_2d(&mapC, box, col0 + 32 * g, ti.i0);
+                        bulk_commit();
+                    }
+                }
+                continue;
+            }
             if (row >= ti.Mz) continue;
             float *cp = a.C + (long long)ti.z * a.c_bstride + (long long)row * a.ldc + col0;
-            const float alpha = a.alpha, beta = a.beta;
+            const float beta = a.beta;
+            float alpha = a.alpha;
+            if (F16) alpha *= a.row_inv ? op_scale * a.row_inv[(long long)ti.z * a.M + row] : op_scale;
             const bool vec_ok = (reinterpret_cast<uintptr_t>(cp) & 15) == 0;
 #pragma unroll
             for (int q = 0; q < TBN / 2 / 4; ++q) {
@@ -275,6 +364,10 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap mapAhi, const __grid_constant
                 if (a.mask == TC_MASK_STRICT_ZERO) {
 #pragma unroll
                     for (int e = 0; e < 4; ++e) if (c + e <= row) v[e] = 0.f;
+                }
+                if (a.amax_out) {
+#pragma unroll
+                    for (int e = 0; e < 4; ++e) if (c + e < ti.Nz) out_max = fmaxf(out_max, fabsf(v[e]));
                 }
                 const bool keep_all = a.mask != TC_MASK_UPPER_KEEP || c >= row;
                 if (vec_ok && c + 3 < ti.Nz && keep_all) {
@@ -300,6 +393,12 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap mapAhi, const __grid_constant
                     }
                 }
             }
+        }
+        if (a.c_tma) bulk_wait0();          // (only the issuing threads have groups outstanding)
+        if (a.amax_out) {
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) out_max = fmaxf(out_max, __shfl_xor_sync(0xffffffffu, out_max, o));
+            if (lane == 0 && out_max > 0.f) atomicMax(a.amax_out, __float_as_uint(out_max));
         }
     }
 
@@ -365,6 +464,133 @@ __global__ void __launch_bounds__(256) split_kernel(SplitArgs a) {
             if (r < rows && c < cols) {
                 hi[(long long)c * a.ldd + r] = th[tx][cc];
                 lo[(long long)c * a.ldd + r] = tl[tx][cc];
+            }
+        }
+    }
+}
+
+// ---------------------------------------------------------------------------
+// FP16 operand preparation.  absmax_kernel (a CTA per row, strided) records max |scale * src| over the
+// (masked) region as a float bit pattern (atomicMax on the bits orders non-negative floats);
+// split16_kernel then writes
+// hi = fp16(s x), lo = fp16(s x - hi), x = scale * src, s = split_scale(recorded maximum), with the
+// same options as split_kernel.  The slot has to be zeroed before the first absmax_kernel into it;
+// several matrices that share a scale are reduced into the same slot.
+// ---------------------------------------------------------------------------
+__global__ void __launch_bounds__(256) absmax_kernel(const float *src, long long lds, int rows, int cols, int mask,
+                                                     float scale, unsigned *slot) {
+    __shared__ float red[8];
+    float m = 0.f;
+    const bool vec = (lds & 3) == 0 && (reinterpret_cast<uintptr_t>(src) & 15) == 0;
+    for (int r = blockIdx.x; r < rows; r += gridDim.x) {
+        const int cb = mask == SPLIT_ALL ? 0 : (mask == SPLIT_UPPER ? r : r + 1);     // first column kept
+        const float *row = src + (long long)r * lds;
+        if (vec) {
+            for (int c4 = (cb >> 2) + threadIdx.x; 4 * c4 < cols; c4 += 256) {
+                const int c = 4 * c4;
+                float v[4] = {0.f, 0.f, 0.f, 0.f};
+                if (c + 3 < cols) {
+                    const float4 q = *reinterpret_cast<const float4 *>(row + c);
+                    v[0] = q.x; v[1] = q.y; v[2] = q.z; v[3] = q.w;
+                } else {
+                    for (int e = 0; c + e < cols; ++e) v[e] = row[c + e];
+                }
+#pragma unroll
+                for (int e = 0; e < 4; ++e) if (c + e >= cb) m = fmaxf(m, fabsf(v[e]));
+            }
+        } else {
+            for (int c = cb + threadIdx.x; c < cols; c += 256) m = fmaxf(m, fabsf(row[c]));
+        }
+    }
+    m *= fabsf(scale);
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
+    if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = m;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        for (int w = 1; w < 8; ++w) m = fmaxf(m, red[w]);
+        if (m > 0.f) atomicMax(slot, __float_as_uint(m));
+    }
+}
+
+struct Split16Args {
+    const float *src; long long lds;
+    __half *hi, *lo; long long ldd;
+    int rows, cols;
+    int transpose, mask;
+    float scale;
+    const unsigned *amax;
+};
+
+__device__ __forceinline__ void split16_pack(const float (&x)[4], uint2 &hi, uint2 &lo) {
+    __half h[4], l[4];
+#pragma unroll
+    for (int e = 0; e < 4; ++e) { h[e] = __float2half_rn(x[e]); l[e] = __float2half_rn(x[e] - __half2float(h[e])); }
+    const __half2 h01 = __halves2half2(h[0], h[1]), h23 = __halves2half2(h[2], h[3]);
+    const __half2 l01 = __halves2half2(l[0], l[1]), l23 = __halves2half2(l[2], l[3]);
+    hi = make_uint2(*reinterpret_cast<const uint32_t *>(&h01), *reinterpret_cast<const uint32_t *>(&h23));
+    lo = make_uint2(*reinterpret_cast<const uint32_t *>(&l01), *reinterpret_cast<const uint32_t *>(&l23));
+}
+
+// 64 x 64 tiles; a thread handles four consecutive source columns (plain) or four consecutive source
+// rows of one column (transposed), so that every store is 8 bytes.  Needs lds, ldd multiples of 4 and
+// 16- / 8-byte aligned bases (the host checks); rows and cols are arbitrary.
+__global__ void __launch_bounds__(256) split16_kernel(Split16Args a) {
+    __shared__ float tile[64][65];
+    const int r0 = blockIdx.y * 64, c0 = blockIdx.x * 64;
+    const float s = a.scale * split_scale(__uint_as_float(*a.amax));
+    const int tq = threadIdx.x & 15, ty = threadIdx.x >> 4;        // 16 quads x 16 rows
+    for (int rr = ty; rr < 64; rr += 16) {
+        const int r = r0 + rr, c = c0 + 4 * tq;
+        float x[4] = {0.f, 0.f, 0.f, 0.f};
+        if (r < a.rows && c < a.cols) {
+            const float *sp = a.src + (long long)r * a.lds + c;
+            if (c + 3 < a.cols) {
+                const float4 q = *reinterpret_cast<const float4 *>(sp);
+                x[0] = q.x; x[1] = q.y; x[2] = q.z; x[3] = q.w;
+            } else {
+                for (int e = 0; c + e < a.cols; ++e) x[e] = sp[e];
+            }
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+                const bool keep = a.mask == SPLIT_ALL || (a.mask == SPLIT_UPPER ? c + e >= r : c + e > r);
+                x[e] = keep ? s * x[e] : 0.f;
+            }
+        }
+        if (!a.transpose) {
+            if (r < a.rows && c < a.cols) {
+                uint2 hi, lo;
+                split16_pack(x, hi, lo);
+                __half *ph = a.hi + (long long)r * a.ldd + c, *pl = a.lo + (long long)r * a.ldd + c;
+                if (c + 3 < a.cols) {
+                    *reinterpret_cast<uint2 *>(ph) = hi;
+                    *reinterpret_cast<uint2 *>(pl) = lo;
+                } else {
+                    const __half *hh = reinterpret_cast<const __half *>(&hi), *ll = reinterpret_cast<const __half *>(&lo);
+                    for (int e = 0; c + e < a.cols; ++e) { ph[e] = hh[e]; pl[e] = ll[e]; }
+                }
+            }
+        } else {
+#pragma unroll
+            for (int e = 0; e < 4; ++e) tile[rr][4 * tq + e] = x[e];
+        }
+    }
+    if (a.transpose) {
+        __syncthreads();
+        // destination row = source column c, destination columns = source rows r0 + 4 * tq ..
+        for (int cc = ty; cc < 64; cc += 16) {
+            const int c = c0 + cc, r = r0 + 4 * tq;
+            if (c >= a.cols || r >= a.rows) continue;
+            const float x[4] = {tile[4 * tq][cc], tile[4 * tq + 1][cc], tile[4 * tq + 2][cc], tile[4 * tq + 3][cc]};
+            uint2 hi, lo;
+            split16_pack(x, hi, lo);
+            __half *ph = a.hi + (long long)c * a.ldd + r, *pl = a.lo + (long long)c * a.ldd + r;
+            if (r + 3 < a.rows) {
+                *reinterpret_cast<uint2 *>(ph) = hi;
+                *reinterpret_cast<uint2 *>(pl) = lo;
+            } else {
+                const __half *hh = reinterpret_cast<const __half *>(&hi), *ll = reinterpret_cast<const __half *>(&lo);
+                for (int e = 0; r + e < a.rows; ++e) { ph[e] = hh[e]; pl[e] = ll[e]; }
             }
         }
     }
