@@ -88,10 +88,15 @@ inline bool tc_shape_ok(int64_t n) { return n >= TC_MIN_N && (n % 4) == 0; }
 struct WsLayout {
     size_t t_off, rinv_off;
     size_t s_off[6];        // split operand matrices (n x n each): S1 hi/lo, S2 hi/lo, S3 hi/lo
-    size_t pan_off[2];      // split copy of one factor panel (n x 128), hi/lo
+    size_t pan_off[2];      // split copy of factor panels, hi/lo: n x 128 float32 (TF32) or n x SUPER_NB fp16
     size_t ew_off, ew_lo_off, rs_off, total;   // [-Err | Wpre] (m x 2B), its second part, one scale per row
     bool tensor;
 };
+
+// FP16-split factorisation: panels are grouped in super-panels of SUPER_NB columns; inside a super-panel
+// the rank-128 update only touches the super-panel's remaining columns, the rest of the matrix receives
+// one rank-SUPER_NB update per super-panel (8x less read-modify-write traffic, longer contractions)
+constexpr int SUPER_NB = 8 * NB;
 
 WsLayout ws_layout(int64_t n, int64_t m_max, int blocksize) {
     WsLayout w;
@@ -102,7 +107,8 @@ WsLayout ws_layout(int64_t n, int64_t m_max, int blocksize) {
     w.rinv_off = w.t_off + mat;
     size_t off = w.rinv_off + round_up(nb * NB * NB * sizeof(float), ALIGN);
     for (int i = 0; i < 6; ++i) { w.s_off[i] = off; if (w.tensor) off += mat; }
-    for (int i = 0; i < 2; ++i) { w.pan_off[i] = off; if (w.tensor) off += round_up((size_t)n * NB * sizeof(float), ALIGN); }
+    const size_t pan = std::max((size_t)n * NB * sizeof(float), (size_t)n * SUPER_NB * sizeof(__half));
+    for (int i = 0; i < 2; ++i) { w.pan_off[i] = off; if (w.tensor) off += round_up(pan, ALIGN); }
     const size_t ew = round_up((size_t)m_max * 2 * (size_t)blocksize * sizeof(float), ALIGN);
     w.ew_off = off;
     w.ew_lo_off = off + ew;
@@ -835,16 +841,19 @@ gptaq_status_t gptaq_factor(gptaq_handle_t h, float damp, gptaq_stream_t stream)
     float *pan_hi = h->tensor ? reinterpret_cast<float *>(h->ws + wl.pan_off[0]) : nullptr;
     float *pan_lo = h->tensor ? reinterpret_cast<float *>(h->ws + wl.pan_off[1]) : nullptr;
     TcMaps pan_maps;
+    const int pan_ld = h->f16 ? SUPER_NB : NB;
     if (h->tensor) {
-        const SplitOperand pan{pan_hi, pan_lo, n, NB, NB, h->f16};
+        const SplitOperand pan{pan_hi, pan_lo, n, pan_ld, pan_ld, h->f16};
         if (!make_tc_maps(&pan_maps, pan, pan, nullptr)) { h->cuda_error = "cuTensorMapEncodeTiled failed"; return GPTAQ_ERR_CUDA; }
     }
     for (int p = nb - 1; p >= 0; --p) {
         const int b0 = p * NB;
+        const int s0 = h->f16 ? b0 / SUPER_NB * SUPER_NB : b0;      // first column of this panel's super-panel
         // diagonal block (factor + inverse) and the panel above it: R[0:b0, blk] = A[0:b0, blk] inv(R_pp)^T
         FactorPanelArgs fa;
         fa.H = H; fa.n = n; fa.b0 = b0; fa.Rdiag = Rinv + (size_t)p * NB * NB;
         fa.pan_hi = pan_hi; fa.pan_lo = pan_lo; fa.pan_f16 = h->f16 ? 1 : 0; fa.hd = h->hd;
+        fa.pan_ld = pan_ld; fa.pan_col0 = b0 - s0;
         // rows above the block in tiles of 32, 64 or 128 rows: the smallest tile that still gives every
         // SM at most one tile spreads a short panel over more SMs (the diagonal block is refactored by
         // every CTA either way)
@@ -856,10 +865,27 @@ gptaq_status_t gptaq_factor(gptaq_handle_t h, float damp, gptaq_stream_t stream)
         factor_panel_kernel<<<fgrid, FP_THREADS, FP_SMEM, s>>>(fa);
         LAUNCHED();
         if (p == 0) break;
+        if (h->f16 && b0 >= TC_MIN_N) {
+            const unsigned *am = h->hd->tc_amax + AMAX_PAN;
+            if (b0 > s0) {
+                // inside the super-panel: A[0:b0, s0:b0] -= R[0:b0, blk] R[s0:b0, blk]^T  (upper part)
+                TcGemmArgs g = tc_args(H + s0, n, b0, b0 - s0, NB, -1.f, 1.f, TC_UPPER_TILES, TC_MASK_UPPER_KEEP, h->hd);
+                g.diag_off = s0; g.a_k0 = g.b_k0 = b0 - s0; g.b_row0 = s0;
+                g.amax_a = g.amax_b = am;
+                CU(launch_tc_gemm(pan_maps, g, h->num_sms, s));
+            } else {
+                // super-panel [s0, s1) done: A[0:s0, 0:s0] -= R[0:s0, s0:s1] R[0:s0, s0:s1]^T  (upper part)
+                const int s1 = std::min(s0 + SUPER_NB, nb * NB);
+                TcGemmArgs g = tc_args(H, n, s0, s0, s1 - s0, -1.f, 1.f, TC_UPPER_TILES, TC_MASK_UPPER_KEEP, h->hd);
+                g.amax_a = g.amax_b = am;
+                CU(launch_tc_gemm(pan_maps, g, h->num_sms, s));
+            }
+            h->launches++;
+            continue;
+        }
         // A[0:b0, 0:b0] -= R[0:b0, blk] R[0:b0, blk]^T  (upper part)
         if (h->tensor && b0 >= TC_MIN_N) {
             TcGemmArgs g = tc_args(H, n, b0, b0, NB, -1.f, 1.f, TC_UPPER_TILES, TC_MASK_UPPER_KEEP, h->hd);
-            if (h->f16) g.amax_a = g.amax_b = h->hd->tc_amax + AMAX_PAN;
             CU(launch_tc_gemm(pan_maps, g, h->num_sms, s));
             h->launches++;
         } else {

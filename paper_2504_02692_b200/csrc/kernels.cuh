@@ -128,7 +128,8 @@ struct FactorPanelArgs {
     float *H; int n; int b0;
     float *Rdiag;              // NB x NB (ld NB): the diagonal factor R_pp (upper, zeros below)
     float *pan_hi, *pan_lo;    // nullptr, or [n][NB]: TF32 parts of the panel rows
-    int pan_f16;               // the two arrays hold __half instead: fp16 parts of split_scale(tc_amax[AMAX_PAN]) * row
+    int pan_f16;               // the two arrays hold __half instead: fp16 parts of split_scale(tc_amax[AMAX_PAN]) * row,
+    int pan_ld, pan_col0;      //   row pitch pan_ld, this panel at columns pan_col0 .. + NB (several panels side by side)
     int rows_per_cta;          // slab of step 2, a multiple of tile_rows
     int tile_rows;             // rows of the slab processed at a time: 32, 64 or 128
     StateHeader *hd;
@@ -396,8 +397,8 @@ __global__ void __launch_bounds__(FP_THREADS, 1) factor_panel_kernel(FactorPanel
                     lv[f] = __halves2half2(__float2half_rn(xs[2 * f] - __half2float(h0)),
                                            __float2half_rn(xs[2 * f + 1] - __half2float(h1)));
                 }
-                __half *ph = reinterpret_cast<__half *>(a.pan_hi) + (int64_t)(r0 + i) * NB + 4 * j4;
-                __half *pl = reinterpret_cast<__half *>(a.pan_lo) + (int64_t)(r0 + i) * NB + 4 * j4;
+                __half *ph = reinterpret_cast<__half *>(a.pan_hi) + (int64_t)(r0 + i) * a.pan_ld + a.pan_col0 + 4 * j4;
+                __half *pl = reinterpret_cast<__half *>(a.pan_lo) + (int64_t)(r0 + i) * a.pan_ld + a.pan_col0 + 4 * j4;
                 *reinterpret_cast<uint2 *>(ph) = make_uint2(*reinterpret_cast<uint32_t *>(&hv[0]), *reinterpret_cast<uint32_t *>(&hv[1]));
                 *reinterpret_cast<uint2 *>(pl) = make_uint2(*reinterpret_cast<uint32_t *>(&lv[0]), *reinterpret_cast<uint32_t *>(&lv[1]));
             } else if (a.pan_hi) {

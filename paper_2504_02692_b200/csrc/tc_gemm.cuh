@@ -42,7 +42,7 @@ constexpr size_t TC_SMEM = (size_t)TSTAGES * TSTAGE_BYTES + TC_STG_BYTES + 1024 
 
 enum TcMode {
     TC_FULL = 0,
-    TC_UPPER_TILES = 1,   // tiles entirely below the diagonal are skipped
+    TC_UPPER_TILES = 1,   // tiles entirely below the diagonal (column j + diag_off = row i) are skipped
     TC_O = 2,             // C[i][a] = sum_{k >= a} ..., lower tiles skipped
     TC_P = 3,             // C[i][j] = sum_{i <= k < j + tile} ..., lower tiles zero-filled
     TC_TRI_RIGHT = 4,     // B upper triangular: k <= j
@@ -50,7 +50,7 @@ enum TcMode {
 };
 enum TcMask {
     TC_MASK_NONE = 0,
-    TC_MASK_UPPER_KEEP = 1,     // elements with j < i are left untouched
+    TC_MASK_UPPER_KEEP = 1,     // elements with j + diag_off < i are left untouched
     TC_MASK_STRICT_ZERO = 2     // elements with j <= i are written as 0
 };
 
@@ -74,6 +74,7 @@ struct TcGemmArgs {
     const float *row_inv;            // FP16 operands with one scale per row of A: 1 / scale of row i (amax_a null)
     unsigned *amax_out;              // if set: receives (atomicMax) the bit pattern of max |C| over what is stored
     int c_tma;                       // beta == 1, one batch entry: C += through bulk tensor reductions (mapC)
+    int diag_off;                    // C is a block of columns of a square matrix: its column j is column j + diag_off there
 };
 
 struct TcTile {
@@ -99,7 +100,7 @@ __device__ __forceinline__ void tc_decode(const TcGemmArgs &a, int t, TcTile &ti
     ti.zero_fill = false;
     int kb = 0, ke = Kz;
     switch (a.mode) {
-        case TC_UPPER_TILES: if (ti.i0 >= ti.j0 + TBN) ti.skip = true; break;
+        case TC_UPPER_TILES: if (ti.i0 >= ti.j0 + a.diag_off + TBN) ti.skip = true; break;
         case TC_O: if (ti.i0 >= ti.j0 + TBN) ti.skip = true; kb = ti.j0; break;
         case TC_P:
             if (!ti.skip && ti.i0 >= ti.j0 + TBN) { ti.skip = true; ti.zero_fill = true; }
@@ -334,7 +335,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap mapAhi, const __grid_constant
 #pragma unroll
                         for (int e = 0; e < 4; ++e) {
                             v[e] = alpha * acc[32 * g + 4 * j + e];
-                            if (a.mask == TC_MASK_UPPER_KEEP && col0 + 32 * g + 4 * j + e < row) v[e] = 0.f;
+                            if (a.mask == TC_MASK_UPPER_KEEP && col0 + 32 * g + 4 * j + e + a.diag_off < row) v[e] = 0.f;
                         }
                         const uint32_t dst = box + r_in * 128 + ((j ^ (r_in & 7)) << 4);
                         asm volatile("st.shared.v4.f32 [%0], {%1, %2, %3, %4};" ::"r"(dst), "f"(v[0]), "f"(v[1]), "f"(v[2]), "f"(v[3]) : "memory");
@@ -369,7 +370,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap mapAhi, const __grid_constant
 #pragma unroll
                     for (int e = 0; e < 4; ++e) if (c + e < ti.Nz) out_max = fmaxf(out_max, fabsf(v[e]));
                 }
-                const bool keep_all = a.mask != TC_MASK_UPPER_KEEP || c >= row;
+                const bool keep_all = a.mask != TC_MASK_UPPER_KEEP || c + a.diag_off >= row;
                 if (vec_ok && c + 3 < ti.Nz && keep_all) {
                     if (beta == 1.f) {
                         // each element belongs to exactly one thread per launch: a reduction without
@@ -388,7 +389,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap mapAhi, const __grid_constant
 #pragma unroll
                     for (int e = 0; e < 4; ++e) {
                         if (c + e >= ti.Nz) continue;
-                        if (a.mask == TC_MASK_UPPER_KEEP && c + e < row) continue;
+                        if (a.mask == TC_MASK_UPPER_KEEP && c + e + a.diag_off < row) continue;
                         cp[4 * q + e] = (beta != 0.f) ? fmaf(beta, cp[4 * q + e], v[e]) : v[e];
                     }
                 }
