@@ -89,7 +89,9 @@ struct WsLayout {
     size_t t_off, rinv_off;
     size_t s_off[6];        // split operand matrices (n x n each): S1 hi/lo, S2 hi/lo, S3 hi/lo
     size_t pan_off[2];      // split copy of factor panels, hi/lo: n x 128 float32 (TF32) or n x SUPER_NB fp16
-    size_t ew_off, ew_lo_off, rs_off, total;   // [-Err | Wpre] (m x 2B), its second part, one scale per row
+    // [-Err | Wpre]: float32 (m x 2B, or m x 2 * QSUPER * B for the FP16-split update), second part
+    // (TF32 remainder, or the fp16 hi / lo parts of the wide matrix), fp16 hi / lo of one block, row scales
+    size_t ew_off, ew_lo_off, ew16_off, rs_off, total;
     bool tensor;
 };
 
@@ -97,6 +99,9 @@ struct WsLayout {
 // the rank-128 update only touches the super-panel's remaining columns, the rest of the matrix receives
 // one rank-SUPER_NB update per super-panel (8x less read-modify-write traffic, longer contractions)
 constexpr int SUPER_NB = 8 * NB;
+// The lazy-batch update of gptaq_quantize likewise: QSUPER blocks form a super-block; a block's errors
+// are applied to the rest of its super-block at once and to everything beyond once per super-block.
+constexpr int QSUPER = 8;
 
 WsLayout ws_layout(int64_t n, int64_t m_max, int blocksize) {
     WsLayout w;
@@ -109,11 +114,14 @@ WsLayout ws_layout(int64_t n, int64_t m_max, int blocksize) {
     for (int i = 0; i < 6; ++i) { w.s_off[i] = off; if (w.tensor) off += mat; }
     const size_t pan = std::max((size_t)n * NB * sizeof(float), (size_t)n * SUPER_NB * sizeof(__half));
     for (int i = 0; i < 2; ++i) { w.pan_off[i] = off; if (w.tensor) off += round_up(pan, ALIGN); }
-    const size_t ew = round_up((size_t)m_max * 2 * (size_t)blocksize * sizeof(float), ALIGN);
+    const bool f16 = w.tensor && (n % 8) == 0;
+    const size_t ew1 = round_up((size_t)m_max * 2 * (size_t)blocksize * sizeof(float), ALIGN);
+    const size_t ew = f16 ? QSUPER * ew1 : ew1;
     w.ew_off = off;
     w.ew_lo_off = off + ew;
-    w.rs_off = off + (w.tensor ? 2 * ew : ew);
-    w.total = w.rs_off + (w.tensor ? round_up((size_t)m_max * sizeof(float), ALIGN) : 0);
+    w.ew16_off = off + (w.tensor ? 2 * ew : ew);
+    w.rs_off = w.ew16_off + (f16 ? ew1 : 0);
+    w.total = w.rs_off + (f16 ? round_up(2 * (size_t)m_max * sizeof(float), ALIGN) : 0);
     return w;
 }
 
@@ -439,6 +447,10 @@ struct QuantizeTarget {
     const __half *UT16 = nullptr, *PT16 = nullptr;
     __half *EW16 = nullptr;
     float *row_inv = nullptr;
+    // ... in super-blocks: EW is then m x 2 * QSUPER * B wide; EWS16 its fp16 hi / lo parts (lo = hi +
+    // m * 2 * QSUPER * B) with the row scales row_inv_s
+    __half *EWS16 = nullptr;
+    float *row_inv_s = nullptr;
     const unsigned *amax_u = nullptr, *amax_p = nullptr;
     int terms = GPTAQ_TERM_ERR | GPTAQ_TERM_ASYM;   // which terms of the weight update are applied
     const int *perm = nullptr;                      // act_order: working column c is the caller's column perm[c]
@@ -513,12 +525,17 @@ gptaq_status_t quantize_core(const QuantizeTarget &t, void *d_W, int w_dtype, in
 
     const bool tensor16 = t.EW16 != nullptr;
     const bool tensor = tensor16 || t.EW_lo != nullptr;
-    TcMaps maps;
+    TcMaps maps, maps_super;
+    const int SBW = QSUPER * blocksize;           // super-block width (FP16-split update)
     if (tensor16) {
         const size_t nn = (size_t)n * n, me = (size_t)m * 2 * blocksize;
         const SplitOperand A{t.EW16, t.EW16 + me, m, 2 * blocksize, 2 * blocksize, true};
+        const SplitOperand AS{t.EWS16, t.EWS16 + (size_t)m * 2 * SBW, m, 2 * SBW, 2 * SBW, true};
         const SplitOperand B{t.UT16, t.UT16 + nn, n, n, n, true}, B2{t.PT16, t.PT16 + nn, n, n, n, true};
-        if (!make_tc_maps(&maps, A, B, &B2)) { *err = cudaErrorUnknown; return GPTAQ_ERR_CUDA; }
+        if (!make_tc_maps(&maps, A, B, &B2) || !make_tc_maps(&maps_super, AS, B, &B2)) {
+            *err = cudaErrorUnknown;
+            return GPTAQ_ERR_CUDA;
+        }
     } else if (tensor) {
         const SplitOperand A{EW, t.EW_lo, m, 2 * blocksize, 2 * blocksize};
         const SplitOperand B{t.UT_hi, t.UT_lo, n, n, n}, B2{t.PT_hi, t.PT_lo, n, n, n};
@@ -530,23 +547,49 @@ gptaq_status_t quantize_core(const QuantizeTarget &t, void *d_W, int w_dtype, in
         a.i0 = i0; a.bw = std::min(blocksize, n - i0);
         a.bits = bits; a.group = group; a.sym = sym;
         a.codes = d_codes; a.scales = d_scales; a.zeros = d_zeros; a.G = G; a.EW = EW; a.EW_lo = tensor16 ? nullptr : t.EW_lo; a.hd = t.hd;
+        a.ew_ld = 2 * blocksize; a.ew_pre = blocksize;
         a.EW16_hi = tensor16 ? t.EW16 : nullptr; a.EW16_lo = tensor16 ? t.EW16 + (size_t)m * 2 * blocksize : nullptr;
         a.row_inv = t.row_inv; a.amax_u = t.amax_u; a.amax_p = t.amax_p;
         a.perm = t.perm; a.clip_steps = t.clip_steps; a.clip_min = t.clip_min; a.err_scale = (t.terms & GPTAQ_TERM_ERR) ? 1.f : 0.f; a.asym_scale = (t.terms & GPTAQ_TERM_ASYM) ? 1.f : 0.f;
         const bool fast = a.bw == blocksize && (group <= 0 || (group % 32) == 0) && (i0 % 4) == 0 &&
                           (reinterpret_cast<uintptr_t>(t.dead) & 3) == 0;
+        const int sb0 = i0 / SBW * SBW, sb_end = std::min(sb0 + SBW, n);
+        if (fast && tensor16) {
+            // this block's columns of the super-block's [-Err | Wpre]
+            a.EW = EW + (i0 - sb0); a.ew_ld = 2 * SBW; a.ew_pre = SBW;
+        }
         if (fast) column_block_kernel<<<cb_grid, CB_THREADS, column_block_smem(cb_rows), s>>>(a, cb_rows, blocksize);
         else if (T == 4) column_loop_kernel<4><<<cl_grid, nw * 32, cl_smem, s>>>(a);
         else if (T == 2) column_loop_kernel<2><<<cl_grid, nw * 32, cl_smem, s>>>(a);
         else column_loop_kernel<1><<<cl_grid, nw * 32, cl_smem, s>>>(a);
         QLAUNCHED();
         const int i2 = i0 + blocksize;
-        if (i2 < n && tensor) {
+        if (tensor16) {
+            if (i2 < sb_end) {
+                // rest of the super-block: W[:, i2:sb_end] += [-Err | Wpre] * [U[blk, i2:sb_end] ; P[blk, i2:sb_end]]
+                TcGemmArgs g = tc_args(Wk + i2, ldk, (int)m, sb_end - i2, 2 * blocksize, 1.f, 1.f, TC_FULL, TC_MASK_NONE, t.hd);
+                g.b_row0 = i2; g.b_k0 = i0; g.k_split = blocksize; g.b2_k0 = i0;
+                g.row_inv = t.row_inv; g.amax_b = t.amax_u;
+                *err = launch_tc_gemm(maps, g, t.num_sms, s);
+                if (*err != cudaSuccess) return GPTAQ_ERR_CUDA;
+                ++*launches;
+            } else if (i2 == sb_end && sb_end < n) {
+                // super-block done: everything to its right receives all of its errors at once
+                rowscale_split16_kernel<<<(unsigned)((m + 7) / 8), 256, 0, s>>>(EW, 2 * SBW, (int)m, 2 * SBW, t.EWS16,
+                                                                              t.EWS16 + (size_t)m * 2 * SBW, t.row_inv_s);
+                QLAUNCHED();
+                TcGemmArgs g = tc_args(Wk + sb_end, ldk, (int)m, n - sb_end, 2 * SBW, 1.f, 1.f, TC_FULL, TC_MASK_NONE, t.hd);
+                g.b_row0 = sb_end; g.b_k0 = sb0; g.k_split = SBW; g.b2_k0 = sb0;
+                g.row_inv = t.row_inv_s; g.amax_b = t.amax_u;
+                *err = launch_tc_gemm(maps_super, g, t.num_sms, s);
+                if (*err != cudaSuccess) return GPTAQ_ERR_CUDA;
+                ++*launches;
+            }
+        } else if (i2 < n && tensor) {
             // W[:, i2:] += [-Err | Wpre] * [U[blk, i2:] ; P[blk, i2:]] on the tensor cores: B operand rows
             // are rows i2.. of U^T (first B contraction steps) and of P^T (the next B)
             TcGemmArgs g = tc_args(Wk + i2, ldk, (int)m, n - i2, 2 * blocksize, 1.f, 1.f, TC_FULL, TC_MASK_NONE, t.hd);
             g.b_row0 = i2; g.b_k0 = i0; g.k_split = blocksize; g.b2_k0 = i0;
-            if (tensor16) { g.row_inv = t.row_inv; g.amax_b = t.amax_u; }
             *err = launch_tc_gemm(maps, g, t.num_sms, s);
             if (*err != cudaSuccess) return GPTAQ_ERR_CUDA;
             ++*launches;
@@ -1075,8 +1118,10 @@ gptaq_status_t gptaq_quantize(gptaq_handle_t h, void *d_W, int w_dtype, int64_t 
     if (f16) {
         t.UT16 = reinterpret_cast<const __half *>(h->ws + wl.s_off[0]);
         t.PT16 = reinterpret_cast<const __half *>(h->ws + wl.s_off[1]);
-        t.EW16 = reinterpret_cast<__half *>(h->ws + wl.ew_lo_off);
+        t.EWS16 = reinterpret_cast<__half *>(h->ws + wl.ew_lo_off);
+        t.EW16 = reinterpret_cast<__half *>(h->ws + wl.ew16_off);
         t.row_inv = reinterpret_cast<float *>(h->ws + wl.rs_off);
+        t.row_inv_s = t.row_inv + m;
         t.amax_u = h->hd->tc_amax + AMAX_U; t.amax_p = h->hd->tc_amax + AMAX_P;
     } else if (h->tensor) {
         float *S[6];

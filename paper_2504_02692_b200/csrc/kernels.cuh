@@ -597,6 +597,8 @@ struct ColumnLoopArgs {
     float *scales, *zeros;     // m x G
     int G;
     float *EW;                 // m x (2 * 32 * T): [-Err | Wpre]
+    int ew_ld, ew_pre;         // column_block_kernel: row pitch of EW / EW_lo and the offset of Wpre in a row (2B and B
+                               //   for the layout above; a block's slice of a wider [-Err | Wpre] otherwise)
     float *EW_lo;              // nullptr, or: EW receives the TF32 value of each entry and EW_lo the remainder
     // FP16 operand for the tensor-core update (column_block_kernel only; EW_lo is null then), or nullptr:
     // row i of [-Err | rho * Wpre] times a power of two s_i, as fp16 hi / lo parts, m x (2 * block) each;
@@ -953,8 +955,8 @@ __global__ void __launch_bounds__(CB_THREADS, 1) column_block_kernel(ColumnLoopA
 #pragma unroll
                 for (int k = 0; k < 32; ++k) crow[k] = (uint8_t)(code[k >> 2] >> (8 * (k & 3)));
             }
-            float *ew = a.EW + (int64_t)row * (2 * B) + o;
-            float *ewl = a.EW_lo ? a.EW_lo + (int64_t)row * (2 * B) + o : nullptr;
+            float *ew = a.EW + (int64_t)row * a.ew_ld + o;
+            float *ewl = a.EW_lo ? a.EW_lo + (int64_t)row * a.ew_ld + o : nullptr;
 #pragma unroll
             for (int k4 = 0; k4 < 8; ++k4) {
                 *reinterpret_cast<float4 *>(&Wt[tid][o + 4 * k4]) = make_float4(x[4 * k4], x[4 * k4 + 1], x[4 * k4 + 2], x[4 * k4 + 3]);
@@ -976,10 +978,10 @@ __global__ void __launch_bounds__(CB_THREADS, 1) column_block_kernel(ColumnLoopA
                         e4[f] = eh; p4[f] = ph;
                     }
                     *reinterpret_cast<float4 *>(ewl + 4 * k4) = make_float4(el[0], el[1], el[2], el[3]);
-                    *reinterpret_cast<float4 *>(ewl + B + 4 * k4) = make_float4(pl[0], pl[1], pl[2], pl[3]);
+                    *reinterpret_cast<float4 *>(ewl + a.ew_pre + 4 * k4) = make_float4(pl[0], pl[1], pl[2], pl[3]);
                 }
                 *reinterpret_cast<float4 *>(ew + 4 * k4) = make_float4(e4[0], e4[1], e4[2], e4[3]);
-                *reinterpret_cast<float4 *>(ew + B + 4 * k4) = make_float4(p4[0], p4[1], p4[2], p4[3]);
+                *reinterpret_cast<float4 *>(ew + a.ew_pre + 4 * k4) = make_float4(p4[0], p4[1], p4[2], p4[3]);
             }
 #pragma unroll
             for (int k = 0; k < 32; ++k) { St[k * sld + tid] = nerr[k]; St[(32 + k) * sld + tid] = pre[k]; }
@@ -1045,7 +1047,9 @@ __global__ void __launch_bounds__(CB_THREADS, 1) column_block_kernel(ColumnLoopA
         for (int idx = tid; idx < nrows * q; idx += CB_THREADS) {
             const int r = idx / q, c4 = idx - r * q;
             const int64_t off = (int64_t)(row0 + r) * (2 * B) + 4 * c4;
-            const float4 v = *reinterpret_cast<const float4 *>(a.EW + off);
+            const int cc = 4 * c4;
+            const float4 v = *reinterpret_cast<const float4 *>(a.EW + (int64_t)(row0 + r) * a.ew_ld +
+                                                               (cc < B ? cc : a.ew_pre + cc - B));
             const float sc = srow[r];
             const float x[4] = {sc * v.x, sc * v.y, sc * v.z, sc * v.w};
             __half h[4], l[4];

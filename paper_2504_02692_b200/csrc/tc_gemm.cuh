@@ -597,4 +597,31 @@ __global__ void __launch_bounds__(256) split16_kernel(Split16Args a) {
     }
 }
 
+// Rows of a float32 matrix [rows][cols] (pitch ld) as fp16 hi / lo parts with one power-of-two scale per
+// row (the row's largest magnitude lands in [2^13, 2^14)); row_inv[r] = 1 / scale.  One warp per row;
+// cols a multiple of 4, 16-byte aligned rows.
+__global__ void __launch_bounds__(256) rowscale_split16_kernel(const float *src, long long ld, int rows, int cols,
+                                                               __half *hi, __half *lo, float *row_inv) {
+    const int r = blockIdx.x * 8 + (threadIdx.x >> 5), lane = threadIdx.x & 31;
+    if (r >= rows) return;
+    const float *row = src + (long long)r * ld;
+    float m = 0.f;
+    for (int c = 4 * lane; c < cols; c += 128) {
+        const float4 q = *reinterpret_cast<const float4 *>(row + c);
+        m = fmaxf(fmaxf(m, fmaxf(fabsf(q.x), fabsf(q.y))), fmaxf(fabsf(q.z), fabsf(q.w)));
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
+    const float sc = split_scale(m);
+    if (lane == 0) row_inv[r] = 1.f / sc;
+    for (int c = 4 * lane; c < cols; c += 128) {
+        const float4 q = *reinterpret_cast<const float4 *>(row + c);
+        const float x[4] = {sc * q.x, sc * q.y, sc * q.z, sc * q.w};
+        uint2 h2, l2;
+        split16_pack(x, h2, l2);
+        *reinterpret_cast<uint2 *>(hi + (long long)r * cols + c) = h2;
+        *reinterpret_cast<uint2 *>(lo + (long long)r * cols + c) = l2;
+    }
+}
+
 }  // namespace gptaq

@@ -64,6 +64,17 @@ def test_tensor_path_block_sizes_and_tails(n, m, B, group, sym, bits):
     hp.assert_parity(out)
 
 
+@pytest.mark.parametrize("n,m,B,group,bits", [(1416, 100, 128, 128, 4), (1160, 40, 64, 64, 3)])
+def test_super_panels_and_super_blocks(n, m, B, group, bits):
+    """Widths beyond one super-panel of the factorisation (1024 columns) and beyond one super-block of the
+    lazy-batch update (8 blocks), with ragged last panels: the rank-1024 update, the updates inside a
+    super-panel at a column offset and the wide update with one scale per row all run."""
+    cfg = wl.scaled(wl.CONFIGS["cfg2"], name="super", n=n, m=m, batch_tokens=3000, n_batches=2, bits=bits, group=group,
+                    blocksize=B, outlier_channels=12)
+    out = hp.check_layer(cfg, wl.make_weight(cfg), batches_of(cfg), rows=np.arange(0, m, 3))
+    hp.assert_parity(out)
+
+
 def test_strided_inputs():
     """Activations and weights given as views with a leading dimension larger than n."""
     cfg = wl.scaled(wl.CONFIGS["cfg2"], name="strided", n=512, m=64, batch_tokens=1024, n_batches=2, outlier_channels=5)
