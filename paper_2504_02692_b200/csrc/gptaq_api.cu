@@ -289,22 +289,25 @@ cudaError_t launch_absmax(const float *src, int64_t lds, int rows, int cols, int
     return cudaGetLastError();
 }
 
-cudaError_t launch_split16(const float *src, int64_t lds, __half *hi, __half *lo, int64_t ldd, int rows, int cols,
-                           bool transpose, int mask, float scale, const unsigned *amax, cudaStream_t s) {
-    if (rows <= 0 || cols <= 0) return cudaSuccess;
-    Split16Args a;
-    a.src = src; a.lds = lds; a.hi = hi; a.lo = lo; a.ldd = ldd; a.rows = rows; a.cols = cols;
-    a.transpose = transpose ? 1 : 0; a.mask = mask; a.scale = scale; a.amax = amax;
-    dim3 grid((cols + 63) / 64, (rows + 63) / 64, 1);
-    split16_kernel<<<grid, 256, 0, s>>>(a);
-    return cudaGetLastError();
-}
-
 struct SplitBatch {
     int nbatch = 1;
     int64_t src_bstride = 0, dst_bstride = 0;
     int rows_last = 0, cols_last = 0;
 };
+
+cudaError_t launch_split16(const float *src, int64_t lds, __half *hi, __half *lo, int64_t ldd, int rows, int cols,
+                           bool transpose, int mask, float scale, const unsigned *amax, cudaStream_t s,
+                           const SplitBatch &b = SplitBatch()) {
+    if (rows <= 0 || cols <= 0 || b.nbatch <= 0) return cudaSuccess;
+    Split16Args a;
+    a.src = src; a.lds = lds; a.src_bstride = b.src_bstride; a.hi = hi; a.lo = lo; a.ldd = ldd;
+    a.dst_bstride = b.dst_bstride;
+    a.rows = rows; a.cols = cols; a.rows_last = b.rows_last; a.cols_last = b.cols_last; a.nbatch = b.nbatch;
+    a.transpose = transpose ? 1 : 0; a.mask = mask; a.scale = scale; a.amax = amax;
+    dim3 grid((cols + 63) / 64, (rows + 63) / 64, b.nbatch);
+    split16_kernel<<<grid, 256, 0, s>>>(a);
+    return cudaGetLastError();
+}
 
 cudaError_t launch_split(const float *src, int64_t lds, float *hi, float *lo, int64_t ldd, int rows, int cols,
                          bool transpose, int mask, float scale, cudaStream_t s, const SplitBatch &b = SplitBatch()) {
@@ -954,6 +957,41 @@ gptaq_status_t gptaq_factor(gptaq_handle_t h, float damp, gptaq_stream_t stream)
         const int np = (int)((n - sz + 2 * sz - 1) / (2 * sz));
         const int tail = (int)(n - (2 * sz * (np - 1) + sz));
         const int64_t bstride = 2 * sz * ((int64_t)n + 1);
+        if (h->f16 && damp > 0.f && sz >= 2 * NB) {
+            // The two products on the tensor cores with FP16-split operands.  Ranges: B holds entries of R
+            // (bounded like the panels), the inverted blocks are bounded by 1 / sqrt(lambda), the
+            // intermediate T records its own maximum in the first product's epilogue.
+            const size_t nn = (size_t)n * n;
+            __half *A1 = reinterpret_cast<__half *>(h->ws + wl.s_off[0]);     // left operands, K-major at their own coordinates
+            __half *B2 = reinterpret_cast<__half *>(h->ws + wl.s_off[1]);     // transposed right operands
+            unsigned *am = h->hd->tc_amax;
+            const SplitOperand Aop{A1, A1 + nn, n, n, n, true}, Bop{B2, B2 + nn, n, n, n, true};
+            TcMaps m16;
+            if (!make_tc_maps(&m16, Aop, Bop, nullptr)) { h->cuda_error = "cuTensorMapEncodeTiled failed"; return GPTAQ_ERR_CUDA; }
+            SplitBatch sb; sb.nbatch = np; sb.src_bstride = sb.dst_bstride = bstride;
+            SplitBatch sbt = sb; sbt.cols_last = tail;
+            SplitBatch sbc = sb; sbc.rows_last = tail; sbc.cols_last = tail;
+            CU(cudaMemsetAsync(am + AMAX_T, 0, sizeof(unsigned), s));
+            CU(launch_split16(H + sz, n, A1 + sz, A1 + nn + sz, n, (int)sz, (int)sz, false, SPLIT_ALL, 1.f, am + AMAX_PAN, s, sbt));
+            CU(launch_split16(H + sz * n + sz, n, B2 + sz * n + sz, B2 + nn + sz * n + sz, n, (int)sz, (int)sz, true,
+                              SPLIT_UPPER, 1.f, am + AMAX_INV, s, sbc));
+            TcGemmArgs g1 = tc_args(T + sz, n, (int)sz, (int)sz, (int)sz, 1.f, 0.f, TC_TRI_RIGHT, TC_MASK_NONE, h->hd);
+            g1.nbatch = np; g1.c_bstride = bstride; g1.N_last = tail; g1.K_last = tail;
+            g1.a_row0 = 0; g1.a_row_bs = (int)(2 * sz); g1.a_k0 = (int)sz; g1.a_k_bs = (int)(2 * sz);
+            g1.b_row0 = (int)sz; g1.b_row_bs = (int)(2 * sz); g1.b_k0 = (int)sz; g1.b_k_bs = (int)(2 * sz);
+            g1.amax_a = am + AMAX_PAN; g1.amax_b = am + AMAX_INV; g1.amax_out = am + AMAX_T;
+            CU(launch_tc_gemm(m16, g1, h->num_sms, s));
+            CU(launch_split16(H, n, A1, A1 + nn, n, (int)sz, (int)sz, false, SPLIT_UPPER, 1.f, am + AMAX_INV, s, sb));
+            CU(launch_split16(T + sz, n, B2 + sz * n, B2 + nn + sz * n, n, (int)sz, (int)sz, true, SPLIT_ALL, 1.f, am + AMAX_T, s, sbt));
+            TcGemmArgs g2 = tc_args(H + sz, n, (int)sz, (int)sz, (int)sz, -1.f, 0.f, TC_TRI_LEFT, TC_MASK_NONE, h->hd);
+            g2.nbatch = np; g2.c_bstride = bstride; g2.N_last = tail;
+            g2.a_row0 = 0; g2.a_row_bs = (int)(2 * sz); g2.a_k0 = 0; g2.a_k_bs = (int)(2 * sz);
+            g2.b_row0 = (int)sz; g2.b_row_bs = (int)(2 * sz); g2.b_k0 = 0; g2.b_k_bs = (int)(2 * sz);
+            g2.amax_a = am + AMAX_INV; g2.amax_b = am + AMAX_T;
+            CU(launch_tc_gemm(m16, g2, h->num_sms, s));
+            h->launches += 6;
+            continue;
+        }
         if (h->tensor && sz >= 2 * NB) {
             // Same two products on the tensor cores.  S1 holds K-major copies of the left operands at
             // their own coordinates (B, then A^-1), S2 the transposed right operands (C^-T, then T^T).

@@ -23,8 +23,9 @@ static_assert(sizeof(StateHeader) == 128, "header size");
 
 constexpr int ST_NOT_SPD = 4, ST_NONFINITE = 5, ST_TIMEOUT = 6;
 
-// Slots of StateHeader::tc_amax: factor panels (an a-priori bound), U, dXX^T / tokens, O, P.
-enum { AMAX_PAN = 0, AMAX_U = 1, AMAX_D = 2, AMAX_O = 3, AMAX_P = 4 };
+// Slots of StateHeader::tc_amax: factor panels (an a-priori bound), U, dXX^T / tokens, O, P, the blocks of
+// the inverse factor while it is built (an a-priori bound), the intermediate product of one doubling level.
+enum { AMAX_PAN = 0, AMAX_U = 1, AMAX_D = 2, AMAX_O = 3, AMAX_P = 4, AMAX_INV = 5, AMAX_T = 6 };
 
 // Scale of an FP16-split operand: a power of two that puts the largest magnitude into [2^13, 2^14).
 __host__ __device__ __forceinline__ float split_scale(float amax) {
@@ -82,6 +83,9 @@ __global__ void __launch_bounds__(1024) diag_stats_kernel(const float *H, int n,
         // every entry of row i of the factor R (H_d = R R^T) is at most sqrt(H_d,ii): the range of the
         // factor panels is known before they exist
         hd->tc_amax[AMAX_PAN] = __float_as_uint(sqrtf(redmax[0] + lambda));
+        // ... and H_d >= lambda I bounds every entry of R^-1 (and of the inverse of any diagonal block of R)
+        // by 1 / sqrt(lambda)
+        hd->tc_amax[AMAX_INV] = lambda > 0.f ? __float_as_uint(rsqrtf(lambda)) : 0u;
     }
 }
 

@@ -515,9 +515,9 @@ __global__ void __launch_bounds__(256) absmax_kernel(const float *src, long long
 }
 
 struct Split16Args {
-    const float *src; long long lds;
-    __half *hi, *lo; long long ldd;
-    int rows, cols;
+    const float *src; long long lds, src_bstride;
+    __half *hi, *lo; long long ldd, dst_bstride;
+    int rows, cols, rows_last, cols_last, nbatch;      // blockIdx.z walks batch entries, as in split_kernel
     int transpose, mask;
     float scale;
     const unsigned *amax;
@@ -539,6 +539,16 @@ __device__ __forceinline__ void split16_pack(const float (&x)[4], uint2 &hi, uin
 __global__ void __launch_bounds__(256) split16_kernel(Split16Args a) {
     __shared__ float tile[64][65];
     const int r0 = blockIdx.y * 64, c0 = blockIdx.x * 64;
+    {
+        const int z = blockIdx.z;
+        const bool last = z == a.nbatch - 1;
+        if (last && a.rows_last) a.rows = a.rows_last;
+        if (last && a.cols_last) a.cols = a.cols_last;
+        if (r0 >= a.rows || c0 >= a.cols) return;
+        a.src += (long long)z * a.src_bstride;
+        a.hi += (long long)z * a.dst_bstride;
+        a.lo += (long long)z * a.dst_bstride;
+    }
     const float s = a.scale * split_scale(__uint_as_float(*a.amax));
     const int tq = threadIdx.x & 15, ty = threadIdx.x >> 4;        // 16 quads x 16 rows
     for (int rr = ty; rr < 64; rr += 16) {
