@@ -321,29 +321,32 @@ def run_ours(args, cfg):
         v, desc, threads = oracle_sample(cfg, args.ref_tokens, args.ref_rows)
         cpu = {"value": v, "unit": "ms", "cores": threads, "kind": "oracle", "sample": desc}
     # Per-stage rooflines (algorithmic work / stage time against the bound that applies): the products of
-    # factor, P and the lazy-batch update run as three TF32 tensor-core products, i.e. at most
-    # (bf16 peak / 2) / 3 of useful flops; the column loop is bound by HBM on paper.
-    tf32x3_peak = peak / 2.0 / 3.0
+    # factor, P and the lazy-batch update run as three tensor-core products on split operands: fp16 hi / lo
+    # parts where the width is a multiple of 8 (at most bf16 peak / 3 of useful flops), TF32 parts otherwise
+    # (bf16 peak / 2 / 3); the column loop is bound by HBM on paper.
+    fp16_split = cfg.n >= 512 and cfg.n % 8 == 0
+    split_peak = peak / 3.0 if fp16_split else peak / 2.0 / 3.0
+    split_name = "tensor (3xFP16 split)" if fp16_split else "tensor (3xTF32)"
     n_, m_, B_ = float(cfg.n), float(cfg.m), float(cfg.blocksize)
     fl_factor, fl_P = 2.0 * n_ ** 3 / 3.0, 2.0 * n_ ** 3 / 3.0
     fl_trail = 2.0 * m_ * n_ * n_ * max(0.0, 1.0 - B_ / n_)
     by_loop = 25.0 * m_ * n_ + 8.0 * n_ * B_
-    layer_roofline_ms = (flops_call * len(batches) / (peak * 1e12) + (fl_factor + fl_P + fl_trail) / (tf32x3_peak * 1e12)
+    layer_roofline_ms = (flops_call * len(batches) / (peak * 1e12) + (fl_factor + fl_P + fl_trail) / (split_peak * 1e12)
                          + by_loop / (pk["hbm_gbs"] * 1e9)) * 1e3
     stage_rooflines = {
-        "factor": {"bound": "tensor (3xTF32)", "achieved": fl_factor / (fac_ms * 1e-3) / 1e12, "peak": tf32x3_peak, "unit": "TFLOP/s"},
-        "build_P": {"bound": "tensor (3xTF32)", "achieved": fl_P / (p_ms * 1e-3) / 1e12, "peak": tf32x3_peak, "unit": "TFLOP/s"},
-        "quantize": {"bound": "tensor (3xTF32) + hbm", "trailing_update_tflops_if_alone": fl_trail / (q_ms * 1e-3) / 1e12,
-                     "column_loop_gbs_if_alone": by_loop / (q_ms * 1e-3) / 1e9, "peak_tflops": tf32x3_peak,
+        "factor": {"bound": split_name, "achieved": fl_factor / (fac_ms * 1e-3) / 1e12, "peak": split_peak, "unit": "TFLOP/s"},
+        "build_P": {"bound": split_name, "achieved": fl_P / (p_ms * 1e-3) / 1e12, "peak": split_peak, "unit": "TFLOP/s"},
+        "quantize": {"bound": split_name + " + hbm", "trailing_update_tflops_if_alone": fl_trail / (q_ms * 1e-3) / 1e12,
+                     "column_loop_gbs_if_alone": by_loop / (q_ms * 1e-3) / 1e9, "peak_tflops": split_peak,
                      "peak_gbs": pk["hbm_gbs"]},
         "layer": {"roofline_ms": layer_roofline_ms, "measured_ms": ms_step, "frac": layer_roofline_ms / ms_step},
     }
     for k in ("factor", "build_P"):
-        stage_rooflines[k]["frac"] = stage_rooflines[k]["achieved"] / tf32x3_peak
+        stage_rooflines[k]["frac"] = stage_rooflines[k]["achieved"] / split_peak
     line = {
         "metric": METRIC, "value": ms_layer, "unit": "ms", "n_gpus": world, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": False, "scaling": "strong" if shard else "weak",
-        "vs_baseline": None, "dtype": "f16 x f16 -> f32 (statistics), f32 (solve)", "data": "synthetic",
+        "vs_baseline": None, "dtype": "f16 x f16 -> f32 (statistics), f32 (solve; its products as 3 x f16 hi/lo -> f32)", "data": "synthetic",
         "config": dict(wl.describe(cfg), parallelism=(f"one layer over {world} GPUs: tokens sharded, one all-reduce of H and dXX^T, rows sharded"
                                     if shard else f"{world} independent layer(s), one per GPU"),
                        l2="inputs (%.1f GB per step) exceed L2" % (2 * cfg.tokens * cfg.n * 4 / 1e9),
