@@ -79,8 +79,8 @@ size_t gptaq_state_bytes(int64_t n);
  * for width n, at most m_max weight rows and the given lazy-batch block size
  * (Algorithm 1, input B).  max_batch_tokens is the largest `tokens` that
  * gptaq_accumulate will be given in one call (larger batches still work: they
- * are processed in chunks that fit).  For n >= 512 the scratch holds TF32 operand copies of
- * U^T and P^T (about 7 n^2 floats in all): the library reads them in every gptaq_quantize, so the
+ * are processed in chunks that fit).  For n >= 512 the scratch holds split (high part / low part)
+ * operand copies of U^T and P^T for the tensor cores (about 7 n^2 floats in all): the library reads them in every gptaq_quantize, so the
  * workspace must be left untouched from gptaq_factor until the last gptaq_quantize on this state. */
 size_t gptaq_workspace_bytes(int64_t n, int64_t m_max, int64_t max_batch_tokens, int blocksize);
 

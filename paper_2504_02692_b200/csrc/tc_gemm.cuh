@@ -1,15 +1,17 @@
 // float32-grade tensor-core GEMM for sm_100a:  C = alpha * A * B^T + beta * C.
 //
-// Every operand is given as two K-major float32 arrays that hold TF32 values, hi = tf32(x)
-// and lo = tf32(x - hi) (split_kernel below makes them), and the product is evaluated as
-// hi*hi + hi*lo + lo*hi with tcgen05.mma.kind::tf32 and float32 accumulation in tensor
-// memory: about 22 significant bits per factor, which is what the factorisation, the
-// correction matrix and the propagation of quantization errors need (single TF32/fp16
-// products flip integer codes).  TMA loads 128 x 32 (A) and 256 x 32 (B) tiles of both
-// parts into 128-byte-swizzled shared memory; one thread issues the MMAs into one of two
-// 128 x 256 accumulators; eight epilogue warps drain them.  Accumulation chains in tensor
-// memory are cut every TCHUNK K-blocks and added into float32 registers with
-// round-to-nearest (the tensor core truncates its accumulator).
+// Every operand is given as two K-major arrays, a high part and a low part of each element
+// (hi = round(x), lo = round(x - hi)), and the product is evaluated as hi*hi + hi*lo + lo*hi
+// on the tensor cores with float32 accumulation in tensor memory: about 22 significant bits
+// per factor, which is what the factorisation, the correction matrix and the propagation of
+// quantization errors need (single TF32/fp16 products flip integer codes).  TMA loads the
+// 128-row (A) and 256-row (B) tiles of both parts, one 128-byte row piece per K-block, into
+// 128-byte-swizzled shared memory; one thread issues the MMAs into one of two 128 x 256
+// accumulators; eight epilogue warps drain them.  Accumulation chains in tensor memory are
+// cut every TCHUNK K-blocks and added into float32 registers with round-to-nearest (the
+// tensor core truncates its accumulator).  "C += ..." results leave through shared memory
+// as bulk tensor reductions (one request per 128 x 32 box) where C qualifies for a tensor
+// map; per-thread 16-byte reductions saturate the L2's reduction rate long before HBM.
 //
 // One kernel serves all shapes of the solve through a small tile description: batches of
 // equally shaped problems inside one matrix (block inversion by doubling), K ranges cut to
