@@ -75,6 +75,15 @@ def test_super_panels_and_super_blocks(n, m, B, group, bits):
     hp.assert_parity(out)
 
 
+def test_no_damping_keeps_the_unbounded_operand_form():
+    """damp = 0: nothing bounds the entries of the inverse factor in advance, so the block inverse runs with
+    TF32-split operands (no range limits) while the other products keep their fp16-split form."""
+    cfg = wl.scaled(wl.CONFIGS["cfg2"], name="nodamp", n=768, m=40, batch_tokens=4096, n_batches=2, damp=0.0,
+                    outlier_channels=6)
+    out = hp.check_layer(cfg, wl.make_weight(cfg), batches_of(cfg))
+    hp.assert_parity(out)
+
+
 def test_strided_inputs():
     """Activations and weights given as views with a leading dimension larger than n."""
     cfg = wl.scaled(wl.CONFIGS["cfg2"], name="strided", n=512, m=64, batch_tokens=1024, n_batches=2, outlier_channels=5)
