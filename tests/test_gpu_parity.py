@@ -84,6 +84,16 @@ def test_no_damping_keeps_the_unbounded_operand_form():
     hp.assert_parity(out)
 
 
+@pytest.mark.parametrize("scale", [1e-3, 250.0])
+def test_activation_units_do_not_matter(scale):
+    """The fp16-split operands of the solve carry power-of-two scales taken from their own ranges: the
+    same layer with its activations in other units (U scales with 1 / unit, P not at all) keeps parity."""
+    cfg = wl.scaled(wl.CONFIGS["cfg2"], name="units", n=640, m=48, batch_tokens=2048, n_batches=2, outlier_channels=6)
+    bt = [(X * scale, Xfp * scale) for X, Xfp in batches_of(cfg)]
+    out = hp.check_layer(cfg, wl.make_weight(cfg), bt)
+    hp.assert_parity(out)
+
+
 def test_strided_inputs():
     """Activations and weights given as views with a leading dimension larger than n."""
     cfg = wl.scaled(wl.CONFIGS["cfg2"], name="strided", n=512, m=64, batch_tokens=1024, n_batches=2, outlier_channels=5)
