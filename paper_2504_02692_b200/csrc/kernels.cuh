@@ -42,6 +42,13 @@ __device__ __forceinline__ float tf32_rn(float x) {
     return __uint_as_float(r);
 }
 
+// Programmatic dependent launch: a kernel launched with the stream-serialization attribute may be
+// scheduled while its predecessor in the stream drains; pdl_wait() returns once the predecessor has
+// completed and its writes are visible (a no-op for a plain launch), pdl_launch_dependents() lets the
+// successor be scheduled from here on.
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
 __device__ __forceinline__ void record_status(StateHeader *hd, int code, long long info) {
     if (atomicCAS(&hd->status, 0, code) == 0) hd->info = info;
 }
@@ -243,6 +250,8 @@ __global__ void __launch_bounds__(FP_THREADS, 1) factor_panel_kernel(FactorPanel
     const int n = a.n, b0 = a.b0;
     const int nv = min(NB, n - b0);
     const bool vec = (n & 3) == 0 && (reinterpret_cast<uintptr_t>(a.H) & 15) == 0 && nv == NB;
+    pdl_launch_dependents();
+    pdl_wait();
 
     // the block, read along rows (all loads in flight before the first store); only j >= i is used
     if (vec) {

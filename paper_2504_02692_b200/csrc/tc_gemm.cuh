@@ -185,9 +185,11 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap mapAhi, const __grid_constant
                      ::"r"(smem_u32(const_cast<uint32_t *>(tmem_slot))), "r"(512u) : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
     }
+    pdl_launch_dependents();
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
+    pdl_wait();                      // everything above is independent of the previous kernel's results
     const uint32_t tmem_base = *tmem_slot;
     const int ntiles = a.nbatch * ((a.M + TBM - 1) / TBM) * ((a.N + TBN - 1) / TBN);
 
