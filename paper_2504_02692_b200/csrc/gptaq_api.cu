@@ -401,7 +401,7 @@ gptaq_status_t accumulate_tc(gptaq_ctx *h, const float *X, const float *Xfp, int
         dim3 cgrid(kp / 64, (n + 63) / 64);
         convert_transpose_kernel<0><<<cgrid, 256, 0, s>>>(ca);
         LAUNCHED();
-        convert_transpose_kernel<1><<<cgrid, 256, 0, s>>>(ca);
+        convert_transpose_kernel<1><<<std::min<unsigned>(cgrid.x * cgrid.y, 4u * (unsigned)h->num_sms), 256, 0, s>>>(ca);
         LAUNCHED();
         CU(cudaEventRecord(h->conv_done[buf], s));
         CU(cudaStreamWaitEvent(gs, h->conv_done[buf], 0));

@@ -61,19 +61,11 @@ struct ConvertArgs {
 __device__ __forceinline__ int cvt_word(int c, int tp) { return c * 33 + 2 * (c >> 5) + tp; }
 constexpr int CVT_WORDS = 64 * 33 + 4;
 
+// One 64-token x 64-channel tile by one CTA of 256 threads.
 template <int PASS>
-__global__ void __launch_bounds__(256) convert_transpose_kernel(ConvertArgs a) {
-    __shared__ uint32_t sx[CVT_WORDS];
-    __shared__ uint32_t sd[CVT_WORDS];
-    __shared__ uint32_t sl[CVT_WORDS];
-    float scx = 1.f, scd = 1.f;
-    if (PASS == 1) {
-        scx = pick_scale(__uint_as_float(a.amax[0]));
-        scd = pick_scale(__uint_as_float(a.amax[1]));
-        if (scx == 1.f && scd == 1.f) return;
-    }
+__device__ __forceinline__ void convert_tile(const ConvertArgs &a, int t0, int c0, float scx, float scd,
+                                             uint32_t *sx, uint32_t *sd, uint32_t *sl) {
     const bool split = a.Xlo != nullptr;
-    const int t0 = blockIdx.x * 64, c0 = blockIdx.y * 64;
     const int tid = threadIdx.x;
     float mx = 0.f, md = 0.f;
     bool nan = false;
@@ -156,6 +148,28 @@ __global__ void __launch_bounds__(256) convert_transpose_kernel(ConvertArgs a) {
             *reinterpret_cast<uint4 *>(a.dXt + off) = make_uint4(sd[w], sd[w + 1], sd[w + 2], sd[w + 3]);
             if (split) *reinterpret_cast<uint4 *>(a.Xlo + off) = make_uint4(sl[w], sl[w + 1], sl[w + 2], sl[w + 3]);
         }
+    }
+}
+
+// PASS 0: grid (kp / 64, ceil(n / 64)), one tile per CTA.  PASS 1: any 1-D grid; the CTAs leave at once
+// unless a maximum was out of range (the usual case: a short grid keeps that exit cheap), else they
+// walk the tiles.
+template <int PASS>
+__global__ void __launch_bounds__(256) convert_transpose_kernel(ConvertArgs a) {
+    __shared__ uint32_t sx[CVT_WORDS];
+    __shared__ uint32_t sd[CVT_WORDS];
+    __shared__ uint32_t sl[CVT_WORDS];
+    if (PASS == 1) {
+        const float scx = pick_scale(__uint_as_float(a.amax[0]));
+        const float scd = pick_scale(__uint_as_float(a.amax[1]));
+        if (scx == 1.f && scd == 1.f) return;
+        const int TX = a.kp / 64, TY = (a.n + 63) / 64;
+        for (int tile = blockIdx.x; tile < TX * TY; tile += gridDim.x) {
+            convert_tile<1>(a, (tile % TX) * 64, (tile / TX) * 64, scx, scd, sx, sd, sl);
+            __syncthreads();
+        }
+    } else {
+        convert_tile<0>(a, blockIdx.x * 64, blockIdx.y * 64, 1.f, 1.f, sx, sd, sl);
     }
 }
 
