@@ -212,9 +212,14 @@ def run_ours(args, cfg):
     st = g.LayerState(cfg.n, cfg.m, cfg.batch_tokens, cfg.blocksize, dev, total_tokens=args.full_tokens)
     h = st.handle
     prec = g.gptaq_recommended_stats_precision(cfg.n, args.full_tokens)
+    if args.full_split_statistics:
+        prec = g.GPTAQ_STATS_FP16_SPLIT_FULL_TENSOR
     prec_name = {g.GPTAQ_STATS_FP16_TENSOR: "fp16 operands, fp32 accumulate",
-                 g.GPTAQ_STATS_FP16_SPLIT_TENSOR: "fp16 hi+lo split for H, fp32 accumulate"}[prec]
+                 g.GPTAQ_STATS_FP16_SPLIT_TENSOR: "fp16 hi+lo split for H, fp32 accumulate",
+                 g.GPTAQ_STATS_FP16_SPLIT_FULL_TENSOR: "fp16 hi+lo split for H and dXX^T, fp32 accumulate"}[prec]
     stream = torch.cuda.current_stream()
+    if args.full_split_statistics:
+        g.gptaq_set_stats_precision(h, prec)
     if args.act_order:
         g.gptaq_set_act_order(h, True)
     if args.clip_search > 0:
@@ -382,6 +387,8 @@ def main():
     ap.add_argument("--clip-search", type=int, default=0,
                     help="clipping-range search of the grids with this many candidates (off in the headline configuration)")
     ap.add_argument("--act-order", action="store_true", help="columns sorted by diag(H) (off in the headline configuration)")
+    ap.add_argument("--full-split-statistics", action="store_true",
+                    help="both statistics with split fp16 operands (float32-grade, 3x the MMAs; off in the headline configuration)")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()

@@ -67,8 +67,15 @@ enum { GPTAQ_W_FP32 = 0, GPTAQ_W_BF16 = 1 };
  *   the factor U keeps its accuracy even with few tokens per input channel.
  * GPTAQ_STATS_FP16_TENSOR: single fp16 term (11 significant bits), 40 % fewer MMAs; accurate
  *   enough for U once total tokens >= 16 n (see gptaq_recommended_stats_precision).
+ * GPTAQ_STATS_FP16_SPLIT_FULL_TENSOR: both sums carry the remainders (dXX^T = dh xh^T + dh xl^T +
+ *   dl xh^T as well): float32-grade statistics at three times the MMAs of the single-term mode.
+ *   The entries of dXX^T are themselves sums of randomly signed products, so the fp16 rounding of
+ *   single terms stays visible in them (about 3e-4 relative, and as much in P); that is far inside the
+ *   tolerances at alpha = 0.25 and 2-4 bits, but shows as rounding-tie flips at 8 bits and in the
+ *   objective once alpha approaches 1 with weak damping: use this mode (or GPTAQ_STATS_FP32) there.
  * GPTAQ_STATS_FP32: float32 products and sums on the plain FMA pipes (exact inputs). */
-enum { GPTAQ_STATS_FP16_TENSOR = 0, GPTAQ_STATS_FP32 = 1, GPTAQ_STATS_FP16_SPLIT_TENSOR = 2 };
+enum { GPTAQ_STATS_FP16_TENSOR = 0, GPTAQ_STATS_FP32 = 1, GPTAQ_STATS_FP16_SPLIT_TENSOR = 2,
+       GPTAQ_STATS_FP16_SPLIT_FULL_TENSOR = 3 };
 
 /* Bytes of the caller-owned device state for layer width n: a header (status
  * word, pivot index), H (n x n), dXX^T (n x n) and the dead-input flags.

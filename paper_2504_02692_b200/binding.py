@@ -29,6 +29,7 @@ GPTAQ_W_BF16 = 1
 GPTAQ_STATS_FP16_TENSOR = 0
 GPTAQ_STATS_FP32 = 1
 GPTAQ_STATS_FP16_SPLIT_TENSOR = 2
+GPTAQ_STATS_FP16_SPLIT_FULL_TENSOR = 3
 GPTAQ_TERM_ERR = 1
 GPTAQ_TERM_ASYM = 2
 

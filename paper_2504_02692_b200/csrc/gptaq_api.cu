@@ -340,10 +340,15 @@ cudaError_t launch_split(const float *src, int64_t lds, float *hi, float *lo, in
 size_t stats_scratch_bytes(int num_sms) { return round_up((size_t)num_sms * UBM * UBN * sizeof(float), ALIGN); }
 constexpr int MAX_SMS_FOR_SIZING = 256;
 
+// fp16 operand arrays per converted batch: X^T, (X~ - X)^T, the low part of X^T, the low part of (X~ - X)^T
+int stats_operand_arrays(int precision) {
+    return precision == GPTAQ_STATS_FP16_SPLIT_FULL_TENSOR ? 4 : (precision == GPTAQ_STATS_FP16_SPLIT_TENSOR ? 3 : 2);
+}
+
 // Largest token chunk (multiple of 64) whose fp16 operand copies fit the workspace next to that scratch.
 int64_t tc_chunk_tokens(const gptaq_ctx *h) {
-    const int nbuf = h->stats_precision == GPTAQ_STATS_FP16_SPLIT_TENSOR ? 3 : 2;
-    int64_t per_token = 2 * nbuf * h->n * 2;   // two buffers of X^T, dX^T (and the low part of X^T), fp16
+    const int nbuf = stats_operand_arrays(h->stats_precision);
+    int64_t per_token = 2 * nbuf * h->n * 2;   // two buffers of X^T, dX^T (and their low parts), fp16
     const size_t reserve = stats_scratch_bytes(h->num_sms);
     if (h->ws_bytes <= reserve + 2 * ALIGN) return 0;
     int64_t cap = (int64_t)((h->ws_bytes - reserve - 2 * ALIGN) / (size_t)per_token);
@@ -380,13 +385,15 @@ gptaq_status_t accumulate_tc(gptaq_ctx *h, const float *X, const float *Xfp, int
     for (int64_t t0 = 0; t0 < tokens; t0 += chunk) {
         const int tk = (int)std::min<int64_t>(chunk, tokens - t0);
         const int kp = (tk + UBK - 1) / UBK * UBK;
-        const bool split = h->stats_precision == GPTAQ_STATS_FP16_SPLIT_TENSOR;
+        const int narr = stats_operand_arrays(h->stats_precision);
+        const bool split = narr >= 3, splitd = narr == 4;
         const int buf = h->next_buf;
         h->next_buf ^= 1;
-        const size_t buf_bytes = round_up((size_t)(split ? 3 : 2) * n * (size_t)(chunk) * 2, ALIGN);
+        const size_t buf_bytes = round_up((size_t)narr * n * (size_t)(chunk) * 2, ALIGN);
         __half *Xt = reinterpret_cast<__half *>(h->ws + (size_t)buf * buf_bytes);
         __half *dXt = Xt + (size_t)n * kp;
         __half *Xlo = split ? dXt + (size_t)n * kp : nullptr;
+        __half *dXlo = splitd ? Xlo + (size_t)n * kp : nullptr;
         unsigned *amax = h->hd->amax[buf];
         cudaStream_t gs = h->gemm_stream;
         // this buffer was last read by the product issued two chunks ago
@@ -397,7 +404,7 @@ gptaq_status_t accumulate_tc(gptaq_ctx *h, const float *X, const float *Xfp, int
         CU(cudaMemsetAsync(amax, 0, 2 * sizeof(unsigned), s));
         ConvertArgs ca;
         ca.X = X + t0 * ld; ca.Xfp = Xfp + t0 * ld; ca.ld = ld; ca.tokens = tk; ca.n = n; ca.kp = kp;
-        ca.Xt = Xt; ca.dXt = dXt; ca.Xlo = Xlo; ca.amax = amax;
+        ca.Xt = Xt; ca.dXt = dXt; ca.Xlo = Xlo; ca.dXlo = dXlo; ca.amax = amax;
         dim3 cgrid(kp / 64, (n + 63) / 64);
         convert_transpose_kernel<0><<<cgrid, 256, 0, s>>>(ca);
         LAUNCHED();
@@ -405,16 +412,17 @@ gptaq_status_t accumulate_tc(gptaq_ctx *h, const float *X, const float *Xfp, int
         LAUNCHED();
         CU(cudaEventRecord(h->conv_done[buf], s));
         CU(cudaStreamWaitEvent(gs, h->conv_done[buf], 0));
-        CUtensorMap mXa, mDa, mXb, mLa, mLb;
+        CUtensorMap mXa, mDa, mXb, mLa, mLb, mDLa;
         const __half *lo = split ? Xlo : Xt;    // unused maps still have to be valid
+        const __half *dlo = splitd ? dXlo : dXt;
         if (!make_kmajor_map(&mXa, Xt, n, kp, UBM) || !make_kmajor_map(&mDa, dXt, n, kp, UBM) ||
             !make_kmajor_map(&mXb, Xt, n, kp, UBN) || !make_kmajor_map(&mLa, lo, n, kp, UBM) ||
-            !make_kmajor_map(&mLb, lo, n, kp, UBN)) {
+            !make_kmajor_map(&mLb, lo, n, kp, UBN) || !make_kmajor_map(&mDLa, dlo, n, kp, UBM)) {
             h->cuda_error = "cuTensorMapEncodeTiled failed";
             return GPTAQ_ERR_CUDA;
         }
         StatsGemmArgs ga;
-        ga.H = h->H; ga.D = h->D; ga.n = n; ga.kblocks = kp / UBK; ga.nseg_h = split ? 3 : 1; ga.amax = amax; ga.hd = h->hd;
+        ga.H = h->H; ga.D = h->D; ga.n = n; ga.kblocks = kp / UBK; ga.nseg_h = split ? 3 : 1; ga.nseg_d = splitd ? 3 : 1; ga.amax = amax; ga.hd = h->hd;
         // the last, partial wave of tiles is cut along K so that every SM has work
         ga.ntiles = (int)ntiles;
         ga.full_tiles = (int)(ntiles / h->num_sms) * h->num_sms;
@@ -430,7 +438,7 @@ gptaq_status_t accumulate_tc(gptaq_ctx *h, const float *X, const float *Xfp, int
         ga.scratch = reinterpret_cast<float *>(h->ws + 2 * buf_bytes);
         const int nitems = ga.full_tiles + ((int)ntiles - ga.full_tiles) * ga.ksplit;
         const int sgrid = std::min(nitems, h->num_sms);
-        stats_umma_kernel<<<sgrid, UMMA_THREADS, UMMA_SMEM, gs>>>(mXa, mDa, mXb, mLa, mLb, ga);
+        stats_umma_kernel<<<sgrid, UMMA_THREADS, UMMA_SMEM, gs>>>(mXa, mDa, mXb, mLa, mLb, mDLa, ga);
         LAUNCHED();
         if (ga.ksplit > 1) {
             stats_fixup_kernel<<<dim3((unsigned)((int)ntiles - ga.full_tiles), FIXUP_SLABS), 256, 0, gs>>>(ga);
@@ -1307,7 +1315,7 @@ gptaq_status_t gptaq_set_tokens(gptaq_handle_t h, int64_t tokens) {
 gptaq_status_t gptaq_set_stats_precision(gptaq_handle_t h, int precision) {
     if (!h) return GPTAQ_ERR_INVALID_ARG;
     if (precision != GPTAQ_STATS_FP16_TENSOR && precision != GPTAQ_STATS_FP32 &&
-        precision != GPTAQ_STATS_FP16_SPLIT_TENSOR)
+        precision != GPTAQ_STATS_FP16_SPLIT_TENSOR && precision != GPTAQ_STATS_FP16_SPLIT_FULL_TENSOR)
         return GPTAQ_ERR_UNSUPPORTED;
     if (h->stage != STAGE_ACCUM) return GPTAQ_ERR_BAD_STATE;
     if (precision != h->stats_precision) h->relayout = true;

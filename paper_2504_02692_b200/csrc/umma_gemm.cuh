@@ -51,6 +51,7 @@ struct ConvertArgs {
     int tokens, n, kp;
     __half *Xt, *dXt;       // [n][kp]
     __half *Xlo;            // [n][kp] or nullptr: fp16(X - float(fp16(X))), the second term of the split
+    __half *dXlo;           // [n][kp] or nullptr: the same for X~ - X
     unsigned *amax;          // [2]: bit patterns of max|X|, max|X~ - X|
 };
 
@@ -64,8 +65,8 @@ constexpr int CVT_WORDS = 64 * 33 + 4;
 // One 64-token x 64-channel tile by one CTA of 256 threads.
 template <int PASS>
 __device__ __forceinline__ void convert_tile(const ConvertArgs &a, int t0, int c0, float scx, float scd,
-                                             uint32_t *sx, uint32_t *sd, uint32_t *sl) {
-    const bool split = a.Xlo != nullptr;
+                                             uint32_t *sx, uint32_t *sd, uint32_t *sl, uint32_t *sdl) {
+    const bool split = a.Xlo != nullptr, splitd = a.dXlo != nullptr;
     const int tid = threadIdx.x;
     float mx = 0.f, md = 0.f;
     bool nan = false;
@@ -97,7 +98,7 @@ __device__ __forceinline__ void convert_tile(const ConvertArgs &a, int t0, int c
         }
 #pragma unroll
         for (int e = 0; e < 4; ++e) {
-            __half hx[2], hd[2], hl[2];
+            __half hx[2], hd[2], hl[2], hdl[2];
 #pragma unroll
             for (int h = 0; h < 2; ++h) {
                 const float xv = x[h][e], d = f[h][e] - xv;
@@ -105,15 +106,17 @@ __device__ __forceinline__ void convert_tile(const ConvertArgs &a, int t0, int c
                     mx = fmaxf(mx, fabsf(xv)); md = fmaxf(md, fabsf(d));
                     nan |= (xv != xv) || (d != d);     // fmaxf drops NaNs
                 }
-                const float xs = xv * scx;
+                const float xs = xv * scx, ds = d * scd;
                 hx[h] = __float2half_rn(xs);
-                hd[h] = __float2half_rn(d * scd);
+                hd[h] = __float2half_rn(ds);
                 hl[h] = __float2half_rn(xs - __half2float(hx[h]));
+                hdl[h] = __float2half_rn(ds - __half2float(hd[h]));
             }
             const int w = cvt_word(cl + e, tp);
             sx[w] = (uint32_t)__half_as_ushort(hx[0]) | ((uint32_t)__half_as_ushort(hx[1]) << 16);
             sd[w] = (uint32_t)__half_as_ushort(hd[0]) | ((uint32_t)__half_as_ushort(hd[1]) << 16);
             if (split) sl[w] = (uint32_t)__half_as_ushort(hl[0]) | ((uint32_t)__half_as_ushort(hl[1]) << 16);
+            if (splitd) sdl[w] = (uint32_t)__half_as_ushort(hdl[0]) | ((uint32_t)__half_as_ushort(hdl[1]) << 16);
         }
     }
     if (PASS == 0) {
@@ -147,6 +150,7 @@ __device__ __forceinline__ void convert_tile(const ConvertArgs &a, int t0, int c
             *reinterpret_cast<uint4 *>(a.Xt + off) = make_uint4(sx[w], sx[w + 1], sx[w + 2], sx[w + 3]);
             *reinterpret_cast<uint4 *>(a.dXt + off) = make_uint4(sd[w], sd[w + 1], sd[w + 2], sd[w + 3]);
             if (split) *reinterpret_cast<uint4 *>(a.Xlo + off) = make_uint4(sl[w], sl[w + 1], sl[w + 2], sl[w + 3]);
+            if (splitd) *reinterpret_cast<uint4 *>(a.dXlo + off) = make_uint4(sdl[w], sdl[w + 1], sdl[w + 2], sdl[w + 3]);
         }
     }
 }
@@ -159,17 +163,18 @@ __global__ void __launch_bounds__(256) convert_transpose_kernel(ConvertArgs a) {
     __shared__ uint32_t sx[CVT_WORDS];
     __shared__ uint32_t sd[CVT_WORDS];
     __shared__ uint32_t sl[CVT_WORDS];
+    __shared__ uint32_t sdl[CVT_WORDS];
     if (PASS == 1) {
         const float scx = pick_scale(__uint_as_float(a.amax[0]));
         const float scd = pick_scale(__uint_as_float(a.amax[1]));
         if (scx == 1.f && scd == 1.f) return;
         const int TX = a.kp / 64, TY = (a.n + 63) / 64;
         for (int tile = blockIdx.x; tile < TX * TY; tile += gridDim.x) {
-            convert_tile<1>(a, (tile % TX) * 64, (tile / TX) * 64, scx, scd, sx, sd, sl);
+            convert_tile<1>(a, (tile % TX) * 64, (tile / TX) * 64, scx, scd, sx, sd, sl, sdl);
             __syncthreads();
         }
     } else {
-        convert_tile<0>(a, blockIdx.x * 64, blockIdx.y * 64, 1.f, 1.f, sx, sd, sl);
+        convert_tile<0>(a, blockIdx.x * 64, blockIdx.y * 64, 1.f, 1.f, sx, sd, sl, sdl);
     }
 }
 
@@ -259,6 +264,7 @@ struct StatsGemmArgs {
     int n;
     int kblocks;             // kp / 64
     int nseg_h;              // 1: H = hi hi^T;  3: H = hi hi^T + hi lo^T + lo hi^T (split operands)
+    int nseg_d;              // 1: dXX^T = dh xh^T;  3: dh xh^T + dh xl^T + dl xh^T
     const unsigned *amax;    // scales are recomputed from the recorded maxima
     StateHeader *hd;
     // Work items: tiles [0, full_tiles) are whole tiles; each of the remaining `ntiles - full_tiles`
@@ -312,7 +318,7 @@ __device__ __forceinline__ bool stats_item(const StatsGemmArgs &a, int w, TileIt
         parts = a.ksplit;
     }
     if (!it.seek_to(tile)) return false;
-    const int kb_total = (it.r >= it.TM) ? a.kblocks : a.kblocks * a.nseg_h;
+    const int kb_total = (it.r >= it.TM) ? a.kblocks * a.nseg_d : a.kblocks * a.nseg_h;
     item.g0 = (int)((long long)kb_total * part / parts);
     item.g1 = (int)((long long)kb_total * (part + 1) / parts);
     item.part = part;
@@ -330,7 +336,8 @@ constexpr int UCHUNK = 8;           // K-blocks (of 64) per TMEM accumulation ch
 __global__ void __launch_bounds__(UMMA_THREADS, 1)
 stats_umma_kernel(const __grid_constant__ CUtensorMap mapXa, const __grid_constant__ CUtensorMap mapDa,
                   const __grid_constant__ CUtensorMap mapXb, const __grid_constant__ CUtensorMap mapLa,
-                  const __grid_constant__ CUtensorMap mapLb, StatsGemmArgs a) {
+                  const __grid_constant__ CUtensorMap mapLb, const __grid_constant__ CUtensorMap mapDLa,
+                  StatsGemmArgs a) {
     extern __shared__ uint8_t smem_raw[];
     // 1024-byte alignment for the swizzled tiles
     const uint32_t raw = smem_u32(smem_raw);
@@ -376,7 +383,7 @@ stats_umma_kernel(const __grid_constant__ CUtensorMap mapXa, const __grid_consta
                 const int row0 = (isD ? it.r - it.TM : it.r) * UBM, col0 = it.tn * UBN;
                 for (int g = item.g0; g < item.g1; ++g) {
                     const int seg = g / KB, kb = g - seg * KB;
-                    const CUtensorMap *mapA = isD ? &mapDa : (seg == 2 ? &mapLa : &mapXa);
+                    const CUtensorMap *mapA = isD ? (seg == 2 ? &mapDLa : &mapDa) : (seg == 2 ? &mapLa : &mapXa);
                     const CUtensorMap *mapB = (seg == 1) ? &mapLb : &mapXb;
                     if (!mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag)) { ok = false; break; }
                     const uint32_t sa = base + stage * USTAGE_BYTES, sb = sa + UA_BYTES;

@@ -35,13 +35,15 @@ def n_groups(n, group):
     return 1 if group <= 0 else (n + group - 1) // group
 
 
-def gpu_layer(cfg: wl.LayerConfig, W: torch.Tensor, batches, keep_stats=True, rows=None) -> GpuRun:
+def gpu_layer(cfg: wl.LayerConfig, W: torch.Tensor, batches, keep_stats=True, rows=None, stats_precision=None) -> GpuRun:
     """Runs create -> accumulate* -> factor -> build_P -> quantize through the binding."""
     dev = "cuda"
     m = W.shape[0]
     # statistics precision as recommended for this width and token count (what bench.py uses)
     st = g.LayerState(cfg.n, m, cfg.batch_tokens, cfg.blocksize, dev, total_tokens=cfg.tokens)
     try:
+        if stats_precision is not None:
+            g.gptaq_set_stats_precision(st.handle, stats_precision)
         for X, Xfp in batches:
             g.gptaq_accumulate(st.handle, X.to(dev), Xfp.to(dev))
         H = D = None
@@ -79,10 +81,10 @@ def rel_fro(a, b):
     return float(np.linalg.norm(a - b) / np.linalg.norm(b))
 
 
-def check_layer(cfg, W, batches, rows=None, report=None):
+def check_layer(cfg, W, batches, rows=None, report=None, stats_precision=None):
     """Full parity of one layer against the oracle; returns a dict of numbers."""
     Wn = W.cpu().numpy().astype(np.float64)
-    run = gpu_layer(cfg, W, batches)
+    run = gpu_layer(cfg, W, batches, stats_precision=stats_precision)
     assert run.status[0] == g.GPTAQ_OK, run.status
     st = oracle_stats(cfg, batches)
     U, dead = orc.factor(st.H, st.tokens, cfg.damp)

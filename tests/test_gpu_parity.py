@@ -477,7 +477,8 @@ def _stats_only(cfg, bt, precision, scale=1.0):
 def test_tensor_core_statistics_against_oracle(n, tokens, nb):
     """Tensor-core sums vs float64.  Elementwise error relative to sqrt(H_ii H_jj) is bounded by
     the rounding of the operands: 2^-11 per fp16 factor in the single-term mode; the split mode
-    keeps ~22 bits of X for H (dXX^T stays single-term in both)."""
+    keeps ~22 bits of X for H (dXX^T stays single-term in both), the full split mode keeps them in
+    dXX^T too."""
     cfg = wl.scaled(wl.CONFIGS["cfg2"], name="stats", n=n, m=8, batch_tokens=tokens, n_batches=nb,
                     outlier_channels=max(1, n // 100))
     bt = batches_of(cfg)
@@ -487,6 +488,7 @@ def test_tensor_core_statistics_against_oracle(n, tokens, nb):
     dd = np.sqrt(np.diag(so.G))
     for prec, tolH, tolD in ((g.GPTAQ_STATS_FP16_TENSOR, 2.0 ** -10, 2.0 ** -10),
                              (g.GPTAQ_STATS_FP16_SPLIT_TENSOR, 1e-5, 2.0 ** -10),
+                             (g.GPTAQ_STATS_FP16_SPLIT_FULL_TENSOR, 1e-5, 1e-5),
                              (g.GPTAQ_STATS_FP32, 1e-5, 1e-5)):
         H, D = _stats_only(cfg, bt, prec)
         errH = np.abs(H - so.H)[iu] / np.outer(d, d)[iu]
@@ -496,7 +498,19 @@ def test_tensor_core_statistics_against_oracle(n, tokens, nb):
         assert hp.rel_fro(D, so.D) < tolD and np.linalg.norm((H - so.H)[iu]) / np.linalg.norm(so.H[iu]) < tolH
 
 
-@pytest.mark.parametrize("prec", [g.GPTAQ_STATS_FP16_TENSOR, g.GPTAQ_STATS_FP16_SPLIT_TENSOR])
+def test_full_split_statistics_carry_a_hard_layer():
+    """Eight bits, alpha = 1, damping 0.001, sparse gated activations: the 3e-4 that single fp16 terms leave
+    in dXX^T (and in P) flips codes outside the tie band here; with both sums split the layer is exact to
+    the tolerances again."""
+    cfg = wl.scaled(wl.CONFIGS["cfg2"], name="hard", n=512, m=64, batch_tokens=3000, n_batches=1, bits=8, group=32,
+                    blocksize=32, damp=0.001, alpha=1.0, act="gated", outlier_channels=3, seed=1002)
+    out = hp.check_layer(cfg, wl.make_weight(cfg), batches_of(cfg), stats_precision=g.GPTAQ_STATS_FP16_SPLIT_FULL_TENSOR)
+    hp.assert_parity(out)
+    assert out["D_rel"] < 1e-5 and out["P_rel"] < 2e-5, out
+
+
+@pytest.mark.parametrize("prec", [g.GPTAQ_STATS_FP16_TENSOR, g.GPTAQ_STATS_FP16_SPLIT_TENSOR,
+                                  g.GPTAQ_STATS_FP16_SPLIT_FULL_TENSOR])
 @pytest.mark.parametrize("scale", [3e5, 1e-7])
 def test_tensor_core_statistics_rescale_out_of_range_batches(scale, prec):
     cfg = wl.scaled(wl.CONFIGS["cfg2"], name="stats", n=512, m=8, batch_tokens=640, n_batches=1, outlier_channels=5)
