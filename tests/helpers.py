@@ -129,4 +129,6 @@ def assert_parity(out):
     # group grids come from weights that carry the factor's error: same order as TOL_FACTOR
     assert rep.grid_rel_err <= 5e-5 and rep.zero_mismatch == 0, rep
     assert out["dequant_consistent"], out
-    assert out["J_gpu"] <= out["J_rtn"], out
+    # never worse than plain rounding, unless the method itself is (the float64 result then is as well:
+    # coarse symmetric grids at 2 bits can do that on the asymmetric objective)
+    assert out["J_gpu"] <= max(out["J_rtn"], out["J_oracle"] * (1.0 + TOL_OBJECTIVE)), out
