@@ -48,6 +48,7 @@ struct gptaq_ctx {
     int stats_precision;   // GPTAQ_STATS_*
     bool tensor;           // float32-grade tensor-core GEMMs for factor / P / trailing update
     bool f16;              // ... with FP16-split operands where the producer can record their range (n % 8 == 0)
+    TcSched sched;         // tile numbering of the float32-grade GEMM launches (see StateHeader::sched_counter)
     bool tf32_copies;      // f16 handles: the TF32 copies of U^T and P^T exist (made on demand by gptaq_quantize)
     int terms;             // GPTAQ_TERM_* switches of gptaq_quantize
     int clip_steps; float clip_min;   // clipping-range search of the grids
@@ -278,13 +279,16 @@ bool make_c_map(CUtensorMap *map, float *C, int64_t M, int64_t N, int64_t ldc) {
               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-cudaError_t launch_tc_gemm(const TcMaps &m, const TcGemmArgs &a_in, int num_sms, cudaStream_t s, bool pdl = true) {
+cudaError_t launch_tc_gemm(const TcMaps &m, const TcGemmArgs &a_in, TcSched &sched, int num_sms, cudaStream_t s, bool pdl = true) {
     if (a_in.M <= 0 || a_in.N <= 0 || a_in.nbatch <= 0) return cudaSuccess;
     TcGemmArgs a = a_in;
     const int64_t tiles = (int64_t)a.nbatch * ((a.M + TBM - 1) / TBM) * ((a.N + TBN - 1) / TBN);
     const int grid = (int)std::min<int64_t>(tiles, num_sms);
     // "C += ...": bulk tensor reductions where the target qualifies for a tensor map (16-byte aligned base
     // and row pitch); scattered per-thread reductions otherwise
+    a.sched = &a.hd->sched_counter;
+    a.sched_base = sched.base;
+    sched.base += (unsigned)tiles;           // (grid <= tiles)
     CUtensorMap mapC = m.a_hi;       // placeholder, not dereferenced unless c_tma is set
     a.c_tma = 0;
     if (a.beta == 1.f && a.nbatch == 1 && !a.amax_out && (a.mask == TC_MASK_NONE || a.mask == TC_MASK_UPPER_KEEP) &&
@@ -460,6 +464,7 @@ struct QuantizeTarget {
     const float *U, *P;
     const uint8_t *dead;
     StateHeader *hd;
+    TcSched *sched;            // host-side count of the tile numbers drawn from hd->sched_counter
     float *EW;
     int num_sms;
     // float32-grade tensor-core trailing update: split copies of U^T and P^T (n x n, ld n) and
@@ -595,7 +600,7 @@ gptaq_status_t quantize_core(const QuantizeTarget &t, void *d_W, int w_dtype, in
                 TcGemmArgs g = tc_args(Wk + i2, ldk, (int)m, sb_end - i2, 2 * blocksize, 1.f, 1.f, TC_FULL, TC_MASK_NONE, t.hd);
                 g.b_row0 = i2; g.b_k0 = i0; g.k_split = blocksize; g.b2_k0 = i0;
                 g.row_inv = t.row_inv; g.amax_b = t.amax_u;
-                *err = launch_tc_gemm(maps, g, t.num_sms, s, false);
+                *err = launch_tc_gemm(maps, g, *t.sched, t.num_sms, s, false);
                 if (*err != cudaSuccess) return GPTAQ_ERR_CUDA;
                 ++*launches;
             } else if (i2 == sb_end && sb_end < n) {
@@ -606,7 +611,7 @@ gptaq_status_t quantize_core(const QuantizeTarget &t, void *d_W, int w_dtype, in
                 TcGemmArgs g = tc_args(Wk + sb_end, ldk, (int)m, n - sb_end, 2 * SBW, 1.f, 1.f, TC_FULL, TC_MASK_NONE, t.hd);
                 g.b_row0 = sb_end; g.b_k0 = sb0; g.k_split = SBW; g.b2_k0 = sb0;
                 g.row_inv = t.row_inv_s; g.amax_b = t.amax_u;
-                *err = launch_tc_gemm(maps_super, g, t.num_sms, s, false);
+                *err = launch_tc_gemm(maps_super, g, *t.sched, t.num_sms, s, false);
                 if (*err != cudaSuccess) return GPTAQ_ERR_CUDA;
                 ++*launches;
             }
@@ -615,7 +620,7 @@ gptaq_status_t quantize_core(const QuantizeTarget &t, void *d_W, int w_dtype, in
             // are rows i2.. of U^T (first B contraction steps) and of P^T (the next B)
             TcGemmArgs g = tc_args(Wk + i2, ldk, (int)m, n - i2, 2 * blocksize, 1.f, 1.f, TC_FULL, TC_MASK_NONE, t.hd);
             g.b_row0 = i2; g.b_k0 = i0; g.k_split = blocksize; g.b2_k0 = i0;
-            *err = launch_tc_gemm(maps, g, t.num_sms, s, false);
+            *err = launch_tc_gemm(maps, g, *t.sched, t.num_sms, s, false);
             if (*err != cudaSuccess) return GPTAQ_ERR_CUDA;
             ++*launches;
         } else if (i2 < n) {
@@ -809,6 +814,7 @@ gptaq_status_t gptaq_reset(gptaq_handle_t h, gptaq_stream_t stream) {
     CU(cudaMemsetAsync(h->state, 0, l.total, static_cast<cudaStream_t>(stream)));
     h->stage = STAGE_ACCUM;
     h->tokens = 0;
+    h->sched.base = 0;           // the counter in the header was zeroed with the rest of the state
     return GPTAQ_OK;
 }
 
@@ -940,13 +946,13 @@ gptaq_status_t gptaq_factor(gptaq_handle_t h, float damp, gptaq_stream_t stream)
                 TcGemmArgs g = tc_args(H + s0, n, b0, b0 - s0, NB, -1.f, 1.f, TC_UPPER_TILES, TC_MASK_UPPER_KEEP, h->hd);
                 g.diag_off = s0; g.a_k0 = g.b_k0 = b0 - s0; g.b_row0 = s0;
                 g.amax_a = g.amax_b = am;
-                CU(launch_tc_gemm(pan_maps, g, h->num_sms, s));
+                CU(launch_tc_gemm(pan_maps, g, h->sched, h->num_sms, s));
             } else {
                 // super-panel [s0, s1) done: A[0:s0, 0:s0] -= R[0:s0, s0:s1] R[0:s0, s0:s1]^T  (upper part)
                 const int s1 = std::min(s0 + SUPER_NB, nb * NB);
                 TcGemmArgs g = tc_args(H, n, s0, s0, s1 - s0, -1.f, 1.f, TC_UPPER_TILES, TC_MASK_UPPER_KEEP, h->hd);
                 g.amax_a = g.amax_b = am;
-                CU(launch_tc_gemm(pan_maps, g, h->num_sms, s));
+                CU(launch_tc_gemm(pan_maps, g, h->sched, h->num_sms, s));
             }
             h->launches++;
             continue;
@@ -954,7 +960,7 @@ gptaq_status_t gptaq_factor(gptaq_handle_t h, float damp, gptaq_stream_t stream)
         // A[0:b0, 0:b0] -= R[0:b0, blk] R[0:b0, blk]^T  (upper part)
         if (h->tensor && b0 >= TC_MIN_N) {
             TcGemmArgs g = tc_args(H, n, b0, b0, NB, -1.f, 1.f, TC_UPPER_TILES, TC_MASK_UPPER_KEEP, h->hd);
-            CU(launch_tc_gemm(pan_maps, g, h->num_sms, s));
+            CU(launch_tc_gemm(pan_maps, g, h->sched, h->num_sms, s));
             h->launches++;
         } else {
             Operand rp = make_operand(H + b0, n, 1);
@@ -1002,7 +1008,7 @@ gptaq_status_t gptaq_factor(gptaq_handle_t h, float damp, gptaq_stream_t stream)
             g1.a_row0 = 0; g1.a_row_bs = (int)(2 * sz); g1.a_k0 = (int)sz; g1.a_k_bs = (int)(2 * sz);
             g1.b_row0 = (int)sz; g1.b_row_bs = (int)(2 * sz); g1.b_k0 = (int)sz; g1.b_k_bs = (int)(2 * sz);
             g1.amax_a = am + AMAX_PAN; g1.amax_b = am + AMAX_INV; g1.amax_out = am + AMAX_T;
-            CU(launch_tc_gemm(m16, g1, h->num_sms, s));
+            CU(launch_tc_gemm(m16, g1, h->sched, h->num_sms, s));
             CU(launch_split16(H, n, A1, A1 + nn, n, (int)sz, (int)sz, false, SPLIT_UPPER, 1.f, am + AMAX_INV, s, sb));
             CU(launch_split16(T + sz, n, B2 + sz * n, B2 + nn + sz * n, n, (int)sz, (int)sz, true, SPLIT_ALL, 1.f, am + AMAX_T, s, sbt));
             TcGemmArgs g2 = tc_args(H + sz, n, (int)sz, (int)sz, (int)sz, -1.f, 0.f, TC_TRI_LEFT, TC_MASK_NONE, h->hd);
@@ -1010,7 +1016,7 @@ gptaq_status_t gptaq_factor(gptaq_handle_t h, float damp, gptaq_stream_t stream)
             g2.a_row0 = 0; g2.a_row_bs = (int)(2 * sz); g2.a_k0 = 0; g2.a_k_bs = (int)(2 * sz);
             g2.b_row0 = (int)sz; g2.b_row_bs = (int)(2 * sz); g2.b_k0 = 0; g2.b_k_bs = (int)(2 * sz);
             g2.amax_a = am + AMAX_INV; g2.amax_b = am + AMAX_T;
-            CU(launch_tc_gemm(m16, g2, h->num_sms, s));
+            CU(launch_tc_gemm(m16, g2, h->sched, h->num_sms, s));
             h->launches += 6;
             continue;
         }
@@ -1029,7 +1035,7 @@ gptaq_status_t gptaq_factor(gptaq_handle_t h, float damp, gptaq_stream_t stream)
             g1.nbatch = np; g1.c_bstride = bstride; g1.N_last = tail; g1.K_last = tail;
             g1.a_row0 = 0; g1.a_row_bs = (int)(2 * sz); g1.a_k0 = (int)sz; g1.a_k_bs = (int)(2 * sz);
             g1.b_row0 = (int)sz; g1.b_row_bs = (int)(2 * sz); g1.b_k0 = (int)sz; g1.b_k_bs = (int)(2 * sz);
-            CU(launch_tc_gemm(inv_maps, g1, h->num_sms, s));
+            CU(launch_tc_gemm(inv_maps, g1, h->sched, h->num_sms, s));
             h->launches++;
             CU(launch_split(H, n, S1h, S1l, n, (int)sz, (int)sz, false, SPLIT_UPPER, 1.f, s, sb));
             h->launches++;
@@ -1039,7 +1045,7 @@ gptaq_status_t gptaq_factor(gptaq_handle_t h, float damp, gptaq_stream_t stream)
             g2.nbatch = np; g2.c_bstride = bstride; g2.N_last = tail;
             g2.a_row0 = 0; g2.a_row_bs = (int)(2 * sz); g2.a_k0 = 0; g2.a_k_bs = (int)(2 * sz);
             g2.b_row0 = (int)sz; g2.b_row_bs = (int)(2 * sz); g2.b_k0 = 0; g2.b_k_bs = (int)(2 * sz);
-            CU(launch_tc_gemm(inv_maps, g2, h->num_sms, s));
+            CU(launch_tc_gemm(inv_maps, g2, h->sched, h->num_sms, s));
             h->launches++;
             continue;
         }
@@ -1102,13 +1108,13 @@ gptaq_status_t gptaq_build_P(gptaq_handle_t h, float alpha, gptaq_stream_t strea
         if (!make_tc_maps(&maps, Aop, Uop, nullptr)) { h->cuda_error = "cuTensorMapEncodeTiled failed"; return GPTAQ_ERR_CUDA; }
         TcGemmArgs go = tc_args(O, n, n, n, n, 1.f, 0.f, TC_O, TC_MASK_STRICT_ZERO, h->hd);
         go.amax_a = am + AMAX_D; go.amax_b = am + AMAX_U; go.amax_out = am + AMAX_O;
-        CU(launch_tc_gemm(maps, go, h->num_sms, s));
+        CU(launch_tc_gemm(maps, go, h->sched, h->num_sms, s));
         CU(launch_split16(O, n, A16, A16 + nn, n, n, n, false, SPLIT_STRICT_UPPER, 1.f, am + AMAX_O, s));
         // P = alpha * O U  (B operand rows are rows of U^T)
         if (!make_tc_maps(&maps, Aop, UTop, nullptr)) { h->cuda_error = "cuTensorMapEncodeTiled failed"; return GPTAQ_ERR_CUDA; }
         TcGemmArgs gp = tc_args(h->D, n, n, n, n, alpha, 0.f, TC_P, TC_MASK_STRICT_ZERO, h->hd);
         gp.amax_a = am + AMAX_O; gp.amax_b = am + AMAX_U; gp.amax_out = am + AMAX_P;
-        CU(launch_tc_gemm(maps, gp, h->num_sms, s));
+        CU(launch_tc_gemm(maps, gp, h->sched, h->num_sms, s));
         // P^T for the lazy-batch updates of gptaq_quantize, over the copy of U that is no longer needed
         CU(launch_split16(h->D, n, U16, U16 + nn, n, n, n, true, SPLIT_STRICT_UPPER, 1.f, am + AMAX_P, s));
         h->launches += 4;
@@ -1124,13 +1130,13 @@ gptaq_status_t gptaq_build_P(gptaq_handle_t h, float alpha, gptaq_stream_t strea
         CU(launch_split(h->D, n, S[4], S[5], n, n, n, false, SPLIT_ALL, (float)(1.0 / (double)h->tokens), s));
         h->launches++;
         if (!make_tc_maps(&maps, S3, Us, nullptr)) { h->cuda_error = "cuTensorMapEncodeTiled failed"; return GPTAQ_ERR_CUDA; }
-        CU(launch_tc_gemm(maps, tc_args(O, n, n, n, n, 1.f, 0.f, TC_O, TC_MASK_STRICT_ZERO, h->hd), h->num_sms, s));
+        CU(launch_tc_gemm(maps, tc_args(O, n, n, n, n, 1.f, 0.f, TC_O, TC_MASK_STRICT_ZERO, h->hd), h->sched, h->num_sms, s));
         h->launches++;
         // S3 = split(O);  P = alpha * O U  (B operand rows are rows of U^T)
         CU(launch_split(O, n, S[4], S[5], n, n, n, false, SPLIT_STRICT_UPPER, 1.f, s));
         h->launches++;
         if (!make_tc_maps(&maps, S3, UTs, nullptr)) { h->cuda_error = "cuTensorMapEncodeTiled failed"; return GPTAQ_ERR_CUDA; }
-        CU(launch_tc_gemm(maps, tc_args(h->D, n, n, n, n, alpha, 0.f, TC_P, TC_MASK_STRICT_ZERO, h->hd), h->num_sms, s));
+        CU(launch_tc_gemm(maps, tc_args(h->D, n, n, n, n, alpha, 0.f, TC_P, TC_MASK_STRICT_ZERO, h->hd), h->sched, h->num_sms, s));
         h->launches++;
         // S3 = split(P^T) for the lazy-batch updates of gptaq_quantize
         CU(launch_split(h->D, n, S[4], S[5], n, n, n, true, SPLIT_STRICT_UPPER, 1.f, s));
@@ -1163,7 +1169,7 @@ gptaq_status_t gptaq_quantize(gptaq_handle_t h, void *d_W, int w_dtype, int64_t 
     WsLayout wl = ws_layout(h->n, m, blocksize);
     if (h->ws_bytes < wl.total) return GPTAQ_ERR_WORKSPACE;
     QuantizeTarget t;
-    t.n = (int)h->n; t.U = h->H; t.P = h->D; t.dead = h->dead; t.hd = h->hd;
+    t.n = (int)h->n; t.U = h->H; t.P = h->D; t.dead = h->dead; t.hd = h->hd; t.sched = &h->sched;
     t.EW = reinterpret_cast<float *>(h->ws + wl.ew_off);
     t.num_sms = h->num_sms;
     t.terms = h->terms;
@@ -1261,7 +1267,8 @@ gptaq_status_t gptaq_quantize_static(const float *d_U, const float *d_P, int64_t
     e = cudaMemsetAsync(sc->base, 0, STATIC_EW_OFFSET, s);
     if (e != cudaSuccess) return GPTAQ_ERR_CUDA;
     QuantizeTarget t;
-    t.n = (int)n; t.U = d_U; t.P = d_P;
+    TcSched static_sched;        // (the header is zeroed at every call; this path launches no tensor-core GEMM)
+    t.n = (int)n; t.U = d_U; t.P = d_P; t.sched = &static_sched;
     t.hd = reinterpret_cast<StateHeader *>(sc->base);
     t.dead = sc->base + STATIC_FLAGS_OFFSET;
     t.EW = reinterpret_cast<float *>(sc->base + STATIC_EW_OFFSET);

@@ -17,7 +17,8 @@ struct StateHeader {
     float inv_tokens;
     unsigned amax[2][2]; // per operand buffer: bit patterns of max|X| and max|X~ - X| of the batch converted into it
     unsigned tc_amax[8]; // largest magnitudes of FP16-split operands of the float32-grade GEMMs (see tc_gemm.cuh)
-    int pad1[14];
+    unsigned sched_counter; // tile numbers drawn by the float32-grade GEMM launches so far (never reset between launches)
+    int pad1[13];
 };
 static_assert(sizeof(StateHeader) == 128, "header size");
 

@@ -77,7 +77,16 @@ struct TcGemmArgs {
     unsigned *amax_out;              // if set: receives (atomicMax) the bit pattern of max |C| over what is stored
     int c_tma;                       // beta == 1, one batch entry: C += through bulk tensor reductions (mapC)
     int diag_off;                    // C is a block of columns of a square matrix: its column j is column j + diag_off there
+    // Tile scheduler: CTA b starts with tile b; further tile numbers come from a counter in global
+    // memory that is never reset: this launch owns its values sched_base .. sched_base + tiles - 1
+    // (tiles - grid numbers of tiles, and every CTA draws exactly one number beyond the last tile before
+    // it stops), the host advances the base by `tiles` per launch.
+    unsigned *sched;
+    unsigned sched_base;
 };
+
+// Host-side twin of StateHeader::sched_counter: the first tile number of the next launch.
+struct TcSched { unsigned base = 0; };
 
 struct TcTile {
     bool skip, zero_fill, work;
@@ -87,11 +96,12 @@ struct TcTile {
 __device__ __forceinline__ void tc_decode(const TcGemmArgs &a, int t, TcTile &ti, int bk) {
     const int TM = (a.M + TBM - 1) / TBM, TN = (a.N + TBN - 1) / TBN;
     const int per = TM * TN;
+    // tiles are handed out in the order of t: long K ranges first (column tiles ascending where the
+    // range shrinks with the column, descending where it grows), so that the last tiles drawn are short
+    if (a.mode == TC_P || a.mode == TC_TRI_RIGHT) t = a.nbatch * per - 1 - t;
     ti.z = t / per;
     const int rem = t - ti.z * per;
-    // row tile fastest: the tiles a CTA meets as it strides through the list then cover all column
-    // tiles, i.e. all lengths of the triangular K ranges, evenly (column-tile-fastest order gives
-    // every CTA the same few column tiles again and again: up to 2x imbalance)
+    // row tile fastest: the CTAs that run at the same time share a column panel of B
     const int tn = rem / TM, tm = rem - tn * TM;
     ti.i0 = tm * TBM; ti.j0 = tn * TBN;
     const bool last = ti.z == a.nbatch - 1;
@@ -172,10 +182,16 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap mapAhi, const __grid_constant
     auto tempty_bar = [&](int b) { return bar0 + 8u * (2 * TSTAGES + 2 + b); };
     volatile uint32_t *tmem_slot = reinterpret_cast<volatile uint32_t *>(aligned + TSTAGES * TSTAGE_BYTES + TC_STG_BYTES + 8 * (2 * TSTAGES + 4));
     volatile int *abort_flag = reinterpret_cast<volatile int *>(tmem_slot + 1);
+    // tile scheduler ring (at byte 128 of the barrier block): sfull[4], sempty[4], then the four tile numbers
+    constexpr int NR = 4;
+    auto sfull_bar = [&](int s) { return bar0 + 128u + 8u * s; };
+    auto sempty_bar = [&](int s) { return bar0 + 128u + 8u * (NR + s); };
+    volatile int *ring = reinterpret_cast<volatile int *>(aligned + TSTAGES * TSTAGE_BYTES + TC_STG_BYTES + 128 + 8 * 2 * NR);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     if (threadIdx.x == 0) {
         for (int s = 0; s < TSTAGES; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
+        for (int s = 0; s < NR; ++s) { mbar_init(sfull_bar(s), 1); mbar_init(sempty_bar(s), 1 + UEPI_WARPS); }
         for (int b = 0; b < 2; ++b) { mbar_init(tfull_bar(b), 1); mbar_init(tempty_bar(b), UEPI_WARPS); }
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -196,12 +212,29 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap mapAhi, const __grid_constant
     if (warp == 0) {
         // ------------------------------------------------------------ TMA producer
         if (lane == 0) {
-            uint32_t stage = 0, phase = 0;
+            uint32_t stage = 0, phase = 0, pushed = 0;
             int issued = 0;
             bool ok = true;
             TcTile ti;
-            for (int t = blockIdx.x; t < ntiles && ok; t += gridDim.x) {
-                tc_decode(a, t, ti, BK);
+            bool first = true;
+            while (ok) {
+                // next tile for this CTA; -1 once the list is exhausted.  The first one needs no round trip
+                // to the counter: tile number = CTA number; the counter hands out the numbers from gridDim.x on.
+                const unsigned ticket = first ? blockIdx.x : gridDim.x + (atomicAdd(a.sched, 1u) - a.sched_base);
+                first = false;
+                const int t = ticket < (unsigned)ntiles ? (int)ticket : -1;
+                if (t >= 0) {
+                    tc_decode(a, t, ti, BK);
+                    if (ti.skip && !ti.zero_fill) continue;          // nothing to do for any role
+                }
+                {   // hand the number to the MMA issuer and the epilogue warps
+                    const uint32_t slot = pushed % NR, sph = (pushed / NR) & 1u;
+                    if (!mbar_wait(sempty_bar(slot), sph ^ 1u, abort_flag)) { ok = false; break; }
+                    ring[slot] = t;
+                    mbar_arrive(sfull_bar(slot));
+                    ++pushed;
+                }
+                if (t < 0) break;
                 if (!ti.work) continue;
                 const int arow = a.a_row0 + ti.z * a.a_row_bs + ti.i0;
                 const int brow = a.b_row0 + ti.z * a.b_row_bs + ti.j0;
@@ -238,7 +271,12 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap mapAhi, const __grid_constant
             uint32_t stage = 0, phase = 0, ccount = 0;
             bool ok = true;
             TcTile ti;
-            for (int t = blockIdx.x; t < ntiles && ok; t += gridDim.x) {
+            for (uint32_t taken = 0; ok; ++taken) {
+                const uint32_t slot = taken % NR, sph = (taken / NR) & 1u;
+                if (!mbar_wait(sfull_bar(slot), sph, abort_flag)) break;
+                const int t = ring[slot];
+                mbar_arrive(sempty_bar(slot));
+                if (t < 0) break;
                 tc_decode(a, t, ti, BK);
                 if (!ti.work) continue;
                 for (int kc = ti.kb0; kc < ti.kb1 && ok; kc += TCHUNK) {
@@ -289,9 +327,14 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap mapAhi, const __grid_constant
             if (a.amax_b) op_scale /= split_scale(__uint_as_float(*a.amax_b));
         }
         TcTile ti;
-        for (int t = blockIdx.x; t < ntiles && ok; t += gridDim.x) {
+        for (uint32_t taken = 0; ok; ++taken) {
+            const uint32_t slot = taken % NR, sph = (taken / NR) & 1u;
+            if (!mbar_wait(sfull_bar(slot), sph, abort_flag)) break;
+            const int t = ring[slot];
+            __syncwarp();
+            if (lane == 0) mbar_arrive(sempty_bar(slot));
+            if (t < 0) break;
             tc_decode(a, t, ti, BK);
-            if (ti.skip && !ti.zero_fill) continue;
 #pragma unroll
             for (int i = 0; i < TBN / 2; ++i) acc[i] = 0.f;
             if (ti.work) {
