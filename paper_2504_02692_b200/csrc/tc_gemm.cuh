@@ -598,22 +598,34 @@ __global__ void __launch_bounds__(256) split16_kernel(Split16Args a) {
     }
     const float s = a.scale * split_scale(__uint_as_float(*a.amax));
     const int tq = threadIdx.x & 15, ty = threadIdx.x >> 4;        // 16 quads x 16 rows
-    for (int rr = ty; rr < 64; rr += 16) {
-        const int r = r0 + rr, c = c0 + 4 * tq;
-        float x[4] = {0.f, 0.f, 0.f, 0.f};
-        if (r < a.rows && c < a.cols) {
+    // all four loads of the thread first (a store in between would serialise them), none for quads that
+    // the mask empties
+    float xs[4][4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        const int r = r0 + ty + 16 * i, c = c0 + 4 * tq;
+#pragma unroll
+        for (int e = 0; e < 4; ++e) xs[i][e] = 0.f;
+        const bool any = a.mask == SPLIT_ALL || (a.mask == SPLIT_UPPER ? c + 3 >= r : c + 3 > r);
+        if (r < a.rows && c < a.cols && any) {
             const float *sp = a.src + (long long)r * a.lds + c;
             if (c + 3 < a.cols) {
-                const float4 q = *reinterpret_cast<const float4 *>(sp);
-                x[0] = q.x; x[1] = q.y; x[2] = q.z; x[3] = q.w;
+                const float4 q = __ldcs(reinterpret_cast<const float4 *>(sp));
+                xs[i][0] = q.x; xs[i][1] = q.y; xs[i][2] = q.z; xs[i][3] = q.w;
             } else {
-                for (int e = 0; c + e < a.cols; ++e) x[e] = sp[e];
+                for (int e = 0; c + e < a.cols; ++e) xs[i][e] = sp[e];
             }
+        }
+    }
 #pragma unroll
-            for (int e = 0; e < 4; ++e) {
-                const bool keep = a.mask == SPLIT_ALL || (a.mask == SPLIT_UPPER ? c + e >= r : c + e > r);
-                x[e] = keep ? s * x[e] : 0.f;
-            }
+    for (int i = 0; i < 4; ++i) {
+        const int rr = ty + 16 * i;
+        const int r = r0 + rr, c = c0 + 4 * tq;
+        float x[4];
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+            const bool keep = a.mask == SPLIT_ALL || (a.mask == SPLIT_UPPER ? c + e >= r : c + e > r);
+            x[e] = keep ? s * xs[i][e] : 0.f;
         }
         if (!a.transpose) {
             if (r < a.rows && c < a.cols) {
