@@ -134,7 +134,7 @@ constexpr int NB = 128;
 constexpr int FP_THREADS = 256;
 constexpr int FP_WARPS = FP_THREADS / 32;
 constexpr int FP_LD = NB + 4;
-constexpr size_t FP_SMEM = (2 * NB * FP_LD + 32 * FP_LD + NB) * sizeof(float);
+constexpr size_t FP_SMEM = (2 * NB * FP_LD + 32 * FP_LD + NB + 64) * sizeof(float);
 
 struct FactorPanelArgs {
     float *H; int n; int b0;
@@ -176,14 +176,16 @@ __device__ __forceinline__ void solve_row(float (&a)[LEN], const float *Rt, int 
 // One column step (K, then K - 1, ... 0) of the 32 x 32 reverse Cholesky held one row per lane.
 // `piv` is the pivot of this step, already broadcast: the dependent chain from one pivot to the
 // next runs through lane K - 1 alone (its own c), the other lanes' updates overlap with it.
+// The scaled column c reaches the other lanes through shared memory (cv: two buffers of 32 floats,
+// read back as broadcast float4s): K shuffles per step, one per element, cost three times as much.
+// A pivot that is not positive (or not finite) is replaced by 1 without a branch; the first such
+// column is remembered in bad_col (-1: none) and reported after the block.
 template <int K>
 struct Chol32Step {
-    static __device__ __forceinline__ void run(float (&d)[32], float piv, int lane, float *dinv,
-                                               StateHeader *hd, bool report, int col0) {
-        if (!(piv > 0.f) || !isfinite(piv)) {
-            if (lane == 0 && report) record_status(hd, ST_NOT_SPD, col0 + K);
-            piv = 1.f;
-        }
+    static __device__ __forceinline__ void run(float (&d)[32], float piv, int lane, float *dinv, float *cv, int &bad_col) {
+        const bool bad = !(piv > 0.f) || !isfinite(piv);
+        bad_col = (bad && bad_col < 0) ? K : bad_col;
+        piv = bad ? 1.f : piv;
         // 1/sqrt(piv): hardware estimate plus one Newton step (to about one ulp)
         float rinv = rsqrtf(piv);
         rinv = rinv * fmaf(-0.5f * piv, rinv * rinv, 1.5f);
@@ -193,15 +195,24 @@ struct Chol32Step {
         float next = 0.f;
         if (K > 0) {
             next = __shfl_sync(0xffffffffu, fmaf(-c, c, d[K - 1]), K - 1);
+            float *buf = cv + 32 * (K & 1);
+            buf[lane] = c;
+            __syncwarp();
 #pragma unroll
-            for (int j = K - 1; j >= 0; --j) d[j] = fmaf(-c, __shfl_sync(0xffffffffu, c, j), d[j]);
+            for (int j4 = (K - 1) / 4; j4 >= 0; --j4) {
+                const float4 cj = *reinterpret_cast<const float4 *>(buf + 4 * j4);
+                if (4 * j4 + 3 < K) d[4 * j4 + 3] = fmaf(-c, cj.w, d[4 * j4 + 3]);
+                if (4 * j4 + 2 < K) d[4 * j4 + 2] = fmaf(-c, cj.z, d[4 * j4 + 2]);
+                if (4 * j4 + 1 < K) d[4 * j4 + 1] = fmaf(-c, cj.y, d[4 * j4 + 1]);
+                if (4 * j4 + 0 < K) d[4 * j4 + 0] = fmaf(-c, cj.x, d[4 * j4 + 0]);
+            }
         }
-        Chol32Step<K - 1>::run(d, next, lane, dinv, hd, report, col0);
+        Chol32Step<K - 1>::run(d, next, lane, dinv, cv, bad_col);
     }
 };
 template <>
 struct Chol32Step<-1> {
-    static __device__ __forceinline__ void run(float (&)[32], float, int, float *, StateHeader *, bool, int) {}
+    static __device__ __forceinline__ void run(float (&)[32], float, int, float *, float *, int &) {}
 };
 
 // C[0:rows, 0:o] -= Xt^T * Rt  with Xt[k][row] (32 x rows) and Rt[k][j] (32 x o), both in shared
@@ -247,6 +258,7 @@ __global__ void __launch_bounds__(FP_THREADS, 1) factor_panel_kernel(FactorPanel
     float (*At)[FP_LD] = reinterpret_cast<float (*)[FP_LD]>(smem_f + NB * FP_LD);         // step 2: a tile of panel rows
     float (*Pt)[FP_LD] = reinterpret_cast<float (*)[FP_LD]>(smem_f + 2 * NB * FP_LD);     // Pt[k][i]: 32 solved columns, transposed
     float *dinv = smem_f + 2 * NB * FP_LD + 32 * FP_LD;
+    float *cv = dinv + NB;                 // 2 x 32: the scaled column of the running 32 x 32 step
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int n = a.n, b0 = a.b0;
     const int nv = min(NB, n - b0);
@@ -286,7 +298,9 @@ __global__ void __launch_bounds__(FP_THREADS, 1) factor_panel_kernel(FactorPanel
             float d[32];
 #pragma unroll
             for (int j = 0; j < 32; ++j) d[j] = (j >= lane) ? S[o + lane][o + j] : S[o + j][o + lane];
-            Chol32Step<31>::run(d, __shfl_sync(0xffffffffu, d[31], 31), lane, dinv + o, a.hd, blockIdx.x == 0, b0 + o);
+            int bad_col = -1;
+            Chol32Step<31>::run(d, __shfl_sync(0xffffffffu, d[31], 31), lane, dinv + o, cv, bad_col);
+            if (bad_col >= 0 && lane == 0 && blockIdx.x == 0) record_status(a.hd, ST_NOT_SPD, b0 + o + bad_col);
             // R_ss to the upper part, its transpose to the lower part
 #pragma unroll
             for (int j = 0; j < 32; ++j)
