@@ -131,7 +131,7 @@ __global__ void __launch_bounds__(256) scale_damp_kernel(float *H, int n, const 
 // Rows/columns beyond n are padded with the identity.
 // ---------------------------------------------------------------------------
 constexpr int NB = 128;
-constexpr int FP_THREADS = 256;
+constexpr int FP_THREADS = 512;
 constexpr int FP_WARPS = FP_THREADS / 32;
 constexpr int FP_LD = NB + 4;
 constexpr size_t FP_SMEM = (2 * NB * FP_LD + 32 * FP_LD + NB + 64) * sizeof(float);
