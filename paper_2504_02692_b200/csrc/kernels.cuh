@@ -786,6 +786,15 @@ __host__ __device__ inline size_t column_block_smem(int rows) {
     return ((size_t)rows * CB_LD + 2 * 2 * 32 * CB_LD + 64 * (rows + 4) + 2 * 32) * sizeof(float);
 }
 
+// Round to nearest, ties to even, for a value that is clamped to [0, 255] afterwards: adding and
+// subtracting 1.5 * 2^23 rounds exactly like rintf wherever |v| < 2^22 and leaves larger values large
+// (the clamp decides those), in two additions instead of a trip through the conversion unit, which
+// was 30 of the 154 cycles of a column step.
+__device__ __forceinline__ float round_for_clamp(float v) {
+    const float magic = 12582912.f;
+    return __fsub_rn(__fadd_rn(v, magic), magic);
+}
+
 template <int K>
 struct QuantStep {
     // x: the row's 32 columns (already-updated weights in, dequantized values out)
@@ -796,7 +805,7 @@ struct QuantStep {
         const float w0 = x[K];
         // w / scale as w * (1 / scale): one rounding more (about 1e-7 of a step, far inside the tie band)
         // for a much shorter dependent chain
-        const float cq = fminf(fmaxf(rintf(w0 * inv_scale) + zero, 0.f), maxq);
+        const float cq = fminf(fmaxf(round_for_clamp(w0 * inv_scale) + zero, 0.f), maxq);
         const float q = scale * (cq - zero);
         const float ne = err_scale * ((q - w0) * udinv[K]);           // -(w - q) / U_kk
         const float w = asym_scale * w0;
