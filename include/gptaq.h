@@ -24,7 +24,10 @@
  *    errors are returned at once, conditions found on the device (a
  *    non-positive pivot, a non-finite value, a bounded wait that ran out) are
  *    recorded in a device status word that gptaq_sync_status() reads.  Nothing
- *    traps or asserts on the device.
+ *    traps or asserts on the device.  The calls on one handle are one sequence of
+ *    work: give them one stream, or order the streams yourself (an event between
+ *    calls); the handle keeps host-side counters that mirror device-side ones in
+ *    the order of the calls, and one call's kernels read what the previous call's wrote.
  *  - Call order: create -> accumulate* -> factor -> build_P -> quantize*.
  *    Anything else returns GPTAQ_ERR_BAD_STATE.  gptaq_reset() returns a
  *    handle to the state right after create.  quantize may be called many
