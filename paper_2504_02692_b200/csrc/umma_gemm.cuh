@@ -276,29 +276,42 @@ struct StatsGemmArgs {
     float *scratch;
 };
 
-// Tile enumeration shared by all roles: row-major over (row tile, column tile);
-// rows [0, TM) belong to H (tiles entirely below the diagonal are not
-// enumerated), rows [TM, 2 TM) to dXX^T.
+// Tile enumeration shared by all roles.  Rows [0, TM) belong to H (tiles entirely below the
+// diagonal are not enumerated), rows [TM, 2 TM) to dXX^T.  Order: bands of UBAND row tiles; inside a
+// band column tile by column tile, first the band's tiles of H, then its tiles of dXX^T.  The 148
+// tiles that are in flight together then share about 2 x 16 row panels (X and X~ - X) and a handful
+// of column panels of X through the L2, and X streams from HBM once per band instead of once per
+// 2.6 row tiles (row-major order over the whole matrix: 15 GB of HBM reads per 8192-token batch at
+// n = 14336).
+constexpr int UBAND = 16;
 struct TileIter {
-    int TM, TN, r, tn, ord;       // ord: ordinal of the current tile (r, tn)
-    __device__ TileIter(int n) : TM((n + UBM - 1) / UBM), TN((n + UBN - 1) / UBN), r(0), tn(0), ord(0) {
-        tn = first_tn(0);
-    }
-    __device__ int first_tn(int row) const { return row < TM ? (row * UBM) / UBN : 0; }
+    int TM, TN, r, tn, ord;       // (r, tn): the current tile; ord: its ordinal
+    int band, k;                  // band of row tiles, position inside the group (band, tn)
+    __device__ TileIter(int n) : TM((n + UBM - 1) / UBM), TN((n + UBN - 1) / UBN), r(0), tn(0), ord(0), band(0), k(0) {}
+    __device__ int band_rows() const { return min(UBAND, TM - band * UBAND); }
+    // row tiles r of the band whose tile (r, tn) of H is not entirely below the diagonal: r <= 2 tn + 1
+    __device__ int h_count() const { return max(0, min(band * UBAND + band_rows(), (2 * tn + 2) * (UBN / (2 * UBM))) - band * UBAND); }
     // Advances to the tile with ordinal `target` >= ord; false when the list is exhausted.
     __device__ bool seek_to(int target) {
         int left = target - ord;
-        while (r < 2 * TM) {
-            int avail = TN - tn;
-            if (left < avail) { tn += left; ord = target; return true; }
+        while (band * UBAND < TM) {
+            const int hc = h_count();
+            const int avail = hc + band_rows() - k;
+            if (left < avail) {
+                k += left;
+                ord = target;
+                r = k < hc ? band * UBAND + k : TM + band * UBAND + (k - hc);
+                return true;
+            }
             left -= avail;
             ord += avail;
-            ++r;
-            tn = first_tn(r);
+            k = 0;
+            if (++tn == TN) { tn = 0; ++band; }
         }
         return false;
     }
 };
+static_assert(UBN == 2 * UBM, "the diagonal test of TileIter assumes 128 x 256 tiles");
 
 // One work item of a CTA: a tile and a range of its K-blocks (all segments concatenated).
 struct StatsItem {
