@@ -34,7 +34,7 @@ METRIC = "ms per layer (GPTAQ solve: accumulate + factor + P + quantize)"
 # dram__bytes_read.sum + dram__bytes_write.sum of one stats_umma_kernel launch (one token batch), from
 # the ncu capture summarised in profiles/stats_umma_kernel_cfg2_batch.md; keyed by (workload, statistics
 # arithmetic).  Entries are dropped when the kernel changes.
-STATS_KERNEL_TRAFFIC = {("cfg2", 0): 636.7e6}
+STATS_KERNEL_TRAFFIC = {("cfg2", 0): 597.2e6}
 
 
 def peaks():
