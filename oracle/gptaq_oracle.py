@@ -177,8 +177,8 @@ def dequant(code: np.ndarray, scale: np.ndarray, zero: np.ndarray) -> np.ndarray
 
 
 def clip_candidates(w: np.ndarray, bits: int, sym: bool, steps: int, min_ratio: float):
-    """All candidate grids of the clipping-range search (setup of Section 5; the paper only says the
-    range "is searched by minimizing mean squared error"): candidate k shrinks the min/max range by
+    """All candidate grids of the clipping-range search (setup of Section 5; the paper says only that
+    the range is chosen for the least squared error): candidate k shrinks the min/max range by
     p_k = 1 - k (1 - min_ratio) / steps.  Returns (scales, zeros, errors), each ``[steps, rows]``;
     errors are the sums of squared rounding errors of ``w`` on the candidate grid."""
     w = np.asarray(w, dtype=F64)
@@ -427,7 +427,9 @@ def follow(W: np.ndarray, U: np.ndarray, P: np.ndarray | None, dead,
         bad = got != want
         if bad.any():
             frac = np.abs(t[bad] - np.floor(t[bad]) - 0.5)   # distance to x.5
-            near = (frac <= band) & (np.abs(got[bad] - want[bad]) <= 1.0)
+            # the tie's other choice: of floor(t) and floor(t) + 1, the one that rint did not take
+            other = np.clip(2.0 * np.floor(t[bad]) + 1.0 - np.rint(t[bad]) + z[bad], 0.0, maxq)
+            near = (frac <= band) & (got[bad] == other)
             mism += int(bad.sum())
             allowed += int(near.sum())
             disallowed += int((~near).sum())
