@@ -5,7 +5,7 @@
  * the quantized layer fed with the quantized model's input X reproduces the
  * full-precision layer fed with the full-precision input X~ (the paper's
  * asymmetric calibration objective, Eq. "asym obj", Section 4).  The calls
- * follow Algorithm 1 of the paper line by line:
+ * map to the steps of Algorithm 1 of the paper:
  *
  *   gptaq_accumulate   line 2   H += X X^T,  dXX^T += (X~ - X) X^T
  *   gptaq_factor       line 3   L = Inverse_Cholesky(H + lambda_1 I), kept as U = L^T
@@ -128,7 +128,7 @@ gptaq_status_t gptaq_accumulate_host(gptaq_handle_t h, const float *h_X, const f
                                      int64_t tokens, int64_t ld, void *d_stage, size_t stage_bytes,
                                      gptaq_stream_t stream);
 
-/* Algorithm 1, line 3 with the "standard GPTQ procedure" of Section 4:
+/* Algorithm 1, line 3, with the customary GPTQ preprocessing that Section 4 refers to:
  * H <- H / tokens; inputs with H_qq == 0 get H_qq = 1 (their weight columns
  * are zeroed by gptaq_quantize); H_d = H + damp * mean(diag H) * I; then the
  * upper factor U of H_d^-1 = U^T U (U = L^T of the paper) overwrites H
@@ -185,7 +185,12 @@ gptaq_status_t gptaq_quantize_host(gptaq_handle_t h, const float *h_W, int64_t m
  * any library.
  *   d_U, d_P   [n x n] float32, leading dimension n: U (upper, H_d^-1 = U^T U) and P (strictly
  *              upper), e.g. gptaq_H / gptaq_D of a handle after gptaq_build_P, or restored
- *              copies of them.  All n inputs are taken as live (no dead-input flags).
+ *              copies of them.  All n inputs are taken as live: there are no dead-input flags
+ *              here, so a caller whose layer has inputs that never fired (H_qq = 0) zeroes those
+ *              columns of W itself before the call, as gptaq_quantize would.  U and P of a
+ *              handle with act_order enabled are in SORTED column order: such a caller passes W
+ *              with its columns gathered by gptaq_perm and scatters the codes and dequantized
+ *              weights back; this entry point does not permute.
  *   d_status   device int64[2] or NULL: receives the status a handle would record
  *              (GPTAQ_OK or GPTAQ_ERR_NONFINITE) and the row index that goes with it.
  *   All other arguments as in gptaq_quantize.
@@ -228,7 +233,7 @@ gptaq_status_t gptaq_set_stats_precision(gptaq_handle_t h, int precision);
  * layer of width n calibrated on total_tokens tokens. */
 int gptaq_recommended_stats_precision(int64_t n, int64_t total_tokens);
 
-/* act_order (Section 5, experimental setup: "act_order, which sorts the columns by the Hessian diagonal"):
+/* act_order (Section 5, experimental setup: columns processed in the order of the Hessian's diagonal):
  * when enabled (before gptaq_factor), gptaq_factor orders the inputs by decreasing diag(H) (dead inputs
  * count as 1; ties keep the lower index first), permutes H and dXX^T accordingly, and gptaq_quantize
  * processes the weight columns in that order.  Outputs: d_codes and d_Wq in the CALLER's column order;
@@ -240,8 +245,8 @@ int gptaq_recommended_stats_precision(int64_t n, int64_t total_tokens);
 gptaq_status_t gptaq_set_act_order(gptaq_handle_t h, int enable);
 const int32_t *gptaq_perm(gptaq_handle_t h);
 
-/* Clipping-range search of the quantization grids (Section 5, setup: "the weight clipping range is
- * searched by minimizing mean squared error"; the paper gives no further detail).  With steps > 0 every
+/* Clipping-range search of the quantization grids by least squared rounding error (experimental
+ * setup of Section 5; the paper gives no further detail).  With steps > 0 every
  * grid -- per output channel, or per group at the group's first column -- is chosen among `steps`
  * candidates that shrink the min/max range by p_k = 1 - k (1 - min_ratio) / steps, k = 0 .. steps - 1:
  * the candidate with the smallest sum of squared rounding errors over the grid's weights, the widest one

@@ -16,6 +16,12 @@ TOL_OBJECTIVE = 1e-3      # relative difference of the layer objective
 TOL_FACTOR = 1e-4         # relative Frobenius error of U
 TOL_FLIP_BAND = 1e-4      # distance to a rounding boundary that excuses a flip
 TOL_FLIP_RATE = 1e-3      # at most 0.1 % excused flips
+# Group scales and zero points are functions of already-updated weights.  In follow mode the oracle
+# replays a row with its own float64 U and P, so its group extremes differ from the device's by what the
+# device's U and P contribute to the accumulated update: at most TOL_FACTOR of the update's size, and
+# the update of a weight stays below half the group's range.  Hence TOL_FACTOR / 2 relative on the scale
+# (observed: 1e-6 .. 1.3e-5); a replay from the device's own U and P would see float32 rounding only.
+TOL_GRID = 0.5 * TOL_FACTOR
 
 
 @dataclasses.dataclass
@@ -126,9 +132,9 @@ def assert_parity(out):
     assert out["J_rel"] <= TOL_OBJECTIVE, out
     assert rep.disallowed == 0, rep
     assert rep.allowed <= TOL_FLIP_RATE * rep.total, rep
-    # group grids come from weights that carry the factor's error: same order as TOL_FACTOR
-    assert rep.grid_rel_err <= 5e-5 and rep.zero_mismatch == 0, rep
+    assert rep.grid_rel_err <= TOL_GRID and rep.zero_mismatch == 0, rep
     assert out["dequant_consistent"], out
-    # never worse than plain rounding, unless the method itself is (the float64 result then is as well:
-    # coarse symmetric grids at 2 bits can do that on the asymmetric objective)
+    # never worse than plain rounding, unless the float64 method itself is: the ordering is empirical, and
+    # tests/test_oracle_pins.py::test_two_bit_symmetric_group_grids_can_lose_to_plain_rounding names a layer
+    # (2-bit symmetric group grids, outlier channels) where the oracle ends 3.7 % above plain rounding
     assert out["J_gpu"] <= max(out["J_rtn"], out["J_oracle"] * (1.0 + TOL_OBJECTIVE)), out

@@ -7,13 +7,19 @@ cfg3 (n = 14,336) and cfg5 (n = 53,248) are too large for that (2e14 / 1.5e15 fl
 there the oracle checks sampled outputs it can compute one by one and properties that hold at
 any size, stage by stage:
   statistics   sampled entries H[i, j], dXX^T[i, j] against float64 sums over all tokens;
-  factor       U upper with positive diagonal and  u_i H_d u_j^T = delta_ij  for sampled rows
-               (H_d from the device's own H, widened to float64): orthonormality of the rows of
-               U in the H_d inner product is the definition of the factor, and its defect is
-               twice the relative error of U;
-  P            sampled rows against Theorem 4.2 evaluated in float64 from the device's D and U;
-  loop         sampled rows of W replayed in follow mode and free-running from the device's U
-               and P (rows are independent), with the flip accounting and the objective bound.
+  factor       cfg3: the whole of U against the oracle's factor of the device's sums widened to
+               float64 (relative Frobenius error, the bound of the benchmark spec), stage-wise.
+               cfg5: a float64 factorisation of a 53,248-wide matrix (four 22.7 GB matrices, 6e14
+               flops) is out of reach of a test; there U is checked to be upper with a positive
+               diagonal and  u_i H_d u_j^T = delta_ij  for 77 sampled rows, the first row of every
+               1024-column super-panel of the factorisation among them (H_d from the device's own
+               H, widened to float64): orthonormality of the rows of U in the H_d inner product is
+               the definition of the factor, and its defect is twice the relative error of U;
+  P            cfg3: the whole of P against Theorem 4.2 evaluated by the oracle from the device's
+               dXX^T and the oracle's U; cfg5: sampled rows, from the device's dXX^T and U;
+  loop         sampled rows of W replayed in follow mode and free-running (rows are independent),
+               with the flip accounting and the objective bound: from the oracle's U and P on
+               cfg3, from the device's U and P on cfg5.
 """
 import time
 
@@ -78,7 +84,7 @@ def _check_rows(cfg, W_rows, U, P, codes, scales, zeros, Wq_rows, objective):
     rep = orc.follow(W_rows, U, P, dead, cfg.bits, cfg.group, cfg.sym, codes, scales, zeros, band=hp.TOL_FLIP_BAND)
     assert rep.disallowed == 0, rep
     assert rep.allowed <= hp.TOL_FLIP_RATE * rep.total, rep
-    assert rep.grid_rel_err <= 5e-5 and rep.zero_mismatch == 0, rep
+    assert rep.grid_rel_err <= hp.TOL_GRID and rep.zero_mismatch == 0, rep
     res = orc.quantize(W_rows, U, P, dead, cfg.bits, cfg.group, cfg.sym)
     rtn = orc.quantize(W_rows, U, None, dead, cfg.bits, cfg.group, cfg.sym, update=False)
     J_gpu, J_orc, J_rtn = objective(Wq_rows), objective(res.Wq), objective(rtn.Wq)
@@ -182,12 +188,27 @@ def test_large_configs_sampled_parity(name, n_rows, n_cols):
         assert float(torch.tril(blk, diagonal=r0 - 1).abs().max()) == 0.0
     assert float(torch.diagonal(Ud).min()) > 0.0
     U_host = Ud.cpu().numpy()
-    urows = np.sort(rng.choice(cfg.n, 12, replace=False))
-    urows[0], urows[-1] = 0, cfg.n - 1
-    Gm = _upper_quadratic(H_host, U_host[urows].astype(np.float64), lam, 1.0 / tokens)
-    defect = np.abs(Gm - np.eye(len(urows))).max()
-    assert defect <= 2 * hp.TOL_FACTOR, defect
-    # ---- P: sampled rows against Theorem 4.2 in float64
+    U_ref = P_ref = None
+    if name == "cfg3":
+        # the whole factor against the oracle's, from the same (device) sums widened to float64
+        H64 = np.triu(H_host).astype(np.float64)
+        H64 += np.triu(H64, 1).T
+        U_ref, dead = orc.factor(H64, tokens, cfg.damp)
+        del H64
+        assert not dead.any()
+        U_rel = hp.rel_fro(np.triu(U_host).astype(np.float64), U_ref)
+        assert U_rel <= hp.TOL_FACTOR, U_rel
+        defect = U_rel
+    else:
+        # rows of U: the first row of every super-panel of the factorisation (1024 columns), the last
+        # row of the matrix and 24 random ones
+        urows = np.unique(np.concatenate([np.arange(0, cfg.n, 1024), [cfg.n - 1],
+                                          rng.choice(cfg.n, 24, replace=False)]))
+        assert len(urows) >= 64
+        Gm = _upper_quadratic(H_host, U_host[urows].astype(np.float64), lam, 1.0 / tokens)
+        defect = np.abs(Gm - np.eye(len(urows))).max()
+        assert defect <= 2 * hp.TOL_FACTOR, defect
+    # ---- P
     g.gptaq_build_P(st.handle, cfg.alpha)
     assert g.gptaq_sync_status(st.handle)[0] == g.GPTAQ_OK
     Pd = st.D()
@@ -195,19 +216,26 @@ def test_large_configs_sampled_parity(name, n_rows, n_cols):
         blk = Pd[r0:r0 + 4096, :r0 + 4096]
         assert float(torch.tril(blk, diagonal=r0).abs().max()) == 0.0
     P_host = Pd.cpu().numpy()
-    prow = np.sort(rng.choice(cfg.n - 1, 6, replace=False))
-    prow[0] = 0
-    P_want = orc.build_P_rows(D_host[prow], prow, tokens, U_host, cfg.alpha)
-    P_err = np.linalg.norm(P_host[prow] - P_want) / np.linalg.norm(P_want)
+    if name == "cfg3":
+        # the whole of P by Theorem 4.2 from the oracle's factor
+        P_ref = orc.build_P(D_host, tokens, U_ref, cfg.alpha)
+        P_err = hp.rel_fro(np.triu(P_host, 1).astype(np.float64), P_ref)
+    else:
+        # sampled rows against Theorem 4.2 in float64
+        prow = np.sort(rng.choice(cfg.n - 1, 6, replace=False))
+        prow[0] = 0
+        P_want = orc.build_P_rows(D_host[prow], prow, tokens, U_host, cfg.alpha)
+        P_err = np.linalg.norm(P_host[prow] - P_want) / np.linalg.norm(P_want)
     assert P_err <= 1e-4, P_err
     # ---- loop: sampled rows
     W = wl.make_weight(cfg, "cuda")
     codes, scales, zeros, Wq = _quantize_on_device(cfg, st, W)
     del W
     rep, J_gpu, J_orc, J_rtn, free = _check_rows(
-        cfg, W_rows, U_host, P_host, *_rows_to_host(rows, codes, scales, zeros, Wq),
+        cfg, W_rows, U_host if U_ref is None else U_ref, P_host if P_ref is None else P_ref,
+        *_rows_to_host(rows, codes, scales, zeros, Wq),
         lambda q: orc.objective_terms_chunked(W_rows, q, H_host, D_host) + resid)
-    print(f"{name} full size: H err {errH:.2e}, D err {errD:.2e}, U defect {defect:.2e}, P rows rel {P_err:.2e}, "
+    print(f"{name} full size: H err {errH:.2e}, D err {errD:.2e}, U {'rel' if U_ref is not None else 'defect'} {defect:.2e}, P rel {P_err:.2e}, "
           f"flips {rep.mismatches}/{rep.total} (excused {rep.allowed}), free-running mismatch {free:.2e}, "
           f"J gpu/oracle/rtn {J_gpu:.6g}/{J_orc:.6g}/{J_rtn:.6g}, {time.time() - t0:.0f} s")
     st.close()

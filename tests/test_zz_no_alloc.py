@@ -6,7 +6,9 @@ they cannot size a per-layer workspace for the lazy-batch update.  For them the 
 a fixed scratch array of its own.  This file checks, through the C ABI, that the entry point
 built on that array gives exactly what gptaq_quantize gives on the same factor, correction
 matrix and weights, on two calls in a row (the second finds the first call's leftovers in the
-shared array), and that sizes beyond the array are refused on the host.
+shared array), that a layer wide enough for gptaq_quantize to switch to its tensor-core update
+(which this entry point never uses) still matches the float64 oracle, and that sizes beyond the
+array are refused on the host.
 
 The file name sorts last on purpose: a run that stops at the first failure has then already
 been through every other test.
@@ -17,6 +19,8 @@ import torch
 
 import paper_2504_02692_b200 as g
 import workloads as wl
+from oracle import gptaq_oracle as orc
+from tests import helpers as hp
 
 pytestmark = pytest.mark.gpu
 
@@ -64,6 +68,45 @@ def test_static_scratch_entry_point_matches_gptaq_quantize_twice_in_a_row():
         assert np.array_equal(zeros2.cpu().numpy(), zeros.cpu().numpy())
         assert np.array_equal(scales2.cpu().numpy(), scales.cpu().numpy())
         assert np.array_equal(Wq2.cpu().numpy(), Wq.cpu().numpy())
+    st.close()
+
+
+def test_static_scratch_entry_point_against_the_oracle_on_a_wide_layer():
+    """n = 640: gptaq_quantize takes the split-fp16 tensor-core update from this width on, the entry
+    point without a workspace keeps the float32 FMA update, so the two no longer agree bit for bit.
+    Both have to match the oracle: codes in follow mode, objective, and never worse than plain
+    rounding -- on two calls in a row, the second on fewer rows."""
+    cfg = wl.scaled(wl.CONFIGS["cfg2"], name="static_wide", n=640, m=104, batch_tokens=2560, n_batches=2,
+                    outlier_channels=6, group=128, blocksize=128)
+    batches = [wl.make_batch(cfg, b) for b in range(cfg.n_batches)]
+    st = _factored_state(cfg)
+    Ud, Pd = st.H().clone(), st.D().clone()
+    ost = hp.oracle_stats(cfg, batches)
+    U, dead = orc.factor(ost.H, ost.tokens, cfg.damp)
+    P = orc.build_P(ost.D, ost.tokens, U, cfg.alpha)
+    assert not dead.any()
+    assert hp.rel_fro(np.triu(Ud.cpu().numpy().astype(np.float64)), U) <= hp.TOL_FACTOR
+    W_all = wl.make_weight(cfg)
+    status = torch.full((2,), -1, dtype=torch.int64, device="cuda")
+    for W in (W_all, W_all[11:80].contiguous() * 0.7):
+        m = W.shape[0]
+        Wn = W.numpy().astype(np.float64)
+        codes, scales, zeros, Wq = _outputs(m, cfg.n, cfg.group)
+        g.gptaq_quantize_static(Ud, Pd, W.cuda(), cfg.bits, cfg.group, cfg.sym, cfg.blocksize, codes, scales, zeros,
+                                Wq, status)
+        torch.cuda.synchronize()
+        assert status.tolist() == [g.GPTAQ_OK, 0]
+        rep = orc.follow(Wn, U, P, dead, cfg.bits, cfg.group, cfg.sym, codes.cpu().numpy(),
+                         scales.cpu().numpy().astype(np.float64), zeros.cpu().numpy().astype(np.float64),
+                         band=hp.TOL_FLIP_BAND)
+        assert rep.disallowed == 0 and rep.allowed <= hp.TOL_FLIP_RATE * rep.total, rep
+        assert rep.grid_rel_err <= hp.TOL_GRID and rep.zero_mismatch == 0, rep
+        res = orc.quantize(Wn, U, P, dead, cfg.bits, cfg.group, cfg.sym)
+        rtn = orc.quantize(Wn, U, None, dead, cfg.bits, cfg.group, cfg.sym, update=False)
+        J_gpu = orc.objective(Wn, Wq.cpu().numpy().astype(np.float64), ost)
+        J_orc, J_rtn = orc.objective(Wn, res.Wq, ost), orc.objective(Wn, rtn.Wq, ost)
+        assert abs(J_gpu - J_orc) <= hp.TOL_OBJECTIVE * J_orc, (J_gpu, J_orc)
+        assert J_gpu <= J_rtn, (J_gpu, J_rtn)
     st.close()
 
 
