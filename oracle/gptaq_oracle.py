@@ -231,9 +231,27 @@ def _ngroups(n: int, group: int) -> int:
     return 1 if group <= 0 else (n + group - 1) // group
 
 
+def static_group_grids(W: np.ndarray, dead: np.ndarray | None, bits: int, group: int, sym: bool, clip=None):
+    """Static groups (the companion of act_order in the setup of Section 5: per-group grids that survive a
+    column permutation): one grid per output channel and per group of ``group`` consecutive columns of the
+    ORIGINAL column order, taken from the original weights before the loop starts.  Returns
+    (scales, zeros), each ``[m, ceil(n / group)]``."""
+    W = np.array(W, dtype=F64)
+    if dead is not None and dead.any():
+        W[:, dead] = 0.0
+    m, n = W.shape
+    ng = _ngroups(n, group)
+    make = _grid_fn(bits, sym, clip)
+    scales = np.zeros((m, ng), F64)
+    zeros = np.zeros((m, ng), F64)
+    for g in range(ng):
+        scales[:, g], zeros[:, g] = make(W[:, g * group:(g + 1) * group])
+    return scales, zeros
+
+
 def quantize(W: np.ndarray, U: np.ndarray, P: np.ndarray | None, dead: np.ndarray | None,
              bits: int, group: int, sym: bool, update: bool = True,
-             keep_pre: bool = False, error_term: bool = True, clip=None) -> QuantResult:
+             keep_pre: bool = False, error_term: bool = True, clip=None, static=None) -> QuantResult:
     """Unblocked column loop (Eq. "divided update"), all rows at once.
 
     For column j: quantize the current column, e = (w - q) / U[j, j], then
@@ -241,6 +259,9 @@ def quantize(W: np.ndarray, U: np.ndarray, P: np.ndarray | None, dead: np.ndarra
     just before it was quantized.  ``P = None`` drops the second term (GPTQ);
     ``error_term = False`` drops the first (the ablation's GPTAQ');
     ``update = False`` drops both (round to nearest).
+    ``static = (scales, zeros, group_of_column)``: static groups -- the grids are given (see
+    static_group_grids) and column j uses grid number ``group_of_column[j]``; nothing is re-taken from
+    updated weights.
     """
     W = np.array(W, dtype=F64)
     m, n = W.shape
@@ -253,11 +274,16 @@ def quantize(W: np.ndarray, U: np.ndarray, P: np.ndarray | None, dead: np.ndarra
     Wq = np.zeros((m, n), F64)
     pre = np.zeros((m, n), F64) if keep_pre else None
     make = _grid_fn(bits, sym, clip)      # ``clip = (steps, min_ratio)``: clipping-range search of every grid
-    if group <= 0:
+    if static is not None:
+        scales, zeros = np.array(static[0], F64), np.array(static[1], F64)
+        gidx = np.asarray(static[2])
+    elif group <= 0:
         s, z = make(W)
         scales[:, 0], zeros[:, 0] = s, z
     for j in range(n):
-        if group > 0 and j % group == 0:
+        if static is not None:
+            s, z = scales[:, gidx[j]], zeros[:, gidx[j]]
+        elif group > 0 and j % group == 0:
             s, z = make(W[:, j:j + group])
             scales[:, j // group], zeros[:, j // group] = s, z
         w = W[:, j].copy()
@@ -378,7 +404,10 @@ class FollowReport:
 def follow(W: np.ndarray, U: np.ndarray, P: np.ndarray | None, dead,
            bits: int, group: int, sym: bool,
            cand_codes: np.ndarray, cand_scales: np.ndarray, cand_zeros: np.ndarray,
-           band: float = 1e-4, error_term: bool = True, clip=None) -> FollowReport:
+           band: float = 1e-4, error_term: bool = True, clip=None, static=None) -> FollowReport:
+    """``static = (W_original, group_of_column)``: static groups -- the candidate's grids are judged once,
+    against the grids of the original weights in their original column order (``W`` is then the working copy
+    in processing order), and column j uses the candidate's grid number ``group_of_column[j]``."""
     W = np.array(W, dtype=F64)
     m, n = W.shape
     if dead is not None and dead.any():
@@ -415,10 +444,17 @@ def follow(W: np.ndarray, U: np.ndarray, P: np.ndarray | None, dead,
             zero_mis += int(bad.sum())
         return s_c, z_c
 
-    if group <= 0:
+    if static is not None:
+        W0 = np.array(static[0], dtype=F64)
+        gidx = np.asarray(static[1])
+        for g in range(cand_scales.shape[1]):
+            check_grid(W0[:, g * group:(g + 1) * group], g)
+    elif group <= 0:
         s, z = check_grid(W, 0)
     for j in range(n):
-        if group > 0 and j % group == 0:
+        if static is not None:
+            s, z = cand_scales[:, gidx[j]], cand_zeros[:, gidx[j]]
+        elif group > 0 and j % group == 0:
             s, z = check_grid(W[:, j:j + group], j // group)
         w = W[:, j].copy()
         t = w / s
@@ -470,11 +506,13 @@ def act_order_perm(H_sum: np.ndarray, tokens: int) -> np.ndarray:
     return np.argsort(-d, kind="stable")
 
 
-def solve_act_order(W, H_sum, D_sum, tokens, damp, alpha, bits, group, sym, perm=None):
+def solve_act_order(W, H_sum, D_sum, tokens, damp, alpha, bits, group, sym, perm=None, static_groups=False):
     """Algorithm 1 on the layer with its inputs relabelled by ``perm`` (default: act_order_perm):
     H and dXX^T are permuted on both sides, W on its columns; codes and dequantized weights are
-    returned in the original column order, group grids belong to groups of consecutive columns of
-    the sorted order.  Returns (U, P, dead, result, perm), U / P / dead in sorted order."""
+    returned in the original column order.  Group grids belong to groups of consecutive columns of
+    the sorted order, or, with ``static_groups``, to groups of consecutive columns of the ORIGINAL order
+    (taken from the original weights; the column at sorted position j uses group ``perm[j] // group``).
+    Returns (U, P, dead, result, perm), U / P / dead in sorted order."""
     W = np.asarray(W, F64)
     if perm is None:
         perm = act_order_perm(H_sum, tokens)
@@ -483,7 +521,13 @@ def solve_act_order(W, H_sum, D_sum, tokens, damp, alpha, bits, group, sym, perm
     Dp = np.asarray(D_sum, F64)[np.ix_(perm, perm)]
     U, dead = factor(Hp, tokens, damp)
     P = build_P(Dp, tokens, U, alpha)
-    res = quantize(W[:, perm], U, P, dead, bits, group, sym)
+    static = None
+    if static_groups and group > 0:
+        dead0 = np.zeros(W.shape[1], bool)
+        dead0[perm] = dead
+        sc, zr = static_group_grids(W, dead0, bits, group, sym)
+        static = (sc, zr, perm // group)
+    res = quantize(W[:, perm], U, P, dead, bits, group, sym, static=static)
     codes = np.empty_like(res.codes)
     Wq = np.empty_like(res.Wq)
     codes[:, perm] = res.codes

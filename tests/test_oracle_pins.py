@@ -438,6 +438,50 @@ def test_objective_identity():
     assert abs(orc.objective(W, W, st) - np.sum(((Xfp - X) @ W.T) ** 2)) < 1e-10
 
 
+def test_static_groups_index_original_columns_and_survive_relabelling():
+    """Static groups: (i) without weight updates they are plain per-group rounding, whatever the processing
+    order; (ii) under act_order the outputs, returned in the original column order, dequantize with the grid of
+    group column // group -- the layout that needs no index table; (iii) the grids are those of the original
+    weights; (iv) relabelling the inputs inside their groups relabels the result and changes nothing else."""
+    n, m, group, bits = 32, 6, 8, 4
+    W, X, Xfp = tiny(n=n, m=m, k=300)
+    X *= np.linspace(0.5, 2.5, n)[None, ::-1] ** 0.5 * (1.0 + 0.37 * np.sin(np.arange(n)))[None, :]   # distinct diag(H)
+    Xfp *= np.linspace(0.5, 2.5, n)[None, ::-1] ** 0.5 * (1.0 + 0.37 * np.sin(np.arange(n)))[None, :]
+    st = stats_of(X, Xfp)
+    # (i) round to nearest: static grids in any order == dynamic grids in the natural order
+    U, dead = orc.factor(st.H, st.tokens, 0.01)
+    sc, zr = orc.static_group_grids(W, dead, bits, group, False)
+    rtn = orc.quantize(W, U, None, dead, bits, group, False, update=False)
+    assert np.array_equal(sc, rtn.scales) and np.array_equal(zr, rtn.zeros)
+    perm = orc.act_order_perm(st.H, st.tokens)
+    assert not np.array_equal(perm, np.arange(n))
+    rtn_p = orc.quantize(W[:, perm], U, None, dead, bits, group, False, update=False, static=(sc, zr, perm // group))
+    assert np.array_equal(rtn_p.codes, rtn.codes[:, perm])
+    # (ii), (iii)
+    Us, Ps, deads, res, perm2 = orc.solve_act_order(W, st.H, st.D, st.tokens, 0.01, 0.25, bits, group, False,
+                                                    static_groups=True)
+    assert np.array_equal(perm2, perm)
+    assert np.array_equal(res.scales, sc) and np.array_equal(res.zeros, zr)
+    g_of = np.arange(n) // group
+    assert np.allclose(res.Wq, res.scales[:, g_of] * (res.codes.astype(float) - res.zeros[:, g_of]), atol=0, rtol=0)
+    dyn = orc.solve_act_order(W, st.H, st.D, st.tokens, 0.01, 0.25, bits, group, False)[3]
+    assert not np.array_equal(dyn.codes, res.codes)          # the sorted-order groups are something else
+    # (iv) swap columns inside groups (a relabelling that keeps every column in its group)
+    rel = np.arange(n).reshape(-1, group)[:, ::-1].reshape(-1)
+    st_r = stats_of(X[:, rel], Xfp[:, rel])
+    res_r = orc.solve_act_order(W[:, rel], st_r.H, st_r.D, st_r.tokens, 0.01, 0.25, bits, group, False,
+                                static_groups=True)[3]
+    assert np.array_equal(res_r.codes, res.codes[:, rel])
+    assert np.array_equal(res_r.scales, res.scales) and np.array_equal(res_r.zeros, res.zeros)
+    # follow mode accepts the result and refuses a grid from updated weights
+    rep = orc.follow(W[:, perm], Us, Ps, deads, bits, group, False, res.codes[:, perm], res.scales, res.zeros,
+                     static=(W, perm // group))
+    assert rep.mismatches == 0 and rep.grid_rel_err == 0.0 and rep.zero_mismatch == 0
+    rep = orc.follow(W[:, perm], Us, Ps, deads, bits, group, False, res.codes[:, perm], dyn.scales, dyn.zeros,
+                     static=(W, perm // group))
+    assert rep.grid_rel_err > 1e-3
+
+
 # ---------------------------------------------------------------- follow mode
 def test_follow_mode_accepts_own_output_and_flags_planted_errors():
     W, X, Xfp = tiny(n=32, m=12)
