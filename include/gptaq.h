@@ -90,8 +90,10 @@ size_t gptaq_state_bytes(int64_t n);
  * (Algorithm 1, input B).  max_batch_tokens is the largest `tokens` that
  * gptaq_accumulate will be given in one call (larger batches still work: they
  * are processed in chunks that fit).  For n >= 512 the scratch holds split (high part / low part)
- * operand copies of U^T and P^T for the tensor cores (about 7 n^2 floats in all): the library reads them in every gptaq_quantize, so the
- * workspace must be left untouched from gptaq_factor until the last gptaq_quantize on this state. */
+ * operand copies of U^T and P^T for the tensor cores: about 4 n^2 floats in all where n is a multiple
+ * of 8 (fp16 parts), about 7 n^2 where it is a multiple of 4 only (TF32 parts).  The library reads them
+ * in every gptaq_quantize, so the workspace must be left untouched from gptaq_factor until the last
+ * gptaq_quantize on this state. */
 size_t gptaq_workspace_bytes(int64_t n, int64_t m_max, int64_t max_batch_tokens, int blocksize);
 
 /* Creates a handle over caller-owned device buffers (both 256-byte aligned)
@@ -140,6 +142,14 @@ gptaq_status_t gptaq_factor(gptaq_handle_t h, float damp, gptaq_stream_t stream)
  * alpha = 1 is the paper's P; alpha = 0 reduces the solve to GPTQ.
  * P overwrites dXX^T (lower triangle and diagonal zero). */
 gptaq_status_t gptaq_build_P(gptaq_handle_t h, float alpha, gptaq_stream_t stream);
+
+/* The same P computed row by row, Eq. "unparallel" (Section 4, Step 3):
+ *   P[q, q+1:] = alpha * dXX^T[q, q+1:] L[q+1:, q+1:] L[q+1:, q+1:]^T,   L = U^T,
+ * i.e. two passes over the trailing triangle of U for every row q: the form that Theorem 4.2 replaces by
+ * two matrix products.  It exists as the slow side of the latency comparison of Section 5 ("Efficiency")
+ * and gives the same P up to rounding; the solve itself uses gptaq_build_P.  Same call order and effects
+ * as gptaq_build_P; n <= 16384 (GPTAQ_ERR_UNSUPPORTED beyond). */
+gptaq_status_t gptaq_build_P_rowwise(gptaq_handle_t h, float alpha, gptaq_stream_t stream);
 
 /* Algorithm 1, lines 5-13, for one weight matrix sharing this state.
  *   d_W      [m x ldw], float32 or bf16 (w_dtype).  If d_Wq is given, d_W is read
@@ -244,6 +254,15 @@ int gptaq_recommended_stats_precision(int64_t n, int64_t total_tokens);
  * gptaq_perm: device array of n int32, sorted position -> caller column; NULL unless enabled and factored. */
 gptaq_status_t gptaq_set_act_order(gptaq_handle_t h, int enable);
 const int32_t *gptaq_perm(gptaq_handle_t h);
+
+/* Static groups (Section 5, setup of the per-group results with act_order): when enabled, later gptaq_quantize
+ * calls with group > 0 take every group grid BEFORE the loop, from the original weights, for groups of
+ * `group` consecutive columns of the CALLER's column order; a column keeps the grid of its own group wherever
+ * act_order moves it in the processing order.  d_scales / d_zeros [m x G] then index caller column c by
+ * c / group, with or without act_order -- no index table is needed to dequantize.  Without act_order the
+ * only difference from the default is that grids come from the original instead of the updated weights.
+ * Such calls take the general column kernel (one warp per row), not the 32-columns-per-thread one. */
+gptaq_status_t gptaq_set_static_groups(gptaq_handle_t h, int enable);
 
 /* Clipping-range search of the quantization grids by least squared rounding error (experimental
  * setup of Section 5; the paper gives no further detail).  With steps > 0 every

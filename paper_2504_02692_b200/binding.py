@@ -47,6 +47,7 @@ SIGNATURES = {
     "gptaq_accumulate_host": (_int, [_vp, _vp, _vp, _i64, _i64, _vp, _sz, _vp]),
     "gptaq_factor": (_int, [_vp, _f, _vp]),
     "gptaq_build_P": (_int, [_vp, _f, _vp]),
+    "gptaq_build_P_rowwise": (_int, [_vp, _f, _vp]),
     "gptaq_quantize": (_int, [_vp, _vp, _int, _i64, _i64, _int, _int, _int, _int, _vp, _vp, _vp, _vp, _vp]),
     "gptaq_quantize_stage_bytes": (_sz, [_i64, _i64, _int]),
     "gptaq_quantize_host": (_int, [_vp, _vp, _i64, _i64, _int, _int, _int, _int, _vp, _vp, _vp, _vp, _vp, _sz, _vp]),
@@ -64,6 +65,7 @@ SIGNATURES = {
     "gptaq_set_update_terms": (_int, [_vp, _int]),
     "gptaq_set_clip_search": (_int, [_vp, _int, _f]),
     "gptaq_set_act_order": (_int, [_vp, _int]),
+    "gptaq_set_static_groups": (_int, [_vp, _int]),
     "gptaq_perm": (_vp, [_vp]),
     "gptaq_recommended_stats_precision": (_int, [_i64, _i64]),
     "gptaq_launch_count": (_i64, [_vp]),
@@ -197,6 +199,11 @@ def gptaq_build_P(h, alpha: float, stream=None):
     _check(load_library().gptaq_build_P(h, alpha, _stream(stream)), "gptaq_build_P", h)
 
 
+def gptaq_build_P_rowwise(h, alpha: float, stream=None):
+    """P row by row (the comparison form of the paper's latency discussion); same result as gptaq_build_P."""
+    _check(load_library().gptaq_build_P_rowwise(h, alpha, _stream(stream)), "gptaq_build_P_rowwise", h)
+
+
 def gptaq_quantize(h, d_W: torch.Tensor, bits: int, group: int, sym: bool, blocksize: int,
                    d_codes: torch.Tensor, d_scales: torch.Tensor, d_zeros: torch.Tensor,
                    d_Wq: torch.Tensor | None = None, stream=None):
@@ -295,6 +302,11 @@ def gptaq_set_act_order(h, enable: bool):
     _check(load_library().gptaq_set_act_order(h, int(bool(enable))), "gptaq_set_act_order", h)
 
 
+def gptaq_set_static_groups(h, enable: bool):
+    """Group grids from the original weights, per group of the caller's columns (they survive act_order)."""
+    _check(load_library().gptaq_set_static_groups(h, int(bool(enable))), "gptaq_set_static_groups", h)
+
+
 def gptaq_perm_ptr(h) -> int | None:
     return load_library().gptaq_perm(h)
 
@@ -361,6 +373,13 @@ class LayerState:
         """View of dXX^T (before build_P) / P (after), current on torch's stream."""
         gptaq_flush(self.handle)
         return self._view(gptaq_D_ptr(self.handle))
+
+    def tokens(self) -> int:
+        """Tokens accumulated so far (the divisor gptaq_factor will use)."""
+        return gptaq_tokens(self.handle)
+
+    def set_tokens(self, tokens: int):
+        gptaq_set_tokens(self.handle, tokens)
 
     def perm(self) -> torch.Tensor | None:
         """act_order: int32 ``[n]``, sorted position -> caller column (None unless enabled and factored)."""

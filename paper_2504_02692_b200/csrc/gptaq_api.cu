@@ -25,6 +25,7 @@ inline size_t round_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 
 enum Stage { STAGE_ACCUM = 0, STAGE_FACTORED = 1, STAGE_P = 2 };
 constexpr int64_t ACT_ORDER_MAX_N = 57344;     // a weight row (float32) has to fit the shared memory of one CTA
+constexpr int64_t P_ROWWISE_MAX_N = 16384;     // two rows (float32) in the shared memory of one CTA
 
 }  // namespace
 
@@ -49,8 +50,8 @@ struct gptaq_ctx {
     bool tensor;           // float32-grade tensor-core GEMMs for factor / P / trailing update
     bool f16;              // ... with FP16-split operands where the producer can record their range (n % 8 == 0)
     TcSched sched;         // tile numbering of the float32-grade GEMM launches (see StateHeader::sched_counter)
-    bool tf32_copies;      // f16 handles: the TF32 copies of U^T and P^T exist (made on demand by gptaq_quantize)
     int terms;             // GPTAQ_TERM_* switches of gptaq_quantize
+    bool static_groups;    // group grids from the original weights, per group of the caller's columns
     int clip_steps; float clip_min;   // clipping-range search of the grids
     // Statistics pipeline: the conversion of a token batch runs on the caller's stream, the
     // tensor-core product on `gemm_stream`, so that the (memory-bound) conversion of the next
@@ -112,10 +113,15 @@ WsLayout ws_layout(int64_t n, int64_t m_max, int blocksize) {
     w.t_off = 0;
     w.rinv_off = w.t_off + mat;
     size_t off = w.rinv_off + round_up(nb * NB * NB * sizeof(float), ALIGN);
-    for (int i = 0; i < 6; ++i) { w.s_off[i] = off; if (w.tensor) off += mat; }
+    const bool f16 = w.tensor && (n % 8) == 0;
+    // split operand copies: six float32-sized regions for TF32 parts; fp16 hi / lo parts use three
+    // (S0 = U^T, S1 = U then P^T, S4 = dXX^T then O; hi and lo of one matrix fill one region)
+    for (int i = 0; i < 6; ++i) {
+        w.s_off[i] = off;
+        if (w.tensor && (!f16 || i == 0 || i == 1 || i == 4)) off += mat;
+    }
     const size_t pan = std::max((size_t)n * NB * sizeof(float), (size_t)n * SUPER_NB * sizeof(__half));
     for (int i = 0; i < 2; ++i) { w.pan_off[i] = off; if (w.tensor) off += round_up(pan, ALIGN); }
-    const bool f16 = w.tensor && (n % 8) == 0;
     const size_t ew1 = round_up((size_t)m_max * 2 * (size_t)blocksize * sizeof(float), ALIGN);
     const size_t ew = f16 ? QSUPER * ew1 : ew1;
     w.ew_off = off;
@@ -383,9 +389,8 @@ gptaq_status_t accumulate_tc(gptaq_ctx *h, const float *X, const float *Xfp, int
         h->relayout = false;
     }
     const int64_t chunk = tc_chunk_tokens(h);
-    const int TM = (n + UBM - 1) / UBM, TN = (n + UBN - 1) / UBN;
-    int64_t ntiles = (int64_t)TM * TN;
-    for (int tm = 0; tm < TM; ++tm) ntiles += TN - (tm * UBM) / UBN;
+    const int64_t ntiles = TileIter::total(n);              // 256 x 256 tiles of H (upper) and dXX^T
+    const int npairs = std::max(1, h->num_sms / 2);         // CTA pairs (clusters of two)
     for (int64_t t0 = 0; t0 < tokens; t0 += chunk) {
         const int tk = (int)std::min<int64_t>(chunk, tokens - t0);
         const int kp = (tk + UBK - 1) / UBK * UBK;
@@ -416,33 +421,32 @@ gptaq_status_t accumulate_tc(gptaq_ctx *h, const float *X, const float *Xfp, int
         LAUNCHED();
         CU(cudaEventRecord(h->conv_done[buf], s));
         CU(cudaStreamWaitEvent(gs, h->conv_done[buf], 0));
-        CUtensorMap mXa, mDa, mXb, mLa, mLb, mDLa;
+        CUtensorMap mX, mD, mL, mDL;
         const __half *lo = split ? Xlo : Xt;    // unused maps still have to be valid
         const __half *dlo = splitd ? dXlo : dXt;
-        if (!make_kmajor_map(&mXa, Xt, n, kp, UBM) || !make_kmajor_map(&mDa, dXt, n, kp, UBM) ||
-            !make_kmajor_map(&mXb, Xt, n, kp, UBN) || !make_kmajor_map(&mLa, lo, n, kp, UBM) ||
-            !make_kmajor_map(&mLb, lo, n, kp, UBN) || !make_kmajor_map(&mDLa, dlo, n, kp, UBM)) {
+        if (!make_kmajor_map(&mX, Xt, n, kp, UBM) || !make_kmajor_map(&mD, dXt, n, kp, UBM) ||
+            !make_kmajor_map(&mL, lo, n, kp, UBM) || !make_kmajor_map(&mDL, dlo, n, kp, UBM)) {
             h->cuda_error = "cuTensorMapEncodeTiled failed";
             return GPTAQ_ERR_CUDA;
         }
         StatsGemmArgs ga;
         ga.H = h->H; ga.D = h->D; ga.n = n; ga.kblocks = kp / UBK; ga.nseg_h = split ? 3 : 1; ga.nseg_d = splitd ? 3 : 1; ga.amax = amax; ga.hd = h->hd;
-        // the last, partial wave of tiles is cut along K so that every SM has work
+        // the last, partial wave of tiles is cut along K so that every pair has work
         ga.ntiles = (int)ntiles;
-        ga.full_tiles = (int)(ntiles / h->num_sms) * h->num_sms;
+        ga.full_tiles = (int)(ntiles / npairs) * npairs;
         ga.ksplit = 1;
         const int cut = (int)ntiles - ga.full_tiles;
         if (cut > 0) {
-            const int by_sms = h->num_sms / cut, by_k = ga.kblocks / (2 * UCHUNK);
-            ga.ksplit = std::max(1, std::min(std::min(by_sms, by_k), 8));
+            const int by_pairs = npairs / cut, by_k = ga.kblocks / (2 * UCHUNK);
+            ga.ksplit = std::max(1, std::min(std::min(by_pairs, by_k), 8));
         }
         if (ga.ksplit == 1) ga.full_tiles = (int)ntiles;
-        // scratch behind the two operand buffers (one partial tile per SM at most; the products run
-        // one after the other on the internal stream, so one scratch serves both buffers)
+        // scratch behind the two operand buffers (one partial 128 x 256 tile per CTA at most; the products
+        // run one after the other on the internal stream, so one scratch serves both buffers)
         ga.scratch = reinterpret_cast<float *>(h->ws + 2 * buf_bytes);
         const int nitems = ga.full_tiles + ((int)ntiles - ga.full_tiles) * ga.ksplit;
-        const int sgrid = std::min(nitems, h->num_sms);
-        stats_umma_kernel<<<sgrid, UMMA_THREADS, UMMA_SMEM, gs>>>(mXa, mDa, mXb, mLa, mLb, mDLa, ga);
+        const int sgrid = 2 * std::min(nitems, npairs);
+        stats_umma_kernel<<<sgrid, UMMA_THREADS, UMMA_SMEM, gs>>>(mX, mD, mL, mDL, ga);
         LAUNCHED();
         if (ga.ksplit > 1) {
             stats_fixup_kernel<<<dim3((unsigned)((int)ntiles - ga.full_tiles), FIXUP_SLABS), 256, 0, gs>>>(ga);
@@ -485,6 +489,8 @@ struct QuantizeTarget {
     int terms = GPTAQ_TERM_ERR | GPTAQ_TERM_ASYM;   // which terms of the weight update are applied
     const int *perm = nullptr;                      // act_order: working column c is the caller's column perm[c]
     int clip_steps = 0; float clip_min = 1.f;       // clipping-range search of the grids (0 steps: min/max)
+    const uint8_t *dead_orig = nullptr;             // static groups: dead-input flags in the caller's column order
+    bool static_groups = false;
 };
 
 gptaq_status_t check_quantize_args(int64_t n, const void *d_W, int w_dtype, int64_t m, int64_t ldw, int bits,
@@ -538,6 +544,20 @@ gptaq_status_t quantize_core(const QuantizeTarget &t, void *d_W, int w_dtype, in
     }
 
     const int G = group > 0 ? (n + group - 1) / group : 1;
+    const bool static_groups = t.static_groups && group > 0;
+    if (static_groups) {
+        // grids of the original weights (the caller's d_W in its own column order is still untouched)
+        const unsigned sg_grid = (unsigned)(((int64_t)m * G + 7) / 8);
+        if (w_dtype == GPTAQ_W_BF16)
+            static_group_grid_kernel<__nv_bfloat16><<<sg_grid, 256, 0, s>>>(static_cast<const __nv_bfloat16 *>(d_W), ldw, (int)m, n,
+                                                                           group, G, t.dead_orig, bits, sym, d_scales, d_zeros,
+                                                                           t.clip_steps, t.clip_min);
+        else
+            static_group_grid_kernel<float><<<sg_grid, 256, 0, s>>>(static_cast<const float *>(d_W), ldw, (int)m, n, group, G,
+                                                                   t.dead_orig, bits, sym, d_scales, d_zeros, t.clip_steps,
+                                                                   t.clip_min);
+        QLAUNCHED();
+    }
     if (group <= 0) {
         row_grid_kernel<<<(unsigned)((m + 7) / 8), 256, 0, s>>>(Wk, ldk, (int)m, n, t.dead, bits, sym,
                                                                d_scales, d_zeros, t.clip_steps, t.clip_min);
@@ -581,8 +601,10 @@ gptaq_status_t quantize_core(const QuantizeTarget &t, void *d_W, int w_dtype, in
         a.EW16_hi = tensor16 ? t.EW16 : nullptr; a.EW16_lo = tensor16 ? t.EW16 + (size_t)m * 2 * blocksize : nullptr;
         a.row_inv = t.row_inv; a.amax_u = t.amax_u; a.amax_p = t.amax_p;
         a.perm = t.perm; a.clip_steps = t.clip_steps; a.clip_min = t.clip_min; a.err_scale = (t.terms & GPTAQ_TERM_ERR) ? 1.f : 0.f; a.asym_scale = (t.terms & GPTAQ_TERM_ASYM) ? 1.f : 0.f;
+        a.static_groups = static_groups ? 1 : 0;
+        // (every full block of one call takes the same kernel: the conditions do not depend on the block)
         const bool fast = a.bw == blocksize && (group <= 0 || (group % 32) == 0) && (i0 % 4) == 0 &&
-                          (reinterpret_cast<uintptr_t>(t.dead) & 3) == 0;
+                          (reinterpret_cast<uintptr_t>(t.dead) & 3) == 0 && !static_groups;
         const int sb0 = i0 / SBW * SBW, sb_end = std::min(sb0 + SBW, n);
         if (fast && tensor16) {
             // this block's columns of the super-block's [-Err | Wpre]
@@ -594,7 +616,22 @@ gptaq_status_t quantize_core(const QuantizeTarget &t, void *d_W, int w_dtype, in
         else column_loop_kernel<1><<<cl_grid, nw * 32, cl_smem, s>>>(a);
         QLAUNCHED();
         const int i2 = i0 + blocksize;
-        if (tensor16) {
+        if (tensor16 && !fast) {
+            // grids per group of fewer than 32 columns: every full block takes column_loop_kernel, which
+            // leaves [-Err | rho Wpre] in float32; scaled row by row and split here, then applied to all
+            // columns to the right (the ragged last block has none)
+            if (i2 < n) {
+                rowscale_split16_kernel<<<(unsigned)((m + 7) / 8), 256, 0, s>>>(EW, 2 * blocksize, (int)m, 2 * blocksize, t.EW16,
+                                                                              t.EW16 + (size_t)m * 2 * blocksize, t.row_inv);
+                QLAUNCHED();
+                TcGemmArgs g = tc_args(Wk + i2, ldk, (int)m, n - i2, 2 * blocksize, 1.f, 1.f, TC_FULL, TC_MASK_NONE, t.hd);
+                g.b_row0 = i2; g.b_k0 = i0; g.k_split = blocksize; g.b2_k0 = i0;
+                g.row_inv = t.row_inv; g.amax_b = t.amax_u;
+                *err = launch_tc_gemm(maps, g, *t.sched, t.num_sms, s, false);
+                if (*err != cudaSuccess) return GPTAQ_ERR_CUDA;
+                ++*launches;
+            }
+        } else if (tensor16) {
             if (i2 < sb_end) {
                 // rest of the super-block: W[:, i2:sb_end] += [-Err | Wpre] * [U[blk, i2:sb_end] ; P[blk, i2:sb_end]]
                 TcGemmArgs g = tc_args(Wk + i2, ldk, (int)m, sb_end - i2, 2 * blocksize, 1.f, 1.f, TC_FULL, TC_MASK_NONE, t.hd);
@@ -750,6 +787,7 @@ gptaq_status_t gptaq_create(gptaq_handle_t *out, int64_t n, void *d_state, size_
     h->f16 = h->tensor && (n % 8) == 0;
     h->terms = GPTAQ_TERM_ERR | GPTAQ_TERM_ASYM;
     h->clip_steps = 0; h->clip_min = 1.f;
+    h->static_groups = false;
     cudaError_t e = cudaGetDevice(&h->device);
     if (e == cudaSuccess) e = cudaDeviceGetAttribute(&h->num_sms, cudaDevAttrMultiProcessorCount, h->device);
     if (e == cudaSuccess)
@@ -975,7 +1013,7 @@ gptaq_status_t gptaq_factor(gptaq_handle_t h, float damp, gptaq_stream_t stream)
     LAUNCHED();
     float *S1h = nullptr, *S1l = nullptr, *S2h = nullptr, *S2l = nullptr;
     TcMaps inv_maps;
-    if (h->tensor) {
+    if (h->tensor && !h->f16) {
         S1h = reinterpret_cast<float *>(h->ws + wl.s_off[0]); S1l = reinterpret_cast<float *>(h->ws + wl.s_off[1]);
         S2h = reinterpret_cast<float *>(h->ws + wl.s_off[2]); S2l = reinterpret_cast<float *>(h->ws + wl.s_off[3]);
         const SplitOperand A{S1h, S1l, n, n, n}, B{S2h, S2l, n, n, n};
@@ -1020,8 +1058,9 @@ gptaq_status_t gptaq_factor(gptaq_handle_t h, float damp, gptaq_stream_t stream)
             h->launches += 6;
             continue;
         }
-        if (h->tensor && sz >= 2 * NB) {
-            // Same two products on the tensor cores.  S1 holds K-major copies of the left operands at
+        if (h->tensor && !h->f16 && sz >= 2 * NB) {
+            // Same two products on the tensor cores, TF32-split operands (widths that are multiples of 4
+            // only).  S1 holds K-major copies of the left operands at
             // their own coordinates (B, then A^-1), S2 the transposed right operands (C^-T, then T^T).
             SplitBatch sb; sb.nbatch = np; sb.src_bstride = sb.dst_bstride = bstride;
             SplitBatch sbt = sb; sbt.cols_last = tail;                 // blocks with `tail` columns
@@ -1049,6 +1088,8 @@ gptaq_status_t gptaq_factor(gptaq_handle_t h, float damp, gptaq_stream_t stream)
             h->launches++;
             continue;
         }
+        // the 128-wide level, and every level of an fp16-split handle without damping (nothing bounds the
+        // inverse in advance then): plain float32 products
         // T = B * C^-1
         GemmProblem p1 = make_problem(make_operand(H + sz, n, 1),
                                       make_operand(H + sz * n + sz, 1, n), T + sz, n,
@@ -1071,7 +1112,6 @@ gptaq_status_t gptaq_factor(gptaq_handle_t h, float damp, gptaq_stream_t stream)
         CU(launch_split(H, n, S2h, S2l, n, n, n, true, SPLIT_UPPER, 1.f, s));
         h->launches++;
     }
-    h->tf32_copies = false;
     h->stage = STAGE_FACTORED;
     return GPTAQ_OK;
 }
@@ -1156,6 +1196,37 @@ gptaq_status_t gptaq_build_P(gptaq_handle_t h, float alpha, gptaq_stream_t strea
     return GPTAQ_OK;
 }
 
+gptaq_status_t gptaq_build_P_rowwise(gptaq_handle_t h, float alpha, gptaq_stream_t stream) {
+    if (!h || !std::isfinite(alpha)) return GPTAQ_ERR_INVALID_ARG;
+    if (h->stage != STAGE_FACTORED) return GPTAQ_ERR_BAD_STATE;
+    if (h->n > P_ROWWISE_MAX_N) return GPTAQ_ERR_UNSUPPORTED;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    const int n = (int)h->n;
+    CU(cudaFuncSetAttribute(p_rowwise_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)(2 * P_ROWWISE_MAX_N * sizeof(float))));
+    p_rowwise_kernel<<<n, PR_THREADS, 2 * (size_t)n * sizeof(float), s>>>(h->D, h->H, n, (float)((double)alpha / (double)h->tokens));
+    LAUNCHED();
+    // the operand copies that gptaq_quantize reads, as gptaq_build_P leaves them
+    WsLayout wl = ws_layout(h->n, 0, 32);
+    if (h->tensor && h->f16) {
+        const size_t nn = (size_t)n * n;
+        __half *UT16 = reinterpret_cast<__half *>(h->ws + wl.s_off[0]);
+        __half *PT16 = reinterpret_cast<__half *>(h->ws + wl.s_off[1]);
+        unsigned *am = h->hd->tc_amax;
+        CU(cudaMemsetAsync(am + AMAX_U, 0, 4 * sizeof(unsigned), s));
+        CU(launch_absmax(h->H, n, n, n, SPLIT_UPPER, 1.f, am + AMAX_U, h->num_sms, s));
+        CU(launch_absmax(h->D, n, n, n, SPLIT_STRICT_UPPER, 1.f, am + AMAX_P, h->num_sms, s));
+        CU(launch_split16(h->H, n, UT16, UT16 + nn, n, n, n, true, SPLIT_UPPER, 1.f, am + AMAX_U, s));
+        CU(launch_split16(h->D, n, PT16, PT16 + nn, n, n, n, true, SPLIT_STRICT_UPPER, 1.f, am + AMAX_P, s));
+        h->launches += 4;
+    } else if (h->tensor) {
+        float *S4 = reinterpret_cast<float *>(h->ws + wl.s_off[4]), *S5 = reinterpret_cast<float *>(h->ws + wl.s_off[5]);
+        CU(launch_split(h->D, n, S4, S5, n, n, n, true, SPLIT_STRICT_UPPER, 1.f, s));
+        h->launches++;
+    }
+    h->stage = STAGE_P;
+    return GPTAQ_OK;
+}
+
 gptaq_status_t gptaq_quantize(gptaq_handle_t h, void *d_W, int w_dtype, int64_t m, int64_t ldw,
                               int bits, int group, int sym, int blocksize,
                               uint8_t *d_codes, float *d_scales, float *d_zeros, float *d_Wq,
@@ -1175,12 +1246,11 @@ gptaq_status_t gptaq_quantize(gptaq_handle_t h, void *d_W, int w_dtype, int64_t 
     t.terms = h->terms;
     t.perm = h->act_order ? h->perm : nullptr;
     t.clip_steps = h->clip_steps; t.clip_min = h->clip_min;
+    t.static_groups = h->static_groups; t.dead_orig = h->dead_raw;
     t.UT_hi = t.UT_lo = t.PT_hi = t.PT_lo = nullptr; t.EW_lo = nullptr;
-    // FP16-split trailing update: every block that has columns to its right goes through
-    // column_block_kernel (which writes the row-scaled fp16 operand) and the block is a whole number of
-    // 64-step K-blocks
-    const bool f16 = h->f16 && (blocksize % 64) == 0 && (group <= 0 || (group % 32) == 0) &&
-                     (reinterpret_cast<uintptr_t>(h->dead) & 3) == 0;
+    // FP16-split trailing update where a block is a whole number of 64-step K-blocks; TF32-split for
+    // widths that are multiples of 4 only; plain float32 products otherwise (blocks of 32 columns)
+    const bool f16 = h->f16 && (blocksize % 64) == 0;
     if (f16) {
         t.UT16 = reinterpret_cast<const __half *>(h->ws + wl.s_off[0]);
         t.PT16 = reinterpret_cast<const __half *>(h->ws + wl.s_off[1]);
@@ -1189,17 +1259,9 @@ gptaq_status_t gptaq_quantize(gptaq_handle_t h, void *d_W, int w_dtype, int64_t 
         t.row_inv = reinterpret_cast<float *>(h->ws + wl.rs_off);
         t.row_inv_s = t.row_inv + m;
         t.amax_u = h->hd->tc_amax + AMAX_U; t.amax_p = h->hd->tc_amax + AMAX_P;
-    } else if (h->tensor) {
+    } else if (h->tensor && !h->f16) {
         float *S[6];
         for (int i = 0; i < 6; ++i) S[i] = reinterpret_cast<float *>(h->ws + wl.s_off[i]);
-        if (h->f16 && !h->tf32_copies) {
-            const int n = (int)h->n;
-            cudaStream_t s = static_cast<cudaStream_t>(stream);
-            CU(launch_split(h->H, n, S[2], S[3], n, n, n, true, SPLIT_UPPER, 1.f, s));
-            CU(launch_split(h->D, n, S[4], S[5], n, n, n, true, SPLIT_STRICT_UPPER, 1.f, s));
-            h->launches += 2;
-            h->tf32_copies = true;
-        }
         t.UT_hi = S[2]; t.UT_lo = S[3]; t.PT_hi = S[4]; t.PT_lo = S[5];
         t.EW_lo = reinterpret_cast<float *>(h->ws + wl.ew_lo_off);
     }
@@ -1335,6 +1397,12 @@ gptaq_status_t gptaq_set_act_order(gptaq_handle_t h, int enable) {
     if (h->stage != STAGE_ACCUM) return GPTAQ_ERR_BAD_STATE;
     if (enable && h->n > ACT_ORDER_MAX_N) return GPTAQ_ERR_UNSUPPORTED;
     h->act_order = enable != 0;
+    return GPTAQ_OK;
+}
+
+gptaq_status_t gptaq_set_static_groups(gptaq_handle_t h, int enable) {
+    if (!h) return GPTAQ_ERR_INVALID_ARG;
+    h->static_groups = enable != 0;
     return GPTAQ_OK;
 }
 

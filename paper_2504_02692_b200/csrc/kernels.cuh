@@ -558,8 +558,8 @@ __device__ __forceinline__ void make_grid(float lo, float hi, float amax, int bi
     }
 }
 
-// Clipping-range search (setup of Section 5: "the weight clipping range is searched by minimizing mean
-// squared error"): candidate k of `steps` shrinks the min/max range by p_k = 1 - k (1 - min_ratio) / steps;
+// Clipping-range search of a grid by least squared rounding error (experimental setup of Section 5):
+// candidate k of `steps` shrinks the min/max range by p_k = 1 - k (1 - min_ratio) / steps;
 // the candidate with the least squared rounding error of the group's weights wins, the widest one on ties.
 __device__ __forceinline__ float clip_ratio(int k, int steps, float min_ratio) {
     return 1.f - (float)k * ((1.f - min_ratio) / (float)steps);
@@ -608,6 +608,49 @@ __global__ void __launch_bounds__(256) row_grid_kernel(const float *W, int64_t l
     if (lane == 0) { scales[row] = s; zeros[row] = z; }
 }
 
+// Static groups: one grid per output channel and per group of `group` consecutive columns of W in the
+// caller's column order, from the original weights (dead inputs count as zero weights).  One warp per
+// (row, group); W float32 or bf16.
+template <typename T>
+__global__ void __launch_bounds__(256) static_group_grid_kernel(const T *W, int64_t ldw, int m, int n, int group, int G,
+                                                                const uint8_t *dead, int bits, int sym, float *scales,
+                                                                float *zeros, int clip_steps, float clip_min) {
+    const int64_t wid = (int64_t)blockIdx.x * 8 + (threadIdx.x >> 5);
+    const int lane = threadIdx.x & 31;
+    if (wid >= (int64_t)m * G) return;
+    const int row = (int)(wid / G), g = (int)(wid - (int64_t)row * G);
+    const T *w = W + (int64_t)row * ldw;
+    const int c0 = g * group, c1 = min(n, c0 + group);
+    float lo = 0.f, hi = 0.f, am = 0.f;
+    for (int c = c0 + lane; c < c1; c += 32) {
+        const float v = dead[c] ? 0.f : (float)w[c];
+        lo = fminf(lo, v); hi = fmaxf(hi, v); am = fmaxf(am, fabsf(v));
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+        lo = fminf(lo, __shfl_xor_sync(0xffffffffu, lo, o));
+        hi = fmaxf(hi, __shfl_xor_sync(0xffffffffu, hi, o));
+        am = fmaxf(am, __shfl_xor_sync(0xffffffffu, am, o));
+    }
+    float s, z;
+    make_grid(lo, hi, am, bits, sym, s, z);
+    if (clip_steps > 0) {
+        const float maxq = (float)((1 << bits) - 1);
+        float best = INFINITY;
+        for (int k = 0; k < clip_steps; ++k) {
+            const float p = clip_ratio(k, clip_steps, clip_min);
+            float sk, zk;
+            make_grid(p * lo, p * hi, p * am, bits, sym, sk, zk);
+            float err = 0.f;
+            for (int c = c0 + lane; c < c1; c += 32) err += rounding_error_sq(dead[c] ? 0.f : (float)w[c], sk, zk, maxq);
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) err += __shfl_xor_sync(0xffffffffu, err, o);
+            if (err < best) { best = err; s = sk; z = zk; }
+        }
+    }
+    if (lane == 0) { scales[(int64_t)row * G + g] = s; zeros[(int64_t)row * G + g] = z; }
+}
+
 // ---------------------------------------------------------------------------
 // Column loop over one lazy-batch block [i0, i0 + bw) (Algorithm 1, inner
 // loop).  One warp per weight row; the row's block lives in registers (lane
@@ -639,6 +682,8 @@ struct ColumnLoopArgs {
     float err_scale, asym_scale;   // 1 or 0: switches of the two terms of the weight update (ablation)
     const int *perm;               // nullptr, or: working column c is original column perm[c] (codes go there)
     int clip_steps; float clip_min; // clipping-range search of the group grids (0: plain min/max)
+    int static_groups;             // column_loop_kernel: scales / zeros hold ready grids per group of ORIGINAL columns
+                                   //   (static_group_grid_kernel); column c uses group (perm ? perm[c] : c) / group
 };
 
 template <int T>
@@ -675,6 +720,8 @@ __global__ void __launch_bounds__(1024) column_loop_kernel(ColumnLoopArgs a) {
         float v = 0.f;
         if (c < bw && !a.dead[i0 + c]) v = wrow[c];
         w[t] = v; nerr[t] = 0.f; pre[t] = 0.f; code[t] = 0;
+        // reported from the value that was read: the clamp of the quantizer would absorb a NaN or Inf
+        if (!isfinite(v)) record_status(a.hd, ST_NONFINITE, row);
     }
 
     const float maxq = (float)((1 << a.bits) - 1);
@@ -686,7 +733,11 @@ __global__ void __launch_bounds__(1024) column_loop_kernel(ColumnLoopArgs a) {
         for (int jj = 0; jj < 32; ++jj) {
             const int j = t * 32 + jj;
             if (j >= bw) break;
-            if (a.group > 0 && ((i0 + j) % a.group) == 0) {
+            if (a.static_groups) {
+                const int cj = a.perm ? a.perm[i0 + j] : i0 + j;
+                scale = a.scales[(int64_t)row * a.G + cj / a.group];
+                zero = a.zeros[(int64_t)row * a.G + cj / a.group];
+            } else if (a.group > 0 && ((i0 + j) % a.group) == 0) {
                 // grid of the group that starts here, from the current values
                 const int gend = min(j + a.group, bw);
                 float lo = 0.f, hi = 0.f, am = 0.f;
@@ -743,6 +794,13 @@ __global__ void __launch_bounds__(1024) column_loop_kernel(ColumnLoopArgs a) {
     }
 
     bool bad = false;
+    // fp16-split handles (row_inv set): Wpre is stored times rho = scale of U^T / scale of P^T, like
+    // column_block_kernel does, so that the two halves of the update's B operand keep scales of their own
+    float rho = 1.f;
+    if (a.row_inv) {
+        const float ap = __uint_as_float(*a.amax_p);
+        rho = ap > 0.f ? split_scale(__uint_as_float(*a.amax_u)) / split_scale(ap) : 0.f;
+    }
     float *ew = a.EW + (int64_t)row * (2 * BW);
     float *ewl = a.EW_lo ? a.EW_lo + (int64_t)row * (2 * BW) : nullptr;
     uint8_t *crow = a.codes + (int64_t)row * n + i0;
@@ -755,7 +813,7 @@ __global__ void __launch_bounds__(1024) column_loop_kernel(ColumnLoopArgs a) {
             ew[BW + c] = ph; ewl[BW + c] = tf32_rn(pre[t] - ph);
         } else {
             ew[c] = nerr[t];
-            ew[BW + c] = pre[t];
+            ew[BW + c] = rho * pre[t];
         }
         if (c < bw) {
             wrow[c] = w[t];
@@ -869,6 +927,10 @@ __global__ void __launch_bounds__(CB_THREADS, 1) column_block_kernel(ColumnLoopA
             if (dd.y) v[u].y = 0.f;
             if (dd.z) v[u].z = 0.f;
             if (dd.w) v[u].w = 0.f;
+            // a non-finite weight is reported from the value that was read: its code and dequantized value
+            // come out finite (the clamp absorbs NaN and Inf), so the results alone would not show it
+            if (r < nrows && (!isfinite(v[u].x) || !isfinite(v[u].y) || !isfinite(v[u].z) || !isfinite(v[u].w)))
+                record_status(a.hd, ST_NONFINITE, row0 + r);
             *reinterpret_cast<float4 *>(&Wt[r][4 * c4]) = v[u];
         }
     }
@@ -1061,11 +1123,10 @@ __global__ void __launch_bounds__(CB_THREADS, 1) column_block_kernel(ColumnLoopA
     }
     __syncthreads();
     // dequantized block back to W
-    bool bad = false;
     for (int idx = tid; idx < nrows * bq; idx += CB_THREADS) {
         const int r = idx / bq, c4 = idx - r * bq;
         const float4 v = *reinterpret_cast<const float4 *>(&Wt[r][4 * c4]);
-        bad |= !isfinite(v.x) || !isfinite(v.y) || !isfinite(v.z) || !isfinite(v.w);
+        const bool bad = !isfinite(v.x) || !isfinite(v.y) || !isfinite(v.z) || !isfinite(v.w);
         float *dst = a.W + (int64_t)(row0 + r) * a.ldw + i0 + 4 * c4;
         if ((reinterpret_cast<uintptr_t>(dst) & 15) == 0) *reinterpret_cast<float4 *>(dst) = v;
         else { dst[0] = v.x; dst[1] = v.y; dst[2] = v.z; dst[3] = v.w; }
@@ -1099,6 +1160,44 @@ __global__ void __launch_bounds__(CB_THREADS, 1) column_block_kernel(ColumnLoopA
             *reinterpret_cast<uint2 *>(a.EW16_lo + off) =
                 make_uint2(*reinterpret_cast<const uint32_t *>(&l01), *reinterpret_cast<const uint32_t *>(&l23));
         }
+    }
+}
+
+// ---------------------------------------------------------------------------
+// Row-by-row form of P (Eq. "unparallel"):  P[q, f] = scale * (D[q, f] U[f, f]^T) U[f, f],  f = q + 1 .. n - 1
+// (L[f, f] of the paper is U[f, f]^T).  One CTA per row q, two passes over the trailing triangle of U:
+//   v_a     = sum_{k >= a} D[q, k] U[a, k]      a in f   (a warp per a, along row a of U)
+//   P[q, j] = sum_{q < a <= j} v_a U[a, j]      j in f   (a thread per j, coalesced across j)
+// This is the form that Theorem 4.2 replaces by two matrix products; it is kept as the comparison of the
+// latency discussion of Section 5, not as a path of the solve.  In place: row q of P overwrites row q of D.
+// ---------------------------------------------------------------------------
+constexpr int PR_THREADS = 1024;
+__global__ void __launch_bounds__(PR_THREADS) p_rowwise_kernel(float *D, const float *U, int n, float scale) {
+    extern __shared__ float pr_smem[];
+    float *d = pr_smem, *v = pr_smem + n;
+    const int q = blockIdx.x;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    float *row = D + (int64_t)q * n;
+    for (int c = tid; c < n; c += PR_THREADS) d[c] = c > q ? row[c] : 0.f;
+    __syncthreads();
+    for (int a = q + 1 + warp; a < n; a += PR_THREADS / 32) {
+        const float *ur = U + (int64_t)a * n;
+        float s = 0.f;
+        for (int k = a + lane; k < n; k += 32) s = fmaf(d[k], ur[k], s);
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
+        if (lane == 0) v[a] = s;
+    }
+    __syncthreads();
+    for (int j = tid; j < n; j += PR_THREADS) {
+        float s0 = 0.f, s1 = 0.f;
+        int a = q + 1;
+        for (; a + 1 <= j; a += 2) {
+            s0 = fmaf(v[a], U[(int64_t)a * n + j], s0);
+            s1 = fmaf(v[a + 1], U[(int64_t)(a + 1) * n + j], s1);
+        }
+        if (a <= j) s0 = fmaf(v[a], U[(int64_t)a * n + j], s0);
+        row[j] = j > q ? scale * (s0 + s1) : 0.f;
     }
 }
 

@@ -1,14 +1,24 @@
 // Tensor-core statistics kernel for sm_100a: C += A * B^T with fp16 operands in
 // K-major shared-memory tiles (TMA, 128-byte swizzle), tcgen05.mma with fp32
 // accumulators in tensor memory, and a read-modify-write epilogue into the fp32
-// sums.  Persistent, warp-specialised: warp 0 issues TMA loads, warp 1 issues
-// the MMAs and owns the TMEM allocation, warps 2-9 drain the accumulators.
-// Two 128 x 256 accumulators are kept in TMEM so that draining one overlaps the
-// MMAs into the other.
+// sums.  Persistent and warp-specialised; the CTAs work in pairs (clusters of
+// two, the two SMs of one TPC) on 256 x 256 output tiles with
+// tcgen05.mma.cta_group::2: each CTA loads its own 128 rows of the A operand
+// and its own 128 of the 256 rows of the B operand into its own shared memory
+// (plain TMA loads, no multicast), the tensor cores of both SMs read both halves
+// of B, and each CTA's tensor memory receives its 128 rows of the tile.  Per
+// K-block a CTA takes in 32 KB of operands for 128 x 256 outputs instead of the
+// 48 KB of a single-CTA tile: the L2 -> SM operand traffic, which bounded the
+// single-CTA form at 69 % tensor-pipe activity, drops by a third.
+// In each CTA warp 0 issues the TMA loads and warps 2-9 drain the accumulators;
+// warp 1 owns the TMEM allocation, and in the pair's first CTA its first lane
+// issues the MMAs for both.  Two 256-column accumulators are kept in TMEM so
+// that draining one overlaps the MMAs into the other.
 //
 // Every wait on an mbarrier is bounded by a clock limit; when it runs out the
-// kernel records GPTAQ_ERR_TIMEOUT in the state header, lets outstanding copies
-// land (bounded as well), frees its tensor memory and returns.
+// kernel records GPTAQ_ERR_TIMEOUT in the state header, tells the other CTA of
+// the pair, lets outstanding copies land (bounded as well), and both CTAs meet
+// at a cluster barrier, free their tensor memory and return.
 #pragma once
 #include <cuda.h>
 #include <cuda_fp16.h>
@@ -19,9 +29,13 @@
 
 namespace gptaq {
 
-constexpr int UBM = 128, UBN = 256, UBK = 64, USTAGES = 4;
-constexpr int UA_BYTES = UBM * UBK * 2;
-constexpr int UB_BYTES = UBN * UBK * 2;
+// UBM x UBN: the output tile of one CTA (float32-grade GEMM: one CTA per tile; statistics: the pair's
+// tile is 2 UBM x UBN, one half of the rows per CTA).
+constexpr int UBM = 128, UBN = 256, UBK = 64;
+constexpr int UPM = 2 * UBM;                    // rows of a pair's tile
+constexpr int USTAGES = 6;
+constexpr int UA_BYTES = UBM * UBK * 2;         // this CTA's rows of A
+constexpr int UB_BYTES = (UBN / 2) * UBK * 2;   // this CTA's half of the rows of B
 constexpr int USTAGE_BYTES = UA_BYTES + UB_BYTES;
 constexpr int UEPI_WARPS = 8;
 constexpr int UMMA_THREADS = 64 + 32 * UEPI_WARPS;
@@ -245,6 +259,67 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
 }
 __device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 
+// ---- CTA pairs (clusters of two)
+__device__ __forceinline__ uint32_t cluster_ctarank() {
+    uint32_t r;
+    asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+    return r;
+}
+// The address, in the cluster's shared-memory window, of the location that has shared::cta address
+// `addr` in the CTA with rank `rank`.
+__device__ __forceinline__ uint32_t map_to_cta(uint32_t addr, uint32_t rank) {
+    uint32_t r;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(addr), "r"(rank));
+    return r;
+}
+__device__ __forceinline__ void cluster_sync_all() {
+    asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+    asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_addr) {
+    asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
+}
+__device__ __forceinline__ void st_cluster_u32(uint32_t cluster_addr, uint32_t v) {
+    asm volatile("st.shared::cluster.u32 [%0], %1;" ::"r"(cluster_addr), "r"(v) : "memory");
+}
+// Bounded wait of a CTA pair: as mbar_wait, and a wait that gives up also raises the other CTA's flag
+// (at cluster address peer_abort), so that the pair winds down together instead of one timeout at a time.
+__device__ __forceinline__ bool mbar_wait_pair(uint32_t bar, uint32_t parity, volatile int *abort_flag,
+                                               uint32_t peer_abort, long long limit_cycles = WAIT_LIMIT_CYCLES) {
+    if (mbar_try(bar, parity)) return true;
+    const long long t0 = clock64();
+    for (uint32_t it = 1;; ++it) {
+        if (mbar_try(bar, parity)) return true;
+        if ((it & 63) == 0) {
+            if (*abort_flag) return false;
+            if (clock64() - t0 > limit_cycles) { *abort_flag = 1; st_cluster_u32(peer_abort, 1u); return false; }
+        }
+    }
+}
+// TMA load of one CTA of a pair: the tile lands in this CTA's shared memory, its bytes are counted by the
+// mbarrier at cluster address `bar` (the pair's first CTA keeps the barriers of the operand ring).  No multicast.
+__device__ __forceinline__ void tma_load_2d_pair(uint32_t dst, const CUtensorMap *map, int c0, int c1, uint32_t bar) {
+    asm volatile(
+        "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
+        ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(bar), "r"(c0), "r"(c1) : "memory");
+}
+// One MMA over both CTAs of the pair: D (256 x N, 128 rows in each CTA's tensor memory) += A (128 rows from
+// each CTA's shared memory) * B^T (N / 2 rows from each CTA's shared memory); the descriptors address the
+// same offsets in both CTAs.
+__device__ __forceinline__ void umma_f16_pair(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t acc) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(acc) : "memory");
+}
+// Completion of the pair's MMAs issued so far, signalled to the mbarrier at this shared-memory offset in
+// both CTAs (the commit's own multicast; no data moves).
+__device__ __forceinline__ void umma_commit_pair(uint32_t bar) {
+    asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
+                 ::"r"(bar), "h"((uint16_t)3) : "memory");
+}
+
 // K-major, 128-byte-swizzled operand tile: rows of 128 bytes, 8-row groups 1024 bytes apart.
 __device__ __forceinline__ uint64_t make_kmajor_desc(uint32_t smem_addr) {
     uint64_t d = 0;
@@ -258,6 +333,8 @@ __device__ __forceinline__ uint64_t make_kmajor_desc(uint32_t smem_addr) {
 
 // kind::f16 instruction descriptor: fp16 A and B (both K-major), fp32 D, M = 128, N = 256.
 constexpr uint32_t UMMA_IDESC_F16 = (1u << 4) | (0u << 7) | (0u << 10) | ((UBN >> 3) << 17) | ((UBM >> 4) << 24);
+// ... and for the pair: M = 256 (128 rows per CTA), N = 256.
+constexpr uint32_t UMMA_IDESC_F16_PAIR = (1u << 4) | (0u << 7) | (0u << 10) | ((UBN >> 3) << 17) | ((UPM >> 4) << 24);
 
 struct StatsGemmArgs {
     float *H, *D;            // n x n, ld n
@@ -267,53 +344,54 @@ struct StatsGemmArgs {
     int nseg_d;              // 1: dXX^T = dh xh^T;  3: dh xh^T + dh xl^T + dl xh^T
     const unsigned *amax;    // scales are recomputed from the recorded maxima
     StateHeader *hd;
-    // Work items: tiles [0, full_tiles) are whole tiles; each of the remaining `ntiles - full_tiles`
-    // tiles (the last, partial wave) is cut along K into `ksplit` items so that every SM has work.
-    // Item 0 of a cut tile adds into the sums like a whole tile; items c > 0 store their partial
-    // result at scratch[((tile - full_tiles) * (ksplit - 1) + c - 1) * UBM * UBN] and
-    // stats_fixup_kernel adds those in a fixed order (the result does not depend on timing).
+    // Work items of a CTA pair: tiles [0, full_tiles) are whole 256 x 256 tiles; each of the remaining
+    // `ntiles - full_tiles` tiles (the last, partial wave) is cut along K into `ksplit` items so that every
+    // pair has work.  Item 0 of a cut tile adds into the sums like a whole tile; items c > 0 store their
+    // partial result (128 x 256 per CTA) at scratch[(((tile - full_tiles) * (ksplit - 1) + c - 1) * 2 + rank)
+    // * UBM * UBN] and stats_fixup_kernel adds those in a fixed order (the result does not depend on timing).
     int ntiles, full_tiles, ksplit;
     float *scratch;
 };
 
-// Tile enumeration shared by all roles.  Rows [0, TM) belong to H (tiles entirely below the
-// diagonal are not enumerated), rows [TM, 2 TM) to dXX^T.  Order: bands of UBAND row tiles; inside a
-// band column tile by column tile, first the band's tiles of H, then its tiles of dXX^T.  The 148
-// tiles that are in flight together then share about 2 x 16 row panels (X and X~ - X) and a handful
+// Tile enumeration shared by all roles, in units of the pair's 256 x 256 tiles.  Rows [0, T) belong to H
+// (tiles entirely below the diagonal are not enumerated), rows [T, 2 T) to dXX^T.  Order: bands of UBAND
+// row tiles; inside a band column tile by column tile, first the band's tiles of H, then its tiles of dXX^T.
+// The tiles that are in flight together then share about 2 x 8 row panels (X and X~ - X) and a handful
 // of column panels of X through the L2, and X streams from HBM once per band instead of once per
-// 2.6 row tiles (row-major order over the whole matrix: 15 GB of HBM reads per 8192-token batch at
+// 1.3 row tiles (row-major order over the whole matrix: 15 GB of HBM reads per 8192-token batch at
 // n = 14336).
-constexpr int UBAND = 16;
+constexpr int UBAND = 8;
 struct TileIter {
-    int TM, TN, r, tn, ord;       // (r, tn): the current tile; ord: its ordinal
+    int T, r, tn, ord;            // (r, tn): the current tile; ord: its ordinal
     int band, k;                  // band of row tiles, position inside the group (band, tn)
-    __device__ TileIter(int n) : TM((n + UBM - 1) / UBM), TN((n + UBN - 1) / UBN), r(0), tn(0), ord(0), band(0), k(0) {}
-    __device__ int band_rows() const { return min(UBAND, TM - band * UBAND); }
-    // row tiles r of the band whose tile (r, tn) of H is not entirely below the diagonal: r <= 2 tn + 1
-    __device__ int h_count() const { return max(0, min(band * UBAND + band_rows(), (2 * tn + 2) * (UBN / (2 * UBM))) - band * UBAND); }
+    __host__ __device__ TileIter(int n) : T((n + UPM - 1) / UPM), r(0), tn(0), ord(0), band(0), k(0) {}
+    __host__ __device__ int band_rows() const { return min(UBAND, T - band * UBAND); }
+    // row tiles r of the band whose tile (r, tn) of H is not entirely below the diagonal: r <= tn
+    __host__ __device__ int h_count() const { return max(0, min(band_rows(), tn + 1 - band * UBAND)); }
+    __host__ __device__ static int total(int n) { const int t = (n + UPM - 1) / UPM; return t * (t + 1) / 2 + t * t; }
     // Advances to the tile with ordinal `target` >= ord; false when the list is exhausted.
-    __device__ bool seek_to(int target) {
+    __host__ __device__ bool seek_to(int target) {
         int left = target - ord;
-        while (band * UBAND < TM) {
+        while (band * UBAND < T) {
             const int hc = h_count();
             const int avail = hc + band_rows() - k;
             if (left < avail) {
                 k += left;
                 ord = target;
-                r = k < hc ? band * UBAND + k : TM + band * UBAND + (k - hc);
+                r = k < hc ? band * UBAND + k : T + band * UBAND + (k - hc);
                 return true;
             }
             left -= avail;
             ord += avail;
             k = 0;
-            if (++tn == TN) { tn = 0; ++band; }
+            if (++tn == T) { tn = 0; ++band; }
         }
         return false;
     }
 };
-static_assert(UBN == 2 * UBM, "the diagonal test of TileIter assumes 128 x 256 tiles");
+static_assert(UBN == UPM, "the diagonal test of TileIter assumes square pair tiles");
 
-// One work item of a CTA: a tile and a range of its K-blocks (all segments concatenated).
+// One work item of a pair: a tile and a range of its K-blocks (all segments concatenated).
 struct StatsItem {
     int g0, g1;          // K-block range
     int part;            // 0: adds into H / dXX^T;  c > 0: partial result number c of a cut tile
@@ -331,7 +409,7 @@ __device__ __forceinline__ bool stats_item(const StatsGemmArgs &a, int w, TileIt
         parts = a.ksplit;
     }
     if (!it.seek_to(tile)) return false;
-    const int kb_total = (it.r >= it.TM) ? a.kblocks * a.nseg_d : a.kblocks * a.nseg_h;
+    const int kb_total = (it.r >= it.T) ? a.kblocks * a.nseg_d : a.kblocks * a.nseg_h;
     item.g0 = (int)((long long)kb_total * part / parts);
     item.g1 = (int)((long long)kb_total * (part + 1) / parts);
     item.part = part;
@@ -346,18 +424,24 @@ __device__ __forceinline__ bool stats_item(const StatsGemmArgs &a, int w, TileIt
 // of the epilogue warps; HBM is touched once per tile.
 constexpr int UCHUNK = 8;           // K-blocks (of 64) per TMEM accumulation chain
 
-__global__ void __launch_bounds__(UMMA_THREADS, 1)
-stats_umma_kernel(const __grid_constant__ CUtensorMap mapXa, const __grid_constant__ CUtensorMap mapDa,
-                  const __grid_constant__ CUtensorMap mapXb, const __grid_constant__ CUtensorMap mapLa,
-                  const __grid_constant__ CUtensorMap mapLb, const __grid_constant__ CUtensorMap mapDLa,
+// Launched as clusters of two CTAs (grid = 2 x number of pairs).  Tensor maps: X^T, (X~ - X)^T and their
+// low parts, [n][kp] fp16, boxes of 64 tokens x 128 channels; they serve as A and as B operand alike.
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(UMMA_THREADS, 1)
+stats_umma_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ CUtensorMap mapD,
+                  const __grid_constant__ CUtensorMap mapL, const __grid_constant__ CUtensorMap mapDL,
                   StatsGemmArgs a) {
     extern __shared__ uint8_t smem_raw[];
-    // 1024-byte alignment for the swizzled tiles
+    // 1024-byte alignment for the swizzled tiles (the same offsets in both CTAs of the pair: the MMA's
+    // shared-memory descriptors are applied to both)
     const uint32_t raw = smem_u32(smem_raw);
     const uint32_t base = (raw + 1023u) & ~1023u;
     uint8_t *aligned = smem_raw + (base - raw);
     const uint32_t bar0 = base + USTAGES * USTAGE_BYTES;
-    // barrier slots (8 bytes each): full[4], empty[4], tfull[2], tempty[2]; then tmem slot, abort flag
+    // barrier slots (8 bytes each): full[USTAGES], empty[USTAGES], tfull[2], tempty[2]; then tmem slot, abort flag.
+    //   full    first CTA only: its own arrive.expect_tx + the bytes of both CTAs' loads
+    //   empty   each CTA its own: one arrival per use, from the commit of the MMAs that read the stage
+    //   tfull   each CTA its own: one arrival, from the commit of an accumulation chain
+    //   tempty  first CTA only: the epilogue warps of both CTAs
     auto full_bar = [&](int s) { return bar0 + 8u * s; };
     auto empty_bar = [&](int s) { return bar0 + 8u * (USTAGES + s); };
     auto tfull_bar = [&](int b) { return bar0 + 8u * (2 * USTAGES + b); };
@@ -366,43 +450,50 @@ stats_umma_kernel(const __grid_constant__ CUtensorMap mapXa, const __grid_consta
     volatile int *abort_flag = reinterpret_cast<volatile int *>(tmem_slot + 1);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const uint32_t rank = cluster_ctarank();              // 0: issues the MMAs, keeps full / tempty
+    const int pair = blockIdx.x >> 1, npairs = gridDim.x >> 1;
+    const uint32_t peer_abort = map_to_cta(smem_u32(const_cast<int *>(abort_flag)), rank ^ 1u);
     if (threadIdx.x == 0) {
         for (int s = 0; s < USTAGES; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
-        for (int b = 0; b < 2; ++b) { mbar_init(tfull_bar(b), 1); mbar_init(tempty_bar(b), UEPI_WARPS); }
+        for (int b = 0; b < 2; ++b) { mbar_init(tfull_bar(b), 1); mbar_init(tempty_bar(b), 2 * UEPI_WARPS); }
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     if (warp == 1) {
-        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
+        // one warp of each CTA, the same warp in both: the allocation spans the pair
+        asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;"
                      ::"r"(smem_u32(const_cast<uint32_t *>(tmem_slot))), "r"(512u) : "memory");
-        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
     }
     tc_fence_before();
     __syncthreads();
+    cluster_sync_all();              // the other CTA's barriers exist before anything signals them
     tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
     const int KB = a.kblocks;
 
     if (warp == 0) {
-        // ------------------------------------------------------------ TMA producer
+        // ------------------------------------------------------------ TMA producer (each CTA its own halves)
         if (lane == 0) {
             TileIter it(a.n);
             StatsItem item;
             uint32_t stage = 0, phase = 0;
             int issued = 0;
             bool ok = true;
-            for (int w = blockIdx.x; ok && stats_item(a, w, it, item); w += gridDim.x) {
-                const bool isD = it.r >= it.TM;
-                const int row0 = (isD ? it.r - it.TM : it.r) * UBM, col0 = it.tn * UBN;
+            for (int w = pair; ok && stats_item(a, w, it, item); w += npairs) {
+                const bool isD = it.r >= it.T;
+                const int row0 = (isD ? it.r - it.T : it.r) * UPM + (int)rank * UBM;      // this CTA's rows of the tile
+                const int col0 = it.tn * UBN + (int)rank * (UBN / 2);                     // this CTA's half of the columns' operand
                 for (int g = item.g0; g < item.g1; ++g) {
                     const int seg = g / KB, kb = g - seg * KB;
-                    const CUtensorMap *mapA = isD ? (seg == 2 ? &mapDLa : &mapDa) : (seg == 2 ? &mapLa : &mapXa);
-                    const CUtensorMap *mapB = (seg == 1) ? &mapLb : &mapXb;
-                    if (!mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag)) { ok = false; break; }
+                    const CUtensorMap *mapA = isD ? (seg == 2 ? &mapDL : &mapD) : (seg == 2 ? &mapL : &mapX);
+                    const CUtensorMap *mapB = (seg == 1) ? &mapL : &mapX;
+                    if (!mbar_wait_pair(empty_bar(stage), phase ^ 1u, abort_flag, peer_abort)) { ok = false; break; }
                     const uint32_t sa = base + stage * USTAGE_BYTES, sb = sa + UA_BYTES;
-                    mbar_expect_tx(full_bar(stage), USTAGE_BYTES);
-                    tma_load_2d(sa, mapA, kb * UBK, row0, full_bar(stage));
-                    tma_load_2d(sb, mapB, kb * UBK, col0, full_bar(stage));
+                    const uint32_t fb = map_to_cta(full_bar(stage), 0u);
+                    if (rank == 0) mbar_expect_tx(full_bar(stage), 2 * USTAGE_BYTES);
+                    tma_load_2d_pair(sa, mapA, kb * UBK, row0, fb);
+                    tma_load_2d_pair(sb, mapB, kb * UBK, col0, fb);
                     ++issued;
                     if (++stage == USTAGES) { stage = 0; phase ^= 1u; }
                 }
@@ -414,39 +505,39 @@ stats_umma_kernel(const __grid_constant__ CUtensorMap mapXa, const __grid_consta
             }
         }
     } else if (warp == 1) {
-        // ------------------------------------------------------------ MMA issuer
-        if (lane == 0) {
+        // ------------------------------------------------------------ MMA issuer (first CTA of the pair)
+        if (lane == 0 && rank == 0) {
             TileIter it(a.n);
             StatsItem item;
             uint32_t stage = 0, phase = 0, ccount = 0;     // ccount: chunks issued so far
             bool ok = true;
-            for (int w = blockIdx.x; ok && stats_item(a, w, it, item); w += gridDim.x) {
+            for (int w = pair; ok && stats_item(a, w, it, item); w += npairs) {
                 for (int kb0 = item.g0; kb0 < item.g1 && ok; kb0 += UCHUNK) {
                     const uint32_t buf = ccount & 1u, cphase = (ccount >> 1) & 1u;
-                    if (!mbar_wait(tempty_bar(buf), cphase ^ 1u, abort_flag)) { ok = false; break; }
+                    if (!mbar_wait_pair(tempty_bar(buf), cphase ^ 1u, abort_flag, peer_abort)) { ok = false; break; }
                     tc_fence_after();
                     const uint32_t d_tmem = tmem_base + buf * UBN;
                     const int kb1 = min(kb0 + UCHUNK, item.g1);
                     for (int kb = kb0; kb < kb1; ++kb) {
-                        if (!mbar_wait(full_bar(stage), phase, abort_flag)) { ok = false; break; }
+                        if (!mbar_wait_pair(full_bar(stage), phase, abort_flag, peer_abort)) { ok = false; break; }
                         tc_fence_after();
                         const uint32_t sa = base + stage * USTAGE_BYTES, sb = sa + UA_BYTES;
                         const uint64_t ad = make_kmajor_desc(sa), bd = make_kmajor_desc(sb);
 #pragma unroll
                         for (int k = 0; k < UBK / 16; ++k)
-                            umma_f16(d_tmem, ad + (uint64_t)(k * 2), bd + (uint64_t)(k * 2), UMMA_IDESC_F16,
-                                     (kb != kb0 || k != 0) ? 1u : 0u);
-                        umma_commit(empty_bar(stage));
+                            umma_f16_pair(d_tmem, ad + (uint64_t)(k * 2), bd + (uint64_t)(k * 2), UMMA_IDESC_F16_PAIR,
+                                          (kb != kb0 || k != 0) ? 1u : 0u);
+                        umma_commit_pair(empty_bar(stage));
                         if (++stage == USTAGES) { stage = 0; phase ^= 1u; }
                     }
                     if (!ok) break;
-                    umma_commit(tfull_bar(buf));
+                    umma_commit_pair(tfull_bar(buf));
                     ++ccount;
                 }
             }
         }
     } else {
-        // ------------------------------------------------------------ epilogue (warps 2..9)
+        // ------------------------------------------------------------ epilogue (warps 2..9): this CTA's 128 rows
         const int quarter = warp & 3;                 // TMEM lanes 32 * quarter .. + 31
         const int half = (warp - 2) >> 2;             // columns [128 * half, 128 * half + 128)
         TileIter it(a.n);
@@ -456,13 +547,13 @@ stats_umma_kernel(const __grid_constant__ CUtensorMap mapXa, const __grid_consta
         const float sx = pick_scale(__uint_as_float(a.amax[0]));
         const float sd = pick_scale(__uint_as_float(a.amax[1]));
         float acc[UBN / 2];
-        for (int w = blockIdx.x; ok && stats_item(a, w, it, item); w += gridDim.x) {
-            const bool isD = it.r >= it.TM;
+        for (int w = pair; ok && stats_item(a, w, it, item); w += npairs) {
+            const bool isD = it.r >= it.T;
 #pragma unroll
             for (int i = 0; i < UBN / 2; ++i) acc[i] = 0.f;
             for (int kb0 = item.g0; kb0 < item.g1; kb0 += UCHUNK) {
                 const uint32_t buf = ccount & 1u, cphase = (ccount >> 1) & 1u;
-                if (!mbar_wait(tfull_bar(buf), cphase, abort_flag)) { ok = false; break; }
+                if (!mbar_wait_pair(tfull_bar(buf), cphase, abort_flag, peer_abort)) { ok = false; break; }
                 tc_fence_after();
                 const uint32_t taddr = tmem_base + buf * UBN + half * (UBN / 2) + ((uint32_t)(quarter * 32) << 16);
 #pragma unroll
@@ -475,14 +566,14 @@ stats_umma_kernel(const __grid_constant__ CUtensorMap mapXa, const __grid_consta
                 }
                 tc_fence_before();
                 __syncwarp();
-                if (lane == 0) mbar_arrive(tempty_bar(buf));
+                if (lane == 0) mbar_arrive_cluster(map_to_cta(tempty_bar(buf), 0u));
                 ++ccount;
             }
             if (!ok) break;
             const float inv = 1.f / (sx * (isD ? sd : sx));
             if (item.part > 0) {
                 // partial result of a cut tile: plain stores into its slot, all 128 x 256 entries
-                float *sp = a.scratch + ((int64_t)item.cut_index * (a.ksplit - 1) + item.part - 1) * (UBM * UBN) +
+                float *sp = a.scratch + (((int64_t)item.cut_index * (a.ksplit - 1) + item.part - 1) * 2 + (int)rank) * (UBM * UBN) +
                             (quarter * 32 + lane) * UBN + half * (UBN / 2);
 #pragma unroll
                 for (int q = 0; q < UBN / 2 / 4; ++q)
@@ -490,7 +581,7 @@ stats_umma_kernel(const __grid_constant__ CUtensorMap mapXa, const __grid_consta
                                                                          acc[4 * q + 2] * inv, acc[4 * q + 3] * inv);
                 continue;
             }
-            const int row = (isD ? it.r - it.TM : it.r) * UBM + quarter * 32 + lane;
+            const int row = (isD ? it.r - it.T : it.r) * UPM + (int)rank * UBM + quarter * 32 + lane;
             const int col0 = it.tn * UBN + half * (UBN / 2);
             float *C = isD ? a.D : a.H;
             if (row < a.n) {
@@ -512,12 +603,15 @@ stats_umma_kernel(const __grid_constant__ CUtensorMap mapXa, const __grid_consta
         }
     }
 
+    // Both CTAs leave together: neither frees tensor memory, nor lets its shared memory go, while the
+    // other may still signal its barriers or its MMAs read its operands.
     tc_fence_before();
     __syncthreads();
+    cluster_sync_all();
     if (*abort_flag && threadIdx.x == 0) record_status(a.hd, ST_TIMEOUT, blockIdx.x);
     if (warp == 1) {
         tc_fence_after();
-        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(512u) : "memory");
+        asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(512u) : "memory");
     }
 }
 
@@ -538,16 +632,17 @@ __global__ void bounded_wait_selftest_kernel(StateHeader *hd, long long limit_cy
 }
 
 // Adds the partial results of the cut tiles (see StatsGemmArgs) into H / dXX^T, partial 1 first, then 2, ...:
-// one CTA per cut tile, after stats_umma_kernel of the same batch.
-constexpr int FIXUP_SLABS = 16;     // CTAs per cut tile, UBM / FIXUP_SLABS rows each
+// FIXUP_SLABS CTAs per cut tile, after stats_umma_kernel of the same batch.
+constexpr int FIXUP_SLABS = 32;     // CTAs per cut tile, UPM / FIXUP_SLABS rows each
 __global__ void __launch_bounds__(256) stats_fixup_kernel(StatsGemmArgs a) {
     TileIter it(a.n);
     if (!it.seek_to(a.full_tiles + blockIdx.x)) return;
-    const bool isD = it.r >= it.TM;
-    const int row0 = (isD ? it.r - it.TM : it.r) * UBM, col0 = it.tn * UBN;
+    const bool isD = it.r >= it.T;
+    const int row0 = (isD ? it.r - it.T : it.r) * UPM, col0 = it.tn * UBN;
     float *C = isD ? a.D : a.H;
-    const float *sp = a.scratch + (int64_t)blockIdx.x * (a.ksplit - 1) * (UBM * UBN);
-    constexpr int ROWS = UBM / FIXUP_SLABS;
+    // slot of partial c, CTA rank r: ((blockIdx.x * (ksplit - 1) + c) * 2 + r) * UBM * UBN
+    const float *sp = a.scratch + (int64_t)blockIdx.x * (a.ksplit - 1) * 2 * (UBM * UBN);
+    constexpr int ROWS = UPM / FIXUP_SLABS;
     const bool vec = (a.n & 3) == 0 && (reinterpret_cast<uintptr_t>(C) & 15) == 0;
 #pragma unroll
     for (int it4 = 0; it4 < ROWS * UBN / 4 / 256; ++it4) {
@@ -555,18 +650,19 @@ __global__ void __launch_bounds__(256) stats_fixup_kernel(StatsGemmArgs a) {
         const int i = blockIdx.y * ROWS + e4 / (UBN / 4), j = (e4 % (UBN / 4)) * 4;
         if (row0 + i >= a.n || col0 + j >= a.n) continue;
         float *cp = C + (int64_t)(row0 + i) * a.n + col0 + j;
-        const float *pp = sp + i * UBN + j;
+        const float *pp = sp + (int64_t)(i / UBM) * (UBM * UBN) + (i % UBM) * UBN + j;
+        const int64_t pstride = 2 * (int64_t)(UBM * UBN);
         if (vec && col0 + j + 3 < a.n) {
             float4 v = *reinterpret_cast<const float4 *>(cp);
             for (int c = 0; c < a.ksplit - 1; ++c) {
-                const float4 p = *reinterpret_cast<const float4 *>(pp + (int64_t)c * (UBM * UBN));
+                const float4 p = *reinterpret_cast<const float4 *>(pp + c * pstride);
                 v.x += p.x; v.y += p.y; v.z += p.z; v.w += p.w;
             }
             *reinterpret_cast<float4 *>(cp) = v;
         } else {
             for (int f = 0; f < 4 && col0 + j + f < a.n; ++f) {
                 float v = cp[f];
-                for (int c = 0; c < a.ksplit - 1; ++c) v += pp[(int64_t)c * (UBM * UBN) + f];
+                for (int c = 0; c < a.ksplit - 1; ++c) v += pp[c * pstride + f];
                 cp[f] = v;
             }
         }

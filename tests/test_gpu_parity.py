@@ -233,6 +233,48 @@ def test_update_term_switches(terms, n, group, B):
     st.close()
 
 
+@pytest.mark.parametrize("n,m,group,B", [(160, 24, 0, 32), (640, 40, 128, 128), (516, 16, 0, 64)])
+def test_rowwise_P_matches_the_row_by_row_form(n, m, group, B):
+    """gptaq_build_P_rowwise (Eq. "unparallel") against the oracle's row-by-row form: stage-wise from the device's
+    own dXX^T and U widened to float64, end to end through the codes that the loop then produces (which shows
+    that the operand copies of the lazy-batch update were made from this P)."""
+    cfg = wl.scaled(wl.CONFIGS["cfg2"], name="rowwise", n=n, m=m, batch_tokens=2048, n_batches=2, group=group,
+                    blocksize=B, outlier_channels=5)
+    batches = batches_of(cfg)
+    st = g.LayerState(cfg.n, m, cfg.batch_tokens, cfg.blocksize, total_tokens=cfg.tokens)
+    h = st.handle
+    for X, Xfp in batches:
+        g.gptaq_accumulate(h, X.cuda(), Xfp.cuda())
+    D_dev = st.D().cpu().numpy().astype(np.float64)
+    g.gptaq_factor(h, cfg.damp)
+    U_dev = np.triu(st.H().cpu().numpy().astype(np.float64))
+    g.gptaq_build_P_rowwise(h, cfg.alpha)
+    assert g.gptaq_sync_status(h)[0] == g.GPTAQ_OK
+    P_dev = st.D().cpu().numpy().astype(np.float64)
+    assert np.abs(np.tril(P_dev)).max() == 0.0
+    want = orc.build_P_rowwise(D_dev, cfg.tokens, U_dev, cfg.alpha)
+    assert hp.rel_fro(P_dev, want) <= 1e-5
+    # the loop on this P against the oracle's end-to-end U and P
+    ost = hp.oracle_stats(cfg, batches)
+    U, dead = orc.factor(ost.H, ost.tokens, cfg.damp)
+    P = orc.build_P_rowwise(ost.D, ost.tokens, U, cfg.alpha)
+    W = wl.make_weight(cfg)
+    G = hp.n_groups(n, group)
+    codes = torch.empty((m, n), dtype=torch.uint8, device="cuda")
+    scales = torch.empty((m, G), device="cuda"); zeros = torch.empty((m, G), device="cuda")
+    Wq = torch.empty((m, n), device="cuda")
+    g.gptaq_quantize(h, W.cuda(), cfg.bits, group, cfg.sym, B, codes, scales, zeros, Wq)
+    assert g.gptaq_sync_status(h)[0] == g.GPTAQ_OK
+    rep = orc.follow(W.numpy().astype(np.float64), U, P, dead, cfg.bits, group, cfg.sym, codes.cpu().numpy(),
+                     scales.cpu().numpy().astype(np.float64), zeros.cpu().numpy().astype(np.float64), band=hp.TOL_FLIP_BAND)
+    assert rep.disallowed == 0 and rep.allowed <= hp.TOL_FLIP_RATE * rep.total, rep
+    assert rep.grid_rel_err <= hp.TOL_GRID and rep.zero_mismatch == 0, rep
+    # wrong call order and the width limit are refused on the host
+    with pytest.raises(g.GptaqError):
+        g.gptaq_build_P_rowwise(h, cfg.alpha)
+    st.close()
+
+
 @pytest.mark.parametrize("n,m,group,B,bf16", [(160, 40, 0, 32, False), (200, 24, 32, 64, False),
                                                 (640, 96, 128, 128, False), (768, 64, 0, 128, True)])
 def test_act_order(n, m, group, B, bf16):
@@ -278,13 +320,57 @@ def test_act_order(n, m, group, B, bf16):
     rep = orc.follow(Wn[:, perm], U, P, dead, cfg.bits, cfg.group, cfg.sym, cg[:, perm],
                      sc.cpu().numpy().astype(np.float64), zp.cpu().numpy().astype(np.float64), band=hp.TOL_FLIP_BAND)
     assert rep.disallowed == 0 and rep.allowed <= hp.TOL_FLIP_RATE * rep.total, rep
-    assert rep.grid_rel_err <= 5e-5 and rep.zero_mismatch == 0, rep
+    assert rep.grid_rel_err <= hp.TOL_GRID and rep.zero_mismatch == 0, rep
     # dequantized weights come back in the caller's column order and match codes and grids
     gsz = cfg.group if cfg.group > 0 else n
     scp = np.repeat(sc.cpu().numpy(), gsz, axis=1)[:, :n]
     zpp = np.repeat(zp.cpu().numpy(), gsz, axis=1)[:, :n]
     deq_sorted = scp * (cg[:, perm].astype(np.float32) - zpp)
     assert np.array_equal(Wq.cpu().numpy()[:, perm], deq_sorted.astype(np.float32))
+    J_gpu, J_orc = orc.objective(Wn, Wq.cpu().numpy().astype(np.float64), so), orc.objective(Wn, res.Wq, so)
+    assert abs(J_gpu - J_orc) <= hp.TOL_OBJECTIVE * J_orc
+    st.close()
+
+
+@pytest.mark.parametrize("n,m,group,B,act,bf16", [(192, 24, 32, 64, True, False), (640, 40, 128, 128, True, False),
+                                                  (768, 33, 64, 128, True, True), (640, 20, 128, 128, False, False)])
+def test_static_groups(n, m, group, B, act, bf16):
+    """Static groups, with and without act_order: grids per group of the caller's columns from the original
+    weights; the loop replayed by the oracle in the device's processing order with those grids."""
+    cfg = wl.scaled(wl.CONFIGS["cfg2"], name="static_groups", n=n, m=m, batch_tokens=2048, n_batches=2, group=group,
+                    blocksize=B, outlier_channels=4, w_bf16=bf16)
+    bt = batches_of(cfg)
+    W = wl.make_weight(cfg)
+    st = g.LayerState(cfg.n, cfg.m, cfg.batch_tokens, cfg.blocksize, total_tokens=cfg.tokens)
+    g.gptaq_set_act_order(st.handle, act)
+    g.gptaq_set_static_groups(st.handle, True)
+    for X, Xfp in bt:
+        g.gptaq_accumulate(st.handle, X.cuda(), Xfp.cuda())
+    g.gptaq_factor(st.handle, cfg.damp)
+    g.gptaq_build_P(st.handle, cfg.alpha)
+    perm = st.perm().cpu().numpy().astype(np.int64) if act else np.arange(n)
+    G = hp.n_groups(n, group)
+    codes = torch.empty((m, n), dtype=torch.uint8, device="cuda")
+    sc = torch.empty((m, G), dtype=torch.float32, device="cuda")
+    zp = torch.empty((m, G), dtype=torch.float32, device="cuda")
+    Wq = torch.empty((m, n), dtype=torch.float32, device="cuda")
+    Wd = W.cuda().to(torch.bfloat16) if bf16 else W.cuda()
+    g.gptaq_quantize(st.handle, Wd, cfg.bits, group, cfg.sym, B, codes, sc, zp, Wq)
+    assert g.gptaq_sync_status(st.handle)[0] == g.GPTAQ_OK
+    so = hp.oracle_stats(cfg, bt)
+    Wn = W.numpy().astype(np.float64)
+    U, P, dead, res, _ = orc.solve_act_order(Wn, so.H, so.D, so.tokens, cfg.damp, cfg.alpha, cfg.bits, group, cfg.sym,
+                                             perm=perm, static_groups=True)
+    cg, scn, zpn = codes.cpu().numpy(), sc.cpu().numpy(), zp.cpu().numpy()
+    # the grids are those of the original weights, float32 arithmetic on both sides of a min/max
+    assert np.abs(scn - res.scales).max() <= 1e-6 * np.abs(res.scales).max() and np.array_equal(zpn, res.zeros)
+    rep = orc.follow(Wn[:, perm], U, P, dead, cfg.bits, group, cfg.sym, cg[:, perm], scn.astype(np.float64),
+                     zpn.astype(np.float64), band=hp.TOL_FLIP_BAND, static=(Wn, perm // group))
+    assert rep.disallowed == 0 and rep.allowed <= hp.TOL_FLIP_RATE * rep.total, rep
+    assert rep.grid_rel_err <= 1e-6 and rep.zero_mismatch == 0, rep
+    # the outputs dequantize with the grid of group column // group, in the caller's column order
+    g_of = np.arange(n) // group
+    assert np.array_equal(Wq.cpu().numpy(), (scn[:, g_of] * (cg.astype(np.float32) - zpn[:, g_of])).astype(np.float32))
     J_gpu, J_orc = orc.objective(Wn, Wq.cpu().numpy().astype(np.float64), so), orc.objective(Wn, res.Wq, so)
     assert abs(J_gpu - J_orc) <= hp.TOL_OBJECTIVE * J_orc
     st.close()
@@ -325,7 +411,7 @@ def test_clip_search(n, m, group, B, sym, bits):
                      sc.cpu().numpy().astype(np.float64), zp.cpu().numpy().astype(np.float64),
                      band=hp.TOL_FLIP_BAND, clip=clip)
     assert rep.disallowed == 0 and rep.allowed <= hp.TOL_FLIP_RATE * rep.total, rep
-    assert rep.grid_rel_err <= 5e-5 and rep.zero_mismatch == 0, rep
+    assert rep.grid_rel_err <= hp.TOL_GRID and rep.zero_mismatch == 0, rep
     # the search does change grids on this input, and the objective matches the oracle's
     plain = orc.quantize(Wn, U, P, dead, cfg.bits, cfg.group, cfg.sym)
     res = orc.quantize(Wn, U, P, dead, cfg.bits, cfg.group, cfg.sym, clip=clip)
@@ -427,6 +513,25 @@ def test_device_side_conditions_are_reported_not_trapped():
     status, info = g.gptaq_sync_status(h)
     assert status == g.GPTAQ_ERR_NONFINITE
     st.close()
+    # a NaN / Inf in the LAST column of W propagates nowhere and quantizes to a finite code: it is
+    # reported from the loaded value, with its row, by both column kernels (full blocks with grids per
+    # 32 columns take column_block_kernel, groups of 8 take column_loop_kernel)
+    for group, bad_value, row in ((32, float("nan"), 2), (8, float("inf"), 1), (0, float("nan"), 3)):
+        st = g.LayerState(n, 4, 256, 32)
+        h = st.handle
+        Xb = torch.randn(256, n, device="cuda")
+        g.gptaq_accumulate(h, Xb, Xb + 0.01 * torch.randn_like(Xb))
+        g.gptaq_factor(h, 0.01)
+        g.gptaq_build_P(h, 0.25)
+        W = 0.02 * torch.randn(4, n, device="cuda")
+        W[row, n - 1] = bad_value
+        G = hp.n_groups(n, group)
+        codes = torch.empty((4, n), dtype=torch.uint8, device="cuda")
+        scales = torch.empty((4, G), device="cuda"); zeros = torch.empty((4, G), device="cuda")
+        g.gptaq_quantize(h, W, 4, group, False, 32, codes, scales, zeros)
+        status, info = g.gptaq_sync_status(h)
+        assert status == g.GPTAQ_ERR_NONFINITE and info == row, (group, status, info)
+        st.close()
 
 
 def test_bounded_wait_runs_out_and_is_reported():
