@@ -7,10 +7,12 @@ reset -> accumulate (all token batches) -> factor -> build_P -> quantize.
     python bench.py [--gpus N] [--steps K] [--warmup W] [--workload cfg2]
     python bench.py --impl reference ...     # the float64 CPU oracle, bounded sample
 
-Prints ONE JSON line (rank 0).  With N > 1 (launched by torchrun) every rank
-solves its own independent layer of the same shape (layers are independent
-problems; no data-path collective), and the value is the time per layer of
-the whole job.
+Prints ONE JSON line (rank 0).  With N > 1 (launched by torchrun) the ranks
+share ONE layer: every rank accumulates its share of the token batches, one
+all-reduce sums H and dXX^T, every rank factors and then quantizes its slab
+of the rows of W (strong scaling; the value is the time of that one layer).
+``--replicas`` instead gives every rank an independent layer of the same
+shape (no data-path collective; the value is the time per layer of the job).
 """
 from __future__ import annotations
 
@@ -31,10 +33,11 @@ import workloads as wl  # noqa: E402
 
 METRIC = "ms per layer (GPTAQ solve: accumulate + factor + P + quantize)"
 
-# dram__bytes_read.sum + dram__bytes_write.sum of one stats_umma_kernel launch (one token batch), from
-# the ncu capture summarised in profiles/stats_umma_kernel_cfg2_batch.md; keyed by (workload, statistics
-# arithmetic).  Entries are dropped when the kernel changes.
-STATS_KERNEL_TRAFFIC = {("cfg2", 0): 597.2e6}
+# dram__bytes_read.sum + dram__bytes_write.sum of one stats_umma_kernel launch (one token batch) from an
+# ncu capture of the kernel as it stands, keyed by (workload, statistics arithmetic); workloads without a
+# capture of the current kernel report null with the reason.
+STATS_KERNEL_TRAFFIC = {}
+TRAFFIC_MISSING = "no ncu capture of the current statistics kernel for this workload and arithmetic"
 
 
 def peaks():
@@ -108,7 +111,8 @@ def oracle_sample(cfg: wl.LayerConfig, sample_tokens: int, sample_rows: int):
     orc.accumulate(st, X, Xfp)
     t_acc = time.perf_counter() - t0
     t0 = time.perf_counter()
-    U, dead = orc.factor(st.H, st.tokens, max(cfg.damp, 0.05))   # few tokens: keep the sample SPD
+    sample_damp = max(cfg.damp, 0.05)                            # few tokens: keep the sample SPD
+    U, dead = orc.factor(st.H, st.tokens, sample_damp)
     t_fac = time.perf_counter() - t0
     t0 = time.perf_counter()
     P = orc.build_P(st.D, st.tokens, U, cfg.alpha)
@@ -118,8 +122,9 @@ def oracle_sample(cfg: wl.LayerConfig, sample_tokens: int, sample_rows: int):
     t_q = time.perf_counter() - t0
     total = t_acc * (cfg.tokens / sample_tokens) + t_fac + t_p + t_q * (cfg.m / sample_rows)
     desc = (f"accumulate on {sample_tokens} of {cfg.tokens} tokens ({t_acc:.2f} s, scaled by tokens); "
-            f"factor ({t_fac:.2f} s) and P ({t_p:.2f} s) in full; column loop on {sample_rows} of {cfg.m} rows "
-            f"({t_q:.2f} s, scaled by rows)")
+            f"factor ({t_fac:.2f} s; damp raised from {cfg.damp} to {sample_damp} so that the sample's H, from fewer "
+            f"tokens than input channels, stays positive definite) and P ({t_p:.2f} s) in full; column loop on "
+            f"{sample_rows} of {cfg.m} rows ({t_q:.2f} s, scaled by rows)")
     return total * 1e3, desc, threads
 
 
@@ -178,6 +183,10 @@ def run_ours(args, cfg):
     dev = torch.device("cuda", local)
     if world > 1:
         import torch.distributed as dist
+        # the communicator's own log lines (ranks, transport) stay on: they are the record of what the
+        # all-reduce ran over
+        os.environ.setdefault("NCCL_DEBUG", "INFO")
+        os.environ.setdefault("NCCL_DEBUG_SUBSYS", "INIT")
         dist.init_process_group("nccl", device_id=dev)
     if rank == 0:
         gbuild.build()
@@ -187,7 +196,7 @@ def run_ours(args, cfg):
     pk = peaks()
 
     # inputs resident in HBM before the timed region (each rank its own layer: seed = rank)
-    shard = bool(args.shard_layer) and world > 1
+    shard = world > 1 and not args.replicas
     if shard:
         # ONE layer across the ranks: this rank's share of the token batches and of the rows of W
         from paper_2504_02692_b200 import sharded
@@ -360,14 +369,59 @@ def run_ours(args, cfg):
                       "layer_quantize": fac_ms + p_ms + q_ms},
         "accumulate_tflops": achieved, "stage_rooflines": stage_rooflines,
         "roofline": {"kernel": "gptaq_accumulate (one token batch)", "bound": "tensor", "achieved": achieved,
-                     "peak": peak, "unit": "TFLOP/s", "frac": achieved / peak, "traffic": STATS_KERNEL_TRAFFIC.get((cfg.name, prec)),
-                     "peak_source": pk["source"] + " bf16 cuBLAS, sustained",
+                     "peak": peak, "unit": "TFLOP/s", "frac": achieved / peak,
+                     "traffic": STATS_KERNEL_TRAFFIC.get((cfg.name, prec)),
+                     "traffic_note": None if (cfg.name, prec) in STATS_KERNEL_TRAFFIC else TRAFFIC_MISSING,
+                     "peak_source": pk["source"] + " bf16 cuBLAS, sustained (the accumulate stage runs for "
+                                    "milliseconds under the power cap)",
+                     "peak_burst": pk["bf16_burst"], "frac_of_burst": achieved / pk["bf16_burst"],
                      "algorithmic_flops_per_launch": flops_call},
         "cpu_baseline": cpu, "e2e": e2e, "gpu_launches": launches, "clocks": clk.summary(),
     }
     if args.batches > 0:
         line["truncated"] = f"{cfg.n_batches} token batches only: not a benchmark value"
     print(json.dumps(line), flush=True)
+
+
+def run_p_rowwise(args):
+    """Latency of P in its two forms (Theorem 4.2 as two matrix products vs. Eq. "unparallel" row by row),
+    the comparison of the paper's Section 5 ("Efficiency"), on synthetic layers of width 1024 and 4096."""
+    import paper_2504_02692_b200 as g
+    from paper_2504_02692_b200 import build as gbuild
+    torch.cuda.set_device(0)
+    gbuild.build()
+    g.load_library()
+    stream = torch.cuda.current_stream()
+    out = {}
+    for n in (1024, 4096):
+        cfg = wl.scaled(wl.CONFIGS["cfg2"], name=f"p{n}", n=n, m=128, n_batches=2)
+        batches = [wl.make_batch(cfg, b, "cuda") for b in range(cfg.n_batches)]
+        st = g.LayerState(cfg.n, cfg.m, cfg.batch_tokens, cfg.blocksize, "cuda", total_tokens=cfg.tokens)
+        h = st.handle
+        times = {"theorem_4_2": [], "row_by_row": []}
+        for name, fn in (("theorem_4_2", g.gptaq_build_P), ("row_by_row", g.gptaq_build_P_rowwise)):
+            for i in range(args.warmup + args.steps):
+                g.gptaq_reset(h)
+                for X, Xfp in batches:
+                    g.gptaq_accumulate(h, X, Xfp)
+                g.gptaq_factor(h, cfg.damp)
+                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                e0.record(stream)
+                fn(h, cfg.alpha)
+                e1.record(stream)
+                torch.cuda.synchronize()
+                if i >= args.warmup:
+                    times[name].append(e0.elapsed_time(e1))
+        status = g.gptaq_sync_status(h)
+        if status[0] != g.GPTAQ_OK:
+            raise RuntimeError(f"device status {status}")
+        med = {k: sorted(v)[len(v) // 2] for k, v in times.items()}
+        out[f"n{n}"] = {"theorem_4_2_ms": med["theorem_4_2"], "row_by_row_ms": med["row_by_row"],
+                        "ratio": med["row_by_row"] / med["theorem_4_2"]}
+        st.close()
+    print(json.dumps({"metric": "ms to build P, two forms (includes the operand copies for the loop)", "unit": "ms",
+                      "steps": args.steps, "warmup": args.warmup, "p_rowwise": out, "data": "synthetic",
+                      "truncated": "comparison of two forms of one stage: not a benchmark value"}), flush=True)
 
 
 def main():
@@ -381,14 +435,18 @@ def main():
     ap.add_argument("--ref-rows", type=int, default=512)
     ap.add_argument("--batches", type=int, default=0,
                     help="profiler captures only: keep this many token batches (the line is marked truncated)")
-    ap.add_argument("--shard-layer", action="store_true",
-                    help="N > 1: one layer across the ranks (token-sharded statistics, one all-reduce, row-sharded "
-                         "quantize; strong scaling) instead of one independent layer per rank")
+    ap.add_argument("--replicas", action="store_true",
+                    help="N > 1: one independent layer per rank (weak scaling, no collective) instead of the default, "
+                         "one layer across the ranks (token-sharded statistics, one all-reduce, row-sharded quantize)")
+    ap.add_argument("--shard-layer", action="store_true", help="(default for N > 1; kept for older command lines)")
     ap.add_argument("--clip-search", type=int, default=0,
                     help="clipping-range search of the grids with this many candidates (off in the headline configuration)")
     ap.add_argument("--act-order", action="store_true", help="columns sorted by diag(H) (off in the headline configuration)")
     ap.add_argument("--full-split-statistics", action="store_true",
                     help="both statistics with split fp16 operands (float32-grade, 3x the MMAs; off in the headline configuration)")
+    ap.add_argument("--p-rowwise", action="store_true",
+                    help="times P as two matrix products (Theorem 4.2) against the row-by-row form at n = 1024 and 4096 "
+                         "and prints that comparison instead of the benchmark line")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()
@@ -399,6 +457,10 @@ def main():
     args.full_tokens = full_tokens
     if args.impl == "reference":
         run_reference(args, cfg)
+    elif args.p_rowwise:
+        if not torch.cuda.is_available():
+            raise SystemExit("bench.py --p-rowwise needs a CUDA device")
+        run_p_rowwise(args)
     else:
         if not torch.cuda.is_available():
             raise SystemExit("bench.py needs a CUDA device (there is no CPU fallback); "

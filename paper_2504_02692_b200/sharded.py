@@ -50,9 +50,10 @@ def allreduce_sums(H: torch.Tensor, D: torch.Tensor, tokens: int, group=None) ->
 def allreduce_statistics(state, group=None) -> int:
     """The exchange step for a ``LayerState`` after this rank's gptaq_accumulate calls: orders the
     stream after the pending products, all-reduces H and dXX^T in the state buffer and sets the total
-    token count on the handle (so that gptaq_factor normalises by it).  Returns the total."""
-    from . import binding as g
+    token count on the handle (so that gptaq_factor normalises by it).  Returns the total.
+    ``state`` needs ``H()``, ``D()`` (views of the sums, current on the stream the collective runs on),
+    ``tokens()`` and ``set_tokens(total)``."""
     H, D = state.H(), state.D()          # views; H() / D() flush the handle's internal stream first
-    total = allreduce_sums(H, D, g.gptaq_tokens(state.handle), group)
-    g.gptaq_set_tokens(state.handle, total)
+    total = allreduce_sums(H, D, state.tokens(), group)
+    state.set_tokens(total)
     return total

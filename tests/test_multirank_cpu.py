@@ -80,7 +80,18 @@ def _shard_worker(rank, world, port, out):
         X, Xfp = wl.make_batch(cfg, b)
         orc.accumulate(st, X.numpy(), Xfp.numpy())
     H, D = torch.from_numpy(st.H.astype(np.float32)), torch.from_numpy(st.D.astype(np.float32))
-    total = sharded.allreduce_sums(H, D, st.tokens)
+
+    class HostState:
+        """What allreduce_statistics needs of a LayerState, over plain CPU tensors."""
+        def __init__(self, tokens): self._tokens, self.views = tokens, 0
+        def H(self): self.views += 1; return H
+        def D(self): self.views += 1; return D
+        def tokens(self): return self._tokens
+        def set_tokens(self, t): self._tokens = t
+
+    hs = HostState(st.tokens)
+    total = sharded.allreduce_statistics(hs)
+    assert hs.tokens() == total and hs.views == 2
     full = orc.new_stats(cfg.n)
     for b in range(cfg.n_batches):
         X, Xfp = wl.make_batch(cfg, b)
