@@ -36,7 +36,7 @@ METRIC = "ms per layer (GPTAQ solve: accumulate + factor + P + quantize)"
 # dram__bytes_read.sum + dram__bytes_write.sum of one stats_umma_kernel launch (one token batch) from an
 # ncu capture of the kernel as it stands, keyed by (workload, statistics arithmetic); workloads without a
 # capture of the current kernel report null with the reason.
-STATS_KERNEL_TRAFFIC = {}
+STATS_KERNEL_TRAFFIC = {("cfg2", 0): 589.6e6}
 TRAFFIC_MISSING = "no ncu capture of the current statistics kernel for this workload and arithmetic"
 
 
@@ -97,16 +97,21 @@ class ClockSampler:
 
 # --------------------------------------------------------------------------- CPU oracle leg
 def oracle_sample(cfg: wl.LayerConfig, sample_tokens: int, sample_rows: int):
-    """Times the float64 oracle, as it stands, on a bounded sample of the
-    workload and scales linearly to the whole layer (statistics are linear in
-    tokens, rows of W are independent).  Returns (ms per layer, description)."""
+    """Times the float64 oracle, as it stands, on a bounded sample of the workload and scales to the whole
+    layer: statistics are linear in tokens, rows of W are independent.  Beyond n = 4096 the sample shrinks so
+    that it stays near 10-30 s of CPU work (fewer tokens and rows), and beyond n = 16384 -- where a float64
+    factorisation of the whole n x n matrix takes hours -- factor, P and the loop run on the leading 8192
+    input channels and are scaled by the cubes / squares of the width ratio.  Returns (ms per layer,
+    description, threads)."""
     from oracle import gptaq_oracle as orc
     threads = torch.get_num_threads()
-    sample_tokens = min(sample_tokens, cfg.batch_tokens)
-    sample_rows = min(sample_rows, cfg.m)
-    X, Xfp = (t.numpy() for t in wl.make_batch(cfg, 0, "cpu", sample_tokens))
-    W = wl.make_weight(cfg, "cpu", rows=sample_rows).numpy()
-    st = orc.new_stats(cfg.n)
+    n_s = cfg.n if cfg.n <= 16384 else 8192
+    shrink = min(1.0, 4096.0 / n_s)
+    sample_tokens = min(max(256, int(sample_tokens * shrink)), cfg.batch_tokens)
+    sample_rows = min(max(8, int(sample_rows * shrink * shrink)), cfg.m)
+    X, Xfp = (t.numpy()[:, :n_s] for t in wl.make_batch(cfg, 0, "cpu", sample_tokens))
+    W = wl.make_weight(cfg, "cpu", rows=sample_rows).numpy()[:, :n_s]
+    st = orc.new_stats(n_s)
     t0 = time.perf_counter()
     orc.accumulate(st, X, Xfp)
     t_acc = time.perf_counter() - t0
@@ -120,11 +125,14 @@ def oracle_sample(cfg: wl.LayerConfig, sample_tokens: int, sample_rows: int):
     t0 = time.perf_counter()
     orc.quantize(W, U, P, dead, cfg.bits, cfg.group, cfg.sym)
     t_q = time.perf_counter() - t0
-    total = t_acc * (cfg.tokens / sample_tokens) + t_fac + t_p + t_q * (cfg.m / sample_rows)
+    w = cfg.n / n_s                                              # width ratio of the layer to the sample
+    total = t_acc * (cfg.tokens / sample_tokens) * w * w + (t_fac + t_p) * w ** 3 + t_q * (cfg.m / sample_rows) * w * w
+    width = "" if n_s == cfg.n else (f"; all of it on the leading {n_s} of {cfg.n} input channels, statistics and loop scaled "
+                                     f"by the width ratio squared, factor and P by its cube")
     desc = (f"accumulate on {sample_tokens} of {cfg.tokens} tokens ({t_acc:.2f} s, scaled by tokens); "
             f"factor ({t_fac:.2f} s; damp raised from {cfg.damp} to {sample_damp} so that the sample's H, from fewer "
             f"tokens than input channels, stays positive definite) and P ({t_p:.2f} s) in full; column loop on "
-            f"{sample_rows} of {cfg.m} rows ({t_q:.2f} s, scaled by rows)")
+            f"{sample_rows} of {cfg.m} rows ({t_q:.2f} s, scaled by rows){width}")
     return total * 1e3, desc, threads
 
 
@@ -269,6 +277,8 @@ def run_ours(args, cfg):
 
     marks = []
     sync_all()
+    g.gptaq_set_kernel_timing(h, True)       # event pairs around the statistics kernel on its own stream
+    g.gptaq_stats_kernel_time(h)
     l0 = g.gptaq_launch_count(h)
     t_beg, t_end = ev(), ev()
     with ClockSampler(local) as clk:
@@ -278,6 +288,8 @@ def run_ours(args, cfg):
         t_end.record(stream)
         sync_all()
     launches = g.gptaq_launch_count(h) - l0
+    kern_ms_total, kern_launches = g.gptaq_stats_kernel_time(h)
+    g.gptaq_set_kernel_timing(h, False)
     ms_total = t_beg.elapsed_time(t_end)
     ms_total = max_over_ranks(ms_total, world, dev)
     ms_step = ms_total / args.steps
@@ -289,8 +301,18 @@ def run_ours(args, cfg):
     p_ms = sum(m[2].elapsed_time(m[3]) for m in marks) / args.steps
     q_ms = sum(m[3].elapsed_time(m[4]) for m in marks) / args.steps
     flops_call = 3.0 * cfg.n * cfg.n * cfg.batch_tokens
-    achieved = flops_call / (acc_call_ms * 1e-3) / 1e12
+    stage_achieved = flops_call / (acc_call_ms * 1e-3) / 1e12     # whole accumulate call: conversion, product, fix-up
     peak = pk["bf16_sustained"]
+    if kern_launches > 0:
+        # the dominant kernel by itself: algorithmic flops of the timed region / the sum of its launch durations
+        kern_us = kern_ms_total * 1e3 / kern_launches
+        flops_launch = 3.0 * cfg.n * cfg.n * cfg.batch_tokens * len(batches) * args.steps / kern_launches
+        achieved = flops_launch / (kern_us * 1e-6) / 1e12
+        kern_name = "stats_umma_kernel (tcgen05 kind::f16, cta_group::2), one token batch per launch"
+    else:
+        # widths below 256 accumulate on the float32 FMA kernel: the stage is the unit
+        kern_us, flops_launch, achieved = acc_call_ms * 1e3, flops_call, stage_achieved
+        kern_name = "gptaq_accumulate (one token batch; float32 FMA path below n = 256)"
 
     # end to end through the host entry points: pinned host buffers in, host results out
     e2e = None
@@ -367,15 +389,19 @@ def run_ours(args, cfg):
                        statistics=prec_name, act_order=bool(args.act_order), clip_search=args.clip_search),
         "stages_ms": {"accumulate": acc_step_ms, "factor": fac_ms, "build_P": p_ms, "quantize": q_ms,
                       "layer_quantize": fac_ms + p_ms + q_ms},
-        "accumulate_tflops": achieved, "stage_rooflines": stage_rooflines,
-        "roofline": {"kernel": "gptaq_accumulate (one token batch)", "bound": "tensor", "achieved": achieved,
+        "accumulate_tflops": stage_achieved, "stage_rooflines": stage_rooflines,
+        "roofline": {"kernel": kern_name, "bound": "tensor", "achieved": achieved,
                      "peak": peak, "unit": "TFLOP/s", "frac": achieved / peak,
+                     "kernel_us_per_launch": kern_us, "kernel_launches": kern_launches,
+                     "accumulate_stage": {"what": "whole gptaq_accumulate call (conversion prologue + product + fix-up)",
+                                          "us_per_batch": acc_call_ms * 1e3, "achieved": stage_achieved,
+                                          "frac": stage_achieved / peak, "frac_of_burst": stage_achieved / pk["bf16_burst"]},
                      "traffic": STATS_KERNEL_TRAFFIC.get((cfg.name, prec)),
                      "traffic_note": None if (cfg.name, prec) in STATS_KERNEL_TRAFFIC else TRAFFIC_MISSING,
                      "peak_source": pk["source"] + " bf16 cuBLAS, sustained (the accumulate stage runs for "
                                     "milliseconds under the power cap)",
                      "peak_burst": pk["bf16_burst"], "frac_of_burst": achieved / pk["bf16_burst"],
-                     "algorithmic_flops_per_launch": flops_call},
+                     "algorithmic_flops_per_launch": flops_launch},
         "cpu_baseline": cpu, "e2e": e2e, "gpu_launches": launches, "clocks": clk.summary(),
     }
     if args.batches > 0:

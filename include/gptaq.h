@@ -284,6 +284,14 @@ gptaq_status_t gptaq_set_update_terms(gptaq_handle_t h, int terms);
 /* Number of kernels this handle has launched since create (bookkeeping for benchmarks). */
 int64_t gptaq_launch_count(gptaq_handle_t h);
 
+/* Timing of the dominant kernel by itself (bookkeeping for benchmarks).  While enabled, every launch of the
+ * tensor-core statistics kernel (Algorithm 1, line 2) is bracketed by a pair of CUDA events on the stream it
+ * runs on -- the handle's own stream, which events of the caller cannot reach.  gptaq_stats_kernel_time waits
+ * (on the host) for the recorded launches, returns the sum of their durations in milliseconds and their number,
+ * and starts a new record.  The conversion prologue and the fix-up of K-split tiles are not included. */
+gptaq_status_t gptaq_set_kernel_timing(gptaq_handle_t h, int enable);
+gptaq_status_t gptaq_stats_kernel_time(gptaq_handle_t h, double *ms_total, int64_t *launches);
+
 /* Failure-path self-test: enqueues one warp that waits, with the bounded wait of the tensor-core
  * kernels, for a barrier that nothing completes; after `seconds` (0 < seconds <= 2, in SM clock
  * cycles at the nominal clock) it gives up and records GPTAQ_ERR_TIMEOUT (info 2000000) for

@@ -69,6 +69,8 @@ SIGNATURES = {
     "gptaq_perm": (_vp, [_vp]),
     "gptaq_recommended_stats_precision": (_int, [_i64, _i64]),
     "gptaq_launch_count": (_i64, [_vp]),
+    "gptaq_set_kernel_timing": (_int, [_vp, _int]),
+    "gptaq_stats_kernel_time": (_int, [_vp, C.POINTER(C.c_double), C.POINTER(_i64)]),
     "gptaq_status_string": (C.c_char_p, [_int]),
     "gptaq_last_cuda_error": (C.c_char_p, [_vp]),
 }
@@ -327,6 +329,18 @@ def gptaq_recommended_stats_precision(n: int, total_tokens: int) -> int:
 
 def gptaq_launch_count(h) -> int:
     return load_library().gptaq_launch_count(h)
+
+
+def gptaq_set_kernel_timing(h, enable: bool):
+    """Brackets every launch of the statistics kernel with events on its own stream (see gptaq_stats_kernel_time)."""
+    _check(load_library().gptaq_set_kernel_timing(h, int(bool(enable))), "gptaq_set_kernel_timing", h)
+
+
+def gptaq_stats_kernel_time(h):
+    """``(total ms, launches)`` of the statistics kernel since the last call; waits for those launches."""
+    ms, n = C.c_double(0.0), _i64(0)
+    _check(load_library().gptaq_stats_kernel_time(h, C.byref(ms), C.byref(n)), "gptaq_stats_kernel_time", h)
+    return ms.value, n.value
 
 
 def gptaq_status_string(status: int) -> str:

@@ -10,6 +10,8 @@
 #include <mutex>
 #include <new>
 #include <string>
+#include <utility>
+#include <vector>
 
 #include "kernels.cuh"
 #include "simt_gemm.cuh"
@@ -61,6 +63,10 @@ struct gptaq_ctx {
     bool gemm_pending[2];
     bool relayout;         // the operand buffers change size: wait for the products in flight first
     int next_buf;
+    // optional timing of the statistics kernel alone: one event pair per launch, on the stream it runs on
+    bool kernel_timing;
+    std::vector<std::pair<cudaEvent_t, cudaEvent_t>> timing_events;   // pool; the first timing_used are recorded
+    size_t timing_used;
     std::string cuda_error;
 };
 
@@ -446,8 +452,20 @@ gptaq_status_t accumulate_tc(gptaq_ctx *h, const float *X, const float *Xfp, int
         ga.scratch = reinterpret_cast<float *>(h->ws + 2 * buf_bytes);
         const int nitems = ga.full_tiles + ((int)ntiles - ga.full_tiles) * ga.ksplit;
         const int sgrid = 2 * std::min(nitems, npairs);
+        std::pair<cudaEvent_t, cudaEvent_t> *tev = nullptr;
+        if (h->kernel_timing) {
+            if (h->timing_used == h->timing_events.size()) {
+                std::pair<cudaEvent_t, cudaEvent_t> ev{nullptr, nullptr};
+                CU(cudaEventCreate(&ev.first));
+                CU(cudaEventCreate(&ev.second));
+                h->timing_events.push_back(ev);
+            }
+            tev = &h->timing_events[h->timing_used++];
+            CU(cudaEventRecord(tev->first, gs));
+        }
         stats_umma_kernel<<<sgrid, UMMA_THREADS, UMMA_SMEM, gs>>>(mX, mD, mL, mDL, ga);
         LAUNCHED();
+        if (tev) CU(cudaEventRecord(tev->second, gs));
         if (ga.ksplit > 1) {
             stats_fixup_kernel<<<dim3((unsigned)((int)ntiles - ga.full_tiles), FIXUP_SLABS), 256, 0, gs>>>(ga);
             LAUNCHED();
@@ -788,6 +806,8 @@ gptaq_status_t gptaq_create(gptaq_handle_t *out, int64_t n, void *d_state, size_
     h->terms = GPTAQ_TERM_ERR | GPTAQ_TERM_ASYM;
     h->clip_steps = 0; h->clip_min = 1.f;
     h->static_groups = false;
+    h->kernel_timing = false;
+    h->timing_used = 0;
     cudaError_t e = cudaGetDevice(&h->device);
     if (e == cudaSuccess) e = cudaDeviceGetAttribute(&h->num_sms, cudaDevAttrMultiProcessorCount, h->device);
     if (e == cudaSuccess)
@@ -866,6 +886,7 @@ gptaq_status_t gptaq_destroy(gptaq_handle_t h) {
         if (h->conv_done[i]) cudaEventDestroy(h->conv_done[i]);
         if (h->gemm_done[i]) cudaEventDestroy(h->gemm_done[i]);
     }
+    for (auto &ev : h->timing_events) { cudaEventDestroy(ev.first); cudaEventDestroy(ev.second); }
     delete h;
     return GPTAQ_OK;
 }
@@ -1431,6 +1452,27 @@ int gptaq_recommended_stats_precision(int64_t n, int64_t total_tokens) {
 }
 
 int64_t gptaq_launch_count(gptaq_handle_t h) { return h ? h->launches : -1; }
+
+gptaq_status_t gptaq_set_kernel_timing(gptaq_handle_t h, int enable) {
+    if (!h) return GPTAQ_ERR_INVALID_ARG;
+    h->kernel_timing = enable != 0;
+    return GPTAQ_OK;
+}
+
+gptaq_status_t gptaq_stats_kernel_time(gptaq_handle_t h, double *ms_total, int64_t *launches) {
+    if (!h || !ms_total || !launches) return GPTAQ_ERR_INVALID_ARG;
+    double total = 0.0;
+    for (size_t i = 0; i < h->timing_used; ++i) {
+        CU(cudaEventSynchronize(h->timing_events[i].second));
+        float ms = 0.f;
+        CU(cudaEventElapsedTime(&ms, h->timing_events[i].first, h->timing_events[i].second));
+        total += ms;
+    }
+    *ms_total = total;
+    *launches = (int64_t)h->timing_used;
+    h->timing_used = 0;
+    return GPTAQ_OK;
+}
 
 const char *gptaq_status_string(gptaq_status_t s) {
     switch (s) {
