@@ -54,10 +54,12 @@ def test_ragged_shapes(n, m, tokens, nb, bits, group, sym, B):
 
 
 @pytest.mark.parametrize("n,m,B,group,sym,bits", [(576, 70, 64, 64, True, 4), (640, 33, 32, 32, False, 3),
-                                                   (516, 129, 128, 0, False, 4)])
+                                                   (516, 129, 128, 0, False, 4), (576, 40, 64, 16, False, 3),
+                                                   (648, 50, 128, 8, True, 4)])
 def test_tensor_path_block_sizes_and_tails(n, m, B, group, sym, bits):
     """Widths >= 512 (float32-grade tensor-core products) with the smaller lazy-batch blocks, a width that is
-    a multiple of 4 only, and row counts that do not fill the last CTA."""
+    a multiple of 4 only, row counts that do not fill the last CTA, and grids per group of fewer than 32 columns
+    (the general column kernel feeding the fp16-split tensor-core update)."""
     cfg = wl.scaled(wl.CONFIGS["cfg2"], name="tails", n=n, m=m, batch_tokens=1500, n_batches=2, bits=bits, group=group,
                     sym=sym, blocksize=B, outlier_channels=5)
     out = hp.check_layer(cfg, wl.make_weight(cfg), batches_of(cfg))
