@@ -282,14 +282,25 @@ __device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_addr) {
 __device__ __forceinline__ void st_cluster_u32(uint32_t cluster_addr, uint32_t v) {
     asm volatile("st.shared::cluster.u32 [%0], %1;" ::"r"(cluster_addr), "r"(v) : "memory");
 }
+// try_wait with acquire semantics at cluster scope: what the other CTA of the pair wrote (to this CTA's
+// shared memory, or through the commit of its MMAs) before it signalled the barrier is visible afterwards.
+__device__ __forceinline__ bool mbar_try_cluster(uint32_t bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+    return ok != 0;
+}
 // Bounded wait of a CTA pair: as mbar_wait, and a wait that gives up also raises the other CTA's flag
 // (at cluster address peer_abort), so that the pair winds down together instead of one timeout at a time.
 __device__ __forceinline__ bool mbar_wait_pair(uint32_t bar, uint32_t parity, volatile int *abort_flag,
                                                uint32_t peer_abort, long long limit_cycles = WAIT_LIMIT_CYCLES) {
-    if (mbar_try(bar, parity)) return true;
+    if (mbar_try_cluster(bar, parity)) return true;
     const long long t0 = clock64();
     for (uint32_t it = 1;; ++it) {
-        if (mbar_try(bar, parity)) return true;
+        if (mbar_try_cluster(bar, parity)) return true;
         if ((it & 63) == 0) {
             if (*abort_flag) return false;
             if (clock64() - t0 > limit_cycles) { *abort_flag = 1; st_cluster_u32(peer_abort, 1u); return false; }

@@ -54,7 +54,7 @@ def test_ragged_shapes(n, m, tokens, nb, bits, group, sym, B):
 
 
 @pytest.mark.parametrize("n,m,B,group,sym,bits", [(576, 70, 64, 64, True, 4), (640, 33, 32, 32, False, 3),
-                                                   (516, 129, 128, 0, False, 4), (576, 40, 64, 16, False, 3),
+                                                   (516, 129, 128, 0, False, 4), (576, 120, 64, 16, False, 4),
                                                    (648, 50, 128, 8, True, 4)])
 def test_tensor_path_block_sizes_and_tails(n, m, B, group, sym, bits):
     """Widths >= 512 (float32-grade tensor-core products) with the smaller lazy-batch blocks, a width that is
