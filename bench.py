@@ -204,10 +204,12 @@ def run_ours(args, cfg):
     pk = peaks()
 
     # inputs resident in HBM before the timed region (each rank its own layer: seed = rank)
-    shard = world > 1 and not args.replicas
+    shard = (world > 1 and not args.replicas) or args.shard_layer
     if shard:
         # ONE layer across the ranks: this rank's share of the token batches and of the rows of W
         from paper_2504_02692_b200 import sharded
+        if world > 1 and cfg.n_batches < world:
+            raise SystemExit(f"{cfg.n_batches} token batches cannot be shared by {world} ranks")
         cfg_r = cfg
         my_batches = sharded.token_shard(cfg.n_batches, rank, world)
         r0, r1 = sharded.row_shard(cfg.m, rank, world)
@@ -464,7 +466,9 @@ def main():
     ap.add_argument("--replicas", action="store_true",
                     help="N > 1: one independent layer per rank (weak scaling, no collective) instead of the default, "
                          "one layer across the ranks (token-sharded statistics, one all-reduce, row-sharded quantize)")
-    ap.add_argument("--shard-layer", action="store_true", help="(default for N > 1; kept for older command lines)")
+    ap.add_argument("--shard-layer", action="store_true",
+                    help="the default for N > 1; at N = 1 it forces the same code path with one rank holding every shard "
+                         "(the all-reduce is a no-op), as a check of that path on one GPU")
     ap.add_argument("--clip-search", type=int, default=0,
                     help="clipping-range search of the grids with this many candidates (off in the headline configuration)")
     ap.add_argument("--act-order", action="store_true", help="columns sorted by diag(H) (off in the headline configuration)")
