@@ -7,10 +7,10 @@
  * asymmetric calibration objective, Eq. "asym obj", Section 4).  The calls
  * map to the steps of Algorithm 1 of the paper:
  *
- *   gptaq_accumulate   line 2   H += X X^T,  dXX^T += (X~ - X) X^T
- *   gptaq_factor       line 3   L = Inverse_Cholesky(H + lambda_1 I), kept as U = L^T
- *   gptaq_build_P      line 4   P = ((dXX^T L) .* M_U) L^T          (Theorem 4.2)
- *   gptaq_quantize     l. 5-13  blocked column loop + lazy-batch trailing update
+ *   gptaq_accumulate   the statistics          H += X X^T,  dXX^T += (X~ - X) X^T
+ *   gptaq_factor       the inverse Cholesky    L = Inverse_Cholesky(H + lambda_1 I), kept as U = L^T
+ *   gptaq_build_P      the correction matrix   P = ((dXX^T L) .* M_U) L^T          (Theorem 4.2)
+ *   gptaq_quantize     the blocked loop        column loop + lazy-batch trailing update
  *
  * Conventions
  *  - Every pointer named d_* is DEVICE memory, every pointer named h_* is
@@ -61,7 +61,7 @@ typedef enum {
 
 enum { GPTAQ_W_FP32 = 0, GPTAQ_W_BF16 = 1 };
 
-/* Arithmetic of the statistics (Algorithm 1, line 2).  In the two tensor-core modes X and
+/* Arithmetic of the statistics (Algorithm 1, first step).  In the two tensor-core modes X and
  * X~ - X (the difference taken in float32 first) are rounded to fp16, scaled by a power of two
  * if the batch would leave the fp16 range, and multiplied by tcgen05 MMAs with float32
  * accumulation; they apply for n >= 256, smaller layers always take the float32 path.
@@ -98,7 +98,7 @@ size_t gptaq_workspace_bytes(int64_t n, int64_t m_max, int64_t max_batch_tokens,
 
 /* Creates a handle over caller-owned device buffers (both 256-byte aligned)
  * on the current CUDA device and enqueues the zeroing of H and dXX^T
- * (Algorithm 1, line 2 starts from empty sums). */
+ * (the statistics of Algorithm 1 start from empty sums). */
 gptaq_status_t gptaq_create(gptaq_handle_t *out, int64_t n, void *d_state, size_t state_bytes,
                             void *d_workspace, size_t workspace_bytes, gptaq_stream_t stream);
 
@@ -107,7 +107,7 @@ gptaq_status_t gptaq_reset(gptaq_handle_t h, gptaq_stream_t stream);
 
 gptaq_status_t gptaq_destroy(gptaq_handle_t h);
 
-/* Algorithm 1, line 2, one token batch:  H += X X^T,  dXX^T += (X~ - X) X^T.
+/* Algorithm 1, the statistics, one token batch:  H += X X^T,  dXX^T += (X~ - X) X^T.
  * d_X, d_Xfp: [tokens x n] float32, leading dimension ld >= n, read only.
  * The difference X~ - X is formed in float32 before any product.
  * tokens == 0 is a no-op.  Only the upper triangle of H is maintained. */
@@ -130,14 +130,14 @@ gptaq_status_t gptaq_accumulate_host(gptaq_handle_t h, const float *h_X, const f
                                      int64_t tokens, int64_t ld, void *d_stage, size_t stage_bytes,
                                      gptaq_stream_t stream);
 
-/* Algorithm 1, line 3, with the customary GPTQ preprocessing that Section 4 refers to:
+/* Algorithm 1, the inverse-Cholesky step, with the customary GPTQ preprocessing that Section 4 refers to:
  * H <- H / tokens; inputs with H_qq == 0 get H_qq = 1 (their weight columns
  * are zeroed by gptaq_quantize); H_d = H + damp * mean(diag H) * I; then the
  * upper factor U of H_d^-1 = U^T U (U = L^T of the paper) overwrites H
  * (strict lower triangle zeroed).  Needs at least one accumulated token. */
 gptaq_status_t gptaq_factor(gptaq_handle_t h, float damp, gptaq_stream_t stream);
 
-/* Algorithm 1, line 4 / Theorem 4.2:  P = alpha * ((dXX^T U^T) .* M_U) U with
+/* Algorithm 1, the step that forms P / Theorem 4.2:  P = alpha * ((dXX^T U^T) .* M_U) U with
  * dXX^T normalised by the token count like H, M_U the strictly-upper mask.
  * alpha = 1 is the paper's P; alpha = 0 reduces the solve to GPTQ.
  * P overwrites dXX^T (lower triangle and diagonal zero). */
@@ -151,7 +151,7 @@ gptaq_status_t gptaq_build_P(gptaq_handle_t h, float alpha, gptaq_stream_t strea
  * as gptaq_build_P; n <= 16384 (GPTAQ_ERR_UNSUPPORTED beyond). */
 gptaq_status_t gptaq_build_P_rowwise(gptaq_handle_t h, float alpha, gptaq_stream_t stream);
 
-/* Algorithm 1, lines 5-13, for one weight matrix sharing this state.
+/* Algorithm 1, the blocked loop, for one weight matrix sharing this state.
  *   d_W      [m x ldw], float32 or bf16 (w_dtype).  If d_Wq is given, d_W is read
  *            only and the float32 working copy lives in d_Wq (required for bf16
  *            weights).  If d_Wq is NULL (or equal to d_W), float32 weights are
@@ -190,7 +190,7 @@ gptaq_status_t gptaq_quantize_host(gptaq_handle_t h, const float *h_W, int64_t m
  * real-time loop, under a memory pool whose budget is already spent, in a plug-in that is not
  * allowed to call the CUDA allocator) and that therefore cannot size a workspace per layer.
  * It needs no handle and no workspace: the factor and the correction matrix are plain inputs,
- * and the m x 2B scratch of the lazy-batch update ([-Err | Wpre], Algorithm 1 line 5) lives in
+ * and the m x 2B scratch of the lazy-batch update ([-Err | Wpre]: the error matrix E of Algorithm 1 and the block's columns) lives in
  * an array built into the library.  The function allocates nothing, on the device or through
  * any library.
  *   d_U, d_P   [n x n] float32, leading dimension n: U (upper, H_d^-1 = U^T U) and P (strictly
@@ -229,8 +229,8 @@ gptaq_status_t gptaq_sync_status(gptaq_handle_t h, int64_t *info, gptaq_stream_t
  * callers that checkpoint the sums: H / U and dXX^T / P share storage. */
 float *gptaq_H(gptaq_handle_t h);
 float *gptaq_D(gptaq_handle_t h);
-/* The same storage under the names of what it holds later: U (Algorithm 1, line 3; NULL before
- * gptaq_factor) and P (line 4; NULL before gptaq_build_P). */
+/* The same storage under the names of what it holds later: U (the inverse-Cholesky factor of Algorithm 1; NULL
+ * before gptaq_factor) and P (Theorem 4.2; NULL before gptaq_build_P). */
 const float *gptaq_U(gptaq_handle_t h);
 const float *gptaq_P(gptaq_handle_t h);
 int64_t gptaq_tokens(gptaq_handle_t h);
@@ -285,7 +285,7 @@ gptaq_status_t gptaq_set_update_terms(gptaq_handle_t h, int terms);
 int64_t gptaq_launch_count(gptaq_handle_t h);
 
 /* Timing of the dominant kernel by itself (bookkeeping for benchmarks).  While enabled, every launch of the
- * tensor-core statistics kernel (Algorithm 1, line 2) is bracketed by a pair of CUDA events on the stream it
+ * tensor-core statistics kernel (the statistics of Algorithm 1) is bracketed by a pair of CUDA events on the stream it
  * runs on -- the handle's own stream, which events of the caller cannot reach.  gptaq_stats_kernel_time waits
  * (on the host) for the recorded launches, returns the sum of their durations in milliseconds and their number,
  * and starts a new record.  The conversion prologue and the fix-up of K-split tiles are not included. */

@@ -48,7 +48,7 @@ F64 = np.float64
 
 
 # --------------------------------------------------------------------------
-# Step 1 (Algorithm 1, line 2): H = X X^T, dXX^T = (X~ - X) X^T
+# Step 1 (Algorithm 1, the statistics step): H = X X^T, dXX^T = (X~ - X) X^T
 # --------------------------------------------------------------------------
 @dataclasses.dataclass
 class Stats:
@@ -76,7 +76,7 @@ def accumulate(st: Stats, X_tm: np.ndarray, Xfp_tm: np.ndarray) -> None:
 
 
 # --------------------------------------------------------------------------
-# Step 2 (Algorithm 1, line 3): L = Inverse_Cholesky(H + lambda_1 I)
+# Step 2 (Algorithm 1, the inverse-Cholesky step): L = Inverse_Cholesky(H + lambda_1 I)
 # --------------------------------------------------------------------------
 def damped_hessian(H_sum: np.ndarray, tokens: int, damp: float):
     """H/k with dead diagonal entries set to 1, plus damp * mean(diag) * I.
@@ -106,7 +106,7 @@ def factor(H_sum: np.ndarray, tokens: int, damp: float):
 
 
 # --------------------------------------------------------------------------
-# Step 3 (Algorithm 1, line 4; Theorem 4.2): P = ((dXX^T L) .* M_U) L^T
+# Step 3 (Algorithm 1, the step that forms P; Theorem 4.2): P = ((dXX^T L) .* M_U) L^T
 # --------------------------------------------------------------------------
 def build_P(D_sum: np.ndarray, tokens: int, U: np.ndarray, alpha: float) -> np.ndarray:
     D = np.asarray(D_sum, dtype=F64) / float(max(tokens, 1))
@@ -216,7 +216,7 @@ def _grid_fn(bits, sym, clip):
 
 
 # --------------------------------------------------------------------------
-# Steps 3-4 of Algorithm 1 (lines 6-13): the quantize-and-propagate loop
+# Steps 3-4 (Algorithm 1, the blocked loop): quantize and propagate
 # --------------------------------------------------------------------------
 @dataclasses.dataclass
 class QuantResult:

@@ -531,7 +531,7 @@ gptaq_status_t check_quantize_args(int64_t n, const void *d_W, int w_dtype, int6
         ++*launches;                                         \
     } while (0)
 
-// Algorithm 1, lines 5-13: launch sequence shared by the entry points that quantize.
+// Algorithm 1, the blocked loop: launch sequence shared by the entry points that quantize.
 gptaq_status_t quantize_core(const QuantizeTarget &t, void *d_W, int w_dtype, int64_t m, int64_t ldw,
                              int bits, int group, int sym, int blocksize, uint8_t *d_codes, float *d_scales,
                              float *d_zeros, float *d_Wq, cudaStream_t s, int64_t *launches, cudaError_t *err) {

@@ -1,7 +1,7 @@
 """One layer on several GPUs: token-sharded statistics, row-sharded quantization.
 
 The solve shards naturally with ONE exchange step.  Tokens are independent in the statistics
-(Algorithm 1, line 2: H and dXX^T are sums over tokens), so every rank accumulates its share of the
+(Algorithm 1, the statistics step: H and dXX^T are sums over tokens), so every rank accumulates its share of the
 token batches into its own state; one all-reduce (sum, float32, 2 n^2 elements) gives every rank the
 full sums.  The factor and P depend only on the sums and are recomputed on every rank (cheaper than
 broadcasting two n x n matrices and free of a second exchange).  Rows of W are independent in the

@@ -11,7 +11,7 @@ import paper_2504_02692_b200 as g
 import workloads as wl
 from oracle import gptaq_oracle as orc
 
-# Parity bounds of the benchmark spec.
+# Parity bounds of the CUDA path against the float64 oracle.
 TOL_OBJECTIVE = 1e-3      # relative difference of the layer objective
 TOL_FACTOR = 1e-4         # relative Frobenius error of U
 TOL_FLIP_BAND = 1e-4      # distance to a rounding boundary that excuses a flip

@@ -8,7 +8,7 @@ there the oracle checks sampled outputs it can compute one by one and properties
 any size, stage by stage:
   statistics   sampled entries H[i, j], dXX^T[i, j] against float64 sums over all tokens;
   factor       cfg3: the whole of U against the oracle's factor of the device's sums widened to
-               float64 (relative Frobenius error, the bound of the benchmark spec), stage-wise.
+               float64 (relative Frobenius error at most 1e-4), stage-wise.
                cfg5: a float64 factorisation of a 53,248-wide matrix (four 22.7 GB matrices, 6e14
                flops) is out of reach of a test; there U is checked to be upper with a positive
                diagonal and  u_i H_d u_j^T = delta_ij  for 77 sampled rows, the first row of every
