@@ -312,9 +312,9 @@ def run_ours(args, cfg):
         achieved = flops_launch / (kern_us * 1e-6) / 1e12
         kern_name = "stats_umma_kernel (tcgen05 kind::f16, cta_group::2), one token batch per launch"
     else:
-        # widths below 256 accumulate on the float32 FMA kernel: the stage is the unit
+        # small widths accumulate on the float32 FMA kernel: the stage is the unit
         kern_us, flops_launch, achieved = acc_call_ms * 1e3, flops_call, stage_achieved
-        kern_name = "gptaq_accumulate (one token batch; float32 FMA path below n = 256)"
+        kern_name = "gptaq_accumulate (one token batch; float32 FMA path of small widths)"
 
     # end to end through the host entry points: pinned host buffers in, host results out
     e2e = None

@@ -64,7 +64,7 @@ enum { GPTAQ_W_FP32 = 0, GPTAQ_W_BF16 = 1 };
 /* Arithmetic of the statistics (Algorithm 1, first step).  In the two tensor-core modes X and
  * X~ - X (the difference taken in float32 first) are rounded to fp16, scaled by a power of two
  * if the batch would leave the fp16 range, and multiplied by tcgen05 MMAs with float32
- * accumulation; they apply for n >= 256, smaller layers always take the float32 path.
+ * accumulation; they apply for n >= 256 and for n = 128, other small layers always take the float32 path.
  * GPTAQ_STATS_FP16_SPLIT_TENSOR (default): H additionally carries the rounding remainder of X
  *   as a second fp16 term (H = hi hi^T + hi lo^T + lo hi^T, about 22 significant bits), so that
  *   the factor U keeps its accuracy even with few tokens per input channel.

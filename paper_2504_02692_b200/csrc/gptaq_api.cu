@@ -373,7 +373,9 @@ int64_t tc_chunk_tokens(const gptaq_ctx *h) {
 }
 
 bool tc_eligible(const gptaq_ctx *h) {
-    return h->stats_precision != GPTAQ_STATS_FP32 && h->n >= UBN && tc_chunk_tokens(h) >= UBK &&
+    // from 256 input channels on, and for exactly 128 (one half-empty pair tile per sum; the TMA boxes of 128
+    // channels then cover the operand exactly)
+    return h->stats_precision != GPTAQ_STATS_FP32 && (h->n >= UBN || h->n == UBM) && tc_chunk_tokens(h) >= UBK &&
            encode_tiled_fn() != nullptr;
 }
 
@@ -628,7 +630,12 @@ gptaq_status_t quantize_core(const QuantizeTarget &t, void *d_W, int w_dtype, in
             // this block's columns of the super-block's [-Err | Wpre]
             a.EW = EW + (i0 - sb0); a.ew_ld = 2 * SBW; a.ew_pre = SBW;
         }
-        if (fast) column_block_kernel<<<cb_grid, CB_THREADS, column_block_smem(cb_rows), s>>>(a, cb_rows, blocksize);
+        if (fast) {
+            const int lanes = column_block_lanes(cb_rows);
+            if (lanes == 4) column_block_kernel<4><<<cb_grid, CB_THREADS, column_block_smem(cb_rows), s>>>(a, cb_rows, blocksize);
+            else if (lanes == 2) column_block_kernel<2><<<cb_grid, CB_THREADS, column_block_smem(cb_rows), s>>>(a, cb_rows, blocksize);
+            else column_block_kernel<1><<<cb_grid, CB_THREADS, column_block_smem(cb_rows), s>>>(a, cb_rows, blocksize);
+        }
         else if (T == 4) column_loop_kernel<4><<<cl_grid, nw * 32, cl_smem, s>>>(a);
         else if (T == 2) column_loop_kernel<2><<<cl_grid, nw * 32, cl_smem, s>>>(a);
         else column_loop_kernel<1><<<cl_grid, nw * 32, cl_smem, s>>>(a);
@@ -748,8 +755,11 @@ cudaError_t static_scratch_for_current_device(StaticScratch **out) {
         e = cudaFuncSetAttribute(column_loop_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                  2 * 64 * 64 * (int)sizeof(float));
         if (e != cudaSuccess) return e;
-        e = cudaFuncSetAttribute(column_block_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                 (int)column_block_smem(128));
+        e = cudaFuncSetAttribute(column_block_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)column_block_smem(128));
+        if (e != cudaSuccess) return e;
+        e = cudaFuncSetAttribute(column_block_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)column_block_smem(128));
+        if (e != cudaSuccess) return e;
+        e = cudaFuncSetAttribute(column_block_kernel<4>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)column_block_smem(128));
         if (e != cudaSuccess) return e;
         sc.base = static_cast<uint8_t *>(ptr);
         sc.ready = true;
@@ -835,8 +845,11 @@ gptaq_status_t gptaq_create(gptaq_handle_t *out, int64_t n, void *d_state, size_
         e = cudaFuncSetAttribute(column_loop_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                  2 * 64 * 64 * (int)sizeof(float));
     if (e == cudaSuccess)
-        e = cudaFuncSetAttribute(column_block_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                 (int)column_block_smem(128));
+        e = cudaFuncSetAttribute(column_block_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)column_block_smem(128));
+    if (e == cudaSuccess)
+        e = cudaFuncSetAttribute(column_block_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)column_block_smem(128));
+    if (e == cudaSuccess)
+        e = cudaFuncSetAttribute(column_block_kernel<4>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)column_block_smem(128));
     if (e == cudaSuccess)
         e = cudaFuncSetAttribute(unpermute_rows_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)ACT_ORDER_MAX_N * 4);
     if (e != cudaSuccess) {

@@ -830,9 +830,13 @@ __global__ void __launch_bounds__(1024) column_loop_kernel(ColumnLoopArgs a) {
 // output channel or per group of a multiple of 32 columns.  One CTA owns `rows` weight rows
 // (a multiple of 32); their block lives in shared memory.  The block is processed 32 columns
 // at a time:
-//   - one thread per row takes the 32 columns into registers and runs the sequential part
-//     (quantize column k, scaled error, rank-1 update of the later columns of the 32) with
-//     the rows k of U and P read from shared memory as broadcasts;
+//   - LANES threads per row (4 for 32 rows per CTA, 2 for 64, 1 beyond) take the 32 columns into
+//     registers, 32 / LANES consecutive columns each, and run the sequential part (quantize column
+//     k, scaled error, rank-1 update of the later columns of the 32): the lane that holds column k
+//     quantizes it and passes the scaled error and the pre-quantization value to the row's other
+//     lanes by shuffles, every lane updates its own later columns from the rows k of U and P in
+//     shared memory.  The dependent chain of a column is then the quantizer plus one update, not
+//     the up to 31 updates of one thread (154 cycles per column with one thread per row);
 //   - all threads then apply the 32 columns' errors and pre-quantization values to the rest
 //     of the block, a (rows x 64) x (64 x rest) product out of shared memory.
 // Same outputs as column_loop_kernel.
@@ -841,8 +845,11 @@ constexpr int CB_THREADS = 256;
 constexpr int CB_LD = 128 + 4;
 
 __host__ __device__ inline size_t column_block_smem(int rows) {
-    return ((size_t)rows * CB_LD + 2 * 2 * 32 * CB_LD + 64 * (rows + 4) + 2 * 32) * sizeof(float);
+    // the block, two buffers of 32 rows of U and P, [-Err | Wpre] of 32 columns transposed, two sets of 32
+    // reciprocal pivots, and per row: the chosen clipping candidate and the largest operand magnitude
+    return ((size_t)rows * CB_LD + 2 * 2 * 32 * CB_LD + 64 * (rows + 4) + 2 * 32 + 2 * rows) * sizeof(float);
 }
+__host__ __device__ inline int column_block_lanes(int rows) { return rows <= 32 ? 4 : (rows <= 64 ? 2 : 1); }
 
 // Round to nearest, ties to even, for a value that is clamped to [0, 255] afterwards: adding and
 // subtracting 1.5 * 2^23 rounds exactly like rintf wherever |v| < 2^22 and leaves larger values large
@@ -853,41 +860,62 @@ __device__ __forceinline__ float round_for_clamp(float v) {
     return __fsub_rn(__fadd_rn(v, magic), magic);
 }
 
-template <int K>
+// Step K of the sequential part for one row held by LANES lanes (lane `sub` of the row holds columns
+// sub * CPL .. + CPL - 1 of the 32 in x).  The arithmetic of every column is that of a single thread per
+// row: the results do not depend on LANES.
+template <int LANES, int K>
 struct QuantStep {
-    // x: the row's 32 columns (already-updated weights in, dequantized values out)
-    static __device__ __forceinline__ void run(float (&x)[32], float (&nerr)[32], float (&pre)[32], uint32_t (&code)[8],
-                                               const float *Us, const float *Ps, const float *udinv,
+    static constexpr int CPL = 32 / LANES;
+    static __device__ __forceinline__ void run(float (&x)[CPL], float (&nerr)[CPL], float (&pre)[CPL], uint32_t (&code)[CPL / 4],
+                                               int sub, const float *Us, const float *Ps, const float *udinv,
                                                float scale, float inv_scale, float zero, float maxq, float err_scale,
                                                float asym_scale) {
-        const float w0 = x[K];
+        constexpr int OWNER = K / CPL, KK = K % CPL;
+        // Straight-line code for all lanes (no divergent branches, so that the loads of U and P for the next
+        // steps can move ahead of this step's arithmetic): every lane quantizes its own column KK, the owner's
+        // result is the one that is kept and passed on.
+        const bool own = LANES == 1 || sub == OWNER;
+        const float w0 = x[KK];
         // w / scale as w * (1 / scale): one rounding more (about 1e-7 of a step, far inside the tie band)
         // for a much shorter dependent chain
         const float cq = fminf(fmaxf(round_for_clamp(w0 * inv_scale) + zero, 0.f), maxq);
         const float q = scale * (cq - zero);
-        const float ne = err_scale * ((q - w0) * udinv[K]);           // -(w - q) / U_kk
-        const float w = asym_scale * w0;
-        x[K] = q; nerr[K] = ne; pre[K] = w;
-        code[K >> 2] |= (uint32_t)cq << (8 * (K & 3));
-        const float *ur = Us + K * CB_LD, *pr = Ps + K * CB_LD;
+        float ne = err_scale * ((q - w0) * udinv[K]);           // -(w - q) / U_kk
+        float w = asym_scale * w0;
+        if (own) { x[KK] = q; nerr[KK] = ne; pre[KK] = w; code[KK >> 2] |= (uint32_t)cq << (8 * (KK & 3)); }
+        if (LANES > 1) {
+            ne = __shfl_sync(0xffffffffu, ne, OWNER, LANES);
+            w = __shfl_sync(0xffffffffu, w, OWNER, LANES);
+        }
+        // this lane's columns beyond K
+        const float *ur = Us + K * CB_LD + sub * CPL, *pr = Ps + K * CB_LD + sub * CPL;
 #pragma unroll
-        for (int j4 = (K + 1) / 4; j4 < 8; ++j4) {
+        for (int j4 = 0; j4 < CPL / 4; ++j4) {
+            // (compile-time skip of the quads that no lane needs any more)
+            if ((LANES - 1) * CPL + 4 * j4 + 3 <= K) continue;
             const float4 u = *reinterpret_cast<const float4 *>(ur + 4 * j4);
             const float4 p = *reinterpret_cast<const float4 *>(pr + 4 * j4);
-            if (4 * j4 + 0 > K) x[4 * j4 + 0] = fmaf(w, p.x, fmaf(ne, u.x, x[4 * j4 + 0]));
-            if (4 * j4 + 1 > K) x[4 * j4 + 1] = fmaf(w, p.y, fmaf(ne, u.y, x[4 * j4 + 1]));
-            if (4 * j4 + 2 > K) x[4 * j4 + 2] = fmaf(w, p.z, fmaf(ne, u.z, x[4 * j4 + 2]));
-            if (4 * j4 + 3 > K) x[4 * j4 + 3] = fmaf(w, p.w, fmaf(ne, u.w, x[4 * j4 + 3]));
+            const int c0 = sub * CPL + 4 * j4;
+            const float y0 = fmaf(w, p.x, fmaf(ne, u.x, x[4 * j4 + 0]));
+            const float y1 = fmaf(w, p.y, fmaf(ne, u.y, x[4 * j4 + 1]));
+            const float y2 = fmaf(w, p.z, fmaf(ne, u.z, x[4 * j4 + 2]));
+            const float y3 = fmaf(w, p.w, fmaf(ne, u.w, x[4 * j4 + 3]));
+            x[4 * j4 + 0] = c0 + 0 > K ? y0 : x[4 * j4 + 0];
+            x[4 * j4 + 1] = c0 + 1 > K ? y1 : x[4 * j4 + 1];
+            x[4 * j4 + 2] = c0 + 2 > K ? y2 : x[4 * j4 + 2];
+            x[4 * j4 + 3] = c0 + 3 > K ? y3 : x[4 * j4 + 3];
         }
-        QuantStep<K + 1>::run(x, nerr, pre, code, Us, Ps, udinv, scale, inv_scale, zero, maxq, err_scale, asym_scale);
+        QuantStep<LANES, K + 1>::run(x, nerr, pre, code, sub, Us, Ps, udinv, scale, inv_scale, zero, maxq, err_scale, asym_scale);
     }
 };
-template <>
-struct QuantStep<32> {
-    static __device__ __forceinline__ void run(float (&)[32], float (&)[32], float (&)[32], uint32_t (&)[8],
+template <int LANES>
+struct QuantStep<LANES, 32> {
+    static constexpr int CPL = 32 / LANES;
+    static __device__ __forceinline__ void run(float (&)[CPL], float (&)[CPL], float (&)[CPL], uint32_t (&)[CPL / 4], int,
                                                const float *, const float *, const float *, float, float, float, float, float, float) {}
 };
 
+template <int LANES>
 __global__ void __launch_bounds__(CB_THREADS, 1) column_block_kernel(ColumnLoopArgs a, int rows, int B) {
     extern __shared__ __align__(16) float smem_f[];
     float (*Wt)[CB_LD] = reinterpret_cast<float (*)[CB_LD]>(smem_f);                       // [rows][B]
@@ -897,11 +925,18 @@ __global__ void __launch_bounds__(CB_THREADS, 1) column_block_kernel(ColumnLoopA
     float *St = smem_f + rows * CB_LD + 2 * 2 * 32 * CB_LD;                                // [64][rows + 4]: -Err, then Wpre
     const int sld = rows + 4;
     float *udinv2 = St + 64 * sld;                                                         // [2][32]
+    int *bsel = reinterpret_cast<int *>(udinv2 + 2 * 32);                                  // [rows]: chosen clipping candidate
+    float *rmax_s = reinterpret_cast<float *>(bsel + rows);                                // [rows]: largest |operand| of the row
     const int tid = threadIdx.x;
     const int n = a.n, i0 = a.i0;
     const int row0 = blockIdx.x * rows;
     const int nrows = min(rows, a.m - row0);
     const int bq = B / 4;
+    // sequential part: thread tid < rows * LANES holds columns sub * CPL .. of row lrow (whole warps take part,
+    // rows beyond the matrix run on zeros and store nothing)
+    constexpr int CPL = 32 / LANES;
+    const int lrow = tid / LANES, sub = tid % LANES;
+    const bool chain = tid < rows * LANES;
 
     // the block of W (dead inputs read as zero), along rows; four loads in flight per thread
     for (int base = 0; base < rows * bq; base += 4 * CB_THREADS) {
@@ -937,8 +972,8 @@ __global__ void __launch_bounds__(CB_THREADS, 1) column_block_kernel(ColumnLoopA
 
     const float maxq = (float)((1 << a.bits) - 1);
     float scale = 1.f, zero = 0.f;
-    const bool owner = tid < nrows;
-    const int row = row0 + tid;
+    const bool owner = chain && lrow < nrows;
+    const int row = row0 + lrow;
     if (a.group <= 0 && owner) { scale = a.scales[row]; zero = a.zeros[row]; }
     const bool f16 = a.EW16_hi != nullptr;
     float rho = 1.f, rmax = 0.f;
@@ -1006,59 +1041,80 @@ __global__ void __launch_bounds__(CB_THREADS, 1) column_block_kernel(ColumnLoopA
                 bk[cgi * rows + r] = kb;
             }
             __syncthreads();
-            if (owner) {
+            if (tid < rows) {
                 float best = INFINITY;
+                int kbest = 0;
                 for (int c = 0; c < ncg; ++c) {
                     const float e = berr[c * rows + tid];
                     const int k = bk[c * rows + tid];
-                    if (e < best || (e == best && k < best_k)) { best = e; best_k = k; }
+                    if (e < best || (e == best && k < kbest)) { best = e; kbest = k; }
                 }
+                bsel[tid] = kbest;
             }
             __syncthreads();
+            if (chain) best_k = bsel[lrow];
         }
         if (tid >= CB_THREADS / 2 && o + 32 < B) fetch_up(o + 32, buf ^ 1, CB_THREADS / 2, CB_THREADS / 2);
-        if (owner) {
+        if (chain) {
             if (group_start) {
-                // grid of the group that starts here, from the current values
+                // grid of the group that starts here, from the current values (the row's lanes share the scan)
                 float lo = 0.f, hi = 0.f, am = 0.f;
                 const int gend = min(o + a.group, B);
-                for (int c = o; c < gend; ++c) {
-                    const float v = Wt[tid][c];
+                for (int c = o + sub; c < gend; c += LANES) {
+                    const float v = Wt[lrow][c];
                     lo = fminf(lo, v); hi = fmaxf(hi, v); am = fmaxf(am, fabsf(v));
+                }
+#pragma unroll
+                for (int d = 1; d < LANES; d <<= 1) {
+                    lo = fminf(lo, __shfl_xor_sync(0xffffffffu, lo, d));
+                    hi = fmaxf(hi, __shfl_xor_sync(0xffffffffu, hi, d));
+                    am = fmaxf(am, __shfl_xor_sync(0xffffffffu, am, d));
                 }
                 const float p = a.clip_steps > 0 ? clip_ratio(best_k, a.clip_steps, a.clip_min) : 1.f;
                 make_grid(p * lo, p * hi, p * am, a.bits, a.sym, scale, zero);
-                const int g = (i0 + o) / a.group;
-                a.scales[(int64_t)row * a.G + g] = scale;
-                a.zeros[(int64_t)row * a.G + g] = zero;
+                if (owner && sub == 0) {
+                    const int g = (i0 + o) / a.group;
+                    a.scales[(int64_t)row * a.G + g] = scale;
+                    a.zeros[(int64_t)row * a.G + g] = zero;
+                }
             }
-            float x[32], nerr[32], pre[32];
-            uint32_t code[8];
+            float x[CPL], nerr[CPL], pre[CPL];
+            uint32_t code[CPL / 4];
+            const int c_lane = o + sub * CPL;                 // this lane's first column in the block
 #pragma unroll
-            for (int k4 = 0; k4 < 8; ++k4) {
-                const float4 v = *reinterpret_cast<const float4 *>(&Wt[tid][o + 4 * k4]);
+            for (int k4 = 0; k4 < CPL / 4; ++k4) {
+                const float4 v = *reinterpret_cast<const float4 *>(&Wt[lrow][c_lane + 4 * k4]);
                 x[4 * k4] = v.x; x[4 * k4 + 1] = v.y; x[4 * k4 + 2] = v.z; x[4 * k4 + 3] = v.w;
                 code[k4] = 0u;
             }
-            QuantStep<0>::run(x, nerr, pre, code, &Us[0][o], &Ps[0][o], udinv, scale, 1.f / scale, zero, maxq, a.err_scale, a.asym_scale);
-            uint8_t *crow = a.codes + (int64_t)row * n + i0 + o;
-            if (a.perm) {
-                uint8_t *cbase = a.codes + (int64_t)row * n;
-                const int *pp = a.perm + i0 + o;
+            QuantStep<LANES, 0>::run(x, nerr, pre, code, sub, &Us[0][o], &Ps[0][o], udinv, scale, 1.f / scale, zero, maxq,
+                                     a.err_scale, a.asym_scale);
+            if (owner) {
+                uint8_t *crow = a.codes + (int64_t)row * n + i0 + c_lane;
+                if (a.perm) {
+                    uint8_t *cbase = a.codes + (int64_t)row * n;
+                    const int *pp = a.perm + i0 + c_lane;
 #pragma unroll
-                for (int k = 0; k < 32; ++k) cbase[pp[k]] = (uint8_t)(code[k >> 2] >> (8 * (k & 3)));
-            } else if ((reinterpret_cast<uintptr_t>(crow) & 15) == 0) {
-                *reinterpret_cast<uint4 *>(crow) = make_uint4(code[0], code[1], code[2], code[3]);
-                *reinterpret_cast<uint4 *>(crow + 16) = make_uint4(code[4], code[5], code[6], code[7]);
-            } else {
+                    for (int k = 0; k < CPL; ++k) cbase[pp[k]] = (uint8_t)(code[k >> 2] >> (8 * (k & 3)));
+                } else if ((reinterpret_cast<uintptr_t>(crow) & (CPL >= 16 ? 15 : 7)) == 0) {
+                    if constexpr (CPL == 32) {
+                        *reinterpret_cast<uint4 *>(crow) = make_uint4(code[0], code[1], code[2], code[3]);
+                        *reinterpret_cast<uint4 *>(crow + 16) = make_uint4(code[4], code[5], code[6], code[7]);
+                    } else if constexpr (CPL == 16) {
+                        *reinterpret_cast<uint4 *>(crow) = make_uint4(code[0], code[1], code[2], code[3]);
+                    } else {
+                        *reinterpret_cast<uint2 *>(crow) = make_uint2(code[0], code[1]);
+                    }
+                } else {
 #pragma unroll
-                for (int k = 0; k < 32; ++k) crow[k] = (uint8_t)(code[k >> 2] >> (8 * (k & 3)));
+                    for (int k = 0; k < CPL; ++k) crow[k] = (uint8_t)(code[k >> 2] >> (8 * (k & 3)));
+                }
             }
-            float *ew = a.EW + (int64_t)row * a.ew_ld + o;
-            float *ewl = a.EW_lo ? a.EW_lo + (int64_t)row * a.ew_ld + o : nullptr;
+            float *ew = a.EW + (int64_t)row * a.ew_ld + c_lane;
+            float *ewl = a.EW_lo ? a.EW_lo + (int64_t)row * a.ew_ld + c_lane : nullptr;
 #pragma unroll
-            for (int k4 = 0; k4 < 8; ++k4) {
-                *reinterpret_cast<float4 *>(&Wt[tid][o + 4 * k4]) = make_float4(x[4 * k4], x[4 * k4 + 1], x[4 * k4 + 2], x[4 * k4 + 3]);
+            for (int k4 = 0; k4 < CPL / 4; ++k4) {
+                *reinterpret_cast<float4 *>(&Wt[lrow][c_lane + 4 * k4]) = make_float4(x[4 * k4], x[4 * k4 + 1], x[4 * k4 + 2], x[4 * k4 + 3]);
                 float e4[4] = {nerr[4 * k4], nerr[4 * k4 + 1], nerr[4 * k4 + 2], nerr[4 * k4 + 3]};
                 float p4[4] = {pre[4 * k4], pre[4 * k4 + 1], pre[4 * k4 + 2], pre[4 * k4 + 3]};
                 if (f16) {
@@ -1068,6 +1124,7 @@ __global__ void __launch_bounds__(CB_THREADS, 1) column_block_kernel(ColumnLoopA
                         rmax = fmaxf(rmax, fmaxf(fabsf(e4[f]), fabsf(p4[f])));
                     }
                 }
+                if (!owner) continue;
                 if (ewl) {
                     float el[4], pl[4];
 #pragma unroll
@@ -1083,10 +1140,10 @@ __global__ void __launch_bounds__(CB_THREADS, 1) column_block_kernel(ColumnLoopA
                 *reinterpret_cast<float4 *>(ew + a.ew_pre + 4 * k4) = make_float4(p4[0], p4[1], p4[2], p4[3]);
             }
 #pragma unroll
-            for (int k = 0; k < 32; ++k) { St[k * sld + tid] = nerr[k]; St[(32 + k) * sld + tid] = pre[k]; }
-        } else if (tid < rows) {
-#pragma unroll
-            for (int k = 0; k < 64; ++k) St[k * sld + tid] = 0.f;
+            for (int k = 0; k < CPL; ++k) {
+                St[(sub * CPL + k) * sld + lrow] = nerr[k];
+                St[(32 + sub * CPL + k) * sld + lrow] = pre[k];
+            }
         }
         __syncthreads();
         // rest of the block: Wt[:, c] += sum_k (-Err)[:, k] U[o + k][c] + Wpre[:, k] P[o + k][c], c >= o + 32
@@ -1121,6 +1178,12 @@ __global__ void __launch_bounds__(CB_THREADS, 1) column_block_kernel(ColumnLoopA
             }
         }
     }
+    if (f16 && chain) {
+        // the row's largest operand magnitude, over its lanes
+#pragma unroll
+        for (int d = 1; d < LANES; d <<= 1) rmax = fmaxf(rmax, __shfl_xor_sync(0xffffffffu, rmax, d));
+        if (sub == 0) rmax_s[lrow] = rmax;
+    }
     __syncthreads();
     // dequantized block back to W
     for (int idx = tid; idx < nrows * bq; idx += CB_THREADS) {
@@ -1136,9 +1199,10 @@ __global__ void __launch_bounds__(CB_THREADS, 1) column_block_kernel(ColumnLoopA
         // this CTA's rows of [-Err | rho * Wpre], scaled row by row into the fp16 range and split
         float *srow = St;                       // free since the last rank update
         if (tid < rows) {
-            const float sc = owner ? split_scale(rmax) : 1.f;
+            const bool live = tid < nrows;
+            const float sc = live ? split_scale(rmax_s[tid]) : 1.f;
             srow[tid] = sc;
-            if (owner) a.row_inv[row] = 1.f / sc;
+            if (live) a.row_inv[row0 + tid] = 1.f / sc;
         }
         __syncthreads();                        // (also: the rows written above are visible to the whole CTA)
         const int q = 2 * B / 4;

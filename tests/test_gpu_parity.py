@@ -25,7 +25,8 @@ def test_cfg1_full_parity():
     cfg = wl.CONFIGS["cfg1"]
     out = hp.check_layer(cfg, wl.make_weight(cfg), batches_of(cfg))
     hp.assert_parity(out)
-    assert out["H_rel"] < 1e-5 and out["D_rel"] < 1e-5 and out["P_rel"] < 1e-4
+    # tensor-core statistics (split H, single-term fp16 dXX^T): the sums carry the operand rounding, 2^-11 per factor
+    assert out["H_rel"] < 1e-5 and out["D_rel"] < 2.0 ** -10 and out["P_rel"] < 5e-3
 
 
 @pytest.mark.parametrize("alpha", [0.0, 1.0])
