@@ -405,9 +405,10 @@ def follow(W: np.ndarray, U: np.ndarray, P: np.ndarray | None, dead,
            bits: int, group: int, sym: bool,
            cand_codes: np.ndarray, cand_scales: np.ndarray, cand_zeros: np.ndarray,
            band: float = 1e-4, error_term: bool = True, clip=None, static=None) -> FollowReport:
-    """``static = (W_original, group_of_column)``: static groups -- the candidate's grids are judged once,
-    against the grids of the original weights in their original column order (``W`` is then the working copy
-    in processing order), and column j uses the candidate's grid number ``group_of_column[j]``."""
+    """``static = (W_original, group_of_column[, dead_original])``: static groups -- the candidate's grids are
+    judged once, against the grids of the original weights in their original column order with dead inputs
+    counting as zero weights (``W`` is then the working copy in processing order), and column j uses the
+    candidate's grid number ``group_of_column[j]``."""
     W = np.array(W, dtype=F64)
     m, n = W.shape
     if dead is not None and dead.any():
@@ -425,15 +426,29 @@ def follow(W: np.ndarray, U: np.ndarray, P: np.ndarray | None, dead,
         if clip is not None and clip[0] > 0:
             # clipping-range search: the candidate's grid must be one of the candidate grids, and its
             # squared error (in float64) must equal the best one up to rounding: near-ties may fall
-            # either way in float32
+            # either way in float32.  A candidate whose zero point sits on a rounding tie before it is
+            # rounded (-lo / scale within 10 * band of x.5: exact for weights with short mantissas and
+            # symmetric extremes) exists in two versions, zero point rounded down or up; the searcher may
+            # have met either one, so the bar is the best candidate in its worse version.
             S, Z, E = clip_candidates(block, bits, sym, clip[0], clip[1])
+            Zalt, Ealt = Z, E
+            if not sym:
+                pk = 1.0 - np.arange(clip[0]) * (1.0 - clip[1]) / clip[0]
+                t = -pk[:, None] * np.minimum(block.min(axis=1), 0.0)[None, :] / S
+                tie = np.abs(t - np.floor(t) - 0.5) <= 10 * band
+                Zalt = np.where(tie, 2.0 * np.floor(t) + 1.0 - Z, Z)
+                Ealt = E.copy()
+                for kk, rr in zip(*np.nonzero(tie)):
+                    q = dequant(qcode(block[rr], S[kk, rr], Zalt[kk, rr], bits), S[kk, rr], Zalt[kk, rr])
+                    Ealt[kk, rr] = np.sum((q - block[rr]) ** 2)
             rel = np.abs(S - s_c[None, :]) / S
             k = np.argmin(rel, axis=0)
             r = np.arange(S.shape[1])
             grid_err = max(grid_err, float(np.max(rel[k, r])))
-            best = E.min(axis=0)
-            worse = E[k, r] > best * (1.0 + 1e-5) + 1e-30
-            zero_mis += int(np.sum(worse)) + int(np.sum(Z[k, r] != z_c))
+            bar = np.maximum(E, Ealt).min(axis=0)
+            mine = np.where(z_c == Z[k, r], E[k, r], np.where(z_c == Zalt[k, r], Ealt[k, r], np.inf))
+            worse = mine > bar * (1.0 + 1e-5) + 1e-30
+            zero_mis += int(np.sum(worse))
             return s_c, z_c
         s_o, z_o = grid(block, bits, sym)
         grid_err = max(grid_err, float(np.max(np.abs(s_c - s_o) / s_o)))
@@ -447,6 +462,8 @@ def follow(W: np.ndarray, U: np.ndarray, P: np.ndarray | None, dead,
     if static is not None:
         W0 = np.array(static[0], dtype=F64)
         gidx = np.asarray(static[1])
+        if len(static) > 2 and static[2] is not None and np.any(static[2]):
+            W0[:, np.asarray(static[2], bool)] = 0.0
         for g in range(cand_scales.shape[1]):
             check_grid(W0[:, g * group:(g + 1) * group], g)
     elif group <= 0:

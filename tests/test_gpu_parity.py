@@ -335,15 +335,22 @@ def test_act_order(n, m, group, B, bf16):
     st.close()
 
 
-@pytest.mark.parametrize("n,m,group,B,act,bf16", [(192, 24, 32, 64, True, False), (640, 40, 128, 128, True, False),
-                                                  (768, 33, 64, 128, True, True), (640, 20, 128, 128, False, False)])
-def test_static_groups(n, m, group, B, act, bf16):
+@pytest.mark.parametrize("n,m,group,B,act,bf16,ndead", [(192, 24, 32, 64, True, False, 0), (640, 40, 128, 128, True, False, 0),
+                                                        (768, 33, 64, 128, True, True, 0), (640, 20, 128, 128, False, False, 0),
+                                                        (320, 30, 64, 64, True, False, 3), (512, 33, 64, 64, False, True, 3)])
+def test_static_groups(n, m, group, B, act, bf16, ndead):
     """Static groups, with and without act_order: grids per group of the caller's columns from the original
-    weights; the loop replayed by the oracle in the device's processing order with those grids."""
+    weights (inputs that never fired count as zero weights); the loop replayed by the oracle in the device's
+    processing order with those grids."""
     cfg = wl.scaled(wl.CONFIGS["cfg2"], name="static_groups", n=n, m=m, batch_tokens=2048, n_batches=2, group=group,
                     blocksize=B, outlier_channels=4, w_bf16=bf16)
     bt = batches_of(cfg)
     W = wl.make_weight(cfg)
+    if ndead:
+        for X, Xfp in bt:
+            X[:, 7:7 + ndead] = 0.0
+            Xfp[:, 7:7 + ndead] = 0.0
+        W[:, 7] = 30.0 * W.abs().max()          # a dead input's weight must not stretch its group's grid
     st = g.LayerState(cfg.n, cfg.m, cfg.batch_tokens, cfg.blocksize, total_tokens=cfg.tokens)
     g.gptaq_set_act_order(st.handle, act)
     g.gptaq_set_static_groups(st.handle, True)
@@ -367,8 +374,11 @@ def test_static_groups(n, m, group, B, act, bf16):
     cg, scn, zpn = codes.cpu().numpy(), sc.cpu().numpy(), zp.cpu().numpy()
     # the grids are those of the original weights, float32 arithmetic on both sides of a min/max
     assert np.abs(scn - res.scales).max() <= 1e-6 * np.abs(res.scales).max() and np.array_equal(zpn, res.zeros)
+    dead0 = np.zeros(n, bool)
+    dead0[perm] = dead
+    assert dead0.sum() == ndead
     rep = orc.follow(Wn[:, perm], U, P, dead, cfg.bits, group, cfg.sym, cg[:, perm], scn.astype(np.float64),
-                     zpn.astype(np.float64), band=hp.TOL_FLIP_BAND, static=(Wn, perm // group))
+                     zpn.astype(np.float64), band=hp.TOL_FLIP_BAND, static=(Wn, perm // group, dead0))
     assert rep.disallowed == 0 and rep.allowed <= hp.TOL_FLIP_RATE * rep.total, rep
     assert rep.grid_rel_err <= 1e-6 and rep.zero_mismatch == 0, rep
     # the outputs dequantize with the grid of group column // group, in the caller's column order

@@ -480,6 +480,56 @@ def test_static_groups_index_original_columns_and_survive_relabelling():
     rep = orc.follow(W[:, perm], Us, Ps, deads, bits, group, False, res.codes[:, perm], dyn.scales, dyn.zeros,
                      static=(W, perm // group))
     assert rep.grid_rel_err > 1e-3
+    # dead inputs count as zero weights in the static grids, in solve_act_order and in follow alike
+    Xd, Xfd = X.copy(), Xfp.copy()
+    Xd[:, [3, 17]] = 0.0
+    Xfd[:, [3, 17]] = 0.0
+    Wd = W.copy()
+    Wd[:, 3] = 40.0 * np.abs(W).max()          # would stretch its group's grid if it counted
+    st_d = stats_of(Xd, Xfd)
+    Ud, Pd, dead_s, res_d, perm_d = orc.solve_act_order(Wd, st_d.H, st_d.D, st_d.tokens, 0.01, 0.25, bits, group, False,
+                                                        static_groups=True)
+    dead0 = np.zeros(n, bool)
+    dead0[perm_d] = dead_s
+    assert dead0[[3, 17]].all() and dead0.sum() == 2
+    Wz = Wd.copy()
+    Wz[:, dead0] = 0.0
+    sz, zz = orc.grid(Wz[:, 0:group], bits, False)
+    assert np.array_equal(res_d.scales[:, 0], sz) and np.array_equal(res_d.zeros[:, 0], zz)
+    rep = orc.follow(Wd[:, perm_d], Ud, Pd, dead_s, bits, group, False, res_d.codes[:, perm_d], res_d.scales, res_d.zeros,
+                     static=(Wd, perm_d // group, dead0))
+    assert rep.mismatches == 0 and rep.grid_rel_err == 0.0 and rep.zero_mismatch == 0
+    rep = orc.follow(Wd[:, perm_d], Ud, Pd, dead_s, bits, group, False, res_d.codes[:, perm_d], res_d.scales, res_d.zeros,
+                     static=(Wd, perm_d // group))
+    assert rep.grid_rel_err > 1e-2             # without the flags the stretched grid is expected, and refused
+
+
+def test_clip_search_follow_accepts_either_rounding_of_a_tied_zero_point():
+    """Weights with short mantissas and symmetric extremes put -lo / scale exactly on x.5 for every candidate of
+    the clipping-range search; whether float arithmetic lands on 7.4999 or 7.5 is then an accident of rounding.
+    follow accepts a searcher that met the other rounding (and chose accordingly), and still refuses a grid that
+    is worse than every version of the best candidate."""
+    bits, steps, ratio = 4, 6, 0.3
+    r = np.random.default_rng(5)
+    w = np.round(r.standard_normal((4, 16)) * 8.0) / 64.0          # multiples of 1/64
+    w[:, 0], w[:, 1] = -0.75, 0.75                                   # lo = -hi: -lo / scale = 7.5 for every candidate
+    w[:, 2:] = np.clip(w[:, 2:], -0.74, 0.74)
+    S, Z, E = orc.clip_candidates(w, bits, False, steps, ratio)
+    k = np.argmin(E, axis=0)
+    rr = np.arange(4)
+    U = np.eye(16)
+    codes = orc.qcode(w, S[k, rr][:, None], Z[k, rr][:, None], bits).astype(np.uint8)
+    ok = orc.follow(w, U, None, None, bits, 0, False, codes, S[k, rr], Z[k, rr], clip=(steps, ratio))
+    assert ok.zero_mismatch == 0 and ok.mismatches == 0
+    # the same scale with the zero point rounded the other way is a legitimate candidate too
+    Zo = 15.0 - Z[k, rr]                                             # 7 <-> 8
+    codes_o = orc.qcode(w, S[k, rr][:, None], Zo[:, None], bits).astype(np.uint8)
+    other = orc.follow(w, U, None, None, bits, 0, False, codes_o, S[k, rr], Zo, clip=(steps, ratio))
+    assert other.zero_mismatch == 0 and other.disallowed == 0     # (on this fixture both versions beat every other candidate)
+    # a zero point two steps off is no version of any candidate
+    Zbad = Z[k, rr] + 2.0
+    codes_b = orc.qcode(w, S[k, rr][:, None], Zbad[:, None], bits).astype(np.uint8)
+    assert orc.follow(w, U, None, None, bits, 0, False, codes_b, S[k, rr], Zbad, clip=(steps, ratio)).zero_mismatch == 4
 
 
 # ---------------------------------------------------------------- follow mode
