@@ -460,7 +460,9 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="cfg2", choices=sorted(wl.CONFIGS))
     ap.add_argument("--ref-tokens", type=int, default=8192)
-    ap.add_argument("--ref-rows", type=int, default=512)
+    ap.add_argument("--ref-rows", type=int, default=None,
+                    help="rows of W in the oracle's timed sample (default: 512 for the cpu_baseline leg of a GPU run, 128 per "
+                         "step of --impl reference, so that 25 steps stay near two minutes)")
     ap.add_argument("--batches", type=int, default=0,
                     help="profiler captures only: keep this many token batches (the line is marked truncated)")
     ap.add_argument("--replicas", action="store_true",
@@ -485,6 +487,8 @@ def main():
     if args.batches > 0:
         cfg = wl.scaled(cfg, n_batches=min(args.batches, cfg.n_batches))
     args.full_tokens = full_tokens
+    if args.ref_rows is None:
+        args.ref_rows = 128 if args.impl == "reference" else 512
     if args.impl == "reference":
         run_reference(args, cfg)
     elif args.p_rowwise:
