@@ -63,6 +63,10 @@ struct gptaq_ctx {
     bool gemm_pending[2];
     bool relayout;         // the operand buffers change size: wait for the products in flight first
     int next_buf;
+    // partial sums of the cut tiles of the statistics products wait in the workspace (fix_args.scratch) until
+    // the sums are needed or the cut changes; fix_pending: they have not been added to H / dXX^T yet
+    bool fix_pending;
+    StatsGemmArgs fix_args;
     // optional timing of the statistics kernel alone: one event pair per launch, on the stream it runs on
     bool kernel_timing;
     std::vector<std::pair<cudaEvent_t, cudaEvent_t>> timing_events;   // pool; the first timing_used are recorded
@@ -379,8 +383,21 @@ bool tc_eligible(const gptaq_ctx *h) {
            encode_tiled_fn() != nullptr;
 }
 
+// Adds the waiting partial sums of the cut tiles to H / dXX^T, on the internal stream behind the products.
+gptaq_status_t flush_partials(gptaq_ctx *h) {
+    if (!h->fix_pending) return GPTAQ_OK;
+    const StatsGemmArgs &ga = h->fix_args;
+    stats_fixup_kernel<<<dim3((unsigned)(ga.ntiles - ga.full_tiles), FIXUP_SLABS), 256, 0, h->gemm_stream>>>(ga);
+    LAUNCHED();
+    h->fix_pending = false;
+    CU(cudaEventRecord(h->gemm_done[0], h->gemm_stream));
+    h->gemm_pending[0] = true;
+    return GPTAQ_OK;
+}
+
 // Orders `s` after every statistics product still running on the internal stream.
 gptaq_status_t join_statistics(gptaq_ctx *h, cudaStream_t s) {
+    OK(flush_partials(h));
     for (int i = 0; i < 2; ++i)
         if (h->gemm_pending[i]) {
             CU(cudaStreamWaitEvent(s, h->gemm_done[i], 0));
@@ -465,13 +482,17 @@ gptaq_status_t accumulate_tc(gptaq_ctx *h, const float *X, const float *Xfp, int
             tev = &h->timing_events[h->timing_used++];
             CU(cudaEventRecord(tev->first, gs));
         }
+        if (h->fix_pending && (h->fix_args.ksplit != ga.ksplit || h->fix_args.full_tiles != ga.full_tiles ||
+                               h->fix_args.scratch != ga.scratch))
+            OK(flush_partials(h));              // another cut: the slots change meaning
+        if (ga.ksplit > 1 && !h->fix_pending) {
+            CU(cudaMemsetAsync(ga.scratch, 0, (size_t)((int)ntiles - ga.full_tiles) * (ga.ksplit - 1) * 2 * UBM * UBN * sizeof(float), gs));
+            h->fix_args = ga;
+            h->fix_pending = true;
+        }
         stats_umma_kernel<<<sgrid, UMMA_THREADS, UMMA_SMEM, gs>>>(mX, mD, mL, mDL, ga);
         LAUNCHED();
         if (tev) CU(cudaEventRecord(tev->second, gs));
-        if (ga.ksplit > 1) {
-            stats_fixup_kernel<<<dim3((unsigned)((int)ntiles - ga.full_tiles), FIXUP_SLABS), 256, 0, gs>>>(ga);
-            LAUNCHED();
-        }
         CU(cudaEventRecord(h->gemm_done[buf], gs));
         h->gemm_pending[buf] = true;
     }
@@ -859,6 +880,7 @@ gptaq_status_t gptaq_create(gptaq_handle_t *out, int64_t n, void *d_state, size_
     h->gemm_stream = nullptr;
     h->relayout = false;
     h->next_buf = 0;
+    h->fix_pending = false;
     for (int i = 0; i < 2; ++i) { h->conv_done[i] = h->gemm_done[i] = nullptr; h->gemm_pending[i] = false; }
     e = cudaStreamCreateWithFlags(&h->gemm_stream, cudaStreamNonBlocking);
     for (int i = 0; i < 2 && e == cudaSuccess; ++i) {

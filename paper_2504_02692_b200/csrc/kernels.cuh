@@ -120,21 +120,22 @@ __global__ void __launch_bounds__(256) scale_damp_kernel(float *H, int n, const 
 // [b0, b0 + NB):
 //   1. factor the NB x NB diagonal block from its last row/column upwards in shared memory,
 //      32 columns at a time: one warp factors the 32 x 32 diagonal sub-block in registers
-//      (lane = row, shuffles), the rows above it are solved against the sub-block one thread
-//      per row, and the leading part receives the rank-32 update;
-//   2. rows above the block:  R[0:b0, blk] = A[0:b0, blk] * R_pp^-T  by back substitution,
-//      one thread per row with the row in registers (R_pp is read from shared memory as
-//      broadcasts); written back in place and, if asked for, as TF32 hi/lo parts for the
-//      tensor-core rank-NB update.
+//      (lane = row, shuffles), the rows above it are solved against the sub-block one thread per
+//      row, and the leading part receives the rank-32 update (all threads, the tiles of the upper
+//      triangle numbered densely);
+//   2. rows above the block:  R[0:b0, blk] = A[0:b0, blk] * R_pp^-T, 32 columns at a time: a product
+//      with the inverse of the 32 x 32 diagonal sub-block (the four inverses: one warp each, lane =
+//      column), then a rank-32 update of the columns to the left, all threads on both; written back in place and, if asked for, as split parts for the tensor-core rank update.
 // Every CTA repeats step 1 (it is short and the other SMs would idle) and then takes a
-// slab of rows of step 2; CTA 0 stores R_pp for invert_diag_blocks_kernel.
-// Rows/columns beyond n are padded with the identity.
+// slab of rows of step 2, whose first tile is fetched while step 1 runs; CTA 0 stores R_pp for
+// invert_diag_blocks_kernel.  Rows/columns beyond n are padded with the identity.
 // ---------------------------------------------------------------------------
 constexpr int NB = 128;
 constexpr int FP_THREADS = 512;
 constexpr int FP_WARPS = FP_THREADS / 32;
 constexpr int FP_LD = NB + 4;
-constexpr size_t FP_SMEM = (2 * NB * FP_LD + 32 * FP_LD + NB + 64) * sizeof(float);
+constexpr int FP_YLD = 36;
+constexpr size_t FP_SMEM = (2 * NB * FP_LD + 32 * FP_LD + 4 * 32 * FP_YLD + NB + 64) * sizeof(float);
 
 struct FactorPanelArgs {
     float *H; int n; int b0;
@@ -215,54 +216,47 @@ struct Chol32Step<-1> {
     static __device__ __forceinline__ void run(float (&)[32], float, int, float *, float *, int &) {}
 };
 
-// C[0:rows, 0:o] -= Xt^T * Rt  with Xt[k][row] (32 x rows) and Rt[k][j] (32 x o), both in shared
-// memory with leading dimension FP_LD; C row-major with leading dimension FP_LD.  4 x 8 outputs
-// per thread, all threads of the CTA.
-__device__ __forceinline__ void panel_rank32_update(float (*C)[FP_LD], const float (*Xt)[FP_LD],
-                                                    const float (*Rt)[FP_LD], int o, int tid, int rows) {
-    const int tiles_j = o / 8;
-    for (int t = tid; t < (rows / 4) * tiles_j; t += FP_THREADS) {
-        const int ti = t / tiles_j, tj = t - ti * tiles_j;
-        float acc[4][8];
+// One column step (from 31 down to 0) of the inversion of a 32 x 32 upper triangular block held in
+// shared memory as its transpose (Rt[k][i] = R[i][k], leading dimension FP_LD): lane = column of the
+// inverse, y = that column, dinv = reciprocal diagonal of R.
+template <int K>
+struct InvColStep {
+    static __device__ __forceinline__ void run(float (&y)[32], const float *Rt, const float *dinv) {
+        const float x = y[K] * dinv[K];
+        y[K] = x;
+        const float *col = Rt + K * FP_LD;
 #pragma unroll
-        for (int e = 0; e < 4; ++e)
-#pragma unroll
-            for (int f = 0; f < 8; ++f) acc[e][f] = 0.f;
-#pragma unroll 4
-        for (int k = 0; k < 32; ++k) {
-            const float4 xa = *reinterpret_cast<const float4 *>(&Xt[k][4 * ti]);
-            const float4 r0 = *reinterpret_cast<const float4 *>(&Rt[k][8 * tj]);
-            const float4 r1 = *reinterpret_cast<const float4 *>(&Rt[k][8 * tj + 4]);
-            const float av[4] = {xa.x, xa.y, xa.z, xa.w};
-            const float bv[8] = {r0.x, r0.y, r0.z, r0.w, r1.x, r1.y, r1.z, r1.w};
-#pragma unroll
-            for (int e = 0; e < 4; ++e)
-#pragma unroll
-                for (int f = 0; f < 8; ++f) acc[e][f] = fmaf(av[e], bv[f], acc[e][f]);
+        for (int j4 = 0; j4 < (K + 3) / 4; ++j4) {
+            const float4 r = *reinterpret_cast<const float4 *>(col + 4 * j4);
+            if (4 * j4 + 0 < K) y[4 * j4 + 0] = fmaf(-x, r.x, y[4 * j4 + 0]);
+            if (4 * j4 + 1 < K) y[4 * j4 + 1] = fmaf(-x, r.y, y[4 * j4 + 1]);
+            if (4 * j4 + 2 < K) y[4 * j4 + 2] = fmaf(-x, r.z, y[4 * j4 + 2]);
+            if (4 * j4 + 3 < K) y[4 * j4 + 3] = fmaf(-x, r.w, y[4 * j4 + 3]);
         }
-#pragma unroll
-        for (int e = 0; e < 4; ++e) {
-            float4 *c0 = reinterpret_cast<float4 *>(&C[4 * ti + e][8 * tj]);
-            float4 v0 = c0[0], v1 = c0[1];
-            v0.x -= acc[e][0]; v0.y -= acc[e][1]; v0.z -= acc[e][2]; v0.w -= acc[e][3];
-            v1.x -= acc[e][4]; v1.y -= acc[e][5]; v1.z -= acc[e][6]; v1.w -= acc[e][7];
-            c0[0] = v0; c0[1] = v1;
-        }
+        InvColStep<K - 1>::run(y, Rt, dinv);
     }
-}
+};
+template <>
+struct InvColStep<-1> {
+    static __device__ __forceinline__ void run(float (&)[32], const float *, const float *) {}
+};
 
 __global__ void __launch_bounds__(FP_THREADS, 1) factor_panel_kernel(FactorPanelArgs a) {
     extern __shared__ __align__(16) float smem_f[];
-    // S: upper part = the working block, then R; lower part = R^T as it is produced
+    // S: the block as it is read, then R in the upper part and R^T in the lower part
     float (*S)[FP_LD] = reinterpret_cast<float (*)[FP_LD]>(smem_f);
     float (*At)[FP_LD] = reinterpret_cast<float (*)[FP_LD]>(smem_f + NB * FP_LD);         // step 2: a tile of panel rows
     float (*Pt)[FP_LD] = reinterpret_cast<float (*)[FP_LD]>(smem_f + 2 * NB * FP_LD);     // Pt[k][i]: 32 solved columns, transposed
-    float *dinv = smem_f + 2 * NB * FP_LD + 32 * FP_LD;
-    float *cv = dinv + NB;                 // 2 x 32: the scaled column of the running 32 x 32 step
+    float *Yt = smem_f + 2 * NB * FP_LD + 32 * FP_LD;       // [4][32][FP_YLD]: Yt[c][l][j] = inv(R_cc)[j][l]
+    float *dinv = Yt + 4 * 32 * FP_YLD;                     // [NB] 1 / R_jj
+    float *cv = dinv + NB;                                  // 2 x 32: the scaled column of the running 32 x 32 step
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int n = a.n, b0 = a.b0;
     const int nv = min(NB, n - b0);
     const bool vec = (n & 3) == 0 && (reinterpret_cast<uintptr_t>(a.H) & 15) == 0 && nv == NB;
+    const int TR = a.tile_rows;
+    const int r_begin = blockIdx.x * a.rows_per_cta;
+    const int r_end = min(b0, r_begin + a.rows_per_cta);
     pdl_launch_dependents();
     pdl_wait();
 
@@ -274,6 +268,16 @@ __global__ void __launch_bounds__(FP_THREADS, 1) factor_panel_kernel(FactorPanel
             const int idx = tid + it * FP_THREADS, i = idx >> 5, j4 = idx & 31;
             v[it] = *reinterpret_cast<const float4 *>(a.H + (int64_t)(b0 + i) * n + b0 + 4 * j4);
         }
+        // the first tile of this CTA's slab follows asynchronously
+        if (r_begin < r_end) {
+            for (int idx = tid; idx < TR * (NB / 4); idx += FP_THREADS) {
+                const int i = idx >> 5, j4 = idx & 31;
+                const uint32_t dst = (uint32_t)__cvta_generic_to_shared(&At[i][4 * j4]);
+                const float *src = a.H + (int64_t)(r_begin + i) * n + b0 + 4 * j4;
+                asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(src) : "memory");
+            }
+        }
+        asm volatile("cp.async.commit_group;" ::: "memory");
 #pragma unroll
         for (int it = 0; it < NB * NB / 4 / FP_THREADS; ++it) {
             const int idx = tid + it * FP_THREADS, i = idx >> 5, j4 = idx & 31;
@@ -291,10 +295,11 @@ __global__ void __launch_bounds__(FP_THREADS, 1) factor_panel_kernel(FactorPanel
     }
     __syncthreads();
 
+    // ---- step 1
     for (int sb = NB / 32 - 1; sb >= 0; --sb) {
         const int o = 32 * sb;
         if (warp == 0) {
-            // ---- 32 x 32 reverse Cholesky in registers, lane = row
+            // 32 x 32 reverse Cholesky in registers, lane = row
             float d[32];
 #pragma unroll
             for (int j = 0; j < 32; ++j) d[j] = (j >= lane) ? S[o + lane][o + j] : S[o + j][o + lane];
@@ -306,9 +311,10 @@ __global__ void __launch_bounds__(FP_THREADS, 1) factor_panel_kernel(FactorPanel
             for (int j = 0; j < 32; ++j)
                 if (j >= lane) { S[o + lane][o + j] = d[j]; S[o + j][o + lane] = d[j]; }
         }
+        if (o == 0) break;
         __syncthreads();
-        // ---- rows above: x R_ss^T = S[i, sub], one thread per row; results go to the upper part,
-        //      to the lower part (transposed) and to Pt for the update
+        // rows above: x R_ss^T = S[i, sub], one thread per row; results go to the upper part,
+        // to the lower part (transposed) and to Pt for the update
         if (tid < o) {
             const int i = tid;
             float x[32];
@@ -319,12 +325,13 @@ __global__ void __launch_bounds__(FP_THREADS, 1) factor_panel_kernel(FactorPanel
             for (int k = 0; k < 32; ++k) { S[i][o + k] = x[k]; S[o + k][i] = x[k]; Pt[k][i] = x[k]; }
         }
         __syncthreads();
-        // ---- leading part: S[i][j] -= R[i, sub] . R[j, sub] for i <= j < o, 4 x 4 per thread
+        // leading part: S[i][j] -= X[i] . X[j] for i <= j < o, 4 x 4 per thread; the tiles of the upper
+        // triangle are numbered through a (q / 2) x (q + 1) rectangle so that the active threads are dense
         {
-            const int q = o / 4;                    // 4 x 4 tiles per side
-            for (int t = tid; t < q * q; t += FP_THREADS) {
-                const int ti = t / q, tj = t - ti * q;
-                if (tj < ti) continue;
+            const int q = o / 4;
+            for (int t = tid; t < (q / 2) * (q + 1); t += FP_THREADS) {
+                const int r = t / (q + 1), c = t - r * (q + 1);
+                const int ti = c > r ? r : q - 1 - r, tj = c > r ? c - 1 : q - 1 - r + c;
                 float acc[4][4];
 #pragma unroll
                 for (int e = 0; e < 4; ++e)
@@ -341,14 +348,17 @@ __global__ void __launch_bounds__(FP_THREADS, 1) factor_panel_kernel(FactorPanel
                         for (int f = 0; f < 4; ++f) acc[e][f] = fmaf(av[e], bv[f], acc[e][f]);
                 }
 #pragma unroll
-                for (int e = 0; e < 4; ++e)
-#pragma unroll
-                    for (int f = 0; f < 4; ++f)
-                        if (4 * tj + f >= 4 * ti + e) S[4 * ti + e][4 * tj + f] -= acc[e][f];
+                for (int e = 0; e < 4; ++e) {
+                    float4 *cp = reinterpret_cast<float4 *>(&S[4 * ti + e][4 * tj]);
+                    float4 v = *cp;
+                    v.x -= acc[e][0]; v.y -= acc[e][1]; v.z -= acc[e][2]; v.w -= acc[e][3];
+                    *cp = v;
+                }
             }
         }
         __syncthreads();
     }
+    __syncthreads();
 
     if (blockIdx.x == 0)
         for (int idx = tid; idx < NB * NB; idx += FP_THREADS) {
@@ -357,24 +367,30 @@ __global__ void __launch_bounds__(FP_THREADS, 1) factor_panel_kernel(FactorPanel
         }
     if (b0 == 0) return;
 
-    // ---- step 2: rows [r_begin, r_end) of the panel in tiles of NB rows: a blocked triangular
-    //      solve, 32 columns at a time (one thread per row), then a rank-32 update of the
-    //      columns to the left (all threads)
-    const int r_begin = blockIdx.x * a.rows_per_cta;
-    const int r_end = min(b0, r_begin + a.rows_per_cta);
-    const int TR = a.tile_rows;
+    // the inverses of the four 32 x 32 diagonal sub-blocks (one warp each, lane = column)
+    if (warp < NB / 32) {
+        const int o = 32 * warp;
+        float y[32];
+#pragma unroll
+        for (int k = 0; k < 32; ++k) y[k] = (k == lane) ? 1.f : 0.f;
+        InvColStep<31>::run(y, &S[o][o], dinv + o);
+        float *dst = Yt + (warp * 32 + lane) * FP_YLD;
+#pragma unroll
+        for (int k4 = 0; k4 < 8; ++k4)
+            *reinterpret_cast<float4 *>(dst + 4 * k4) = make_float4(y[4 * k4], y[4 * k4 + 1], y[4 * k4 + 2], y[4 * k4 + 3]);
+    }
+
+    // ---- step 2: rows [r_begin, r_end) of the panel in tiles of TR rows
     for (int r0 = r_begin; r0 < r_end; r0 += TR) {        // b0 and the slabs are multiples of TR
         if (vec) {
-            float4 v[NB * NB / 4 / FP_THREADS];
-#pragma unroll
-            for (int it = 0; it < NB * NB / 4 / FP_THREADS; ++it) {
-                const int idx = tid + it * FP_THREADS, i = idx >> 5, j4 = idx & 31;
-                if (i < TR) v[it] = *reinterpret_cast<const float4 *>(a.H + (int64_t)(r0 + i) * n + b0 + 4 * j4);
-            }
-#pragma unroll
-            for (int it = 0; it < NB * NB / 4 / FP_THREADS; ++it) {
-                const int idx = tid + it * FP_THREADS, i = idx >> 5, j4 = idx & 31;
-                if (i < TR) *reinterpret_cast<float4 *>(&At[i][4 * j4]) = v[it];
+            if (r0 != r_begin) {
+                for (int idx = tid; idx < TR * (NB / 4); idx += FP_THREADS) {
+                    const int i = idx >> 5, j4 = idx & 31;
+                    *reinterpret_cast<float4 *>(&At[i][4 * j4]) =
+                        *reinterpret_cast<const float4 *>(a.H + (int64_t)(r0 + i) * n + b0 + 4 * j4);
+                }
+            } else {
+                asm volatile("cp.async.wait_all;" ::: "memory");
             }
         } else {
             for (int i = warp; i < TR; i += FP_WARPS) {
@@ -385,19 +401,61 @@ __global__ void __launch_bounds__(FP_THREADS, 1) factor_panel_kernel(FactorPanel
         __syncthreads();
         for (int sb = NB / 32 - 1; sb >= 0; --sb) {
             const int o = 32 * sb;
-            if (tid < TR) {
-                float x[32];
+            // X = At[:, o : o + 32] * inv(R_ss)^T, a row and four columns per thread; to Pt (transposed)
+            const float *Ys = Yt + sb * 32 * FP_YLD;
+            for (int t = tid; t < TR * 8; t += FP_THREADS) {
+                const int r = t >> 3, j0 = 4 * (t & 7);
+                float acc[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
-                for (int k = 0; k < 32; ++k) x[k] = At[tid][o + k];
-                solve_row<32>(x, &S[o][o], FP_LD, dinv + o);
+                for (int l4 = 0; l4 < 8; ++l4) {
+                    const float4 av = *reinterpret_cast<const float4 *>(&At[r][o + 4 * l4]);
+                    const float al[4] = {av.x, av.y, av.z, av.w};
 #pragma unroll
-                for (int k = 0; k < 32; ++k) { At[tid][o + k] = x[k]; Pt[k][tid] = x[k]; }
+                    for (int e = 0; e < 4; ++e) {
+                        const float4 yv = *reinterpret_cast<const float4 *>(Ys + (4 * l4 + e) * FP_YLD + j0);
+                        acc[0] = fmaf(al[e], yv.x, acc[0]);
+                        acc[1] = fmaf(al[e], yv.y, acc[1]);
+                        acc[2] = fmaf(al[e], yv.z, acc[2]);
+                        acc[3] = fmaf(al[e], yv.w, acc[3]);
+                    }
+                }
+#pragma unroll
+                for (int e = 0; e < 4; ++e) Pt[j0 + e][r] = acc[e];
             }
             __syncthreads();
-            if (o > 0) {
-                panel_rank32_update(At, Pt, reinterpret_cast<const float (*)[FP_LD]>(&S[o][0]), o, tid, TR);
-                __syncthreads();
+            // the solved columns back into the tile; columns to the left: At[r][j] -= sum_l X[r][l] R[j][o + l]
+            for (int t = tid; t < TR * 8; t += FP_THREADS) {
+                const int r = t >> 3, j0 = 4 * (t & 7);
+                *reinterpret_cast<float4 *>(&At[r][o + j0]) = make_float4(Pt[j0][r], Pt[j0 + 1][r], Pt[j0 + 2][r], Pt[j0 + 3][r]);
             }
+            if (o > 0) {
+                const int tj = o / 4;                       // tiles of 2 rows x 4 columns
+                for (int t = tid; t < (TR / 2) * tj; t += FP_THREADS) {
+                    const int ti = t / tj, j0 = 4 * (t - ti * tj);
+                    float acc[2][4];
+#pragma unroll
+                    for (int e = 0; e < 2; ++e)
+#pragma unroll
+                        for (int f = 0; f < 4; ++f) acc[e][f] = 0.f;
+#pragma unroll 8
+                    for (int l = 0; l < 32; ++l) {
+                        const float2 xv = *reinterpret_cast<const float2 *>(&Pt[l][2 * ti]);
+                        const float4 rv = *reinterpret_cast<const float4 *>(&S[o + l][j0]);
+                        acc[0][0] = fmaf(xv.x, rv.x, acc[0][0]); acc[0][1] = fmaf(xv.x, rv.y, acc[0][1]);
+                        acc[0][2] = fmaf(xv.x, rv.z, acc[0][2]); acc[0][3] = fmaf(xv.x, rv.w, acc[0][3]);
+                        acc[1][0] = fmaf(xv.y, rv.x, acc[1][0]); acc[1][1] = fmaf(xv.y, rv.y, acc[1][1]);
+                        acc[1][2] = fmaf(xv.y, rv.z, acc[1][2]); acc[1][3] = fmaf(xv.y, rv.w, acc[1][3]);
+                    }
+#pragma unroll
+                    for (int e = 0; e < 2; ++e) {
+                        float4 *cp = reinterpret_cast<float4 *>(&At[2 * ti + e][j0]);
+                        float4 v = *cp;
+                        v.x -= acc[e][0]; v.y -= acc[e][1]; v.z -= acc[e][2]; v.w -= acc[e][3];
+                        *cp = v;
+                    }
+                }
+            }
+            __syncthreads();
         }
         // store the tile (and its TF32 parts)
 #pragma unroll

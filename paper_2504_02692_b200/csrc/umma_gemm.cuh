@@ -357,9 +357,12 @@ struct StatsGemmArgs {
     StateHeader *hd;
     // Work items of a CTA pair: tiles [0, full_tiles) are whole 256 x 256 tiles; each of the remaining
     // `ntiles - full_tiles` tiles (the last, partial wave) is cut along K into `ksplit` items so that every
-    // pair has work.  Item 0 of a cut tile adds into the sums like a whole tile; items c > 0 store their
-    // partial result (128 x 256 per CTA) at scratch[(((tile - full_tiles) * (ksplit - 1) + c - 1) * 2 + rank)
-    // * UBM * UBN] and stats_fixup_kernel adds those in a fixed order (the result does not depend on timing).
+    // pair has work.  Item 0 of a cut tile adds into the sums like a whole tile; items c > 0 add their
+    // partial result (128 x 256 per CTA) into scratch[(((tile - full_tiles) * (ksplit - 1) + c - 1) * 2 + rank)
+    // * UBM * UBN], which the host zeroes before the first launch that uses it; the slots collect the partial
+    // sums of all launches with the same cut (one addition per slot entry and launch, in stream order), and
+    // stats_fixup_kernel adds them to the sums in a fixed order once, before the sums are read: the result
+    // does not depend on timing.
     int ntiles, full_tiles, ksplit;
     float *scratch;
 };
@@ -583,13 +586,14 @@ stats_umma_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constan
             if (!ok) break;
             const float inv = 1.f / (sx * (isD ? sd : sx));
             if (item.part > 0) {
-                // partial result of a cut tile: plain stores into its slot, all 128 x 256 entries
+                // partial result of a cut tile: added into its slot, all 128 x 256 entries
                 float *sp = a.scratch + (((int64_t)item.cut_index * (a.ksplit - 1) + item.part - 1) * 2 + (int)rank) * (UBM * UBN) +
                             (quarter * 32 + lane) * UBN + half * (UBN / 2);
 #pragma unroll
                 for (int q = 0; q < UBN / 2 / 4; ++q)
-                    *reinterpret_cast<float4 *>(sp + 4 * q) = make_float4(acc[4 * q + 0] * inv, acc[4 * q + 1] * inv,
-                                                                         acc[4 * q + 2] * inv, acc[4 * q + 3] * inv);
+                    asm volatile("red.global.add.v4.f32 [%0], {%1, %2, %3, %4};" ::"l"(sp + 4 * q),
+                                 "f"(acc[4 * q + 0] * inv), "f"(acc[4 * q + 1] * inv),
+                                 "f"(acc[4 * q + 2] * inv), "f"(acc[4 * q + 3] * inv) : "memory");
                 continue;
             }
             const int row = (isD ? it.r - it.T : it.r) * UPM + (int)rank * UBM + quarter * 32 + lane;
@@ -642,8 +646,8 @@ __global__ void bounded_wait_selftest_kernel(StateHeader *hd, long long limit_cy
     if (!ok && threadIdx.x == 0) record_status(hd, ST_TIMEOUT, 2000000);
 }
 
-// Adds the partial results of the cut tiles (see StatsGemmArgs) into H / dXX^T, partial 1 first, then 2, ...:
-// FIXUP_SLABS CTAs per cut tile, after stats_umma_kernel of the same batch.
+// Adds the collected partial sums of the cut tiles (see StatsGemmArgs) into H / dXX^T, partial 1 first, then
+// 2, ...: FIXUP_SLABS CTAs per cut tile, after the last stats_umma_kernel that used these slots.
 constexpr int FIXUP_SLABS = 32;     // CTAs per cut tile, UPM / FIXUP_SLABS rows each
 __global__ void __launch_bounds__(256) stats_fixup_kernel(StatsGemmArgs a) {
     TileIter it(a.n);
