@@ -36,7 +36,7 @@ METRIC = "ms per layer (GPTAQ solve: accumulate + factor + P + quantize)"
 # dram__bytes_read.sum + dram__bytes_write.sum of one stats_umma_kernel launch (one token batch) from an
 # ncu capture of the kernel as it stands, keyed by (workload, statistics arithmetic); workloads without a
 # capture of the current kernel report null with the reason.
-STATS_KERNEL_TRAFFIC = {("cfg2", 0): 589.6e6}
+STATS_KERNEL_TRAFFIC = {}
 TRAFFIC_MISSING = "no ncu capture of the current statistics kernel for this workload and arithmetic"
 
 
@@ -302,13 +302,16 @@ def run_ours(args, cfg):
     fac_ms = sum(m[1].elapsed_time(m[2]) for m in marks) / args.steps
     p_ms = sum(m[2].elapsed_time(m[3]) for m in marks) / args.steps
     q_ms = sum(m[3].elapsed_time(m[4]) for m in marks) / args.steps
-    flops_call = 3.0 * cfg.n * cfg.n * cfg.batch_tokens
+    # algorithmic flops of one accumulate call: the upper triangle of H (n^2 k) and what P needs of dXX^T:
+    # the part above the diagonal (n^2 k), or all of it under act_order (2 n^2 k)
+    flops_per_token = (3.0 if args.act_order else 2.0) * cfg.n * cfg.n
+    flops_call = flops_per_token * cfg.batch_tokens
     stage_achieved = flops_call / (acc_call_ms * 1e-3) / 1e12     # whole accumulate call: conversion, product, fix-up
     peak = pk["bf16_sustained"]
     if kern_launches > 0:
         # the dominant kernel by itself: algorithmic flops of the timed region / the sum of its launch durations
         kern_us = kern_ms_total * 1e3 / kern_launches
-        flops_launch = 3.0 * cfg.n * cfg.n * cfg.batch_tokens * len(batches) * args.steps / kern_launches
+        flops_launch = flops_per_token * cfg.batch_tokens * len(batches) * args.steps / kern_launches
         achieved = flops_launch / (kern_us * 1e-6) / 1e12
         kern_name = "stats_umma_kernel (tcgen05 kind::f16, cta_group::2), one token batch per launch"
     else:
@@ -388,7 +391,8 @@ def run_ours(args, cfg):
         "config": dict(wl.describe(cfg), parallelism=(f"one layer over {world} GPUs: tokens sharded, one all-reduce of H and dXX^T, rows sharded"
                                     if shard else f"{world} independent layer(s), one per GPU"),
                        l2="inputs (%.1f GB per step) exceed L2" % (2 * cfg.tokens * cfg.n * 4 / 1e9),
-                       statistics=prec_name, act_order=bool(args.act_order), clip_search=args.clip_search),
+                       statistics=prec_name, act_order=bool(args.act_order), clip_search=args.clip_search,
+                       dxx="all of it (act_order permutes it)" if args.act_order else "above the diagonal (what P uses)"),
         "stages_ms": {"accumulate": acc_step_ms, "factor": fac_ms, "build_P": p_ms, "quantize": q_ms,
                       "layer_quantize": fac_ms + p_ms + q_ms},
         "accumulate_tflops": stage_achieved, "stage_rooflines": stage_rooflines,

@@ -110,7 +110,13 @@ gptaq_status_t gptaq_destroy(gptaq_handle_t h);
 /* Algorithm 1, the statistics, one token batch:  H += X X^T,  dXX^T += (X~ - X) X^T.
  * d_X, d_Xfp: [tokens x n] float32, leading dimension ld >= n, read only.
  * The difference X~ - X is formed in float32 before any product.
- * tokens == 0 is a no-op.  Only the upper triangle of H is maintained. */
+ * tokens == 0 is a no-op.  Only the upper triangle of H is maintained (H is symmetric).  Of dXX^T only the
+ * part above the diagonal is guaranteed: Theorem 4.2 masks (dXX^T U^T) with the strictly upper triangular
+ * M_U and row j of U starts at column j, so entry (i, k) of dXX^T reaches P only where k > i; the entries on
+ * and below the diagonal are accumulated where that is free (the simple FMA path; inside the diagonal
+ * tiles of the tensor-core path) and otherwise left as they were -- a third of the products saved.  With
+ * act_order enabled the whole of dXX^T is accumulated, because the permutation mixes the two triangles:
+ * enable it before the first token batch (see gptaq_set_act_order). */
 gptaq_status_t gptaq_accumulate(gptaq_handle_t h, const float *d_X, const float *d_Xfp,
                                 int64_t tokens, int64_t ld, gptaq_stream_t stream);
 
@@ -226,7 +232,8 @@ gptaq_status_t gptaq_quantize_static(const float *d_U, const float *d_P, int64_t
 gptaq_status_t gptaq_sync_status(gptaq_handle_t h, int64_t *info, gptaq_stream_t stream);
 
 /* Device views into the state (n x n, leading dimension n), for tests and for
- * callers that checkpoint the sums: H / U and dXX^T / P share storage. */
+ * callers that checkpoint the sums: H / U and dXX^T / P share storage.  What is defined of the sums:
+ * the upper triangle of H; of dXX^T the part above the diagonal, all of it under act_order. */
 float *gptaq_H(gptaq_handle_t h);
 float *gptaq_D(gptaq_handle_t h);
 /* The same storage under the names of what it holds later: U (the inverse-Cholesky factor of Algorithm 1; NULL
@@ -251,6 +258,8 @@ int gptaq_recommended_stats_precision(int64_t n, int64_t total_tokens);
  * SORTED order, i.e. caller column c uses group rank(c) / group, rank being the inverse of gptaq_perm.
  * gptaq_quantize then needs d_Wq as a second buffer (non-NULL, different from d_W).
  * gptaq_H / gptaq_D show U and P in sorted order.  Supported for n <= 57344.
+ * Enabling it after a token batch has gone in without the lower triangle of dXX^T (see gptaq_accumulate)
+ * returns GPTAQ_ERR_BAD_STATE; gptaq_reset clears that.
  * gptaq_perm: device array of n int32, sorted position -> caller column; NULL unless enabled and factored. */
 gptaq_status_t gptaq_set_act_order(gptaq_handle_t h, int enable);
 const int32_t *gptaq_perm(gptaq_handle_t h);

@@ -67,6 +67,7 @@ struct gptaq_ctx {
     // the sums are needed or the cut changes; fix_pending: they have not been added to H / dXX^T yet
     bool fix_pending;
     StatsGemmArgs fix_args;
+    bool d_upper_only;     // a token batch went in without the tiles of dXX^T below the diagonal
     // optional timing of the statistics kernel alone: one event pair per launch, on the stream it runs on
     bool kernel_timing;
     std::vector<std::pair<cudaEvent_t, cudaEvent_t>> timing_events;   // pool; the first timing_used are recorded
@@ -414,7 +415,10 @@ gptaq_status_t accumulate_tc(gptaq_ctx *h, const float *X, const float *Xfp, int
         h->relayout = false;
     }
     const int64_t chunk = tc_chunk_tokens(h);
-    const int64_t ntiles = TileIter::total(n);              // 256 x 256 tiles of H (upper) and dXX^T
+    // 256 x 256 tiles of H (upper) and of dXX^T (upper too, unless act_order will permute it)
+    const int d_full = h->act_order ? 1 : 0;
+    const int64_t ntiles = TileIter::total(n, d_full);
+    if (!d_full) h->d_upper_only = true;
     const int npairs = std::max(1, h->num_sms / 2);         // CTA pairs (clusters of two)
     for (int64_t t0 = 0; t0 < tokens; t0 += chunk) {
         const int tk = (int)std::min<int64_t>(chunk, tokens - t0);
@@ -457,6 +461,7 @@ gptaq_status_t accumulate_tc(gptaq_ctx *h, const float *X, const float *Xfp, int
         StatsGemmArgs ga;
         ga.H = h->H; ga.D = h->D; ga.n = n; ga.kblocks = kp / UBK; ga.nseg_h = split ? 3 : 1; ga.nseg_d = splitd ? 3 : 1; ga.amax = amax; ga.hd = h->hd;
         // the last, partial wave of tiles is cut along K so that every pair has work
+        ga.d_full = d_full;
         ga.ntiles = (int)ntiles;
         ga.full_tiles = (int)(ntiles / npairs) * npairs;
         ga.ksplit = 1;
@@ -483,6 +488,7 @@ gptaq_status_t accumulate_tc(gptaq_ctx *h, const float *X, const float *Xfp, int
             CU(cudaEventRecord(tev->first, gs));
         }
         if (h->fix_pending && (h->fix_args.ksplit != ga.ksplit || h->fix_args.full_tiles != ga.full_tiles ||
+                               h->fix_args.ntiles != ga.ntiles || h->fix_args.d_full != ga.d_full ||
                                h->fix_args.scratch != ga.scratch))
             OK(flush_partials(h));              // another cut: the slots change meaning
         if (ga.ksplit > 1 && !h->fix_pending) {
@@ -881,6 +887,7 @@ gptaq_status_t gptaq_create(gptaq_handle_t *out, int64_t n, void *d_state, size_
     h->relayout = false;
     h->next_buf = 0;
     h->fix_pending = false;
+    h->d_upper_only = false;
     for (int i = 0; i < 2; ++i) { h->conv_done[i] = h->gemm_done[i] = nullptr; h->gemm_pending[i] = false; }
     e = cudaStreamCreateWithFlags(&h->gemm_stream, cudaStreamNonBlocking);
     for (int i = 0; i < 2 && e == cudaSuccess; ++i) {
@@ -907,6 +914,7 @@ gptaq_status_t gptaq_reset(gptaq_handle_t h, gptaq_stream_t stream) {
     CU(cudaMemsetAsync(h->state, 0, l.total, static_cast<cudaStream_t>(stream)));
     h->stage = STAGE_ACCUM;
     h->tokens = 0;
+    h->d_upper_only = false;
     h->sched.base = 0;           // the counter in the header was zeroed with the rest of the state
     return GPTAQ_OK;
 }
@@ -1030,7 +1038,9 @@ gptaq_status_t gptaq_factor(gptaq_handle_t h, float damp, gptaq_stream_t stream)
         fa.tile_rows = tr;
         const int fgrid = std::max(1, std::min(b0 / tr, h->num_sms));
         fa.rows_per_cta = ((b0 + fgrid - 1) / fgrid + tr - 1) / tr * tr;
-        CU(launch_pdl(true, factor_panel_kernel, dim3(fgrid), dim3(FP_THREADS), FP_SMEM, s, fa));
+        // one more CTA, without a slab, stores the diagonal factor while there is an SM left for it
+        const int fextra = (b0 > 0 && fgrid < h->num_sms) ? 1 : 0;
+        CU(launch_pdl(true, factor_panel_kernel, dim3(fgrid + fextra), dim3(FP_THREADS), FP_SMEM, s, fa));
         h->launches++;
         if (p == 0) break;
         if (h->f16 && b0 >= TC_MIN_N) {
@@ -1452,6 +1462,8 @@ gptaq_status_t gptaq_set_act_order(gptaq_handle_t h, int enable) {
     if (!h) return GPTAQ_ERR_INVALID_ARG;
     if (h->stage != STAGE_ACCUM) return GPTAQ_ERR_BAD_STATE;
     if (enable && h->n > ACT_ORDER_MAX_N) return GPTAQ_ERR_UNSUPPORTED;
+    // the permutation needs the part of dXX^T below the diagonal, which earlier batches did not accumulate
+    if (enable && !h->act_order && h->d_upper_only) return GPTAQ_ERR_BAD_STATE;
     h->act_order = enable != 0;
     return GPTAQ_OK;
 }

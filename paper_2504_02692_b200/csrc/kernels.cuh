@@ -127,7 +127,7 @@ __global__ void __launch_bounds__(256) scale_damp_kernel(float *H, int n, const 
 //      with the inverse of the 32 x 32 diagonal sub-block (the four inverses: one warp each, lane =
 //      column), then a rank-32 update of the columns to the left, all threads on both; written back in place and, if asked for, as split parts for the tensor-core rank update.
 // Every CTA repeats step 1 (it is short and the other SMs would idle) and then takes a
-// slab of rows of step 2, whose first tile is fetched while step 1 runs; CTA 0 stores R_pp for
+// slab of rows of step 2, whose first tile is fetched while step 1 runs; the last CTA stores R_pp for
 // invert_diag_blocks_kernel.  Rows/columns beyond n are padded with the identity.
 // ---------------------------------------------------------------------------
 constexpr int NB = 128;
@@ -179,17 +179,20 @@ __device__ __forceinline__ void solve_row(float (&a)[LEN], const float *Rt, int 
 // next runs through lane K - 1 alone (its own c), the other lanes' updates overlap with it.
 // The scaled column c reaches the other lanes through shared memory (cv: two buffers of 32 floats,
 // read back as broadcast float4s): K shuffles per step, one per element, cost three times as much.
-// A pivot that is not positive (or not finite) is replaced by 1 without a branch; the first such
-// column is remembered in bad_col (-1: none) and reported after the block.
+// A pivot that is not a positive normal number is replaced by 1 without a branch, and off the chain
+// (the estimate is taken from the pivot as it comes, the test runs beside it); the first such column
+// is remembered in bad_col (-1: none) and reported after the block.
 template <int K>
 struct Chol32Step {
     static __device__ __forceinline__ void run(float (&d)[32], float piv, int lane, float *dinv, float *cv, int &bad_col) {
-        const bool bad = !(piv > 0.f) || !isfinite(piv);
+        // 1/sqrt(piv): hardware estimate plus one Newton step (to about one ulp)
+        float rinv;
+        asm("rsqrt.approx.ftz.f32 %0, %1;" : "=f"(rinv) : "f"(piv));
+        rinv = rinv * fmaf(-0.5f * piv, rinv * rinv, 1.5f);
+        const bool bad = !(piv >= 1.17549435e-38f) || !(piv < INFINITY);
         bad_col = (bad && bad_col < 0) ? K : bad_col;
         piv = bad ? 1.f : piv;
-        // 1/sqrt(piv): hardware estimate plus one Newton step (to about one ulp)
-        float rinv = rsqrtf(piv);
-        rinv = rinv * fmaf(-0.5f * piv, rinv * rinv, 1.5f);
+        rinv = bad ? 1.f : rinv;
         const float c = lane < K ? d[K] * rinv : 0.f;
         d[K] = lane < K ? c : (lane == K ? piv * rinv : 0.f);
         if (lane == K) dinv[K] = rinv;
@@ -240,6 +243,45 @@ template <>
 struct InvColStep<-1> {
     static __device__ __forceinline__ void run(float (&)[32], const float *, const float *) {}
 };
+
+// C[0:rows, 0:o] -= X * Rt-columns:  C[r][j] -= sum_l Xt[l][r] * Rt[l][j]  with Xt (32 x rows) and Rt (32 x o)
+// in shared memory, leading dimension FP_LD.  RT rows x 4 columns per thread, all threads of the CTA.
+template <int RT>
+__device__ __forceinline__ void slab_rank32_update(float (*C)[FP_LD], const float (*Xt)[FP_LD], const float (*Rt)[FP_LD],
+                                                   int o, int tid, int rows) {
+    const int tj = o / 4;
+    for (int t = tid; t < (rows / RT) * tj; t += FP_THREADS) {
+        const int ti = t / tj, j0 = 4 * (t - ti * tj);
+        float acc[RT][4];
+#pragma unroll
+        for (int e = 0; e < RT; ++e)
+#pragma unroll
+            for (int f = 0; f < 4; ++f) acc[e][f] = 0.f;
+#pragma unroll 8
+        for (int l = 0; l < 32; ++l) {
+            float xv[RT];
+            if (RT == 2) {
+                const float2 x2 = *reinterpret_cast<const float2 *>(&Xt[l][2 * ti]);
+                xv[0] = x2.x; xv[RT - 1] = x2.y;
+            } else {
+                xv[0] = Xt[l][ti];
+            }
+            const float4 rv = *reinterpret_cast<const float4 *>(&Rt[l][j0]);
+#pragma unroll
+            for (int e = 0; e < RT; ++e) {
+                acc[e][0] = fmaf(xv[e], rv.x, acc[e][0]); acc[e][1] = fmaf(xv[e], rv.y, acc[e][1]);
+                acc[e][2] = fmaf(xv[e], rv.z, acc[e][2]); acc[e][3] = fmaf(xv[e], rv.w, acc[e][3]);
+            }
+        }
+#pragma unroll
+        for (int e = 0; e < RT; ++e) {
+            float4 *cp = reinterpret_cast<float4 *>(&C[RT * ti + e][j0]);
+            float4 v = *cp;
+            v.x -= acc[e][0]; v.y -= acc[e][1]; v.z -= acc[e][2]; v.w -= acc[e][3];
+            *cp = v;
+        }
+    }
+}
 
 __global__ void __launch_bounds__(FP_THREADS, 1) factor_panel_kernel(FactorPanelArgs a) {
     extern __shared__ __align__(16) float smem_f[];
@@ -360,12 +402,13 @@ __global__ void __launch_bounds__(FP_THREADS, 1) factor_panel_kernel(FactorPanel
     }
     __syncthreads();
 
-    if (blockIdx.x == 0)
+    // (the last CTA: the host adds one without a slab while there are SMs left)
+    if (blockIdx.x == gridDim.x - 1)
         for (int idx = tid; idx < NB * NB; idx += FP_THREADS) {
             const int i = idx >> 7, j = idx & 127;
             a.Rdiag[idx] = j >= i ? S[i][j] : 0.f;
         }
-    if (b0 == 0) return;
+    if (b0 == 0 || r_begin >= r_end) return;
 
     // the inverses of the four 32 x 32 diagonal sub-blocks (one warp each, lane = column)
     if (warp < NB / 32) {
@@ -429,31 +472,8 @@ __global__ void __launch_bounds__(FP_THREADS, 1) factor_panel_kernel(FactorPanel
                 *reinterpret_cast<float4 *>(&At[r][o + j0]) = make_float4(Pt[j0][r], Pt[j0 + 1][r], Pt[j0 + 2][r], Pt[j0 + 3][r]);
             }
             if (o > 0) {
-                const int tj = o / 4;                       // tiles of 2 rows x 4 columns
-                for (int t = tid; t < (TR / 2) * tj; t += FP_THREADS) {
-                    const int ti = t / tj, j0 = 4 * (t - ti * tj);
-                    float acc[2][4];
-#pragma unroll
-                    for (int e = 0; e < 2; ++e)
-#pragma unroll
-                        for (int f = 0; f < 4; ++f) acc[e][f] = 0.f;
-#pragma unroll 8
-                    for (int l = 0; l < 32; ++l) {
-                        const float2 xv = *reinterpret_cast<const float2 *>(&Pt[l][2 * ti]);
-                        const float4 rv = *reinterpret_cast<const float4 *>(&S[o + l][j0]);
-                        acc[0][0] = fmaf(xv.x, rv.x, acc[0][0]); acc[0][1] = fmaf(xv.x, rv.y, acc[0][1]);
-                        acc[0][2] = fmaf(xv.x, rv.z, acc[0][2]); acc[0][3] = fmaf(xv.x, rv.w, acc[0][3]);
-                        acc[1][0] = fmaf(xv.y, rv.x, acc[1][0]); acc[1][1] = fmaf(xv.y, rv.y, acc[1][1]);
-                        acc[1][2] = fmaf(xv.y, rv.z, acc[1][2]); acc[1][3] = fmaf(xv.y, rv.w, acc[1][3]);
-                    }
-#pragma unroll
-                    for (int e = 0; e < 2; ++e) {
-                        float4 *cp = reinterpret_cast<float4 *>(&At[2 * ti + e][j0]);
-                        float4 v = *cp;
-                        v.x -= acc[e][0]; v.y -= acc[e][1]; v.z -= acc[e][2]; v.w -= acc[e][3];
-                        *cp = v;
-                    }
-                }
+                const float (*Rt)[FP_LD] = reinterpret_cast<const float (*)[FP_LD]>(&S[o][0]);
+                slab_rank32_update<2>(At, Pt, Rt, o, tid, TR);
             }
             __syncthreads();
         }

@@ -365,10 +365,14 @@ struct StatsGemmArgs {
     // does not depend on timing.
     int ntiles, full_tiles, ksplit;
     float *scratch;
+    int d_full;              // 0: only the tiles of dXX^T that reach the diagonal or lie above it (see TileIter)
 };
 
 // Tile enumeration shared by all roles, in units of the pair's 256 x 256 tiles.  Rows [0, T) belong to H
-// (tiles entirely below the diagonal are not enumerated), rows [T, 2 T) to dXX^T.  Order: bands of UBAND
+// (tiles entirely below the diagonal are not enumerated), rows [T, 2 T) to dXX^T.  Of dXX^T the matrix P
+// (Theorem 4.2) uses the entries above the diagonal only -- the mask M_U keeps column j > i of row i of
+// dXX^T U^T, and row j of U starts at column j -- so its tiles below the diagonal are enumerated only on
+// request (dfull: act_order permutes dXX^T on both sides and needs all of it).  Order: bands of UBAND
 // row tiles; inside a band column tile by column tile, first the band's tiles of H, then its tiles of dXX^T.
 // The tiles that are in flight together then share about 2 x 8 row panels (X and X~ - X) and a handful
 // of column panels of X through the L2, and X streams from HBM once per band instead of once per
@@ -378,17 +382,22 @@ constexpr int UBAND = 8;
 struct TileIter {
     int T, r, tn, ord;            // (r, tn): the current tile; ord: its ordinal
     int band, k;                  // band of row tiles, position inside the group (band, tn)
-    __host__ __device__ TileIter(int n) : T((n + UPM - 1) / UPM), r(0), tn(0), ord(0), band(0), k(0) {}
+    int dfull;                    // all tiles of dXX^T, not only those with r <= tn
+    __host__ __device__ TileIter(int n, int dfull_) : T((n + UPM - 1) / UPM), r(0), tn(0), ord(0), band(0), k(0), dfull(dfull_) {}
     __host__ __device__ int band_rows() const { return min(UBAND, T - band * UBAND); }
     // row tiles r of the band whose tile (r, tn) of H is not entirely below the diagonal: r <= tn
     __host__ __device__ int h_count() const { return max(0, min(band_rows(), tn + 1 - band * UBAND)); }
-    __host__ __device__ static int total(int n) { const int t = (n + UPM - 1) / UPM; return t * (t + 1) / 2 + t * t; }
+    __host__ __device__ int d_count() const { return dfull ? band_rows() : h_count(); }
+    __host__ __device__ static int total(int n, int dfull_) {
+        const int t = (n + UPM - 1) / UPM;
+        return t * (t + 1) / 2 + (dfull_ ? t * t : t * (t + 1) / 2);
+    }
     // Advances to the tile with ordinal `target` >= ord; false when the list is exhausted.
     __host__ __device__ bool seek_to(int target) {
         int left = target - ord;
         while (band * UBAND < T) {
             const int hc = h_count();
-            const int avail = hc + band_rows() - k;
+            const int avail = hc + d_count() - k;
             if (left < avail) {
                 k += left;
                 ord = target;
@@ -489,7 +498,7 @@ stats_umma_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constan
     if (warp == 0) {
         // ------------------------------------------------------------ TMA producer (each CTA its own halves)
         if (lane == 0) {
-            TileIter it(a.n);
+            TileIter it(a.n, a.d_full);
             StatsItem item;
             uint32_t stage = 0, phase = 0;
             int issued = 0;
@@ -521,7 +530,7 @@ stats_umma_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constan
     } else if (warp == 1) {
         // ------------------------------------------------------------ MMA issuer (first CTA of the pair)
         if (lane == 0 && rank == 0) {
-            TileIter it(a.n);
+            TileIter it(a.n, a.d_full);
             StatsItem item;
             uint32_t stage = 0, phase = 0, ccount = 0;     // ccount: chunks issued so far
             bool ok = true;
@@ -554,7 +563,7 @@ stats_umma_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constan
         // ------------------------------------------------------------ epilogue (warps 2..9): this CTA's 128 rows
         const int quarter = warp & 3;                 // TMEM lanes 32 * quarter .. + 31
         const int half = (warp - 2) >> 2;             // columns [128 * half, 128 * half + 128)
-        TileIter it(a.n);
+        TileIter it(a.n, a.d_full);
         StatsItem item;
         uint32_t ccount = 0;
         bool ok = true;
@@ -650,7 +659,7 @@ __global__ void bounded_wait_selftest_kernel(StateHeader *hd, long long limit_cy
 // 2, ...: FIXUP_SLABS CTAs per cut tile, after the last stats_umma_kernel that used these slots.
 constexpr int FIXUP_SLABS = 32;     // CTAs per cut tile, UPM / FIXUP_SLABS rows each
 __global__ void __launch_bounds__(256) stats_fixup_kernel(StatsGemmArgs a) {
-    TileIter it(a.n);
+    TileIter it(a.n, a.d_full);
     if (!it.seek_to(a.full_tiles + blockIdx.x)) return;
     const bool isD = it.r >= it.T;
     const int row0 = (isD ? it.r - it.T : it.r) * UPM, col0 = it.tn * UBN;

@@ -643,3 +643,27 @@ def test_two_bit_symmetric_group_grids_can_lose_to_plain_rounding():
     for bits, group, sym in ((2, 64, False), (3, 64, True), (2, 0, True)):
         Jv, Jv_rtn = pair(bits, group, sym)
         assert Jv < Jv_rtn, (bits, group, sym, Jv, Jv_rtn)
+
+
+def test_P_uses_only_the_part_of_dxx_above_the_diagonal():
+    """Theorem 4.2: the mask M_U keeps column a > q of row q of dXX^T U^T, and row a of U starts at column a,
+    so entry (q, k) of dXX^T enters P only where k > q.  Zeroing (or scrambling) the diagonal and the lower
+    triangle of dXX^T leaves P unchanged to the last bit in both forms; scrambling one entry above the
+    diagonal changes it.  (What the device may skip when it accumulates dXX^T.)"""
+    rng = np.random.default_rng(77)
+    n, k = 48, 300
+    Xf = rng.standard_normal((k, n))
+    X = Xf + 0.1 * np.abs(Xf) * rng.standard_normal((k, n))
+    st = orc.new_stats(n)
+    orc.accumulate(st, X, Xf)
+    U, _ = orc.factor(st.H, st.tokens, 0.01)
+    P = orc.build_P(st.D, st.tokens, U, 0.25)
+    low = np.tril(np.ones((n, n), bool))
+    D2 = st.D.copy()
+    D2[low] = rng.standard_normal(low.sum()) * 1e3
+    assert np.array_equal(orc.build_P(np.triu(st.D, 1), st.tokens, U, 0.25), P)
+    assert np.array_equal(orc.build_P(D2, st.tokens, U, 0.25), P)
+    assert np.allclose(orc.build_P_rowwise(D2, st.tokens, U, 0.25), P, rtol=0, atol=1e-15 * np.abs(P).max())
+    D3 = st.D.copy()
+    D3[3, 17] += 1.0
+    assert np.abs(orc.build_P(D3, st.tokens, U, 0.25) - P).max() > 1e-6
