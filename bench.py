@@ -36,7 +36,7 @@ METRIC = "ms per layer (GPTAQ solve: accumulate + factor + P + quantize)"
 # dram__bytes_read.sum + dram__bytes_write.sum of one stats_umma_kernel launch (one token batch) from an
 # ncu capture of the kernel as it stands, keyed by (workload, statistics arithmetic); workloads without a
 # capture of the current kernel report null with the reason.
-STATS_KERNEL_TRAFFIC = {}
+STATS_KERNEL_TRAFFIC = {("cfg2", 0): 462.5e6}
 TRAFFIC_MISSING = "no ncu capture of the current statistics kernel for this workload and arithmetic"
 
 
