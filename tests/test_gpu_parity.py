@@ -337,7 +337,9 @@ def test_act_order(n, m, group, B, bf16):
 
 @pytest.mark.parametrize("n,m,group,B,act,bf16,ndead", [(192, 24, 32, 64, True, False, 0), (640, 40, 128, 128, True, False, 0),
                                                         (768, 33, 64, 128, True, True, 0), (640, 20, 128, 128, False, False, 0),
-                                                        (320, 30, 64, 64, True, False, 3), (512, 33, 64, 64, False, True, 3)])
+                                                        (320, 30, 64, 64, True, False, 3), (512, 33, 64, 64, False, True, 3),
+                                                        (768, 24, 128, 128, True, True, 0), (1024, 24, 32, 64, True, True, 3),
+                                                        (320, 64, 32, 128, True, True, 3)])
 def test_static_groups(n, m, group, B, act, bf16, ndead):
     """Static groups, with and without act_order: grids per group of the caller's columns from the original
     weights (inputs that never fired count as zero weights); the loop replayed by the oracle in the device's
@@ -372,11 +374,28 @@ def test_static_groups(n, m, group, B, act, bf16, ndead):
     U, P, dead, res, _ = orc.solve_act_order(Wn, so.H, so.D, so.tokens, cfg.damp, cfg.alpha, cfg.bits, group, cfg.sym,
                                              perm=perm, static_groups=True)
     cg, scn, zpn = codes.cpu().numpy(), sc.cpu().numpy(), zp.cpu().numpy()
-    # the grids are those of the original weights, float32 arithmetic on both sides of a min/max
-    assert np.abs(scn - res.scales).max() <= 1e-6 * np.abs(res.scales).max() and np.array_equal(zpn, res.zeros)
     dead0 = np.zeros(n, bool)
     dead0[perm] = dead
     assert dead0.sum() == ndead
+    # the grids are those of the original weights, float32 arithmetic on both sides of a min/max.  A zero
+    # point whose pre-rounding value -lo / scale is a tie (x.5: bf16 weights have short mantissas, and a group
+    # whose extremes are symmetric gives exactly maxq / 2) may round either way, to the floor or to the ceiling
+    assert np.abs(scn - res.scales).max() <= 1e-6 * np.abs(res.scales).max()
+    W0 = Wn.copy()
+    W0[:, dead0] = 0.0
+    lo = np.stack([np.minimum(W0[:, k * group:(k + 1) * group].min(axis=1), 0.0) for k in range(G)], axis=1)
+    t = -lo / res.scales
+    tie = np.abs(t - np.floor(t) - 0.5) <= 1e-6
+    differs = zpn != res.zeros
+    assert not (differs & ~tie).any(), int((differs & ~tie).sum())
+    assert np.isin(zpn[differs] - np.floor(t[differs]), (0.0, 1.0)).all()
+    if differs.any():
+        # the oracle's free run again, with the device's choice at the ties
+        r2 = orc.quantize(Wn[:, perm], U, P, dead, cfg.bits, group, cfg.sym,
+                          static=(res.scales, zpn.astype(np.float64), perm // group))
+        Wq2 = np.empty_like(r2.Wq)
+        Wq2[:, perm] = r2.Wq
+        res = orc.QuantResult(None, res.scales, zpn.astype(np.float64), Wq2)
     rep = orc.follow(Wn[:, perm], U, P, dead, cfg.bits, group, cfg.sym, cg[:, perm], scn.astype(np.float64),
                      zpn.astype(np.float64), band=hp.TOL_FLIP_BAND, static=(Wn, perm // group, dead0))
     assert rep.disallowed == 0 and rep.allowed <= hp.TOL_FLIP_RATE * rep.total, rep
