@@ -889,7 +889,14 @@ gptaq_status_t gptaq_create(gptaq_handle_t *out, int64_t n, void *d_state, size_
     h->fix_pending = false;
     h->d_upper_only = false;
     for (int i = 0; i < 2; ++i) { h->conv_done[i] = h->gemm_done[i] = nullptr; h->gemm_pending[i] = false; }
-    e = cudaStreamCreateWithFlags(&h->gemm_stream, cudaStreamNonBlocking);
+    {
+        // highest priority: when a product and the conversion of the next batch become ready together, the
+        // product's CTAs (one per SM, nearly all of its shared memory) are placed first and the conversion
+        // fills the SMs that the product's last round of tiles leaves idle
+        int prio_lo = 0, prio_hi = 0;
+        e = cudaDeviceGetStreamPriorityRange(&prio_lo, &prio_hi);
+        if (e == cudaSuccess) e = cudaStreamCreateWithPriority(&h->gemm_stream, cudaStreamNonBlocking, prio_hi);
+    }
     for (int i = 0; i < 2 && e == cudaSuccess; ++i) {
         e = cudaEventCreateWithFlags(&h->conv_done[i], cudaEventDisableTiming);
         if (e == cudaSuccess) e = cudaEventCreateWithFlags(&h->gemm_done[i], cudaEventDisableTiming);
