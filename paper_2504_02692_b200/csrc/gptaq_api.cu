@@ -1209,10 +1209,11 @@ gptaq_status_t gptaq_build_P(gptaq_handle_t h, float alpha, gptaq_stream_t strea
         const float inv_tokens = (float)(1.0 / (double)h->tokens);
         CU(cudaMemsetAsync(am + AMAX_U, 0, 4 * sizeof(unsigned), s));      // slots U, D, O, P
         CU(launch_absmax(h->H, n, n, n, SPLIT_UPPER, 1.f, am + AMAX_U, h->num_sms, s));
-        CU(launch_absmax(h->D, n, n, n, SPLIT_ALL, inv_tokens, am + AMAX_D, h->num_sms, s));
+        // (of dXX^T only the entries above the diagonal reach O: row j of U starts at column j and M_U keeps j > i)
+        CU(launch_absmax(h->D, n, n, n, SPLIT_STRICT_UPPER, inv_tokens, am + AMAX_D, h->num_sms, s));
         CU(launch_split16(h->H, n, U16, U16 + nn, n, n, n, false, SPLIT_UPPER, 1.f, am + AMAX_U, s));
         CU(launch_split16(h->H, n, UT16, UT16 + nn, n, n, n, true, SPLIT_UPPER, 1.f, am + AMAX_U, s));
-        CU(launch_split16(h->D, n, A16, A16 + nn, n, n, n, false, SPLIT_ALL, inv_tokens, am + AMAX_D, s));
+        CU(launch_split16(h->D, n, A16, A16 + nn, n, n, n, false, SPLIT_STRICT_UPPER, inv_tokens, am + AMAX_D, s));
         h->launches += 5;
         const SplitOperand Uop{U16, U16 + nn, n, n, n, true}, UTop{UT16, UT16 + nn, n, n, n, true};
         const SplitOperand Aop{A16, A16 + nn, n, n, n, true};
