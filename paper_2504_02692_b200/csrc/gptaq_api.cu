@@ -330,15 +330,17 @@ struct SplitBatch {
     int rows_last = 0, cols_last = 0;
 };
 
+// hi_t / lo_t non-null: the transposed form goes there in the same pass (transpose is then ignored)
 cudaError_t launch_split16(const float *src, int64_t lds, __half *hi, __half *lo, int64_t ldd, int rows, int cols,
                            bool transpose, int mask, float scale, const unsigned *amax, cudaStream_t s,
-                           const SplitBatch &b = SplitBatch()) {
+                           const SplitBatch &b = SplitBatch(), __half *hi_t = nullptr, __half *lo_t = nullptr) {
     if (rows <= 0 || cols <= 0 || b.nbatch <= 0) return cudaSuccess;
     Split16Args a;
     a.src = src; a.lds = lds; a.src_bstride = b.src_bstride; a.hi = hi; a.lo = lo; a.ldd = ldd;
     a.dst_bstride = b.dst_bstride;
     a.rows = rows; a.cols = cols; a.rows_last = b.rows_last; a.cols_last = b.cols_last; a.nbatch = b.nbatch;
-    a.transpose = transpose ? 1 : 0; a.mask = mask; a.scale = scale; a.amax = amax;
+    a.transpose = hi_t ? 2 : (transpose ? 1 : 0); a.mask = mask; a.scale = scale; a.amax = amax;
+    a.hi_t = hi_t; a.lo_t = lo_t;
     dim3 grid((cols + 63) / 64, (rows + 63) / 64, b.nbatch);
     split16_kernel<<<grid, 256, 0, s>>>(a);
     return cudaGetLastError();
@@ -1211,10 +1213,10 @@ gptaq_status_t gptaq_build_P(gptaq_handle_t h, float alpha, gptaq_stream_t strea
         CU(launch_absmax(h->H, n, n, n, SPLIT_UPPER, 1.f, am + AMAX_U, h->num_sms, s));
         // (of dXX^T only the entries above the diagonal reach O: row j of U starts at column j and M_U keeps j > i)
         CU(launch_absmax(h->D, n, n, n, SPLIT_STRICT_UPPER, inv_tokens, am + AMAX_D, h->num_sms, s));
-        CU(launch_split16(h->H, n, U16, U16 + nn, n, n, n, false, SPLIT_UPPER, 1.f, am + AMAX_U, s));
-        CU(launch_split16(h->H, n, UT16, UT16 + nn, n, n, n, true, SPLIT_UPPER, 1.f, am + AMAX_U, s));
+        CU(launch_split16(h->H, n, U16, U16 + nn, n, n, n, false, SPLIT_UPPER, 1.f, am + AMAX_U, s, SplitBatch(),
+                          UT16, UT16 + nn));        // U and U^T in one pass
         CU(launch_split16(h->D, n, A16, A16 + nn, n, n, n, false, SPLIT_STRICT_UPPER, inv_tokens, am + AMAX_D, s));
-        h->launches += 5;
+        h->launches += 4;
         const SplitOperand Uop{U16, U16 + nn, n, n, n, true}, UTop{UT16, UT16 + nn, n, n, n, true};
         const SplitOperand Aop{A16, A16 + nn, n, n, n, true};
         TcMaps maps;

@@ -565,9 +565,10 @@ struct Split16Args {
     const float *src; long long lds, src_bstride;
     __half *hi, *lo; long long ldd, dst_bstride;
     int rows, cols, rows_last, cols_last, nbatch;      // blockIdx.z walks batch entries, as in split_kernel
-    int transpose, mask;
+    int transpose, mask;       // transpose 2: both forms, the plain one to (hi, lo), the transposed one to (hi_t, lo_t)
     float scale;
     const unsigned *amax;
+    __half *hi_t, *lo_t;
 };
 
 __device__ __forceinline__ void split16_pack(const float (&x)[4], uint2 &hi, uint2 &lo) {
@@ -595,6 +596,7 @@ __global__ void __launch_bounds__(256) split16_kernel(Split16Args a) {
         a.src += (long long)z * a.src_bstride;
         a.hi += (long long)z * a.dst_bstride;
         a.lo += (long long)z * a.dst_bstride;
+        if (a.transpose == 2) { a.hi_t += (long long)z * a.dst_bstride; a.lo_t += (long long)z * a.dst_bstride; }
     }
     const float s = a.scale * split_scale(__uint_as_float(*a.amax));
     const int tq = threadIdx.x & 15, ty = threadIdx.x >> 4;        // 16 quads x 16 rows
@@ -627,7 +629,7 @@ __global__ void __launch_bounds__(256) split16_kernel(Split16Args a) {
             const bool keep = a.mask == SPLIT_ALL || (a.mask == SPLIT_UPPER ? c + e >= r : c + e > r);
             x[e] = keep ? s * xs[i][e] : 0.f;
         }
-        if (!a.transpose) {
+        if (a.transpose != 1) {
             if (r < a.rows && c < a.cols) {
                 uint2 hi, lo;
                 split16_pack(x, hi, lo);
@@ -640,12 +642,14 @@ __global__ void __launch_bounds__(256) split16_kernel(Split16Args a) {
                     for (int e = 0; c + e < a.cols; ++e) { ph[e] = hh[e]; pl[e] = ll[e]; }
                 }
             }
-        } else {
+        }
+        if (a.transpose) {
 #pragma unroll
             for (int e = 0; e < 4; ++e) tile[rr][4 * tq + e] = x[e];
         }
     }
     if (a.transpose) {
+        __half *th = a.transpose == 2 ? a.hi_t : a.hi, *tl = a.transpose == 2 ? a.lo_t : a.lo;
         __syncthreads();
         // destination row = source column c, destination columns = source rows r0 + 4 * tq ..
         for (int cc = ty; cc < 64; cc += 16) {
@@ -654,7 +658,7 @@ __global__ void __launch_bounds__(256) split16_kernel(Split16Args a) {
             const float x[4] = {tile[4 * tq][cc], tile[4 * tq + 1][cc], tile[4 * tq + 2][cc], tile[4 * tq + 3][cc]};
             uint2 hi, lo;
             split16_pack(x, hi, lo);
-            __half *ph = a.hi + (long long)c * a.ldd + r, *pl = a.lo + (long long)c * a.ldd + r;
+            __half *ph = th + (long long)c * a.ldd + r, *pl = tl + (long long)c * a.ldd + r;
             if (r + 3 < a.rows) {
                 *reinterpret_cast<uint2 *>(ph) = hi;
                 *reinterpret_cast<uint2 *>(pl) = lo;
